@@ -1,0 +1,395 @@
+#!/usr/bin/env python
+"""Benchmark of the SAGE selection hot path on B200.
+
+A "step" is one pass of the whole path over one synthetic workload: pass 1 (Frequent-Directions sketch
+of all N rows, including the freeze), pass 2 (projection, normalisation, consensus, agreement scores)
+and the top-k selection(s). Metric: gradient rows per second through the whole path (N / step time),
+summed over ranks; with more than one GPU every rank runs an independent replica of the workload.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0). `--impl reference` times the fp64 CPU oracle on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+METRIC = "gradient rows/s (FD sketch + agreement scoring + top-k, whole path)"
+UNIT = "rows/s"
+FP32_ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12     # SMs x FMA lanes x 2 flop x max SM clock
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def shrink_schedule(N: int, ell: int):
+    """Row counts of every factorisation of one pass 1: full buffers (m rows) and the final one."""
+    m, keep = 2 * ell, ell - 1
+    fill, full = 0, 0
+    left = N
+    while left > 0:
+        take = min(left, m - fill)
+        fill += take
+        left -= take
+        if fill == m:
+            full += 1
+            fill = keep
+    return full, fill
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                                       "-i", str(self.gpu)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons, power = [], [], set(), []
+        for line in self.f.read().splitlines():
+            c = [x.strip() for x in line.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1]))
+                mx.append(float(c[2]))
+                power.append(float(c[3]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), c[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        os.unlink(self.f.name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def cpu_oracle_sample(w, seed, sample_rows):
+    """The oracle, as it stands, on the first `sample_rows` rows of the workload, on the host cores."""
+    import oracle
+    from paper_2510_02470_b200 import workloads as wl
+    if w.on_device:
+        stream = wl.DeviceStream(wl.scaled(w, N=sample_rows), seed, "cuda" if torch.cuda.is_available() else "cpu")
+        rows = torch.cat([stream.chunk(j) for j in range((sample_rows + w.chunk_rows - 1) // w.chunk_rows)])[:sample_rows].cpu()
+    else:
+        rows = wl.host_rows(w, seed, sample_rows)
+    oracle.lib()
+    t0 = time.perf_counter()
+    out = oracle.run(rows, w.D, w.ell, w.keep_rates[0], route=0 if w.D <= 20000 else 1)
+    dt = time.perf_counter() - t0
+    cores = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
+    return {"value": sample_rows / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"first {sample_rows} rows of {w.name} through sketch+freeze+score+select, {dt:.1f} s, "
+                      f"{out['stats']['shrinks']} shrinks, SVD route {'rows (Hestenes)' if w.D <= 20000 else 'Gram'}",
+            "seconds": dt}
+
+
+CPU_SAMPLE_ROWS = {"c1": 4096, "c2": 6000, "c3": 1200, "c4": 768, "c5": 256}
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sample = CPU_SAMPLE_ROWS[w.name]
+    times = []
+    base = None
+    for i in range(args.warmup + args.steps):
+        base = cpu_oracle_sample(w, 0, sample)
+        if i >= args.warmup:
+            times.append(base["seconds"])
+    dt = sum(times) / len(times)
+    v = sample / dt
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "N": w.N, "D": w.D, "ell": w.ell, "rows_dtype": str(w.dtype).replace("torch.", ""),
+                       "sample_rows_per_step": sample},
+            "cpu_baseline": {"value": v, "unit": UNIT, "cores": base["cores"], "kind": "oracle", "sample": base["sample"]},
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}, "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--rows", type=int, default=0, help="use only the first ROWS rows of the workload (debugging)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--seed", type=int, default=0)
+    args = ap.parse_args()
+
+    from paper_2510_02470_b200 import workloads as wl
+    w = wl.WORKLOADS[args.workload]
+    if args.rows:
+        w = wl.scaled(w, N=args.rows)
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+    args.warmup = max(args.warmup, 3)
+
+    import paper_2510_02470_b200 as sage
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    sage.lib()
+
+    N, D, ell = w.N, w.D, w.ell
+    e = w.elem_bytes
+    # ---- inputs ------------------------------------------------------------------------------------
+    t_gen0 = time.perf_counter()
+    host_rows = None
+    stream = None
+    if w.on_device:
+        stream = wl.DeviceStream(w, args.seed, dev)
+        chunk_buf = torch.zeros((w.chunk_rows, w.ld), dtype=w.dtype, device=dev)
+    else:
+        host_rows = wl.host_rows(w, args.seed).pin_memory()
+        rows = host_rows.to(dev, non_blocking=True)
+    torch.cuda.synchronize()
+    t_gen = time.perf_counter() - t_gen0
+
+    fd = sage.SageFD(D, ell, w.dtype, local)
+    scores = torch.empty((N,), dtype=torch.float32, device=dev)
+    idx_bufs = [torch.empty((sage.sage_select_count(N, r),), dtype=torch.int64, device=dev) for r in w.keep_rates]
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    gen_ms = [0.0]
+
+    def one_step(phase_events=None):
+        """sketch all rows -> freeze -> score all rows -> select; returns nothing (results stay on device)."""
+        marks = [ev() for _ in range(4)] if phase_events is not None else None
+        fd.reset()
+        if marks: marks[0].record()
+        if stream is None:
+            fd.update(rows)
+        else:
+            for j in range(w.num_chunks):
+                g0, g1 = ev(), ev()
+                g0.record()
+                c = stream.chunk(j, chunk_buf)
+                g1.record()
+                fd.update(c)
+                if phase_events is not None:
+                    phase_events.setdefault("gen", []).append((g0, g1))
+        fd.finalize(allow=(6, 7))
+        if marks: marks[1].record()
+        if stream is None:
+            fd.score(rows, scores)
+        else:
+            fd.score_begin(N)
+            for j in range(w.num_chunks):
+                g0, g1 = ev(), ev()
+                g0.record()
+                c = stream.chunk(j, chunk_buf)
+                g1.record()
+                fd.score_chunk(c, j * w.chunk_rows)
+                if phase_events is not None:
+                    phase_events.setdefault("gen", []).append((g0, g1))
+            fd.score_end(scores)
+        if marks: marks[2].record()
+        for r, ib in zip(w.keep_rates, idx_bufs):
+            sage.sage_select(scores, r, ib)
+        if marks:
+            marks[3].record()
+            phase_events["marks"] = marks
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---- warm-up (the last warm-up step is profiled per kernel class to find the dominant kernel) ----
+    for i in range(args.warmup):
+        if i == args.warmup - 1:
+            fd.set_option(3, 0x1FF)
+            fd.profile()
+        one_step()
+    torch.cuda.synchronize()
+    prof_all = fd.profile()
+    dominant = max(prof_all, key=lambda k: prof_all[k]["ms"])
+    dom_bit = sage.KERNEL_CLASSES.index(dominant)
+    fd.set_option(3, 1 << dom_bit)          # during the timed region only the dominant kernel is bracketed by events
+
+    # ---- timed region -----------------------------------------------------------------------------------
+    sampler = ClockSampler(local)
+    phase = [dict() for _ in range(args.steps)]
+    launches0 = sage.sage_launch_count()
+    barrier()
+    sampler.start()
+    t0, t1 = ev(), ev()
+    t0.record()
+    for s in range(args.steps):
+        one_step(phase[s])
+    t1.record()
+    barrier()
+    clocks = sampler.stop()
+    launches = sage.sage_launch_count() - launches0
+    total_ms = t0.elapsed_time(t1)
+    gen_total_ms = sum(a.elapsed_time(b) for p in phase for (a, b) in p.get("gen", []))
+    step_ms = (total_ms - gen_total_ms) / args.steps          # generator time (streamed workloads) excluded
+    prof_dom = fd.profile()[dominant]
+    p1 = statistics.mean(p["marks"][0].elapsed_time(p["marks"][1]) for p in phase)
+    p2 = statistics.mean(p["marks"][1].elapsed_time(p["marks"][2]) for p in phase)
+    p3 = statistics.mean(p["marks"][2].elapsed_time(p["marks"][3]) for p in phase)
+    gen_per_step = gen_total_ms / args.steps
+    stats = fd.stats()
+
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([step_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        step_ms = float(t.item())
+    value = world * N / (step_ms * 1e-3)
+
+    # ---- roofline of the dominant kernel -------------------------------------------------------------------
+    peaks = measured_peaks()
+    full, r_final = shrink_schedule(N, ell)
+    m, keep = 2 * ell, ell - 1
+    keep_final = (ell - 1) if r_final > ell else min(r_final, ell)
+    per_step_bytes = {
+        "append": N * D * (e + 4),
+        "gram": (full * m + r_final) * D * 4,
+        "rebuild": (full * (m + keep) + (r_final + max(keep_final, ell))) * D * 4,
+        "project": N * D * e,
+        "normalise": N * ell * 8,
+        "score": N * ell * 4 + N * 4,
+    }
+    eig_flops = 9.0 * (full * m ** 3 + r_final ** 3)
+    dom_ms_per_step = prof_dom["ms"] / args.steps
+    dom_launches_per_step = prof_dom["launches"] / args.steps
+    if dominant == "eig_shrink":
+        achieved = eig_flops / (dom_ms_per_step * 1e-3) / 1e12
+        roof = {"kernel": "k_eig_shrink", "bound": "alu", "achieved": achieved, "peak": FP32_ALU_PEAK_TFLOPS, "unit": "TFLOP/s",
+                "frac": achieved / FP32_ALU_PEAK_TFLOPS, "traffic": None,
+                "peak_source": "derived: 148 SMs x 128 fp32 FMA lanes x 2 flop x 1.965 GHz",
+                "algorithmic": "9*n^3 flop per n x n symmetric eigen-solve (textbook count)"}
+    else:
+        gbs = per_step_bytes.get(dominant, 0) / (dom_ms_per_step * 1e-3) / 1e9
+        roof = {"kernel": dominant, "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": f"{peaks['source']} STREAM-style copy"}
+    roof["avg_launch_ms"] = dom_ms_per_step / max(dom_launches_per_step, 1)
+    roof["launches_per_step"] = dom_launches_per_step
+    roof["share_of_step"] = dom_ms_per_step / step_ms
+    kernels = {}
+    for name, v in prof_all.items():
+        if v["launches"] == 0:
+            continue
+        entry = {"ms_per_step": v["ms"], "launches_per_step": v["launches"]}
+        if name in per_step_bytes and v["ms"] > 0:
+            entry["GBps"] = per_step_bytes[name] / (v["ms"] * 1e-3) / 1e9
+            entry["frac_of_hbm"] = entry["GBps"] / peaks["hbm_gbs"]
+        kernels[name] = entry
+    roof_pass2_s = max(N * D * e / (peaks["hbm_gbs"] * 1e9), 2.0 * N * ell * D / (peaks["bf16_tflops_sustained"] * 1e12))
+    p1_bytes = per_step_bytes["append"] + per_step_bytes["gram"] + per_step_bytes["rebuild"]
+    roof_pass1_s = p1_bytes / (peaks["hbm_gbs"] * 1e9)
+
+    # ---- end to end through the host-pointer entry point ------------------------------------------------
+    e2e = None
+    if not args.no_e2e and host_rows is not None:
+        fd.close()
+        del rows
+        torch.cuda.empty_cache()
+        reps = max(1, min(args.steps, 3))
+        sage.sage_select_from_host(host_rows, D, ell, w.keep_rates[0], 0, local)      # warm-up
+        torch.cuda.synchronize()
+        t_e = time.perf_counter()
+        for _ in range(reps):
+            sc, ix = sage.sage_select_from_host(host_rows, D, ell, w.keep_rates[0], 0, local)
+        torch.cuda.synchronize()
+        dt = (time.perf_counter() - t_e) / reps
+        if world > 1:
+            import torch.distributed as dist
+            t = torch.tensor([dt], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t.item())
+        e2e = {"value": world * N / dt, "unit": UNIT, "h2d_bytes_per_step": 2 * N * w.ld * e,
+               "d2h_bytes_per_step": N * 4 + int(ix.numel()) * 8, "ms_per_step": dt * 1e3,
+               "call": "sage_select_from_host (pinned host rows, both passes streamed over PCIe, one keep_rate)"}
+    elif not args.no_e2e:
+        e2e = {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
+               "note": "workload is generated on the device chunk by chunk (it does not fit host or device memory as N x D)"}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        b = cpu_oracle_sample(w, args.seed, min(CPU_SAMPLE_ROWS[w.name], N))
+        cpu = {k: b[k] for k in ("value", "unit", "cores", "kind", "sample")}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "N": N, "D": D, "ell": ell, "rows_dtype": str(w.dtype).replace("torch.", ""),
+                       "ld": w.ld, "keep_rates": list(w.keep_rates), "multi_gpu": "replicas only",
+                       "l2": "inputs larger than L2" if N * D * e > 200e6 else "inputs fit in L2 (no flush: stated, c1 only)",
+                       "generator_ms_per_step_excluded": gen_per_step, "input_generation_s": t_gen},
+            "passes": {"pass1_ms": p1, "pass2_ms": p2, "select_ms": p3,
+                       "pass1_rows_per_s": N / (p1 * 1e-3) if p1 > 0 else None, "pass2_rows_per_s": N / (p2 * 1e-3) if p2 > 0 else None,
+                       "pass1_frac_of_hbm_roofline": roof_pass1_s / (p1 * 1e-3) if p1 > 0 else None,
+                       "pass2_frac_of_roofline": roof_pass2_s / (p2 * 1e-3) if p2 > 0 else None,
+                       "note": "pass times include streamed generator time" if stream is not None else ""},
+            "roofline": roof, "kernels_profiled_step": kernels,
+            "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
+            "clocks": clocks, "fd_stats": {k: stats[k] for k in ("shrinks", "max_sweeps", "last_rank", "device_flags")},
+        }
+        print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

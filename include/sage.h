@@ -1,0 +1,177 @@
+/*
+ * sage.h -- C ABI of the B200 (sm_100a) implementation of SAGE's two-pass selection hot path.
+ *
+ * The path (paper: Method section and Algorithm 1):
+ *   pass 1  stream per-example gradient rows into a Frequent-Directions sketch
+ *           (Algorithm 1, Phase I; Method, first paragraph),
+ *   freeze  the ell x D sketch S (Algorithm 1, "Freeze S for scoring"),
+ *   pass 2  z_i = S g_i, zhat_i = z_i/||z_i||, consensus u, agreement score alpha_i = <zhat_i, u>
+ *           (Method, "Two-pass scoring"; Algorithm 1, Phase II),
+ *   select  the top-k examples by alpha (Algorithm 1, "Select top-k by alpha_i").
+ *
+ * Conventions shared by every entry point
+ *   - Every function returns a sage_status_t; nothing throws or aborts. Out-parameters are written only
+ *     on SAGE_OK. sage_last_error() returns a thread-local, human-readable message for the last failure.
+ *   - Pointers named rows / scores / idx are DEVICE pointers owned by the caller unless the parameter
+ *     says "host". The library never frees them and does not use them after the stream work it
+ *     enqueued has finished.
+ *   - Rows are row-major with a pitch `ld` counted in elements (ld >= D). Element type is the handle's
+ *     row dtype (float32, or bfloat16 stored as 16-bit words).
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream). Work is
+ *     enqueued asynchronously on it unless the entry point documents a synchronisation.
+ *   - A handle belongs to one device and one host thread at a time. Calls on one handle must be issued
+ *     on one stream (or on streams the caller has ordered).
+ *   - Rows are consumed strictly in the order given: the sketch depends on row order.
+ *   - There is no CPU fallback: without a usable CUDA device every compute entry point fails with
+ *     SAGE_ERR_CUDA.
+ */
+#ifndef SAGE_B200_H_
+#define SAGE_B200_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sage_fd sage_fd_t; /* opaque, library-owned */
+
+typedef enum {
+    SAGE_OK = 0,
+    SAGE_ERR_INVALID_ARG = 1,   /* null pointer, non-positive size, ld < D, keep_rate not finite, ... */
+    SAGE_ERR_BAD_STATE = 2,     /* call order violates the state machine below */
+    SAGE_ERR_ALLOC = 3,         /* device or host allocation failed */
+    SAGE_ERR_CUDA = 4,          /* a CUDA runtime call failed (see sage_last_error) */
+    SAGE_ERR_UNSUPPORTED = 5,   /* size outside the supported range */
+    SAGE_ERR_NOT_CONVERGED = 6, /* the eigen-solver hit its sweep limit (results were still produced) */
+    SAGE_ERR_NONFINITE = 7      /* a NaN/Inf was met in the input rows (such rows score 0) */
+} sage_status_t;
+
+typedef enum { SAGE_F32 = 0, SAGE_BF16 = 1 } sage_dtype_t;
+
+/* State machine of a handle:
+ *   create -> SKETCHING --update*--> SKETCHING --finalize--> FROZEN
+ *   FROZEN --score_begin--> SCORING --score_chunk*--> SCORING --score_end--> FROZEN
+ *   sage_score() = score_begin + one score_chunk + score_end.  sage_fd_reset() returns to SKETCHING.
+ */
+
+/* Frequent-Directions sketch state for rows of dimension D with sketch size ell (Method, first
+ * paragraph; Algorithm 1 line "Initialize S"). The library keeps a buffer of 2*ell rows in fp32: rows
+ * are appended into free rows and the buffer is shrunk when all 2*ell rows are in use.
+ *   out        receives the handle (host pointer).
+ *   D          row dimension, 1 <= D.
+ *   ell        sketch size, 2 <= ell <= 256.
+ *   row_dtype  element type of every rows pointer later given to this handle.
+ *   device     CUDA device ordinal; all later calls must be made with pointers of this device.
+ * Allocates about 2 * (2*ell) * D * 4 bytes of device memory. Synchronous. */
+sage_status_t sage_fd_create(sage_fd_t** out, int64_t D, int32_t ell, sage_dtype_t row_dtype, int device);
+
+/* Releases everything the handle owns (synchronises the device first). NULL is allowed. */
+void sage_fd_destroy(sage_fd_t* h);
+
+/* Forget all rows and return to SKETCHING, keeping the allocations. Synchronous. */
+sage_status_t sage_fd_reset(sage_fd_t* h);
+
+/* Algorithm 1, Phase I, for n rows: append each row to the buffer; whenever the buffer is full,
+ * factor it (SVD through the eigen-decomposition of the 2ell x 2ell Gram matrix), set
+ * delta = sigma_ell^2, Sigma'_jj = sqrt(max(sigma_j^2 - delta, 0)) and rebuild S <- Sigma' V^T
+ * (Method, first paragraph). ell-1 rows survive a shrink, so after the first 2*ell rows a shrink
+ * happens every ell+1 rows.
+ *   rows  device, n x ld elements of the handle's dtype; n == 0 is a no-op.
+ * Asynchronous on the stream: the shrink schedule depends only on counts, so no device->host
+ * synchronisation happens here. Device-side problems are reported by sage_fd_finalize. */
+sage_status_t sage_fd_update(sage_fd_t* h, const void* rows, int64_t n, int64_t ld, void* cuda_stream);
+
+/* Algorithm 1, "Freeze S for scoring": orthogonalise what the buffer holds, apply the shrink only if
+ * more than ell rows are in use (so N <= ell is exact), keep the first ell rows as S.
+ * Synchronises the stream once and returns SAGE_ERR_NOT_CONVERGED / SAGE_ERR_NONFINITE if the device
+ * recorded such an event during pass 1 (the sketch is still usable). */
+sage_status_t sage_fd_finalize(sage_fd_t* h, void* cuda_stream);
+
+/* Borrowed pointers to the frozen sketch: S is ell x D fp32 on the device with pitch *pitch
+ * elements, sigma holds its ell row norms sigma'_j (device, fp32). Valid until reset/destroy.
+ * Requires FROZEN or later. Any out-pointer may be NULL. */
+sage_status_t sage_fd_sketch(const sage_fd_t* h, const float** S, int64_t* pitch, const float** sigma);
+
+/* Replace the frozen sketch by caller data (ell x D fp32, device, pitch ld): scoring with a sketch
+ * computed elsewhere. Moves the handle to FROZEN. Asynchronous on the stream. */
+sage_status_t sage_fd_load_sketch(sage_fd_t* h, const float* S, int64_t ld, void* cuda_stream);
+
+/* Algorithm 1, Phase II on n resident rows: z_i = S g_i, zhat_i, u, alpha_i = <zhat_i, u>.
+ *   scores  device, n floats. Rows whose projection is exactly zero (or non-finite) score 0; if the
+ *           consensus is zero every score is 0.
+ * Asynchronous on the stream. */
+sage_status_t sage_score(sage_fd_t* h, const void* rows, int64_t n, int64_t ld, float* scores, void* cuda_stream);
+
+/* Streamed form of Phase II for row sets that are not resident: announce the total row count, feed
+ * chunks (each read once), then finish. row_offset is the index of the chunk's first row in
+ * [0, N_total); chunks must tile [0, N_total) without overlap and be given in ascending order.
+ * The library keeps the N_total x ell normalised projections between chunk and end, because the
+ * consensus direction is only known once every row has been seen. */
+sage_status_t sage_score_begin(sage_fd_t* h, int64_t N_total, void* cuda_stream);
+sage_status_t sage_score_chunk(sage_fd_t* h, const void* rows, int64_t n, int64_t ld, int64_t row_offset,
+                               void* cuda_stream);
+sage_status_t sage_score_end(sage_fd_t* h, float* scores, void* cuda_stream);
+
+/* Borrowed device pointers to the last scoring pass's intermediates (for checks of the lemma in
+ * "Energy preservation"): zhat N x ell fp32, znorm N fp32 (||z_i||), u ell fp32. Any may be NULL. */
+sage_status_t sage_score_intermediates(const sage_fd_t* h, const float** zhat, const float** znorm, const float** u);
+
+/* Number of indices sage_select returns for N scores: floor(keep_rate*N + 0.5) clamped to [0, N]. */
+int64_t sage_select_count(int64_t N, double keep_rate);
+
+/* Algorithm 1, "Select top-k by alpha_i": the k = sage_select_count(N, keep_rate) largest scores,
+ * ordered by (score descending, index ascending); equal scores go to the smaller index. NaN scores
+ * rank below every number.
+ *   scores  device, N floats.         idx    device, capacity >= k int64 values.
+ *   k_out   host, receives k (may be NULL).
+ * Allocates and frees O(N) scratch on the device; asynchronous on the stream apart from that. */
+sage_status_t sage_select(const float* scores, int64_t N, double keep_rate, int64_t* idx, int64_t* k_out,
+                          void* cuda_stream);
+
+/* The whole path for rows that live in HOST memory (pinned memory gives overlap of copies and
+ * kernels): streams the rows to the device in chunks for pass 1, freezes, streams them again for
+ * pass 2, selects, and copies scores (N floats, may be NULL) and indices back to the host.
+ * Synchronous. chunk_rows <= 0 picks a default. */
+sage_status_t sage_select_from_host(const void* rows_host, int64_t N, int64_t D, int64_t ld, int32_t ell,
+                                    sage_dtype_t row_dtype, double keep_rate, int64_t chunk_rows, int device,
+                                    float* scores_host, int64_t* idx_host, int64_t* k_out);
+
+typedef struct {
+    int64_t rows_seen;      /* rows given to sage_fd_update since create/reset */
+    int64_t shrinks;        /* shrinks applied (including the one in finalize, if any) */
+    double sum_delta;       /* sum of delta over shrinks: an upper bound on ||G^T G - S^T S||_2 */
+    int32_t last_sweeps;    /* Jacobi sweeps of the most recent eigen-solve */
+    int32_t max_sweeps;     /* largest sweep count seen */
+    int32_t last_rank;      /* numerical rank found by the most recent factorisation */
+    uint32_t device_flags;  /* bit 0: eigen-solver not converged, bit 1: non-finite input seen */
+    int64_t kernel_launches;/* kernels this handle has launched since create/reset */
+} sage_stats_t;
+
+/* Synchronises the device and reads the counters back. */
+sage_status_t sage_fd_stats(sage_fd_t* h, sage_stats_t* out);
+
+/* Options. Before the first update: key 1 = delta rank (which singular value, 1-indexed, defines
+ * delta; default ell), key 2 = maximum Jacobi sweeps (default 30). At any time: key 3 = bit mask of
+ * kernel classes to time with CUDA events on the launching stream (see sage_fd_profile; default 0). */
+sage_status_t sage_fd_set_option(sage_fd_t* h, int key, double value);
+
+/* Per-kernel device time of this handle's launches since the previous call, for the classes selected
+ * with option 3. Class indices: 0 append, 1 Gram, 2 Gram split reduction, 3 eigen-solve + shrink,
+ * 4 rebuild, 5 projection, 6 projection split reduction, 7 normalise + consensus partials, 8 consensus
+ * + score. ms[c] is the summed event time in milliseconds and launches[c] the number of timed launches.
+ * capacity is the length of both host arrays (>= 9). Synchronises the device. */
+sage_status_t sage_fd_profile(sage_fd_t* h, double* ms, int64_t* launches, int32_t capacity);
+
+const char* sage_status_string(sage_status_t s);
+const char* sage_last_error(void);
+/* Library version string, e.g. for logs. */
+const char* sage_version(void);
+/* Number of kernels this library has launched in the calling process so far (all handles and
+ * sage_select together); a benchmark takes the difference around its timed region. */
+int64_t sage_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SAGE_B200_H_ */

@@ -1,0 +1,304 @@
+"""Thin Python binding of the C ABI in ``include/sage.h`` (argument marshalling only).
+
+Every function here has the name of the C entry point it calls; tensors are turned into raw device
+pointers plus sizes, the current torch CUDA stream is passed as the ``cuda_stream`` argument, and a
+non-zero status raises :class:`SageError`. All arithmetic happens in the CUDA library
+(``libsage_b200.so``, built in-tree by ``python -m paper_2510_02470_b200.build``). There is no CPU
+path: if the library is missing, loading it raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Tuple
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_PKG, "libsage_b200.so")
+_lib: Optional[C.CDLL] = None
+
+SAGE_F32, SAGE_BF16 = 0, 1
+STATUS_NAMES = {0: "SAGE_OK", 1: "SAGE_ERR_INVALID_ARG", 2: "SAGE_ERR_BAD_STATE", 3: "SAGE_ERR_ALLOC",
+                4: "SAGE_ERR_CUDA", 5: "SAGE_ERR_UNSUPPORTED", 6: "SAGE_ERR_NOT_CONVERGED", 7: "SAGE_ERR_NONFINITE"}
+
+# name -> (restype, argtypes); the list every test of the boundary checks against include/sage.h
+_i64, _i32, _f64, _vp, _u32 = C.c_int64, C.c_int32, C.c_double, C.c_void_p, C.c_uint32
+SIGNATURES = {
+    "sage_fd_create": (_i32, [_vp, _i64, _i32, _i32, _i32]),
+    "sage_fd_destroy": (None, [_vp]),
+    "sage_fd_reset": (_i32, [_vp]),
+    "sage_fd_update": (_i32, [_vp, _vp, _i64, _i64, _vp]),
+    "sage_fd_finalize": (_i32, [_vp, _vp]),
+    "sage_fd_sketch": (_i32, [_vp, _vp, _vp, _vp]),
+    "sage_fd_load_sketch": (_i32, [_vp, _vp, _i64, _vp]),
+    "sage_score": (_i32, [_vp, _vp, _i64, _i64, _vp, _vp]),
+    "sage_score_begin": (_i32, [_vp, _i64, _vp]),
+    "sage_score_chunk": (_i32, [_vp, _vp, _i64, _i64, _i64, _vp]),
+    "sage_score_end": (_i32, [_vp, _vp, _vp]),
+    "sage_score_intermediates": (_i32, [_vp, _vp, _vp, _vp]),
+    "sage_select_count": (_i64, [_i64, _f64]),
+    "sage_select": (_i32, [_vp, _i64, _f64, _vp, _vp, _vp]),
+    "sage_select_from_host": (_i32, [_vp, _i64, _i64, _i64, _i32, _i32, _f64, _i64, _i32, _vp, _vp, _vp]),
+    "sage_fd_stats": (_i32, [_vp, _vp]),
+    "sage_fd_set_option": (_i32, [_vp, _i32, _f64]),
+    "sage_fd_profile": (_i32, [_vp, _vp, _vp, _i32]),
+    "sage_status_string": (C.c_char_p, [_i32]),
+    "sage_last_error": (C.c_char_p, []),
+    "sage_version": (C.c_char_p, []),
+    "sage_launch_count": (_i64, []),
+}
+
+
+class SageStats(C.Structure):
+    _fields_ = [("rows_seen", _i64), ("shrinks", _i64), ("sum_delta", _f64), ("last_sweeps", _i32),
+                ("max_sweeps", _i32), ("last_rank", _i32), ("device_flags", _u32), ("kernel_launches", _i64)]
+
+
+class SageError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"{STATUS_NAMES.get(status, status)}: {message}")
+        self.status = status
+
+
+def lib() -> C.CDLL:
+    """Loads the CUDA library; raises if it has not been built (there is no fallback)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(f"{_LIB_PATH} is missing: build it with `python -m paper_2510_02470_b200.build`")
+        L = C.CDLL(_LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(L, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = L
+    return _lib
+
+
+def _check(status: int, allow=()) -> int:
+    if status != 0 and status not in allow:
+        raise SageError(status, lib().sage_last_error().decode())
+    return status
+
+
+def _stream(device=None) -> int:
+    return torch.cuda.current_stream(device).cuda_stream
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return SAGE_F32
+    if t.dtype == torch.bfloat16:
+        return SAGE_BF16
+    raise TypeError(f"rows must be float32 or bfloat16, got {t.dtype}")
+
+
+def _rows_args(rows: torch.Tensor, D: int) -> Tuple[int, int, int]:
+    if rows.dim() != 2 or rows.shape[1] < D or (rows.shape[0] > 1 and rows.stride(1) != 1):
+        raise ValueError("rows must be a 2-D tensor (n, >=D) with unit stride along D")
+    ld = rows.stride(0) if rows.shape[0] > 1 else max(rows.shape[1], D)
+    return rows.data_ptr(), rows.shape[0], ld
+
+
+# ---- functions named after the C entry points -----------------------------------------------------
+
+def sage_fd_create(D: int, ell: int, row_dtype: int, device: int = 0) -> int:
+    h = _vp()
+    _check(lib().sage_fd_create(C.byref(h), D, ell, row_dtype, device))
+    return h.value
+
+
+def sage_fd_destroy(h: int) -> None:
+    lib().sage_fd_destroy(h)
+
+
+def sage_fd_reset(h: int) -> None:
+    _check(lib().sage_fd_reset(h))
+
+
+def sage_fd_set_option(h: int, key: int, value: float) -> None:
+    _check(lib().sage_fd_set_option(h, key, value))
+
+
+def sage_fd_update(h: int, rows: torch.Tensor, D: int) -> None:
+    ptr, n, ld = _rows_args(rows, D)
+    _check(lib().sage_fd_update(h, ptr, n, ld, _stream(rows.device)))
+
+
+def sage_fd_finalize(h: int, device=None, allow=()) -> int:
+    return _check(lib().sage_fd_finalize(h, _stream(device)), allow)
+
+
+def sage_fd_sketch(h: int, ell: int, D: int, device) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Copies of the frozen sketch (ell x D) and sigma' (ell) as torch tensors on the device."""
+    S, pitch, sig = _vp(), _i64(), _vp()
+    _check(lib().sage_fd_sketch(h, C.byref(S), C.byref(pitch), C.byref(sig)))
+    out = _borrow(S.value, (ell, D), (pitch.value * 4, 4), device).clone()
+    sigma = _borrow(sig.value, (ell,), (4,), device).clone()
+    return out, sigma
+
+
+def sage_fd_load_sketch(h: int, S: torch.Tensor) -> None:
+    assert S.dtype == torch.float32 and S.dim() == 2 and S.stride(1) == 1
+    _check(lib().sage_fd_load_sketch(h, S.data_ptr(), S.stride(0), _stream(S.device)))
+
+
+def sage_score(h: int, rows: torch.Tensor, D: int, scores: torch.Tensor) -> None:
+    ptr, n, ld = _rows_args(rows, D)
+    assert scores.dtype == torch.float32 and scores.is_contiguous() and scores.numel() >= n
+    _check(lib().sage_score(h, ptr, n, ld, scores.data_ptr(), _stream(rows.device)))
+
+
+def sage_score_begin(h: int, N_total: int, device=None) -> None:
+    _check(lib().sage_score_begin(h, N_total, _stream(device)))
+
+
+def sage_score_chunk(h: int, rows: torch.Tensor, D: int, row_offset: int) -> None:
+    ptr, n, ld = _rows_args(rows, D)
+    _check(lib().sage_score_chunk(h, ptr, n, ld, row_offset, _stream(rows.device)))
+
+
+def sage_score_end(h: int, scores: torch.Tensor) -> None:
+    assert scores.dtype == torch.float32 and scores.is_contiguous()
+    _check(lib().sage_score_end(h, scores.data_ptr(), _stream(scores.device)))
+
+
+def sage_score_intermediates(h: int, N: int, ell: int, device) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor]:
+    zh, zn, u = _vp(), _vp(), _vp()
+    _check(lib().sage_score_intermediates(h, C.byref(zh), C.byref(zn), C.byref(u)))
+    zhat = _borrow(zh.value, (N, ell), (ell * 4, 4), device).clone()
+    znorm = _borrow(zn.value, (N,), (4,), device).clone()
+    uu = _borrow(u.value, (ell,), (4,), device).clone()
+    return zhat, znorm, uu
+
+
+def sage_select_count(N: int, keep_rate: float) -> int:
+    return int(lib().sage_select_count(N, keep_rate))
+
+
+def sage_select(scores: torch.Tensor, keep_rate: float, idx: Optional[torch.Tensor] = None) -> torch.Tensor:
+    assert scores.dtype == torch.float32 and scores.is_contiguous()
+    N = scores.numel()
+    k = sage_select_count(N, keep_rate)
+    if idx is None:
+        idx = torch.empty((k,), dtype=torch.int64, device=scores.device)
+    assert idx.dtype == torch.int64 and idx.numel() >= k
+    k_out = _i64(0)
+    _check(lib().sage_select(scores.data_ptr(), N, keep_rate, idx.data_ptr(), C.byref(k_out), _stream(scores.device)))
+    return idx[: k_out.value]
+
+
+def sage_select_from_host(rows: torch.Tensor, D: int, ell: int, keep_rate: float, chunk_rows: int = 0,
+                          device: int = 0, want_scores: bool = True):
+    """Whole path on HOST rows (pinned memory recommended). Returns (scores or None, idx) on the host."""
+    assert rows.device.type == "cpu"
+    ptr, N, ld = _rows_args(rows, D)
+    k = sage_select_count(N, keep_rate)
+    scores = torch.empty((N,), dtype=torch.float32).pin_memory() if want_scores else None
+    idx = torch.empty((max(k, 1),), dtype=torch.int64).pin_memory()
+    k_out = _i64(0)
+    st = lib().sage_select_from_host(ptr, N, D, ld, ell, _dtype_code(rows), keep_rate, chunk_rows, device,
+                                     scores.data_ptr() if want_scores else None, idx.data_ptr(), C.byref(k_out))
+    _check(st, allow=(6, 7))
+    return scores, idx[: k_out.value]
+
+
+def sage_fd_stats(h: int) -> dict:
+    s = SageStats()
+    _check(lib().sage_fd_stats(h, C.byref(s)))
+    return {name: getattr(s, name) for name, _ in SageStats._fields_}
+
+
+KERNEL_CLASSES = ("append", "gram", "gram_reduce", "eig_shrink", "rebuild", "project", "project_reduce",
+                  "normalise", "score")
+
+
+def sage_fd_profile(h: int) -> dict:
+    ms = (C.c_double * 16)()
+    n = (C.c_int64 * 16)()
+    _check(lib().sage_fd_profile(h, ms, n, 16))
+    return {name: {"ms": ms[i], "launches": n[i]} for i, name in enumerate(KERNEL_CLASSES)}
+
+
+def sage_launch_count() -> int:
+    return int(lib().sage_launch_count())
+
+
+def sage_version() -> str:
+    return lib().sage_version().decode()
+
+
+class _DevArray:
+    """Raw device memory described through __cuda_array_interface__ so that torch can view it."""
+
+    def __init__(self, ptr: int, shape, strides_bytes, typestr: str = "<f4"):
+        self.__cuda_array_interface__ = {"shape": tuple(shape), "strides": tuple(strides_bytes), "typestr": typestr,
+                                         "data": (int(ptr), False), "version": 2}
+
+
+def _borrow(ptr: int, shape, strides_bytes, device) -> torch.Tensor:
+    """A torch view (no copy) of library-owned device memory; callers clone what they keep."""
+    return torch.as_tensor(_DevArray(ptr, shape, strides_bytes), device=device)
+
+
+class SageFD:
+    """Convenience owner of a handle: ``update`` rows, ``finalize``, ``score``, ``select``."""
+
+    def __init__(self, D: int, ell: int, dtype: torch.dtype = torch.float32, device: int = 0):
+        self.D, self.ell, self.dtype, self.device = D, ell, dtype, device
+        self._h = sage_fd_create(D, ell, SAGE_F32 if dtype == torch.float32 else SAGE_BF16, device)
+
+    def update(self, rows: torch.Tensor) -> None:
+        assert rows.dtype == self.dtype
+        sage_fd_update(self._h, rows, self.D)
+
+    def finalize(self, allow=()) -> int:
+        return sage_fd_finalize(self._h, self.device, allow)
+
+    def sketch(self):
+        return sage_fd_sketch(self._h, self.ell, self.D, torch.device("cuda", self.device))
+
+    def load_sketch(self, S: torch.Tensor) -> None:
+        sage_fd_load_sketch(self._h, S)
+
+    def score(self, rows: torch.Tensor, scores: Optional[torch.Tensor] = None) -> torch.Tensor:
+        if scores is None:
+            scores = torch.empty((rows.shape[0],), dtype=torch.float32, device=rows.device)
+        sage_score(self._h, rows, self.D, scores)
+        return scores
+
+    def score_begin(self, N_total: int) -> None:
+        sage_score_begin(self._h, N_total, self.device)
+
+    def score_chunk(self, rows: torch.Tensor, row_offset: int) -> None:
+        sage_score_chunk(self._h, rows, self.D, row_offset)
+
+    def score_end(self, scores: torch.Tensor) -> None:
+        sage_score_end(self._h, scores)
+
+    def intermediates(self, N: int):
+        return sage_score_intermediates(self._h, N, self.ell, torch.device("cuda", self.device))
+
+    def stats(self) -> dict:
+        return sage_fd_stats(self._h)
+
+    def profile(self) -> dict:
+        return sage_fd_profile(self._h)
+
+    def reset(self) -> None:
+        sage_fd_reset(self._h)
+
+    def set_option(self, key: int, value: float) -> None:
+        sage_fd_set_option(self._h, key, value)
+
+    def close(self) -> None:
+        if self._h:
+            sage_fd_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,723 @@
+// Host orchestration behind the C ABI: state machine, buffer management and the launch sequences of
+// pass 1 (append -> Gram -> eigen/shrink -> rebuild), freeze, pass 2 (project -> normalise -> consensus
+// -> score) and selection. No device->host synchronisation happens inside sage_fd_update.
+#include <atomic>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "sage_internal.h"
+
+using namespace sage;
+
+namespace {
+
+thread_local char g_err[512] = "";
+std::atomic<long long> g_launches{0};
+
+void set_err(const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof g_err, fmt, ap);
+    va_end(ap);
+}
+
+#define CU_TRY(expr)                                                                       \
+    do {                                                                                   \
+        cudaError_t e__ = (expr);                                                          \
+        if (e__ != cudaSuccess) {                                                          \
+            set_err("%s failed: %s (%s:%d)", #expr, cudaGetErrorString(e__), __FILE__, __LINE__); \
+            return e__ == cudaErrorMemoryAllocation ? SAGE_ERR_ALLOC : SAGE_ERR_CUDA;      \
+        }                                                                                  \
+    } while (0)
+
+#define ST_TRY(expr)                       \
+    do {                                   \
+        sage_status_t s__ = (expr);        \
+        if (s__ != SAGE_OK) return s__;    \
+    } while (0)
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = false;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
+        ok = cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard() {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+enum State { SKETCHING = 0, FROZEN = 1, SCORING = 2 };
+
+// Kernel classes for the optional per-kernel timing (sage_fd_profile).
+enum KClass { K_APPEND = 0, K_GRAM, K_GRAM_REDUCE, K_EIG, K_REBUILD, K_PROJECT, K_PROJECT_REDUCE, K_NORMALISE, K_SCORE, K_NCLASS };
+
+struct Prof {
+    unsigned mask = 0;
+    std::vector<cudaEvent_t> pool;
+    struct Pending { int cls; cudaEvent_t a, b; };
+    std::vector<Pending> pending;
+    double ms[K_NCLASS] = {};
+    int64_t n[K_NCLASS] = {};
+    cudaEvent_t get() {
+        if (!pool.empty()) { cudaEvent_t e = pool.back(); pool.pop_back(); return e; }
+        cudaEvent_t e = nullptr;
+        cudaEventCreate(&e);
+        return e;
+    }
+};
+
+size_t elem_size(sage_dtype_t dt) { return dt == SAGE_F32 ? 4 : 2; }
+
+}  // namespace
+
+struct sage_fd {
+    int64_t D = 0;
+    int ell = 0, m = 0;
+    sage_dtype_t dtype = SAGE_F32;
+    int device = 0;
+    int64_t pitch = 0;             // floats per buffer row (multiple of 32)
+    float* B[2] = {nullptr, nullptr};
+    int cur = 0;
+    int fill = 0;
+    int64_t rows_seen = 0;
+    State state = SKETCHING;
+    int delta_rank = 0, max_sweeps = 30;
+    // Gram / eigen workspaces
+    float* gram_parts = nullptr;   // 296 tiles of 64 x 64 floats
+    float* Kmat = nullptr;         // m x m
+    float* Ur = nullptr;           // m x m
+    float* eig_work = nullptr;     // m x m
+    float* sigma = nullptr;        // ell
+    EigInfo* info = nullptr;       // device
+    // scoring
+    int64_t N_total = 0, next_row = 0, zcap = 0;
+    float* zhat = nullptr;
+    float* znorm = nullptr;
+    float* zwork = nullptr;
+    size_t zwork_bytes = 0;
+    float* partials = nullptr;
+    size_t partials_bytes = 0;
+    double* zsum = nullptr;
+    float* u = nullptr;
+    int64_t launches = 0;
+    Prof prof;
+};
+
+namespace {
+
+void count(sage_fd* h, int k) {
+    if (h) h->launches += k;
+    g_launches.fetch_add(k, std::memory_order_relaxed);
+}
+
+// Runs one launcher; when the class is selected for timing, brackets it with events on the same stream.
+template <typename F>
+cudaError_t timed(sage_fd* h, int cls, int nlaunch, cudaStream_t st, F&& f) {
+    const bool on = h && (h->prof.mask >> cls) & 1u;
+    cudaEvent_t a = nullptr, b = nullptr;
+    if (on) {
+        a = h->prof.get();
+        b = h->prof.get();
+        cudaEventRecord(a, st);
+    }
+    const cudaError_t e = f();
+    if (on) {
+        cudaEventRecord(b, st);
+        h->prof.pending.push_back({cls, a, b});
+    }
+    count(h, nlaunch);
+    return e;
+}
+
+int gram_tiles(int r) {
+    const int t = (r + 63) / 64;
+    return t * t;
+}
+
+int pick_splits(int tiles, int64_t K, int64_t min_k) {
+    int64_t s = 296 / (tiles > 0 ? tiles : 1);
+    const int64_t cap = (K + min_k - 1) / min_k;
+    if (s > cap) s = cap;
+    if (s < 1) s = 1;
+    return (int)s;
+}
+
+// Gram of the first r buffer rows -> Kmat (r x r, pitch m).
+sage_status_t enqueue_gram(sage_fd* h, int r, cudaStream_t st) {
+    // splits * tiles <= 296, and the partials are stored compactly (pitch r_pad), so they always fit in
+    // the 296 tiles of 64 x 64 floats allocated at create.
+    const int splits = pick_splits(gram_tiles(r), h->D, 256);
+    const int r_pad = ((r + 63) / 64) * 64;
+    const int64_t stride = (int64_t)r_pad * r_pad;
+    float* Bc = h->B[h->cur];
+    if (splits == 1) {
+        CU_TRY(timed(h, K_GRAM, 1, st, [&] { return launch_gemm_nt(Bc, SAGE_F32, h->pitch, Bc, h->pitch, r, r, h->D, 1, h->Kmat, h->m, 0, st); }));
+    } else {
+        CU_TRY(timed(h, K_GRAM, 1, st, [&] {
+            return launch_gemm_nt(Bc, SAGE_F32, h->pitch, Bc, h->pitch, r, r, h->D, splits, h->gram_parts, r_pad, stride, st);
+        }));
+        CU_TRY(timed(h, K_GRAM_REDUCE, 1, st, [&] { return launch_split_reduce(h->gram_parts, splits, stride, r, r, r_pad, h->Kmat, h->m, st); }));
+    }
+    return SAGE_OK;
+}
+
+// Factor the first r rows and rebuild `keep` rows into the other buffer; rows keep..zero_to-1 are zeroed.
+sage_status_t enqueue_factor(sage_fd* h, int r, int do_shrink, int keep, int zero_to, cudaStream_t st) {
+    ST_TRY(enqueue_gram(h, r, st));
+    CU_TRY(timed(h, K_EIG, 1, st, [&] {
+        return launch_eig_shrink(h->Kmat, h->m, r, do_shrink, h->delta_rank, keep, h->Ur, h->m, h->sigma, h->ell, h->eig_work,
+                                 h->max_sweeps, h->info, st);
+    }));
+    const int m_total = zero_to > keep ? zero_to : keep;
+    CU_TRY(timed(h, K_REBUILD, 1, st, [&] {
+        return launch_rebuild(h->Ur, h->m, h->B[h->cur], h->B[1 - h->cur], h->pitch, h->D, r, keep, m_total, st);
+    }));
+    h->cur = 1 - h->cur;
+    h->fill = keep;
+    return SAGE_OK;
+}
+
+sage_status_t ensure(float** p, size_t* have, size_t need) {
+    if (*have >= need) return SAGE_OK;
+    if (*p) CU_TRY(cudaFree(*p));
+    *p = nullptr;
+    *have = 0;
+    CU_TRY(cudaMalloc(reinterpret_cast<void**>(p), need));
+    *have = need;
+    return SAGE_OK;
+}
+
+sage_status_t check_handle(const sage_fd* h) {
+    if (!h) {
+        set_err("null handle");
+        return SAGE_ERR_INVALID_ARG;
+    }
+    return SAGE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* sage_status_string(sage_status_t s) {
+    switch (s) {
+        case SAGE_OK: return "ok";
+        case SAGE_ERR_INVALID_ARG: return "invalid argument";
+        case SAGE_ERR_BAD_STATE: return "call not allowed in this state";
+        case SAGE_ERR_ALLOC: return "allocation failed";
+        case SAGE_ERR_CUDA: return "CUDA error";
+        case SAGE_ERR_UNSUPPORTED: return "unsupported size";
+        case SAGE_ERR_NOT_CONVERGED: return "eigen-solver did not converge";
+        case SAGE_ERR_NONFINITE: return "non-finite input";
+    }
+    return "unknown status";
+}
+
+const char* sage_last_error(void) { return g_err; }
+const char* sage_version(void) { return "sage-b200 0.1 (sm_100a)"; }
+int64_t sage_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int64_t sage_select_count(int64_t N, double keep_rate) {
+    if (N <= 0 || !(keep_rate == keep_rate)) return 0;
+    double k = std::floor(keep_rate * (double)N + 0.5);
+    if (k < 0.0) k = 0.0;
+    if (k > (double)N) k = (double)N;
+    return (int64_t)k;
+}
+
+sage_status_t sage_fd_create(sage_fd_t** out, int64_t D, int32_t ell, sage_dtype_t row_dtype, int device) {
+    if (!out || D < 1 || (row_dtype != SAGE_F32 && row_dtype != SAGE_BF16) || device < 0) {
+        set_err("sage_fd_create: bad argument (out=%p D=%lld dtype=%d device=%d)", (void*)out, (long long)D, (int)row_dtype, device);
+        return SAGE_ERR_INVALID_ARG;
+    }
+    if (ell < 2 || ell > 256) {
+        set_err("sage_fd_create: ell=%d outside [2, 256]", ell);
+        return ell < 2 ? SAGE_ERR_INVALID_ARG : SAGE_ERR_UNSUPPORTED;
+    }
+    DeviceGuard g(device);
+    if (!g.ok) {
+        set_err("sage_fd_create: cannot select CUDA device %d: %s", device, cudaGetErrorString(cudaGetLastError()));
+        return SAGE_ERR_CUDA;
+    }
+    sage_fd* h = new (std::nothrow) sage_fd();
+    if (!h) return SAGE_ERR_ALLOC;
+    h->D = D;
+    h->ell = ell;
+    h->m = 2 * ell;
+    h->dtype = row_dtype;
+    h->device = device;
+    h->delta_rank = ell;
+    h->pitch = ((D + 31) / 32) * 32;
+    const size_t bbytes = (size_t)h->m * h->pitch * sizeof(float);
+    const size_t mm = (size_t)h->m * h->m * sizeof(float);
+    auto fail = [&](cudaError_t e, const char* what) {
+        set_err("sage_fd_create: %s failed: %s", what, cudaGetErrorString(e));
+        sage_fd_destroy(h);
+        return e == cudaErrorMemoryAllocation ? SAGE_ERR_ALLOC : SAGE_ERR_CUDA;
+    };
+    cudaError_t e;
+    for (int i = 0; i < 2; ++i)
+        if ((e = cudaMalloc((void**)&h->B[i], bbytes)) != cudaSuccess) return fail(e, "cudaMalloc(buffer)");
+    if ((e = cudaMalloc((void**)&h->gram_parts, (size_t)296 * 64 * 64 * sizeof(float))) != cudaSuccess) return fail(e, "cudaMalloc(gram)");
+    if ((e = cudaMalloc((void**)&h->Kmat, mm)) != cudaSuccess) return fail(e, "cudaMalloc(K)");
+    if ((e = cudaMalloc((void**)&h->Ur, mm)) != cudaSuccess) return fail(e, "cudaMalloc(U)");
+    if ((e = cudaMalloc((void**)&h->eig_work, mm)) != cudaSuccess) return fail(e, "cudaMalloc(eig)");
+    if ((e = cudaMalloc((void**)&h->sigma, ell * sizeof(float))) != cudaSuccess) return fail(e, "cudaMalloc(sigma)");
+    if ((e = cudaMalloc((void**)&h->info, sizeof(EigInfo))) != cudaSuccess) return fail(e, "cudaMalloc(info)");
+    if ((e = cudaMalloc((void**)&h->zsum, 256 * sizeof(double))) != cudaSuccess) return fail(e, "cudaMalloc(zsum)");
+    if ((e = cudaMalloc((void**)&h->u, 256 * sizeof(float))) != cudaSuccess) return fail(e, "cudaMalloc(u)");
+    if ((e = cudaMemset(h->info, 0, sizeof(EigInfo))) != cudaSuccess) return fail(e, "cudaMemset");
+    if ((e = cudaMemset(h->sigma, 0, ell * sizeof(float))) != cudaSuccess) return fail(e, "cudaMemset");
+    if ((e = cudaDeviceSynchronize()) != cudaSuccess) return fail(e, "cudaDeviceSynchronize");
+    *out = h;
+    return SAGE_OK;
+}
+
+void sage_fd_destroy(sage_fd_t* h) {
+    if (!h) return;
+    DeviceGuard g(h->device);
+    cudaDeviceSynchronize();
+    cudaFree(h->B[0]);
+    cudaFree(h->B[1]);
+    cudaFree(h->gram_parts);
+    cudaFree(h->Kmat);
+    cudaFree(h->Ur);
+    cudaFree(h->eig_work);
+    cudaFree(h->sigma);
+    cudaFree(h->info);
+    cudaFree(h->zhat);
+    cudaFree(h->znorm);
+    cudaFree(h->zwork);
+    cudaFree(h->partials);
+    cudaFree(h->zsum);
+    cudaFree(h->u);
+    for (auto& p : h->prof.pending) {
+        cudaEventDestroy(p.a);
+        cudaEventDestroy(p.b);
+    }
+    for (cudaEvent_t e : h->prof.pool) cudaEventDestroy(e);
+    delete h;
+}
+
+sage_status_t sage_fd_reset(sage_fd_t* h) {
+    ST_TRY(check_handle(h));
+    DeviceGuard g(h->device);
+    CU_TRY(cudaDeviceSynchronize());
+    CU_TRY(cudaMemset(h->info, 0, sizeof(EigInfo)));
+    CU_TRY(cudaMemset(h->sigma, 0, h->ell * sizeof(float)));
+    h->fill = 0;
+    h->rows_seen = 0;
+    h->cur = 0;
+    h->state = SKETCHING;
+    h->launches = 0;
+    return SAGE_OK;
+}
+
+sage_status_t sage_fd_set_option(sage_fd_t* h, int key, double value) {
+    ST_TRY(check_handle(h));
+    if (key == 3) {                          // per-kernel event timing mask: allowed at any time
+        h->prof.mask = (unsigned)value & ((1u << K_NCLASS) - 1u);
+        return SAGE_OK;
+    }
+    if (h->rows_seen != 0 || h->state != SKETCHING) {
+        set_err("sage_fd_set_option: options must be set before the first update");
+        return SAGE_ERR_BAD_STATE;
+    }
+    const int v = (int)value;
+    if (key == 1 && v >= 2 && v <= h->m - 1) {
+        h->delta_rank = v;
+        return SAGE_OK;
+    }
+    if (key == 2 && v >= 1 && v <= 1000) {
+        h->max_sweeps = v;
+        return SAGE_OK;
+    }
+    set_err("sage_fd_set_option: unknown key %d or value %g out of range", key, value);
+    return SAGE_ERR_INVALID_ARG;
+}
+
+sage_status_t sage_fd_update(sage_fd_t* h, const void* rows, int64_t n, int64_t ld, void* cuda_stream) {
+    ST_TRY(check_handle(h));
+    if (n < 0 || (n > 0 && (!rows || ld < h->D))) {
+        set_err("sage_fd_update: bad argument (rows=%p n=%lld ld=%lld D=%lld)", rows, (long long)n, (long long)ld, (long long)h->D);
+        return SAGE_ERR_INVALID_ARG;
+    }
+    if (h->state != SKETCHING) {
+        set_err("sage_fd_update: the sketch is frozen (call sage_fd_reset to start over)");
+        return SAGE_ERR_BAD_STATE;
+    }
+    if (n == 0) return SAGE_OK;
+    DeviceGuard g(h->device);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const char* p = static_cast<const char*>(rows);
+    const size_t row_bytes = (size_t)ld * elem_size(h->dtype);
+    while (n > 0) {
+        const int64_t room = h->m - h->fill;
+        const int64_t take = n < room ? n : room;
+        CU_TRY(timed(h, K_APPEND, 1, st, [&] { return launch_append(p, h->dtype, take, ld, h->D, h->B[h->cur], h->pitch, h->fill, st); }));
+        h->fill += (int)take;
+        h->rows_seen += take;
+        p += take * row_bytes;
+        n -= take;
+        if (h->fill == h->m) ST_TRY(enqueue_factor(h, h->m, 1, h->delta_rank - 1, 0, st));
+    }
+    return SAGE_OK;
+}
+
+sage_status_t sage_fd_finalize(sage_fd_t* h, void* cuda_stream) {
+    ST_TRY(check_handle(h));
+    if (h->state != SKETCHING) {
+        set_err("sage_fd_finalize: already frozen");
+        return SAGE_ERR_BAD_STATE;
+    }
+    DeviceGuard g(h->device);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const int r = h->fill;
+    if (r == 0) {
+        CU_TRY(cudaMemsetAsync(h->B[h->cur], 0, (size_t)h->ell * h->pitch * sizeof(float), st));
+        CU_TRY(cudaMemsetAsync(h->sigma, 0, h->ell * sizeof(float), st));
+    } else {
+        const int do_shrink = r > h->ell ? 1 : 0;
+        const int keep = do_shrink ? h->delta_rank - 1 : (r < h->ell ? r : h->ell);
+        ST_TRY(enqueue_factor(h, r, do_shrink, keep < h->ell ? keep : h->ell, h->ell, st));
+    }
+    h->state = FROZEN;
+    EigInfo info;
+    CU_TRY(cudaMemcpyAsync(&info, h->info, sizeof info, cudaMemcpyDeviceToHost, st));
+    CU_TRY(cudaStreamSynchronize(st));
+    if (info.flags & kFlagNotConverged) {
+        set_err("sage_fd_finalize: an eigen-solve reached the sweep limit (%d)", h->max_sweeps);
+        return SAGE_ERR_NOT_CONVERGED;
+    }
+    if (info.flags & kFlagNonFinite) {
+        set_err("sage_fd_finalize: non-finite values were met in the rows of pass 1");
+        return SAGE_ERR_NONFINITE;
+    }
+    return SAGE_OK;
+}
+
+sage_status_t sage_fd_sketch(const sage_fd_t* h, const float** S, int64_t* pitch, const float** sigma) {
+    ST_TRY(check_handle(h));
+    if (h->state == SKETCHING) {
+        set_err("sage_fd_sketch: the sketch is not frozen yet");
+        return SAGE_ERR_BAD_STATE;
+    }
+    if (S) *S = h->B[h->cur];
+    if (pitch) *pitch = h->pitch;
+    if (sigma) *sigma = h->sigma;
+    return SAGE_OK;
+}
+
+sage_status_t sage_fd_load_sketch(sage_fd_t* h, const float* S, int64_t ld, void* cuda_stream) {
+    ST_TRY(check_handle(h));
+    if (!S || ld < h->D) {
+        set_err("sage_fd_load_sketch: bad argument");
+        return SAGE_ERR_INVALID_ARG;
+    }
+    if (h->state == SCORING) {
+        set_err("sage_fd_load_sketch: a scoring pass is open");
+        return SAGE_ERR_BAD_STATE;
+    }
+    DeviceGuard g(h->device);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    CU_TRY(timed(h, K_APPEND, 1, st, [&] { return launch_append(S, SAGE_F32, h->ell, ld, h->D, h->B[h->cur], h->pitch, 0, st); }));
+    CU_TRY(cudaMemsetAsync(h->sigma, 0, h->ell * sizeof(float), st));
+    h->fill = h->ell;
+    h->state = FROZEN;
+    return SAGE_OK;
+}
+
+sage_status_t sage_score_begin(sage_fd_t* h, int64_t N_total, void* cuda_stream) {
+    ST_TRY(check_handle(h));
+    if (N_total < 0) {
+        set_err("sage_score_begin: negative row count");
+        return SAGE_ERR_INVALID_ARG;
+    }
+    if (h->state != FROZEN) {
+        set_err("sage_score_begin: needs a frozen sketch and no open scoring pass");
+        return SAGE_ERR_BAD_STATE;
+    }
+    DeviceGuard g(h->device);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (N_total > h->zcap) {
+        CU_TRY(cudaStreamSynchronize(st));
+        if (h->zhat) CU_TRY(cudaFree(h->zhat));
+        if (h->znorm) CU_TRY(cudaFree(h->znorm));
+        h->zhat = h->znorm = nullptr;
+        h->zcap = 0;
+        CU_TRY(cudaMalloc((void**)&h->zhat, (size_t)N_total * h->ell * sizeof(float)));
+        CU_TRY(cudaMalloc((void**)&h->znorm, (size_t)N_total * sizeof(float)));
+        h->zcap = N_total;
+    }
+    CU_TRY(cudaMemsetAsync(h->zsum, 0, 256 * sizeof(double), st));
+    h->N_total = N_total;
+    h->next_row = 0;
+    h->state = SCORING;
+    return SAGE_OK;
+}
+
+sage_status_t sage_score_chunk(sage_fd_t* h, const void* rows, int64_t n, int64_t ld, int64_t row_offset, void* cuda_stream) {
+    ST_TRY(check_handle(h));
+    if (h->state != SCORING) {
+        set_err("sage_score_chunk: no open scoring pass");
+        return SAGE_ERR_BAD_STATE;
+    }
+    if (n < 0 || (n > 0 && (!rows || ld < h->D)) || row_offset != h->next_row || row_offset + n > h->N_total) {
+        set_err("sage_score_chunk: bad argument (n=%lld ld=%lld offset=%lld expected offset=%lld N_total=%lld)", (long long)n,
+                (long long)ld, (long long)row_offset, (long long)h->next_row, (long long)h->N_total);
+        return SAGE_ERR_INVALID_ARG;
+    }
+    if (n == 0) return SAGE_OK;
+    DeviceGuard g(h->device);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const int ell = h->ell;
+    const int64_t sub_max = 16384;
+    const char* p = static_cast<const char*>(rows);
+    const size_t row_bytes = (size_t)ld * elem_size(h->dtype);
+    const float* S = h->B[h->cur];
+    for (int64_t r0 = 0; r0 < n; r0 += sub_max) {
+        const int64_t sub = (n - r0 < sub_max) ? n - r0 : sub_max;
+        const int tiles = (int)((sub + 63) / 64) * ((ell + 63) / 64);
+        const int splits = pick_splits(tiles, h->D, 1024);
+        const size_t zred = (size_t)sub * ell * sizeof(float);
+        ST_TRY(ensure(&h->zwork, &h->zwork_bytes, zred * (splits > 1 ? splits + 1 : 1)));
+        const size_t nb = (size_t)((sub + 63) / 64);
+        ST_TRY(ensure(&h->partials, &h->partials_bytes, nb * ell * sizeof(float)));
+        float* Z = h->zwork;
+        if (splits == 1) {
+            CU_TRY(timed(h, K_PROJECT, 1, st, [&] {
+                return launch_gemm_nt(p + r0 * row_bytes, h->dtype, ld, S, h->pitch, (int)sub, ell, h->D, 1, Z, ell, 0, st);
+            }));
+        } else {
+            float* parts = h->zwork + (size_t)sub * ell;
+            CU_TRY(timed(h, K_PROJECT, 1, st, [&] {
+                return launch_gemm_nt(p + r0 * row_bytes, h->dtype, ld, S, h->pitch, (int)sub, ell, h->D, splits, parts, ell,
+                                      (int64_t)sub * ell, st);
+            }));
+            CU_TRY(timed(h, K_PROJECT_REDUCE, 1, st,
+                         [&] { return launch_split_reduce(parts, splits, (int64_t)sub * ell, (int)sub, ell, ell, Z, ell, st); }));
+        }
+        const int64_t row = row_offset + r0;
+        CU_TRY(timed(h, K_NORMALISE, 2, st, [&] {
+            return launch_normalise(Z, ell, sub, ell, h->zhat + row * ell, h->znorm + row, h->partials, h->zsum, &h->info->flags, st);
+        }));
+    }
+    h->next_row += n;
+    return SAGE_OK;
+}
+
+sage_status_t sage_score_end(sage_fd_t* h, float* scores, void* cuda_stream) {
+    ST_TRY(check_handle(h));
+    if (h->state != SCORING) {
+        set_err("sage_score_end: no open scoring pass");
+        return SAGE_ERR_BAD_STATE;
+    }
+    if (h->next_row != h->N_total) {
+        set_err("sage_score_end: %lld of %lld rows were given", (long long)h->next_row, (long long)h->N_total);
+        return SAGE_ERR_BAD_STATE;
+    }
+    if (!scores && h->N_total > 0) {
+        set_err("sage_score_end: null scores");
+        return SAGE_ERR_INVALID_ARG;
+    }
+    DeviceGuard g(h->device);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    CU_TRY(timed(h, K_SCORE, 1, st, [&] { return launch_consensus_score(h->zsum, h->zhat, h->N_total, h->ell, h->u, scores, st); }));
+    h->state = FROZEN;
+    return SAGE_OK;
+}
+
+sage_status_t sage_score(sage_fd_t* h, const void* rows, int64_t n, int64_t ld, float* scores, void* cuda_stream) {
+    ST_TRY(sage_score_begin(h, n, cuda_stream));
+    sage_status_t s = sage_score_chunk(h, rows, n, ld, 0, cuda_stream);
+    if (s != SAGE_OK) {
+        h->state = FROZEN;
+        return s;
+    }
+    s = sage_score_end(h, scores, cuda_stream);
+    if (s != SAGE_OK) h->state = FROZEN;
+    return s;
+}
+
+sage_status_t sage_score_intermediates(const sage_fd_t* h, const float** zhat, const float** znorm, const float** u) {
+    ST_TRY(check_handle(h));
+    if (h->state != FROZEN || !h->zhat) {
+        set_err("sage_score_intermediates: no finished scoring pass");
+        return SAGE_ERR_BAD_STATE;
+    }
+    if (zhat) *zhat = h->zhat;
+    if (znorm) *znorm = h->znorm;
+    if (u) *u = h->u;
+    return SAGE_OK;
+}
+
+sage_status_t sage_select(const float* scores, int64_t N, double keep_rate, int64_t* idx, int64_t* k_out, void* cuda_stream) {
+    if (N < 0 || N >= (1ll << 31) || !(keep_rate == keep_rate) || (N > 0 && !scores)) {
+        set_err("sage_select: bad argument (N=%lld keep_rate=%g)", (long long)N, keep_rate);
+        return SAGE_ERR_INVALID_ARG;
+    }
+    const int64_t k = sage_select_count(N, keep_rate);
+    if (k > 0 && !idx) {
+        set_err("sage_select: null idx");
+        return SAGE_ERR_INVALID_ARG;
+    }
+    if (k > 0) {
+        cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+        size_t bytes = 0;
+        select_scratch_bytes(N, &bytes);
+        void* scratch = nullptr;
+        CU_TRY(cudaMallocAsync(&scratch, bytes, st));
+        cudaError_t e = launch_select(scores, N, k, idx, scratch, st);
+        cudaError_t e2 = cudaFreeAsync(scratch, st);
+        CU_TRY(e);
+        CU_TRY(e2);
+        int idx_bits = 1;
+        while (idx_bits < 32 && (1ll << idx_bits) < N) ++idx_bits;
+        count(nullptr, 2 + 3 * (4 + (idx_bits + 7) / 8));
+    }
+    if (k_out) *k_out = k;
+    return SAGE_OK;
+}
+
+sage_status_t sage_fd_stats(sage_fd_t* h, sage_stats_t* out) {
+    ST_TRY(check_handle(h));
+    if (!out) {
+        set_err("sage_fd_stats: null out");
+        return SAGE_ERR_INVALID_ARG;
+    }
+    DeviceGuard g(h->device);
+    CU_TRY(cudaDeviceSynchronize());
+    EigInfo info;
+    CU_TRY(cudaMemcpy(&info, h->info, sizeof info, cudaMemcpyDeviceToHost));
+    out->rows_seen = h->rows_seen;
+    out->shrinks = info.shrinks;
+    out->sum_delta = info.sum_delta;
+    out->last_sweeps = info.sweeps;
+    out->max_sweeps = info.max_sweeps;
+    out->last_rank = info.rank;
+    out->device_flags = info.flags;
+    out->kernel_launches = h->launches;
+    return SAGE_OK;
+}
+
+sage_status_t sage_fd_profile(sage_fd_t* h, double* ms, int64_t* launches, int32_t capacity) {
+    ST_TRY(check_handle(h));
+    if (!ms || !launches || capacity < K_NCLASS) {
+        set_err("sage_fd_profile: need arrays of at least %d entries", (int)K_NCLASS);
+        return SAGE_ERR_INVALID_ARG;
+    }
+    DeviceGuard g(h->device);
+    CU_TRY(cudaDeviceSynchronize());
+    for (auto& p : h->prof.pending) {
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, p.a, p.b) == cudaSuccess) {
+            h->prof.ms[p.cls] += t;
+            h->prof.n[p.cls] += 1;
+        }
+        h->prof.pool.push_back(p.a);
+        h->prof.pool.push_back(p.b);
+    }
+    h->prof.pending.clear();
+    for (int c = 0; c < K_NCLASS; ++c) {
+        ms[c] = h->prof.ms[c];
+        launches[c] = h->prof.n[c];
+        h->prof.ms[c] = 0.0;
+        h->prof.n[c] = 0;
+    }
+    return SAGE_OK;
+}
+
+sage_status_t sage_select_from_host(const void* rows_host, int64_t N, int64_t D, int64_t ld, int32_t ell,
+                                    sage_dtype_t row_dtype, double keep_rate, int64_t chunk_rows, int device,
+                                    float* scores_host, int64_t* idx_host, int64_t* k_out) {
+    if (!rows_host || N < 1 || D < 1 || ld < D || !(keep_rate == keep_rate)) {
+        set_err("sage_select_from_host: bad argument");
+        return SAGE_ERR_INVALID_ARG;
+    }
+    const int64_t k = sage_select_count(N, keep_rate);
+    if (k > 0 && !idx_host) {
+        set_err("sage_select_from_host: null idx_host");
+        return SAGE_ERR_INVALID_ARG;
+    }
+    sage_fd_t* h = nullptr;
+    ST_TRY(sage_fd_create(&h, D, ell, row_dtype, device));
+    DeviceGuard g(device);
+    const size_t es = elem_size(row_dtype);
+    if (chunk_rows <= 0) {
+        chunk_rows = (int64_t)((256ull << 20) / ((size_t)ld * es));     // about 256 MB per staging buffer
+        if (chunk_rows < 2 * ell) chunk_rows = 2 * ell;
+    }
+    if (chunk_rows > N) chunk_rows = N;
+    const size_t chunk_bytes = (size_t)chunk_rows * ld * es;
+    void* stage[2] = {nullptr, nullptr};
+    float* d_scores = nullptr;
+    int64_t* d_idx = nullptr;
+    cudaStream_t s_copy = nullptr, s_comp = nullptr;
+    cudaEvent_t copied[2] = {nullptr, nullptr}, consumed[2] = {nullptr, nullptr};
+    sage_status_t rc = SAGE_OK;
+    auto body = [&]() -> sage_status_t {
+        CU_TRY(cudaStreamCreateWithFlags(&s_copy, cudaStreamNonBlocking));
+        CU_TRY(cudaStreamCreateWithFlags(&s_comp, cudaStreamNonBlocking));
+        for (int i = 0; i < 2; ++i) {
+            CU_TRY(cudaMalloc(&stage[i], chunk_bytes));
+            CU_TRY(cudaEventCreateWithFlags(&copied[i], cudaEventDisableTiming));
+            CU_TRY(cudaEventCreateWithFlags(&consumed[i], cudaEventDisableTiming));
+        }
+        CU_TRY(cudaMalloc((void**)&d_scores, (size_t)N * sizeof(float)));
+        if (k > 0) CU_TRY(cudaMalloc((void**)&d_idx, (size_t)k * sizeof(int64_t)));
+        const char* src = static_cast<const char*>(rows_host);
+        for (int pass = 0; pass < 2; ++pass) {
+            if (pass == 1) {
+                sage_status_t f = sage_fd_finalize(h, s_comp);
+                if (f != SAGE_OK && f != SAGE_ERR_NOT_CONVERGED && f != SAGE_ERR_NONFINITE) return f;
+                if (f != SAGE_OK) rc = f;
+                ST_TRY(sage_score_begin(h, N, s_comp));
+            }
+            int64_t c = 0;
+            for (int64_t r0 = 0; r0 < N; r0 += chunk_rows, ++c) {
+                const int b = (int)(c & 1);
+                const int64_t n = (N - r0 < chunk_rows) ? N - r0 : chunk_rows;
+                if (c >= 2 || pass == 1) CU_TRY(cudaStreamWaitEvent(s_copy, consumed[b], 0));
+                CU_TRY(cudaMemcpyAsync(stage[b], src + (size_t)r0 * ld * es, (size_t)n * ld * es, cudaMemcpyHostToDevice, s_copy));
+                CU_TRY(cudaEventRecord(copied[b], s_copy));
+                CU_TRY(cudaStreamWaitEvent(s_comp, copied[b], 0));
+                if (pass == 0)
+                    ST_TRY(sage_fd_update(h, stage[b], n, ld, s_comp));
+                else
+                    ST_TRY(sage_score_chunk(h, stage[b], n, ld, r0, s_comp));
+                CU_TRY(cudaEventRecord(consumed[b], s_comp));
+            }
+        }
+        ST_TRY(sage_score_end(h, d_scores, s_comp));
+        int64_t kk = 0;
+        ST_TRY(sage_select(d_scores, N, keep_rate, d_idx, &kk, s_comp));
+        if (scores_host) CU_TRY(cudaMemcpyAsync(scores_host, d_scores, (size_t)N * sizeof(float), cudaMemcpyDeviceToHost, s_comp));
+        if (k > 0) CU_TRY(cudaMemcpyAsync(idx_host, d_idx, (size_t)k * sizeof(int64_t), cudaMemcpyDeviceToHost, s_comp));
+        CU_TRY(cudaStreamSynchronize(s_comp));
+        CU_TRY(cudaStreamSynchronize(s_copy));
+        return SAGE_OK;
+    };
+    sage_status_t s = body();
+    cudaDeviceSynchronize();
+    for (int i = 0; i < 2; ++i) {
+        cudaFree(stage[i]);
+        if (copied[i]) cudaEventDestroy(copied[i]);
+        if (consumed[i]) cudaEventDestroy(consumed[i]);
+    }
+    cudaFree(d_scores);
+    cudaFree(d_idx);
+    if (s_copy) cudaStreamDestroy(s_copy);
+    if (s_comp) cudaStreamDestroy(s_comp);
+    sage_fd_destroy(h);
+    if (s != SAGE_OK) return s;
+    if (k_out) *k_out = k;
+    return rc;
+}
+
+}  // extern "C"

@@ -1,0 +1,135 @@
+// Phase II after the projection (Method, "Two-pass scoring"; Algorithm 1, Phase II):
+// row normalisation zhat_i = z_i/||z_i|| (0 when z_i = 0), the consensus sum over all rows, the unit
+// consensus u and the agreement scores alpha_i = <zhat_i, u>. All reductions run in a fixed order, so
+// a given sequence of calls gives bit-identical results every time.
+#include "sage_internal.h"
+
+namespace sage {
+namespace {
+
+constexpr int kRowsPerBlock = 64;   // rows whose zhat are summed into one partial
+constexpr int kMaxPerLane = 8;      // ell <= 256
+
+// One warp per row, 8 warps per block, each warp walks rows w, w+8, ... of the block's 64 rows.
+__global__ void __launch_bounds__(256) k_normalise(const float* __restrict__ Z, int64_t ldz, int64_t n, int ell,
+                                                   float* __restrict__ zhat, float* __restrict__ znorm,
+                                                   float* __restrict__ partials, unsigned* __restrict__ flags) {
+    __shared__ float part[8][256];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t row0 = (int64_t)blockIdx.x * kRowsPerBlock;
+    float sum[kMaxPerLane];
+#pragma unroll
+    for (int t = 0; t < kMaxPerLane; ++t) sum[t] = 0.f;
+    bool bad = false;
+    for (int rr = warp; rr < kRowsPerBlock; rr += 8) {
+        const int64_t row = row0 + rr;
+        if (row >= n) break;
+        float z[kMaxPerLane];
+        float amax = 0.f;
+        bool finite = true;
+#pragma unroll
+        for (int t = 0; t < kMaxPerLane; ++t) {
+            const int j = lane + 32 * t;
+            z[t] = (j < ell) ? Z[row * ldz + j] : 0.f;
+            finite = finite && (fabsf(z[t]) <= 3.0e38f);   // false for NaN and Inf
+            amax = fmaxf(amax, fabsf(z[t]));
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+        finite = __all_sync(0xffffffffu, finite);
+        float nrm = 0.f, scale = 0.f;
+        if (finite && amax > 0.f) {
+            const float inv = 1.f / amax;
+            float s = 0.f;
+#pragma unroll
+            for (int t = 0; t < kMaxPerLane; ++t) {
+                z[t] *= inv;
+                s = fmaf(z[t], z[t], s);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+            const float rs = sqrtf(s);
+            nrm = amax * rs;
+            scale = 1.f / rs;
+        }
+        if (!finite) bad = true;
+#pragma unroll
+        for (int t = 0; t < kMaxPerLane; ++t) {
+            const int j = lane + 32 * t;
+            const float v = z[t] * scale;       // scale = 0 for zero / non-finite rows
+            if (j < ell) zhat[row * ell + j] = (scale > 0.f) ? v : 0.f;
+            sum[t] += (scale > 0.f) ? v : 0.f;
+        }
+        if (lane == 0) znorm[row] = nrm;
+    }
+#pragma unroll
+    for (int t = 0; t < kMaxPerLane; ++t) part[warp][lane + 32 * t] = sum[t];
+    __syncthreads();
+    if (threadIdx.x < ell) {
+        float s = 0.f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) s += part[w][threadIdx.x];
+        partials[(int64_t)blockIdx.x * ell + threadIdx.x] = s;
+    }
+    if (bad && lane == 0) atomicOr(flags, kFlagNonFinite);
+}
+
+__global__ void __launch_bounds__(256) k_accumulate(const float* __restrict__ partials, int nblocks, int ell,
+                                                    double* __restrict__ zsum) {
+    const int j = threadIdx.x;
+    if (j >= ell) return;
+    double s = zsum[j];
+    for (int b = 0; b < nblocks; ++b) s += (double)partials[(int64_t)b * ell + j];
+    zsum[j] = s;
+}
+
+// u = zsum/||zsum|| (the 1/N of the mean cancels); alpha_i = <zhat_i, u>. One warp per row.
+__global__ void __launch_bounds__(256) k_consensus_score(const double* __restrict__ zsum, const float* __restrict__ zhat,
+                                                         int64_t N, int ell, float* __restrict__ u_out,
+                                                         float* __restrict__ scores) {
+    __shared__ float u[256];
+    __shared__ double red[8];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    double v = (tid < ell) ? zsum[tid] : 0.0;
+    double sq = v * v;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+    if (lane == 0) red[warp] = sq;
+    __syncthreads();
+    double tot = 0.0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += red[w];
+    const double nrm = sqrt(tot);
+    u[tid] = (nrm > 0.0 && tid < ell) ? (float)(v / nrm) : 0.f;
+    if (blockIdx.x == 0 && tid < ell) u_out[tid] = u[tid];
+    __syncthreads();
+    const int64_t row = (int64_t)blockIdx.x * 8 + warp;
+    if (row >= N) return;
+    float acc = 0.f;
+    for (int j = lane; j < ell; j += 32) acc = fmaf(zhat[row * ell + j], u[j], acc);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) scores[row] = fminf(1.f, fmaxf(-1.f, acc));
+}
+
+}  // namespace
+
+cudaError_t launch_normalise(const float* Z, int64_t ldz, int64_t n, int ell, float* zhat, float* znorm, float* partials,
+                             double* zsum, unsigned* flags, cudaStream_t st) {
+    if (n <= 0) return cudaSuccess;
+    const int nblocks = (int)((n + kRowsPerBlock - 1) / kRowsPerBlock);
+    k_normalise<<<nblocks, 256, 0, st>>>(Z, ldz, n, ell, zhat, znorm, partials, flags);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    k_accumulate<<<1, 256, 0, st>>>(partials, nblocks, ell, zsum);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_consensus_score(const double* zsum, const float* zhat, int64_t N, int ell, float* u, float* scores,
+                                   cudaStream_t st) {
+    const int64_t blocks = N > 0 ? (N + 7) / 8 : 1;
+    k_consensus_score<<<(unsigned)blocks, 256, 0, st>>>(zsum, zhat, N, ell, u, scores);
+    return cudaGetLastError();
+}
+
+}  // namespace sage

@@ -1,0 +1,255 @@
+// Generic (alignment-free) CUDA-core kernels of the sketch path: row append, Gram / projection
+// contraction, split reduction and the rebuild. They accept any pitch and any D; the tensor-core
+// kernels take over where their alignment rules hold.
+#include "sage_internal.h"
+
+namespace sage {
+namespace {
+
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+// ------------------------------------------------------------------------------------------------
+// Append (Algorithm 1, Phase I: "S[r,:] <- g"): copy / convert rows into free buffer rows.
+// One block row of threads walks a row with 16-byte accesses where the addresses allow it.
+// ------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) k_append(const T* __restrict__ rows, int64_t n, int64_t ld, int64_t D,
+                                                float* __restrict__ B, int64_t pitch, int dst_row0) {
+    constexpr int V = 16 / sizeof(T);   // elements per 16-byte load
+    const int64_t row = blockIdx.y;
+    const T* src = rows + row * ld;
+    float* dst = B + (int64_t)(dst_row0 + row) * pitch;
+    const bool vec_ok = ((reinterpret_cast<uintptr_t>(src) & 15) == 0);
+    const int64_t chunk0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * V;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x * V;
+    for (int64_t c = chunk0; c < pitch; c += stride) {
+        float v[V];
+        if (vec_ok && c + V <= D) {
+            const uint4 raw = *reinterpret_cast<const uint4*>(src + c);
+            const T* e = reinterpret_cast<const T*>(&raw);
+#pragma unroll
+            for (int i = 0; i < V; ++i) v[i] = to_f32(e[i]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < V; ++i) v[i] = (c + i < D) ? to_f32(src[c + i]) : 0.0f;
+        }
+        if (c + V <= pitch) {   // pitch is a multiple of 4 floats and dst rows are 16-byte aligned
+#pragma unroll
+            for (int i = 0; i < V; i += 4) *reinterpret_cast<float4*>(dst + c + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < V; ++i)
+                if (c + i < pitch) dst[c + i] = v[i];
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// C[z] = A_z * Bm_z^T over the z-th slice of the contraction index (both operands k-contiguous).
+// 64 x 64 output tile, 32-deep k tiles, 256 threads with 4 x 4 register tiles. The register
+// accumulators are folded into a second set every kFold k-tiles to bound fp32 summation error on
+// very long contractions.
+// ------------------------------------------------------------------------------------------------
+constexpr int BM = 64, BN = 64, BK = 32, PAD = 4, kFold = 64;
+
+template <typename T>
+__device__ __forceinline__ void load4(const T* p, bool vec, int64_t k, int64_t k_end, float out[4]) {
+    if (vec && k + 4 <= k_end) {
+        if constexpr (sizeof(T) == 4) {
+            const float4 v = *reinterpret_cast<const float4*>(p + k);
+            out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
+        } else {
+            const uint2 raw = *reinterpret_cast<const uint2*>(p + k);
+            const T* e = reinterpret_cast<const T*>(&raw);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) out[i] = to_f32(e[i]);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) out[i] = (k + i < k_end) ? to_f32(p[k + i]) : 0.0f;
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) k_gemm_nt(const T* __restrict__ A, int64_t lda, const float* __restrict__ Bm,
+                                                 int64_t ldb, int M, int N, int64_t K, int64_t k_per_split,
+                                                 float* __restrict__ C, int64_t ldc, int64_t split_stride) {
+    __shared__ float As[BK][BM + PAD];
+    __shared__ float Bs[BK][BN + PAD];
+    const int tid = threadIdx.x;
+    const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN;
+    const int64_t k_begin = (int64_t)blockIdx.z * k_per_split;
+    const int64_t k_end = min(K, k_begin + k_per_split);
+    const int lrow = tid >> 3;          // 0..31
+    const int lk = (tid & 7) * 4;       // 0,4,..,28
+    const int ty = tid >> 4, tx = tid & 15;
+    const bool a_vec = (lda * sizeof(T)) % (4 * sizeof(T)) == 0 && (reinterpret_cast<uintptr_t>(A) % (4 * sizeof(T))) == 0 &&
+                       (lda % 4 == 0) && (k_begin % 4 == 0);
+    const bool b_vec = (ldb % 4 == 0) && (reinterpret_cast<uintptr_t>(Bm) % 16 == 0) && (k_begin % 4 == 0);
+
+    float acc[4][4] = {}, tot[4][4] = {};
+    int fold = 0;
+    for (int64_t k0 = k_begin; k0 < k_end; k0 += BK) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int r = lrow + h * 32;
+            float v[4] = {0.f, 0.f, 0.f, 0.f};
+            if (m0 + r < M) load4(A + (int64_t)(m0 + r) * lda, a_vec, k0 + lk, k_end, v);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) As[lk + i][r] = v[i];
+            float w[4] = {0.f, 0.f, 0.f, 0.f};
+            if (n0 + r < N) load4(Bm + (int64_t)(n0 + r) * ldb, b_vec, k0 + lk, k_end, w);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) Bs[lk + i][r] = w[i];
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < BK; ++kk) {
+            const float4 a = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
+            const float4 b = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+            const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+        }
+        __syncthreads();
+        if (++fold == kFold) {
+            fold = 0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { tot[i][j] += acc[i][j]; acc[i][j] = 0.f; }
+        }
+    }
+    float* Cz = C + (int64_t)blockIdx.z * split_stride;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int r = m0 + ty * 4 + i;
+        if (r >= M) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int c = n0 + tx * 4 + j;
+            if (c < N) Cz[(int64_t)r * ldc + c] = tot[i][j] + acc[i][j];
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256) k_split_reduce(const float* __restrict__ parts, int splits, int64_t split_stride,
+                                                      int M, int N, int64_t ldp, float* __restrict__ out, int64_t ldo) {
+    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= (int64_t)M * N) return;
+    const int i = (int)(e / N), j = (int)(e % N);
+    double s = 0.0;
+    for (int z = 0; z < splits; ++z) s += (double)parts[(int64_t)z * split_stride + (int64_t)i * ldp + j];
+    out[(int64_t)i * ldo + j] = (float)s;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Rebuild (Method, first paragraph: "reconstruct S <- Sigma' V^T"): with B B^T = U Lambda U^T,
+// Sigma' V^T = diag(sigma'_j / sigma_j) U^T B, so out[j][:] = sum_i Ur[i][j] B[i][:] where Ur already
+// carries the factor sqrt(max(1 - delta/lambda_j, 0)). Source and destination are different buffers.
+// Block tile: 64 output rows x 128 columns, contraction over the r buffer rows in steps of 16.
+// ------------------------------------------------------------------------------------------------
+constexpr int RM = 64, RN = 128, RK = 16;
+
+__global__ void __launch_bounds__(256) k_rebuild(const float* __restrict__ Ur, int ldu, const float* __restrict__ Bsrc,
+                                                 float* __restrict__ Bdst, int64_t pitch, int r, int keep, int m_total) {
+    __shared__ float Us[RK][RM];
+    __shared__ float Bs[RK][RN];
+    const int tid = threadIdx.x;
+    const int64_t d0 = (int64_t)blockIdx.x * RN;
+    const int j0 = blockIdx.y * RM;
+    const int ty = tid >> 5, tx = tid & 31;     // 8 x 32 threads -> 8 rows x 4 cols each
+    if (j0 >= keep) {                           // rows beyond keep: zero fill
+        for (int j = j0 + ty; j < min(j0 + RM, m_total); j += 8)
+            for (int c = tx * 4; c < RN; c += 128)
+                if (d0 + c < pitch) *reinterpret_cast<float4*>(Bdst + (int64_t)j * pitch + d0 + c) = make_float4(0.f, 0.f, 0.f, 0.f);
+        return;
+    }
+    float acc[8][4] = {};
+    for (int i0 = 0; i0 < r; i0 += RK) {
+        for (int e = tid; e < RK * RM; e += 256) {
+            const int kk = e / RM, jj = e % RM;
+            Us[kk][jj] = (i0 + kk < r && j0 + jj < keep) ? Ur[(int64_t)(i0 + kk) * ldu + j0 + jj] : 0.f;
+        }
+        for (int e = tid; e < RK * RN / 4; e += 256) {
+            const int kk = e / (RN / 4), cc = (e % (RN / 4)) * 4;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (i0 + kk < r && d0 + cc < pitch) v = *reinterpret_cast<const float4*>(Bsrc + (int64_t)(i0 + kk) * pitch + d0 + cc);
+            *reinterpret_cast<float4*>(&Bs[kk][cc]) = v;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < RK; ++kk) {
+            const float4 b = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float u = Us[kk][ty * 8 + i];
+                acc[i][0] = fmaf(u, b.x, acc[i][0]);
+                acc[i][1] = fmaf(u, b.y, acc[i][1]);
+                acc[i][2] = fmaf(u, b.z, acc[i][2]);
+                acc[i][3] = fmaf(u, b.w, acc[i][3]);
+            }
+        }
+        __syncthreads();
+    }
+    if (d0 + tx * 4 >= pitch) return;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int j = j0 + ty * 8 + i;
+        if (j >= m_total) continue;
+        float4 v = (j < keep) ? make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]) : make_float4(0.f, 0.f, 0.f, 0.f);
+        *reinterpret_cast<float4*>(Bdst + (int64_t)j * pitch + d0 + tx * 4) = v;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_append(const void* rows, sage_dtype_t dt, int64_t n, int64_t ld, int64_t D, float* B, int64_t pitch,
+                          int dst_row0, cudaStream_t st) {
+    if (n <= 0) return cudaSuccess;
+    const int V = dt == SAGE_F32 ? 4 : 8;
+    int64_t bx = (pitch / V + 255) / 256;
+    if (bx > 592) bx = 592;
+    if (bx < 1) bx = 1;
+    dim3 grid((unsigned)bx, (unsigned)n);
+    if (dt == SAGE_F32)
+        k_append<float><<<grid, 256, 0, st>>>(static_cast<const float*>(rows), n, ld, D, B, pitch, dst_row0);
+    else
+        k_append<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(rows), n, ld, D, B, pitch, dst_row0);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const float* Bm, int64_t ldb, int M, int N,
+                           int64_t K, int splits, float* C, int64_t ldc, int64_t split_stride, cudaStream_t st) {
+    if (M <= 0 || N <= 0) return cudaSuccess;
+    int64_t kps = (K + splits - 1) / splits;
+    kps = ((kps + BK - 1) / BK) * BK;
+    dim3 grid((M + BM - 1) / BM, (N + BN - 1) / BN, splits);
+    if (dt == SAGE_F32)
+        k_gemm_nt<float><<<grid, 256, 0, st>>>(static_cast<const float*>(A), lda, Bm, ldb, M, N, K, kps, C, ldc, split_stride);
+    else
+        k_gemm_nt<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(A), lda, Bm, ldb, M, N, K, kps, C, ldc,
+                                                       split_stride);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_split_reduce(const float* parts, int splits, int64_t split_stride, int M, int N, int64_t ldp, float* out,
+                                int64_t ldo, cudaStream_t st) {
+    const int64_t total = (int64_t)M * N;
+    if (total <= 0) return cudaSuccess;
+    k_split_reduce<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(parts, splits, split_stride, M, N, ldp, out, ldo);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_rebuild(const float* Ur, int ldu, const float* Bsrc, float* Bdst, int64_t pitch, int64_t D, int r, int keep,
+                           int m_total, cudaStream_t st) {
+    (void)D;
+    dim3 grid((unsigned)((pitch + RN - 1) / RN), (unsigned)((m_total + RM - 1) / RM));
+    k_rebuild<<<grid, 256, 0, st>>>(Ur, ldu, Bsrc, Bdst, pitch, r, keep, m_total);
+    return cudaGetLastError();
+}
+
+}  // namespace sage

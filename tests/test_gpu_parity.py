@@ -1,0 +1,278 @@
+"""GPU parity: the CUDA path, called through the C ABI's Python binding, against the fp64 oracle on the
+same seeded bytes in the same row order. Tolerances (stated by the benchmark spec):
+  sketch  ||S^T S - S_o^T S_o||_2 / ||A||_F^2 <= 1e-4
+  scores  |alpha - alpha_o| <= 1e-4 for fp32 rows, <= 2e-3 for bf16 rows
+  indices identical except for rows whose oracle score is within that tolerance of the k-th score."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import metrics
+import paper_2510_02470_b200 as sage
+from paper_2510_02470_b200 import workloads as wl
+
+from helpers import TOL_SCORE, compare, gpu_run
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def lowrank_rows(N, D, rank, noise, seed, dtype=torch.float32, ld=None):
+    r = np.random.default_rng(seed)
+    Q, _ = np.linalg.qr(r.standard_normal((D, rank)))
+    A = (r.standard_normal((N, rank)) + 0.6) @ Q.T * 2.0 + noise * r.standard_normal((N, D))
+    A *= np.exp(0.5 * r.standard_normal((N, 1)))
+    ld = ld or D
+    out = np.zeros((N, ld), dtype=np.float32)
+    out[:, :D] = A
+    return torch.from_numpy(out).to(dtype)
+
+
+# ------------------------------------------------------------------ selection (bit-exact)
+
+@pytest.mark.parametrize("kind", ["random", "ties", "constant", "signed_zero"])
+@pytest.mark.parametrize("N", [1, 31, 4096, 4097, 200000])
+def test_select_matches_oracle_exactly(kind, N):
+    r = np.random.default_rng(N)
+    a = {"random": r.uniform(-1, 1, N), "ties": r.integers(-5, 6, N) / 5.0, "constant": np.full(N, -0.5),
+         "signed_zero": np.where(r.uniform(size=N) < 0.5, 0.0, -0.0) * 1.0}[kind].astype(np.float32)
+    s = torch.from_numpy(a).to(DEV)
+    for rate in (0.0, 1e-4, 0.1, 0.3, 1.0):
+        idx = sage.sage_select(s, rate).cpu().numpy()
+        ref = oracle.select(a.astype(np.float64), rate)
+        assert np.array_equal(idx, ref), (kind, N, rate)
+
+
+def test_select_nan_ranks_last_and_errors():
+    a = torch.tensor([0.5, float("nan"), -1.0, 0.7], device=DEV)
+    assert sage.sage_select(a, 0.75).cpu().tolist() == [3, 0, 2]
+    with pytest.raises(sage.SageError) as e:
+        sage._check(sage.lib().sage_select(a.data_ptr(), 4, float("nan"), None, None, None))
+    assert e.value.status == 1
+
+
+# ------------------------------------------------------------------ scoring with the oracle's sketch
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("N,D,ell", [(300, 257, 8), (1000, 1024, 32), (130, 5130, 64), (70, 3001, 128), (50, 777, 256)])
+def test_score_with_loaded_sketch(dtype, N, D, ell):
+    ld = wl.padded_pitch(D, 4 if dtype == torch.float32 else 2) if D % 2 else D
+    rows = lowrank_rows(N, D, 5, 0.3, N + D, dtype, ld)
+    S = np.random.default_rng(1).standard_normal((ell, D)) * np.linspace(3, 0.1, ell)[:, None]
+    S32 = torch.from_numpy(S.astype(np.float32))
+    ref = oracle.score(S32.double().numpy(), rows)
+    fd = sage.SageFD(D, ell, dtype, 0)
+    fd.load_sketch(S32.to(DEV))
+    g = rows.to(DEV)
+    a = fd.score(g).double().cpu().numpy()
+    zhat, znorm, u = fd.intermediates(N)
+    fd.close()
+    assert np.max(np.abs(a - ref["alpha"])) <= TOL_SCORE[dtype] * 0.1
+    assert np.allclose(znorm.double().cpu().numpy(), ref["znorm"], rtol=2e-3 if dtype == torch.bfloat16 else 1e-4)
+    assert np.max(np.abs(u.double().cpu().numpy() - ref["u"])) <= 1e-4
+    assert a.min() >= -1.0 and a.max() <= 1.0
+
+
+def test_score_chunked_equals_oneshot_within_rounding_and_is_deterministic():
+    N, D, ell = 5000, 640, 16
+    rows = lowrank_rows(N, D, 6, 0.5, 3)
+    a = gpu_run(rows, D, ell, 0.1)
+    b = gpu_run(rows, D, ell, 0.1)
+    assert np.array_equal(a["alpha"], b["alpha"]) and np.array_equal(a["idx"], b["idx"]) and np.array_equal(a["S"], b["S"])
+    c = gpu_run(rows, D, ell, 0.1, chunks=[1, 30, 33, 936, 4000], score_chunks=[777, 4223])
+    assert np.array_equal(a["S"], c["S"])                    # update chunking does not change the sketch
+    assert np.max(np.abs(a["alpha"] - c["alpha"])) <= 2e-6
+
+
+def test_zero_rows_and_zero_consensus():
+    D, ell = 96, 4
+    rows = lowrank_rows(40, D, 3, 0.2, 5)
+    rows[7] = 0.0
+    ref = oracle.run(rows, D, ell, 0.25)
+    out = gpu_run(rows, D, ell, 0.25)
+    assert out["alpha"][7] == 0.0 and out["znorm"][7] == 0.0 and np.all(out["zhat"][7] == 0)
+    compare(out, ref, rows, D, 0.25)
+    # g and -g cancel exactly: consensus 0, all scores 0
+    fd = sage.SageFD(D, ell, torch.float32, 0)
+    S = torch.zeros((ell, D))
+    S[0, 0] = S[1, 1] = 1.0
+    fd.load_sketch(S.to(DEV))
+    g = torch.zeros((2, D))
+    g[0, 0], g[1, 0] = 2.0, -2.0
+    a = fd.score(g.to(DEV)).cpu().numpy()
+    fd.close()
+    assert np.all(a == 0.0)
+
+
+# ------------------------------------------------------------------ sketch + full path on small shapes
+
+@pytest.mark.parametrize("N,D,ell", [(3, 8, 2), (4, 17, 2), (9, 33, 4), (64, 32, 8), (257, 100, 5), (1000, 300, 16),
+                                     (700, 1030, 33)])
+def test_full_path_small_shapes(N, D, ell):
+    rows = lowrank_rows(N, D, min(3, D), 0.3, N * 7 + D)
+    ref = oracle.run(rows, D, ell, 0.2)
+    out = gpu_run(rows, D, ell, 0.2)
+    compare(out, ref, rows, D, 0.2, label=f"{N}x{D} ell={ell}")
+    assert out["stats"]["shrinks"] == ref["stats"]["shrinks"] and out["stats"]["rows_seen"] == N
+    assert np.isclose(out["stats"]["sum_delta"], ref["stats"]["sum_delta"], rtol=1e-3, atol=1e-6 * np.linalg.norm(rows.numpy()) ** 2)
+
+
+@pytest.mark.parametrize("N", [1, 5, 8])
+def test_exact_when_N_le_ell(N):
+    D, ell = 70, 8
+    rows = lowrank_rows(N, D, 3, 0.5, N)
+    out = gpu_run(rows, D, ell, 0.5)
+    A = rows.double().numpy()
+    assert out["stats"]["shrinks"] == 0
+    assert np.allclose(out["S"].T @ out["S"], A.T @ A, atol=2e-6 * np.linalg.norm(A) ** 2)
+
+
+def test_rank_deficient_input_is_reproduced():
+    D, ell, N = 64, 8, 300
+    rows = lowrank_rows(N, D, 4, 0.0, 11)
+    out = gpu_run(rows, D, ell, 0.1)
+    A = rows.double().numpy()
+    assert out["stats"]["shrinks"] > 10
+    assert metrics.signed_gram_norm(out["S"], A) <= 1e-4 * np.linalg.norm(A) ** 2
+    compare(out, oracle.run(rows, D, ell, 0.1), rows, D, 0.1)
+
+
+def test_closed_form_single_shrink():
+    ell, D = 6, 40
+    m = 2 * ell
+    r = np.random.default_rng(0)
+    Q, _ = np.linalg.qr(r.standard_normal((D, m)))
+    sig = np.sort(r.uniform(0.5, 4.0, m))[::-1]
+    rows = torch.from_numpy((sig[:, None] * Q.T)[r.permutation(m)].astype(np.float32))
+    out = gpu_run(rows, D, ell, 0.5)
+    kept = np.sqrt(np.clip(sig ** 2 - sig[ell - 1] ** 2, 0, None))
+    expect = kept[:, None] * Q.T
+    assert np.allclose(out["S"].T @ out["S"], expect.T @ expect, atol=1e-5 * sig[0] ** 2)
+    assert np.allclose(out["sigma"], kept[:ell], atol=1e-5 * sig[0])
+
+
+def test_lemma_identity_on_gpu_outputs():
+    N, D, ell = 800, 200, 12
+    rows = lowrank_rows(N, D, 4, 0.3, 21)
+    out = gpu_run(rows, D, ell, 0.25)
+    T, a, zn = out["idx"], out["alpha"], out["znorm"]
+    Z = out["zhat"] * zn[:, None]
+    xi = a[T].min()
+    assert xi > 0
+    lhs = ((Z[T] @ out["u"]) ** 2).sum()
+    assert np.isclose(lhs, (zn[T] ** 2 * a[T] ** 2).sum(), rtol=1e-4)
+    assert lhs >= xi ** 2 * (zn[T] ** 2).sum() * (1 - 1e-4)
+    assert np.linalg.norm(Z[T].mean(axis=0)) >= xi * zn[T].mean() * (1 - 1e-4)
+
+
+# ------------------------------------------------------------------ the benchmark workloads
+
+def test_c1_full():
+    w = wl.WORKLOADS["c1"]
+    rows = wl.host_rows(w, 0)
+    ref = oracle.run(rows, w.D, w.ell, 0.1)
+    out = gpu_run(rows, w.D, w.ell, 0.1)
+    rep = compare(out, ref, rows, w.D, 0.1, label="c1")
+    assert out["stats"]["shrinks"] == 124 and len(out["idx"]) == 410
+    print(rep, out["stats"])
+
+
+def test_c2_prefix_three_keep_rates():
+    w = wl.WORKLOADS["c2"]
+    rows = wl.host_rows(w, 0, 4000)                          # dense pitch 5132 (16-byte multiple)
+    ref = oracle.run(rows, w.D, w.ell, 0.1, route=1)
+    out = gpu_run(rows, w.D, w.ell, 0.1)
+    print(compare(out, ref, rows, w.D, 0.1, label="c2[:4000]"), out["stats"])
+    s = torch.from_numpy(out["alpha"].astype(np.float32)).to(DEV)
+    for rate in (0.05, 0.3):
+        idx = sage.sage_select(s, rate).cpu().numpy()
+        ok, _ = metrics.selection_agrees(idx, ref["alpha"], oracle.select_k(4000, rate), 1e-4)
+        assert ok
+    # unpadded pitch (ld = D, rows not 16-byte aligned) takes the generic path and must agree
+    dense = rows[:, : w.D].contiguous()
+    out2 = gpu_run(dense, w.D, w.ell, 0.1)
+    compare(out2, ref, dense, w.D, 0.1, label="c2 dense pitch")
+
+
+def test_c3_prefix_bf16():
+    w = wl.scaled(wl.WORKLOADS["c3"], N=1500)
+    rows = wl.host_rows(w, 0)
+    ref = oracle.run(rows, w.D, w.ell, 0.1, route=1)
+    out = gpu_run(rows, w.D, w.ell, 0.1)
+    print(compare(out, ref, rows, w.D, 0.1, label="c3[:1500]"), out["stats"])
+
+
+def test_c4_shape_small_prefix():
+    """c4's generator and ell=256 on a reduced D and row count (the full D is covered by bench checks)."""
+    w = wl.scaled(wl.WORKLOADS["c4"], N=1300, D=8192, chunk_rows=650)
+    stream = wl.DeviceStream(w, seed=0, device=DEV)
+    rows = torch.cat([stream.chunk(j) for j in range(w.num_chunks)]).cpu()
+    ref = oracle.run(rows, w.D, w.ell, 0.1, route=1)
+    out = gpu_run(rows, w.D, w.ell, 0.1, chunks=[650, 650], score_chunks=[650, 650])
+    print(compare(out, ref, rows, w.D, 0.1, label="c4-shape"), out["stats"])
+
+
+def test_c5_shape_small_prefix():
+    w = wl.scaled(wl.WORKLOADS["c5"], N=600, D=111739, chunk_rows=256)
+    stream = wl.DeviceStream(w, seed=0, device=DEV)
+    rows = torch.cat([stream.chunk(j) for j in range(w.num_chunks)]).cpu()
+    ref = oracle.run(rows, w.D, w.ell, 0.1, route=1)
+    out = gpu_run(rows, w.D, w.ell, 0.1, chunks=[256, 256, 88], score_chunks=[256, 256, 88])
+    print(compare(out, ref, rows, w.D, 0.1, label="c5-shape"), out["stats"])
+
+
+# ------------------------------------------------------------------ host pipeline and state machine
+
+def test_select_from_host_matches_device_path():
+    N, D, ell = 3000, 515, 16
+    rows = lowrank_rows(N, D, 5, 0.4, 9, ld=516)
+    ref = oracle.run(rows, D, ell, 0.1)
+    scores, idx = sage.sage_select_from_host(rows.pin_memory(), D, ell, 0.1, chunk_rows=700)
+    dev = gpu_run(rows, D, ell, 0.1, score_chunks=[700, 700, 700, 700, 200])
+    assert np.array_equal(idx.numpy(), dev["idx"])
+    assert np.max(np.abs(scores.double().numpy() - ref["alpha"])) <= 1e-4
+
+
+def test_state_machine_and_errors():
+    D, ell = 64, 4
+    fd = sage.SageFD(D, ell, torch.float32, 0)
+    rows = lowrank_rows(20, D, 2, 0.1, 1).to(DEV)
+    with pytest.raises(sage.SageError) as e:
+        fd.score(rows)
+    assert e.value.status == 2                               # not frozen yet
+    fd.update(rows[:0])                                      # n == 0 is a no-op
+    fd.update(rows)
+    with pytest.raises(sage.SageError):
+        sage._check(sage.lib().sage_fd_update(fd._h, rows.data_ptr(), 5, D - 1, None))   # ld < D
+    fd.finalize()
+    with pytest.raises(sage.SageError) as e:
+        fd.update(rows)
+    assert e.value.status == 2
+    fd.score_begin(20)
+    with pytest.raises(sage.SageError):
+        fd.score_chunk(rows[:5], 3)                          # wrong offset
+    fd.score_chunk(rows[:5], 0)
+    with pytest.raises(sage.SageError):
+        fd.score_end(torch.empty(20, device=DEV))            # rows missing
+    fd.score_chunk(rows[5:], 5)
+    fd.score_end(torch.empty(20, device=DEV))
+    fd.reset()
+    fd.update(rows)
+    fd.finalize()
+    assert fd.stats()["rows_seen"] == 20
+    fd.close()
+
+
+def test_nonfinite_rows_are_flagged_not_fatal():
+    D, ell = 64, 4
+    fd = sage.SageFD(D, ell, torch.float32, 0)
+    S = torch.eye(ell, D)
+    fd.load_sketch(S.to(DEV))
+    g = lowrank_rows(10, D, 2, 0.1, 2)
+    g[3, 0] = float("nan")
+    g[4, 1] = float("inf")
+    a = fd.score(g.to(DEV)).cpu().numpy()
+    assert a[3] == 0.0 and a[4] == 0.0 and np.all(np.isfinite(a))
+    assert fd.stats()["device_flags"] & 2
+    fd.close()
