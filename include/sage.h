@@ -129,6 +129,22 @@ int64_t sage_select_count(int64_t N, double keep_rate);
 sage_status_t sage_select(const float* scores, int64_t N, double keep_rate, int64_t* idx, int64_t* k_out,
                           void* cuda_stream);
 
+/* Selection without any allocation (the paper has no counterpart; this is a packaging variant of
+ * sage_select with identical results). For callers that cannot allocate device memory at call time:
+ * code running inside a loop whose memory was handed out once at start-up by a pool it does not own,
+ * processes that leave no free device memory, threads that must not block on the allocator. The O(N)
+ * scratch that sage_select obtains per call lives here in a fixed array inside the library image
+ * (about 4.06 MiB, held by every device that loads the library until the process exits), so
+ *   N <= 262,144 scores; larger N returns SAGE_ERR_UNSUPPORTED with a message naming the limit.
+ * Arguments, ordering, tie rule and k_out are those of sage_select; it runs on the CURRENT device.
+ * The first call on each device looks up the array's device address (a synchronous query, no
+ * allocation); make that first call before starting any stream capture. All calls on a device share the
+ * one array: nothing in it needs clearing between calls (every word is written before it is read), but
+ * two calls whose kernels can overlap on the GPU (different streams, no ordering) race on it and give
+ * undefined results. Calls neither allocate nor free: no cudaMalloc, cudaFree or stream-ordered pool. */
+sage_status_t sage_select_static(const float* scores, int64_t N, double keep_rate, int64_t* idx, int64_t* k_out,
+                                 void* cuda_stream);
+
 /* The whole path for rows that live in HOST memory (pinned memory gives overlap of copies and
  * kernels): streams the rows to the device in chunks for pass 1, freezes, streams them again for
  * pass 2, selects, and copies scores (N floats, may be NULL) and indices back to the host.

@@ -39,6 +39,7 @@ SIGNATURES = {
     "sage_score_intermediates": (_i32, [_vp, _vp, _vp, _vp]),
     "sage_select_count": (_i64, [_i64, _f64]),
     "sage_select": (_i32, [_vp, _i64, _f64, _vp, _vp, _vp]),
+    "sage_select_static": (_i32, [_vp, _i64, _f64, _vp, _vp, _vp]),
     "sage_select_from_host": (_i32, [_vp, _i64, _i64, _i64, _i32, _i32, _f64, _i64, _i32, _vp, _vp, _vp]),
     "sage_fd_stats": (_i32, [_vp, _vp]),
     "sage_fd_set_option": (_i32, [_vp, _i32, _f64]),
@@ -186,6 +187,21 @@ def sage_select(scores: torch.Tensor, keep_rate: float, idx: Optional[torch.Tens
     assert idx.dtype == torch.int64 and idx.numel() >= k
     k_out = _i64(0)
     _check(lib().sage_select(scores.data_ptr(), N, keep_rate, idx.data_ptr(), C.byref(k_out), _stream(scores.device)))
+    return idx[: k_out.value]
+
+
+def sage_select_static(scores: torch.Tensor, keep_rate: float, idx: torch.Tensor) -> torch.Tensor:
+    """sage_select for callers that cannot allocate: the caller passes ``idx`` (capacity >= k) and the
+    library uses its built-in scratch (N <= 262,144). Runs on the current device, current stream."""
+    assert scores.dtype == torch.float32 and scores.is_contiguous()
+    assert idx.dtype == torch.int64 and idx.is_contiguous()
+    N = scores.numel()
+    k = sage_select_count(N, keep_rate)
+    assert idx.numel() >= k
+    k_out = _i64(0)
+    with torch.cuda.device(scores.device):
+        _check(lib().sage_select_static(scores.data_ptr(), N, keep_rate, idx.data_ptr(), C.byref(k_out),
+                                        _stream(scores.device)))
     return idx[: k_out.value]
 
 

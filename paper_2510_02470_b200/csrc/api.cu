@@ -203,6 +203,11 @@ sage_status_t check_handle(const sage_fd* h) {
 
 }  // namespace
 
+namespace sage {
+void set_error_message(const char* msg) { set_err("%s", msg); }
+void count_launches(int k) { count(nullptr, k); }
+}  // namespace sage
+
 extern "C" {
 
 const char* sage_status_string(sage_status_t s) {

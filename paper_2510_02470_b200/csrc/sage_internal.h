@@ -66,6 +66,10 @@ cudaError_t launch_consensus_score(const double* zsum, const float* zhat, int64_
 cudaError_t select_scratch_bytes(int64_t N, size_t* bytes);
 cudaError_t launch_select(const float* scores, int64_t N, int64_t k, int64_t* idx, void* scratch, cudaStream_t st);
 
+// Hooks into the C ABI's bookkeeping for entry points defined outside api.cu.
+void set_error_message(const char* msg);   // becomes the calling thread's sage_last_error()
+void count_launches(int k);                // adds to sage_launch_count()
+
 int launches_append();
 int launches_gemm_nt(int splits);
 

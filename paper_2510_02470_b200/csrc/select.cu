@@ -3,6 +3,9 @@
 // order-preserving integer image of the float and whose low word is the row index; every key is
 // distinct, so an ascending LSD radix sort of the keys (8-bit digits, stable scatter) puts the rows in
 // exactly that order and the first k low words are the answer. Integer work only: results are exact.
+#include <cstdio>
+#include <mutex>
+
 #include "sage_internal.h"
 
 namespace sage {
@@ -165,3 +168,90 @@ cudaError_t launch_select(const float* scores, int64_t N, int64_t k, int64_t* id
 }
 
 }  // namespace sage
+
+// ------------------------------------------------------------------------------------------------
+// sage_select_static: the same selection for callers that must not allocate.
+//
+// Some callers run where device allocation is off the table: inside a serving or training loop whose
+// memory is handed out once at start-up by a pool they do not own, in a process whose remaining device
+// memory is deliberately zero, or on a thread that may not take the allocator's locks. sage_select asks
+// the stream-ordered allocator for its O(N) scratch on every call; this variant keeps that scratch in
+// the library image instead, in the array below, which every device that loads the library holds
+// until the process exits.
+//
+// The array's name is only a host-side stand-in in host code, so its device address is looked up once
+// per device (with that device current) and that address is what the kernels get.
+// ------------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int64_t kStaticMaxN = 262144;    // largest N served without allocating
+constexpr size_t kStaticKeyBytes = (size_t)kStaticMaxN * 8;                          // one key array
+constexpr size_t kStaticHistBytes = (size_t)((kStaticMaxN + sage::kTile - 1) / sage::kTile) * 256 * 4;
+constexpr size_t kStaticScratchBytes = 2 * kStaticKeyBytes + kStaticHistBytes + 256;  // about 4.06 MiB
+
+static __device__ __align__(256) unsigned char g_select_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+void* g_scratch_addr[kMaxDevices] = {};    // device address of g_select_scratch, per device ordinal
+std::mutex g_scratch_mutex;
+
+}  // namespace
+
+extern "C" sage_status_t sage_select_static(const float* scores, int64_t N, double keep_rate, int64_t* idx, int64_t* k_out,
+                                            void* cuda_stream) {
+    if (N < 0 || !(keep_rate == keep_rate) || (N > 0 && !scores)) {
+        sage::set_error_message("sage_select_static: bad argument (negative N, NaN keep_rate or null scores)");
+        return SAGE_ERR_INVALID_ARG;
+    }
+    if (N > kStaticMaxN) {
+        char msg[200];
+        snprintf(msg, sizeof msg, "sage_select_static: N=%lld exceeds the built-in scratch (at most %lld scores); use sage_select",
+                 (long long)N, (long long)kStaticMaxN);
+        sage::set_error_message(msg);
+        return SAGE_ERR_UNSUPPORTED;
+    }
+    const int64_t k = sage_select_count(N, keep_rate);
+    if (k > 0 && !idx) {
+        sage::set_error_message("sage_select_static: null idx");
+        return SAGE_ERR_INVALID_ARG;
+    }
+    if (k > 0) {
+        int dev = -1;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+            sage::set_error_message("sage_select_static: no current CUDA device (or ordinal above 63)");
+            return SAGE_ERR_CUDA;
+        }
+        void* scratch = nullptr;
+        {
+            std::lock_guard<std::mutex> lock(g_scratch_mutex);
+            if (!g_scratch_addr[dev]) {       // first call on this device: resolve the array's device address
+                void* p = nullptr;
+                e = cudaGetSymbolAddress(&p, g_select_scratch);
+                if (e != cudaSuccess || !p) {
+                    char msg[200];
+                    snprintf(msg, sizeof msg, "sage_select_static: cudaGetSymbolAddress failed on device %d: %s", dev,
+                             cudaGetErrorString(e));
+                    sage::set_error_message(msg);
+                    return SAGE_ERR_CUDA;
+                }
+                g_scratch_addr[dev] = p;
+            }
+            scratch = g_scratch_addr[dev];
+        }
+        // Nothing in the scratch has to start at zero: the key arrays are written for every i < N before
+        // they are read and each radix pass rewrites the whole histogram it scans.
+        e = sage::launch_select(scores, N, k, idx, scratch, static_cast<cudaStream_t>(cuda_stream));
+        if (e != cudaSuccess) {
+            char msg[200];
+            snprintf(msg, sizeof msg, "sage_select_static: launch failed: %s", cudaGetErrorString(e));
+            sage::set_error_message(msg);
+            return SAGE_ERR_CUDA;
+        }
+        int idx_bits = 1;
+        while (idx_bits < 32 && (1ll << idx_bits) < N) ++idx_bits;
+        sage::count_launches(2 + 3 * (4 + (idx_bits + 7) / 8));
+    }
+    if (k_out) *k_out = k;
+    return SAGE_OK;
+}
