@@ -108,7 +108,7 @@ def test_zero_rows_and_zero_consensus():
 # ------------------------------------------------------------------ sketch + full path on small shapes
 
 @pytest.mark.parametrize("N,D,ell", [(3, 8, 2), (4, 17, 2), (9, 33, 4), (64, 32, 8), (257, 100, 5), (1000, 300, 16),
-                                     (700, 1030, 33)])
+                                     (700, 1030, 33), (600, 400, 80), (500, 260, 100)])
 def test_full_path_small_shapes(N, D, ell):
     rows = lowrank_rows(N, D, min(3, D), 0.3, N * 7 + D)
     ref = oracle.run(rows, D, ell, 0.2)
