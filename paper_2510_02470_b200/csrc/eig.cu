@@ -46,18 +46,21 @@ __device__ __forceinline__ void rr_pair(int n_even, int round, int slot, int& p,
 
 // ------------------------------------------------------------------------------------------------
 // Shared-memory solver for n <= 192 (the common case: n = 2*ell <= 128, and partly filled buffers at
-// the freeze). Same mathematics as k_eig_shrink below, restructured for latency:
-//   * Cholesky with diagonal pivoting but WITHOUT data movement: the pivot column stays where it is,
-//     a per-index pivot order replaces the row/column swaps, every warp keeps the running diagonal in
-//     registers and finds the pivot redundantly, so a step costs one block barrier;
-//   * one-sided Jacobi with one pair per HALF-warp: 16 lanes hold both columns in registers (float4
-//     accesses, conflict-free), reduce the three dot products with 4 shuffle steps and rotate;
+// the freeze). Same mathematics as k_eig_shrink below, restructured for instruction count and latency:
+//   * K is scaled by 1/max(diag) on load, so every intermediate is O(1) and fast reciprocal / rsqrt
+//     intrinsics are safe; eigenvalues are scaled back at the end;
+//   * Cholesky with diagonal pivoting but WITHOUT data movement: the pivot column stays where it is and
+//     a per-index pivot order replaces the row/column swaps; every warp keeps the running diagonal in
+//     registers and finds the pivot redundantly with one warp-wide integer max, so a step costs one
+//     block barrier;
+//   * one-sided Jacobi with one pair per QUARTER-warp: 8 lanes hold both columns in registers (float4
+//     accesses, conflict-free), reduce the three dot products with 3 shuffle steps and rotate; warps
+//     without a pair only take part in the barrier;
 //   * a sweep whose largest pre-rotation cosine is below 3e-4 ends the iteration (the next sweep
 //     would find cosines near 1e-7, below the rotation threshold).
 // X is column-major with a row pitch of LD = 64*T floats; column c of the factor stays at the physical
 // position of the c-th pivot, so the rows of U come out in the original buffer order.
 // ------------------------------------------------------------------------------------------------
-constexpr int kHalfWarps = kThreads / 16;
 constexpr int kMaxFast = 192;
 
 template <int T>
@@ -65,7 +68,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 k_eig_shrink_fast(const float* __restrict__ K, int ldk, int n, int do_shrink, int delta_rank, int keep, float* __restrict__ Ur,
                   int ldu, float* __restrict__ sigma_out, int n_sigma, int max_sweeps, EigInfo* __restrict__ info) {
     constexpr int LD = 64 * T;
-    constexpr int R = 2 * T;            // rows per lane when a warp spans a column (32 lanes)
+    constexpr int R = 2 * T;            // rows per lane when 32 lanes span a column
+    constexpr int Q = 2 * T;            // float4 per lane when 8 lanes span a column
     extern __shared__ __align__(16) float smem[];
     float* X = smem;                                    // LD x LD
     float* lam = X + LD * LD;                           // kMaxFast each from here on
@@ -78,44 +82,54 @@ k_eig_shrink_fast(const float* __restrict__ K, int ldk, int n, int do_shrink, in
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    for (int e = tid; e < n * LD; e += kThreads) {
-        const int c = e / LD, i = e - c * LD;
-        X[e] = (i < n) ? K[(size_t)c * ldk + i] : 0.f;  // K is symmetric: row c serves as column c
-    }
-    if (tid < kMaxFast) ord[tid] = -1;
     // running diagonal and liveness of the rows this lane owns (rows lane + 32 t), one copy per warp
     float dg[R];
     bool alive[R];
     bool bad = false;
+    float dmax = 0.f;
 #pragma unroll
     for (int t = 0; t < R; ++t) {
         const int i = lane + 32 * t;
         dg[t] = (i < n) ? K[(size_t)i * ldk + i] : -1.f;
         alive[t] = i < n;
         if (alive[t] && !(fabsf(dg[t]) <= 3.0e38f)) { bad = true; alive[t] = false; }
+        if (alive[t]) dmax = fmaxf(dmax, dg[t]);
     }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) dmax = fmaxf(dmax, __shfl_xor_sync(0xffffffffu, dmax, o));
     if (warp == 0 && bad) atomicOr(&info->flags, kFlagNonFinite);
+    const bool empty = !(dmax >= 1e-30f);              // nothing to factor: rank 0
+    const float kscale = empty ? 0.f : 1.f / dmax;
+    for (int e = tid; e < n * LD; e += kThreads) {
+        const int c = e / LD, i = e - c * LD;
+        X[e] = (i < n) ? K[(size_t)c * ldk + i] * kscale : 0.f;  // K is symmetric: row c serves as column c
+    }
+#pragma unroll
+    for (int t = 0; t < R; ++t) dg[t] *= kscale;
+    if (tid < kMaxFast) ord[tid] = -1;
     __syncthreads();
 
-    // ---- pivoted Cholesky without swaps ----
-    float tol = 0.f;
-    int rank = n;
-    for (int k = 0; k < n; ++k) {
-        ArgMax am{-1.f, 0x7fffffff};
+    // ---- pivoted Cholesky without swaps (scaled matrix: diagonal <= 1) ----
+    constexpr int CW = (kMaxFast + kWarps - 1) / kWarps;       // columns a warp owns: warp + 32 u
+    unsigned colmask = 0u;                                     // bit u: column warp + 32 u is still unpivoted
+#pragma unroll
+    for (int u = 0; u < CW; ++u)
+        if (warp + kWarps * u < n) colmask |= 1u << u;
+    const float tol = 1e-7f;
+    int rank = empty ? 0 : n;
+    for (int k = 0; k < rank; ++k) {
+        unsigned key = 0u;
 #pragma unroll
         for (int t = 0; t < R; ++t)
-            if (alive[t]) am = better(am, ArgMax{dg[t], lane + 32 * t});
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            ArgMax other{__shfl_xor_sync(0xffffffffu, am.v, o), __shfl_xor_sync(0xffffffffu, am.i, o)};
-            am = better(am, other);
-        }
-        const float d = am.v;
-        const int p = am.i;
-        if (k == 0) tol = fmaxf(d * 1e-7f, 1e-37f);
-        if (!(d > tol) || p >= n) { rank = k; break; }            // identical in every warp
-        const float inv = 1.f / sqrtf(d);
+            if (alive[t]) key = max(key, (__float_as_uint(fmaxf(dg[t], 0.f)) & 0xffffff00u) | (unsigned)(255 - (lane + 32 * t)));
+        key = __reduce_max_sync(0xffffffffu, key);                // largest diagonal (24 significant bits), smaller index on ties
+        const int p = 255 - (int)(key & 255u);
+        if (key == 0u || p >= n) { rank = k; break; }             // identical in every warp
         const float* Xp = X + p * LD;
+        const float d = Xp[p];
+        if (!(d > tol)) { rank = k; break; }
+        const float inv = rsqrtf(d);
+        if ((p & (kWarps - 1)) == warp) colmask &= ~(1u << (p / kWarps));
         float li[R];
 #pragma unroll
         for (int t = 0; t < R; ++t) {
@@ -124,15 +138,24 @@ k_eig_shrink_fast(const float* __restrict__ K, int ldk, int n, int do_shrink, in
             li[t] = alive[t] ? Xp[i] * inv : 0.f;
             dg[t] = fmaf(-li[t], li[t], dg[t]);
         }
-        for (int j = warp; j < n; j += kWarps) {
-            if (j == p) continue;
-            if (ord[j] >= 0) continue;                            // ord[p] is written below but never read here
-            const float lj = Xp[j] * inv;
-            float* col = X + j * LD;
+#pragma unroll
+        for (int u0 = 0; u0 < CW; u0 += 2) {                      // two columns at a time: loads first, then stores
+            const bool on0 = (colmask >> u0) & 1u, on1 = (u0 + 1 < CW) && ((colmask >> (u0 + 1)) & 1u);
+            if (!on0 && !on1) continue;
+            float* c0 = X + (warp + kWarps * u0) * LD;
+            float* c1 = X + (warp + kWarps * (u0 + 1)) * LD;
+            const float l0 = on0 ? Xp[warp + kWarps * u0] * inv : 0.f;
+            const float l1 = on1 ? Xp[warp + kWarps * (u0 + 1)] * inv : 0.f;
+            float v0[R], v1[R];
 #pragma unroll
             for (int t = 0; t < R; ++t) {
-                const int i = lane + 32 * t;
-                col[i] = fmaf(-li[t], lj, col[i]);
+                v0[t] = on0 ? c0[lane + 32 * t] : 0.f;
+                v1[t] = on1 ? c1[lane + 32 * t] : 0.f;
+            }
+#pragma unroll
+            for (int t = 0; t < R; ++t) {
+                if (on0) c0[lane + 32 * t] = fmaf(-li[t], l0, v0[t]);
+                if (on1) c1[lane + 32 * t] = fmaf(-li[t], l1, v1[t]);
             }
         }
         if (tid == 0) { ord[p] = k; perm[k] = p; scl[k] = inv; }
@@ -152,79 +175,99 @@ k_eig_shrink_fast(const float* __restrict__ K, int ldk, int n, int do_shrink, in
     }
     __syncthreads();
 
-    // ---- one-sided cyclic Jacobi on the rank pivot columns, one pair per half-warp ----
-    const int hw = tid >> 4, l16 = tid & 15;
-    const float jtol = 1e-6f;
+    // ---- one-sided cyclic Jacobi on the rank pivot columns ----
+    // Columns (in pivot order) form blocks of 4. A block round pairs the blocks round-robin, one block
+    // pair per warp; the warp rotates the 16 cross pairs of its two blocks in 4 local rounds (one pair per
+    // quarter-warp, synchronised inside the warp only), and in the first block round of a sweep also the
+    // pairs inside each block. Only the warps that own a block pair take part, on a named barrier.
+    const int l8 = tid & 7, qd = lane >> 3;
     int sweeps = 0;
-    float worst = 0.f;
+    float worst2 = 0.f;                 // largest squared cosine met in the current sweep
+    int* sh_flag = reinterpret_cast<int*>(sh_f + 2);
+    if (tid < 2) sh_flag[tid] = 0;
+    __syncthreads();
     if (rank >= 2) {
-        const int ne = rank + (rank & 1), nm1 = ne - 1, half = ne >> 1;
-        for (; sweeps < max_sweeps;) {
-            int rotated = 0;
-            worst = 0.f;
-            for (int round = 0; round < nm1; ++round) {
-                for (int base = 0; base < half; base += kHalfWarps) {
-                    const int slot = base + hw;
-                    int p = 0, q = ne;
-                    if (slot < half) {
-                        int a, b;
-                        if (slot == 0) { a = nm1; b = round; }
-                        else {
-                            a = round + slot; if (a >= nm1) a -= nm1;
-                            b = round + nm1 - slot; if (b >= nm1) b -= nm1;
-                        }
-                        p = min(a, b); q = max(a, b);
-                    }
-                    const bool valid = q < rank;
-                    float4* xp = reinterpret_cast<float4*>(X + (valid ? perm[p] : 0) * LD) + l16;
-                    float4* xq = reinterpret_cast<float4*>(X + (valid ? perm[q] : 0) * LD) + l16;
-                    float4 x[T], y[T];
-                    float a = 0.f, b = 0.f, g = 0.f;
+        const int nb = (rank + 3) >> 2, nbe = nb + (nb & 1), nbm1 = nbe - 1, nact = nbe >> 1;   // nact <= 24 warps
+        if (warp < nact) {
+            const int nthreads = nact * 32;
+            auto pair_step = [&](int p, int q) {                  // p, q: pivot-order columns, q >= rank means no pair
+                const bool valid = p < rank && q < rank;
+                float4* xp = reinterpret_cast<float4*>(X + (valid ? perm[p] : 0) * LD) + l8;
+                float4* xq = reinterpret_cast<float4*>(X + (valid ? perm[q] : 0) * LD) + l8;
+                float4 x[Q], y[Q];
+                float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f, g0 = 0.f, g1 = 0.f;
 #pragma unroll
-                    for (int t = 0; t < T; ++t) {
-                        x[t] = xp[16 * t];
-                        y[t] = xq[16 * t];
-                        a = fmaf(x[t].x, x[t].x, a); a = fmaf(x[t].y, x[t].y, a); a = fmaf(x[t].z, x[t].z, a); a = fmaf(x[t].w, x[t].w, a);
-                        b = fmaf(y[t].x, y[t].x, b); b = fmaf(y[t].y, y[t].y, b); b = fmaf(y[t].z, y[t].z, b); b = fmaf(y[t].w, y[t].w, b);
-                        g = fmaf(x[t].x, y[t].x, g); g = fmaf(x[t].y, y[t].y, g); g = fmaf(x[t].z, y[t].z, g); g = fmaf(x[t].w, y[t].w, g);
-                    }
+                for (int t = 0; t < Q; ++t) {
+                    x[t] = xp[8 * t];
+                    y[t] = xq[8 * t];
+                    a0 = fmaf(x[t].x, x[t].x, a0); a1 = fmaf(x[t].y, x[t].y, a1); a0 = fmaf(x[t].z, x[t].z, a0); a1 = fmaf(x[t].w, x[t].w, a1);
+                    b0 = fmaf(y[t].x, y[t].x, b0); b1 = fmaf(y[t].y, y[t].y, b1); b0 = fmaf(y[t].z, y[t].z, b0); b1 = fmaf(y[t].w, y[t].w, b1);
+                    g0 = fmaf(x[t].x, y[t].x, g0); g1 = fmaf(x[t].y, y[t].y, g1); g0 = fmaf(x[t].z, y[t].z, g0); g1 = fmaf(x[t].w, y[t].w, g1);
+                }
+                float a = a0 + a1, b = b0 + b1, g = g0 + g1;
 #pragma unroll
-                    for (int o = 8; o > 0; o >>= 1) {
-                        a += __shfl_xor_sync(0xffffffffu, a, o);
-                        b += __shfl_xor_sync(0xffffffffu, b, o);
-                        g += __shfl_xor_sync(0xffffffffu, g, o);
-                    }
-                    const float lim = sqrtf(a) * sqrtf(b);
-                    const float ag = fabsf(g);
-                    if (valid && lim > 0.f && ag > jtol * lim) {
-                        worst = fmaxf(worst, ag / lim);
-                        const float zeta = (b - a) / (2.f * g);
-                        const float tt = copysignf(1.f, zeta) / (fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.f)));
-                        const float c = rsqrtf(fmaf(tt, tt, 1.f));
-                        const float s = c * tt;
+                for (int o = 4; o > 0; o >>= 1) {
+                    a += __shfl_xor_sync(0xffffffffu, a, o);
+                    b += __shfl_xor_sync(0xffffffffu, b, o);
+                    g += __shfl_xor_sync(0xffffffffu, g, o);
+                }
+                const float ab = a * b, g2 = g * g;
+                if (valid && ab > 0.f && g2 > 1e-12f * ab) {
+                    worst2 = fmaxf(worst2, __fdividef(g2, ab));
+                    const float zeta = __fdividef(b - a, 2.f * g);
+                    const float tt = copysignf(__fdividef(1.f, fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.f))), zeta);
+                    const float c = rsqrtf(fmaf(tt, tt, 1.f));
+                    const float s = c * tt;
 #pragma unroll
-                        for (int t = 0; t < T; ++t) {
-                            float4 nx, ny;
-                            nx.x = c * x[t].x - s * y[t].x; ny.x = fmaf(s, x[t].x, c * y[t].x);
-                            nx.y = c * x[t].y - s * y[t].y; ny.y = fmaf(s, x[t].y, c * y[t].y);
-                            nx.z = c * x[t].z - s * y[t].z; ny.z = fmaf(s, x[t].z, c * y[t].z);
-                            nx.w = c * x[t].w - s * y[t].w; ny.w = fmaf(s, x[t].w, c * y[t].w);
-                            xp[16 * t] = nx;
-                            xq[16 * t] = ny;
-                        }
-                        rotated = 1;
+                    for (int t = 0; t < Q; ++t) {
+                        float4 nx, ny;
+                        nx.x = fmaf(-s, y[t].x, c * x[t].x); ny.x = fmaf(s, x[t].x, c * y[t].x);
+                        nx.y = fmaf(-s, y[t].y, c * x[t].y); ny.y = fmaf(s, x[t].y, c * y[t].y);
+                        nx.z = fmaf(-s, y[t].z, c * x[t].z); ny.z = fmaf(s, x[t].z, c * y[t].z);
+                        nx.w = fmaf(-s, y[t].w, c * x[t].w); ny.w = fmaf(s, x[t].w, c * y[t].w);
+                        xp[8 * t] = nx;
+                        xq[8 * t] = ny;
                     }
                 }
-                __syncthreads();
+                __syncwarp();
+            };
+            int more = 0;
+            while (sweeps < max_sweeps) {
+                worst2 = 0.f;
+                for (int br = 0; br < nbm1; ++br) {
+                    int ba, bb;                                   // the two blocks of this warp in this block round
+                    if (warp == 0) { ba = nbm1; bb = br; }
+                    else {
+                        ba = br + warp; if (ba >= nbm1) ba -= nbm1;
+                        bb = br + nbm1 - warp; if (bb >= nbm1) bb -= nbm1;
+                    }
+                    if (br == 0) {                                // pairs inside each block: quarters 0,1 -> ba, 2,3 -> bb
+                        const int base = 4 * ((qd < 2) ? ba : bb), h = qd & 1;
+                        pair_step(base + (h ? 2 : 0), base + (h ? 3 : 1));
+                        pair_step(base + (h ? 1 : 0), base + (h ? 3 : 2));
+                        pair_step(base + (h ? 1 : 0), base + (h ? 2 : 3));
+                    }
+                    const int lo = min(ba, bb), hi = max(ba, bb);
+#pragma unroll 1
+                    for (int r = 0; r < 4; ++r) pair_step(4 * lo + qd, 4 * hi + ((qd + r) & 3));
+                    asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
+                }
+                ++sweeps;
+                const int par = sweeps & 1;
+                if (__any_sync(0xffffffffu, worst2 > 9e-8f) && lane == 0) atomicOr(&sh_flag[par], 1);
+                if (tid == 0) sh_flag[par ^ 1] = 0;
+                asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
+                more = sh_flag[par];
+                if (!more) break;               // every cosine of this sweep was below 3e-4: converged after it
             }
-            ++sweeps;
-            (void)rotated;
-            if (!__syncthreads_or(worst > 3e-4f)) break;   // every cosine of this sweep was small: converged after it
+            if (tid == 0) { sh_f[1] = (float)sweeps; sh_f[4] = more ? 1.f : 0.f; }
         }
     }
-    const int not_converged = __syncthreads_or(sweeps >= max_sweeps && worst > 1e-4f);
+    __syncthreads();
+    sweeps = rank >= 2 ? (int)sh_f[1] : 0;
+    const int not_converged = rank >= 2 && sh_f[4] != 0.f;     // stopped at the sweep limit while still rotating visibly
 
-    // ---- eigenvalues = squared column norms (pivot-step order); sort descending, stable ----
+    // ---- eigenvalues = squared column norms (pivot-step order), scaled back; sort descending, stable ----
     for (int k = warp; k < n; k += kWarps) {
         float a = 0.f;
         if (k < rank) {
@@ -234,7 +277,7 @@ k_eig_shrink_fast(const float* __restrict__ K, int ldk, int n, int do_shrink, in
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
         }
-        if (lane == 0) lam[k] = a;
+        if (lane == 0) lam[k] = a * dmax;
     }
     __syncthreads();
     if (tid < n) {
@@ -263,13 +306,14 @@ k_eig_shrink_fast(const float* __restrict__ K, int ldk, int n, int do_shrink, in
     }
     __syncthreads();
     const float delta = sh_f[0];
+    const float back = sqrtf(dmax);     // columns of X are sigma_j u_j / sqrt(dmax)
     if (tid < n) {
         const float l = lam[order[tid]];
         float f = 0.f, sp = 0.f;
         if (l > 0.f && tid < keep) {
             const float kept = fmaxf(l - delta, 0.f);
             sp = sqrtf(kept);
-            f = sqrtf(kept / l) * rsqrtf(l);
+            f = sqrtf(kept / l) * rsqrtf(l) * back;   // (sigma'/sigma) / sigma, for the unscaled column
         }
         fac[tid] = f;
         if (tid < n_sigma) sigma_out[tid] = sp;
@@ -502,7 +546,7 @@ cudaError_t launch_eig_shrink(const float* K, int ldk, int n, int do_shrink, int
     if (n <= 0 || n > 512) return cudaErrorInvalidValue;
     if (n <= kMaxFast) {
         const int T = (n + 63) / 64;
-        const size_t bytes = ((size_t)(64 * T) * (64 * T) + 3 * kMaxFast) * sizeof(float) + 3 * kMaxFast * sizeof(int) + 16;
+        const size_t bytes = ((size_t)(64 * T) * (64 * T) + 3 * kMaxFast) * sizeof(float) + 3 * kMaxFast * sizeof(int) + 32;
         cudaError_t e;
 #define SAGE_EIG_FAST(TT)                                                                                              \
     e = cudaFuncSetAttribute(k_eig_shrink_fast<TT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);          \
