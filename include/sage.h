@@ -160,7 +160,8 @@ typedef struct {
     int32_t last_sweeps;    /* Jacobi sweeps of the most recent eigen-solve */
     int32_t max_sweeps;     /* largest sweep count seen */
     int32_t last_rank;      /* numerical rank found by the most recent factorisation */
-    uint32_t device_flags;  /* bit 0: eigen-solver not converged, bit 1: non-finite input seen */
+    uint32_t device_flags;  /* bit 0: eigen-solver not converged, bit 1: non-finite input seen,
+                               bit 2: a tensor-core kernel gave up a bounded wait (results invalid) */
     int64_t kernel_launches;/* kernels this handle has launched since create/reset */
 } sage_stats_t;
 
@@ -169,7 +170,9 @@ sage_status_t sage_fd_stats(sage_fd_t* h, sage_stats_t* out);
 
 /* Options. Before the first update: key 1 = delta rank (which singular value, 1-indexed, defines
  * delta; default ell), key 2 = maximum Jacobi sweeps (default 30). At any time: key 3 = bit mask of
- * kernel classes to time with CUDA events on the launching stream (see sage_fd_profile; default 0). */
+ * kernel classes to time with CUDA events on the launching stream (see sage_fd_profile; default 0); key 4 =
+ * 1 (default) to use the tensor-core kernels wherever the operands meet their alignment rules (16-byte
+ * aligned base, row pitch a multiple of 16 bytes), 0 to use the CUDA-core kernels everywhere. */
 sage_status_t sage_fd_set_option(sage_fd_t* h, int key, double value);
 
 /* Per-kernel device time of this handle's launches since the previous call, for the classes selected

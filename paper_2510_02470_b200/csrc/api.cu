@@ -105,6 +105,11 @@ struct sage_fd {
     size_t partials_bytes = 0;
     double* zsum = nullptr;
     float* u = nullptr;
+    __nv_bfloat16* P16 = nullptr;  // frozen sketch in bf16 (bf16 handles: tensor-core projection operand); with p16_fold
+                                   // rows [0, ell) hold bf16(S) and rows [n_pad, n_pad + ell) hold bf16(S - bf16(S))
+    int p16_fold = 0, p16_npad = 0;
+    int* tc_err = nullptr;         // set by a tensor-core kernel whose bounded wait ran out
+    bool use_tc = true;            // option 4: tensor-core kernels where their alignment rules hold
     int64_t launches = 0;
     Prof prof;
 };
@@ -146,6 +151,32 @@ int pick_splits(int tiles, int64_t K, int64_t min_k) {
     if (s > cap) s = cap;
     if (s < 1) s = 1;
     return (int)s;
+}
+
+// Split count for a grid of `tiles` CTAs per split on 148 SMs: the count (each slice keeping at least
+// min_k of the contraction) that wastes the least of the last wave; ties go to fewer splits.
+int pick_splits_waves(int tiles, int64_t K, int64_t min_k, int max_splits) {
+    int64_t cap = K / min_k;
+    if (cap > max_splits) cap = max_splits;
+    if (cap < 1) cap = 1;
+    int best = 1;
+    double best_eff = 0.0;
+    for (int s = 1; s <= (int)cap; ++s) {
+        const int64_t ctas = (int64_t)tiles * s;
+        const double eff = (double)ctas / (double)(((ctas + 147) / 148) * 148);
+        if (eff > best_eff + 1e-9) { best_eff = eff; best = s; }
+    }
+    return best;
+}
+
+// After the sketch is frozen: the bf16 copy the tensor-core projection reads (bf16 handles only).
+sage_status_t enqueue_freeze_aux(sage_fd* h, cudaStream_t st) {
+    if (h->dtype == SAGE_BF16 && h->P16)
+        CU_TRY(timed(h, K_APPEND, 1, st, [&] {
+            return launch_to_bf16(h->B[h->cur], h->pitch, h->ell, h->pitch, h->P16,
+                                  h->p16_fold ? h->P16 + (size_t)h->p16_npad * h->pitch : nullptr, h->pitch, st);
+        }));
+    return SAGE_OK;
 }
 
 // Gram of the first r buffer rows -> Kmat (r x r, pitch m).
@@ -277,6 +308,17 @@ sage_status_t sage_fd_create(sage_fd_t** out, int64_t D, int32_t ell, sage_dtype
     if ((e = cudaMalloc((void**)&h->info, sizeof(EigInfo))) != cudaSuccess) return fail(e, "cudaMalloc(info)");
     if ((e = cudaMalloc((void**)&h->zsum, 256 * sizeof(double))) != cudaSuccess) return fail(e, "cudaMalloc(zsum)");
     if ((e = cudaMalloc((void**)&h->u, 256 * sizeof(float))) != cudaSuccess) return fail(e, "cudaMalloc(u)");
+    if ((e = cudaMalloc((void**)&h->tc_err, sizeof(int))) != cudaSuccess) return fail(e, "cudaMalloc(err)");
+    if ((e = cudaMemset(h->tc_err, 0, sizeof(int))) != cudaSuccess) return fail(e, "cudaMemset");
+    if (row_dtype == SAGE_BF16) {
+        // Two-term bf16 sketch (16 significant bits) wherever the doubled tensor work stays well below the HBM
+        // time of the rows: ell <= 64, or short rows where rounding errors average over few terms.
+        h->p16_npad = ((ell + 15) / 16) * 16;
+        h->p16_fold = (2 * h->p16_npad <= 256 && (ell <= 64 || D < 16384)) ? 1 : 0;
+        const size_t prow = h->p16_fold ? 2 * (size_t)h->p16_npad : (size_t)ell;
+        if ((e = cudaMalloc((void**)&h->P16, prow * h->pitch * sizeof(__nv_bfloat16))) != cudaSuccess) return fail(e, "cudaMalloc(P16)");
+        if ((e = cudaMemset(h->P16, 0, prow * h->pitch * sizeof(__nv_bfloat16))) != cudaSuccess) return fail(e, "cudaMemset");
+    }
     if ((e = cudaMemset(h->info, 0, sizeof(EigInfo))) != cudaSuccess) return fail(e, "cudaMemset");
     if ((e = cudaMemset(h->sigma, 0, ell * sizeof(float))) != cudaSuccess) return fail(e, "cudaMemset");
     if ((e = cudaDeviceSynchronize()) != cudaSuccess) return fail(e, "cudaDeviceSynchronize");
@@ -302,6 +344,8 @@ void sage_fd_destroy(sage_fd_t* h) {
     cudaFree(h->partials);
     cudaFree(h->zsum);
     cudaFree(h->u);
+    cudaFree(h->P16);
+    cudaFree(h->tc_err);
     for (auto& p : h->prof.pending) {
         cudaEventDestroy(p.a);
         cudaEventDestroy(p.b);
@@ -316,6 +360,7 @@ sage_status_t sage_fd_reset(sage_fd_t* h) {
     CU_TRY(cudaDeviceSynchronize());
     CU_TRY(cudaMemset(h->info, 0, sizeof(EigInfo)));
     CU_TRY(cudaMemset(h->sigma, 0, h->ell * sizeof(float)));
+    CU_TRY(cudaMemset(h->tc_err, 0, sizeof(int)));
     h->fill = 0;
     h->rows_seen = 0;
     h->cur = 0;
@@ -328,6 +373,10 @@ sage_status_t sage_fd_set_option(sage_fd_t* h, int key, double value) {
     ST_TRY(check_handle(h));
     if (key == 3) {                          // per-kernel event timing mask: allowed at any time
         h->prof.mask = (unsigned)value & ((1u << K_NCLASS) - 1u);
+        return SAGE_OK;
+    }
+    if (key == 4) {                          // 0: CUDA-core kernels only, 1: tensor-core kernels where possible
+        h->use_tc = value != 0.0;
         return SAGE_OK;
     }
     if (h->rows_seen != 0 || h->state != SKETCHING) {
@@ -392,10 +441,17 @@ sage_status_t sage_fd_finalize(sage_fd_t* h, void* cuda_stream) {
         const int keep = do_shrink ? h->delta_rank - 1 : (r < h->ell ? r : h->ell);
         ST_TRY(enqueue_factor(h, r, do_shrink, keep < h->ell ? keep : h->ell, h->ell, st));
     }
+    ST_TRY(enqueue_freeze_aux(h, st));
     h->state = FROZEN;
     EigInfo info;
+    int tc_err = 0;
     CU_TRY(cudaMemcpyAsync(&info, h->info, sizeof info, cudaMemcpyDeviceToHost, st));
+    CU_TRY(cudaMemcpyAsync(&tc_err, h->tc_err, sizeof tc_err, cudaMemcpyDeviceToHost, st));
     CU_TRY(cudaStreamSynchronize(st));
+    if (tc_err) {
+        set_err("sage_fd_finalize: a tensor-core kernel gave up waiting on its pipeline (results are not valid)");
+        return SAGE_ERR_CUDA;
+    }
     if (info.flags & kFlagNotConverged) {
         set_err("sage_fd_finalize: an eigen-solve reached the sweep limit (%d)", h->max_sweeps);
         return SAGE_ERR_NOT_CONVERGED;
@@ -433,6 +489,7 @@ sage_status_t sage_fd_load_sketch(sage_fd_t* h, const float* S, int64_t ld, void
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     CU_TRY(timed(h, K_APPEND, 1, st, [&] { return launch_append(S, SAGE_F32, h->ell, ld, h->D, h->B[h->cur], h->pitch, 0, st); }));
     CU_TRY(cudaMemsetAsync(h->sigma, 0, h->ell * sizeof(float), st));
+    ST_TRY(enqueue_freeze_aux(h, st));
     h->fill = h->ell;
     h->state = FROZEN;
     return SAGE_OK;
@@ -482,31 +539,59 @@ sage_status_t sage_score_chunk(sage_fd_t* h, const void* rows, int64_t n, int64_
     DeviceGuard g(h->device);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const int ell = h->ell;
-    const int64_t sub_max = 16384;
+    const int64_t sub_max = 148 * 128;       // one full wave of 128-row tiles
     const char* p = static_cast<const char*>(rows);
     const size_t row_bytes = (size_t)ld * elem_size(h->dtype);
     const float* S = h->B[h->cur];
+    // Tensor-core path: bf16 rows against the bf16 copy of the sketch (a one-term bf16 sketch is only used for
+    // long rows, where its rounding errors average out). fp32 rows keep the CUDA-core kernel.
+    const bool tc_ok = h->use_tc && h->dtype == SAGE_BF16 && h->P16 && (h->p16_fold || h->D >= 16384) &&
+                       (reinterpret_cast<uintptr_t>(rows) & 15u) == 0 && (row_bytes & 15u) == 0;
     for (int64_t r0 = 0; r0 < n; r0 += sub_max) {
         const int64_t sub = (n - r0 < sub_max) ? n - r0 : sub_max;
-        const int tiles = (int)((sub + 63) / 64) * ((ell + 63) / 64);
-        const int splits = pick_splits(tiles, h->D, 1024);
-        const size_t zred = (size_t)sub * ell * sizeof(float);
-        ST_TRY(ensure(&h->zwork, &h->zwork_bytes, zred * (splits > 1 ? splits + 1 : 1)));
         const size_t nb = (size_t)((sub + 63) / 64);
         ST_TRY(ensure(&h->partials, &h->partials_bytes, nb * ell * sizeof(float)));
-        float* Z = h->zwork;
-        if (splits == 1) {
-            CU_TRY(timed(h, K_PROJECT, 1, st, [&] {
-                return launch_gemm_nt(p + r0 * row_bytes, h->dtype, ld, S, h->pitch, (int)sub, ell, h->D, 1, Z, ell, 0, st);
-            }));
-        } else {
-            float* parts = h->zwork + (size_t)sub * ell;
-            CU_TRY(timed(h, K_PROJECT, 1, st, [&] {
-                return launch_gemm_nt(p + r0 * row_bytes, h->dtype, ld, S, h->pitch, (int)sub, ell, h->D, splits, parts, ell,
-                                      (int64_t)sub * ell, st);
-            }));
-            CU_TRY(timed(h, K_PROJECT_REDUCE, 1, st,
-                         [&] { return launch_split_reduce(parts, splits, (int64_t)sub * ell, (int)sub, ell, ell, Z, ell, st); }));
+        const size_t zred = (size_t)sub * ell * sizeof(float);
+        bool done = false;
+        float* Z = nullptr;
+        if (tc_ok) {
+            const int splits = pick_splits_waves((int)((sub + 127) / 128), h->D, 4096, 64);
+            ST_TRY(ensure(&h->zwork, &h->zwork_bytes, zred * (splits > 1 ? splits + 1 : 1)));
+            Z = h->zwork;
+            float* out = splits > 1 ? h->zwork + (size_t)sub * ell : Z;
+            cudaError_t e = timed(h, K_PROJECT, 1, st, [&] {
+                return launch_tc_gemm_nt(p + r0 * row_bytes, SAGE_BF16, ld, h->P16, h->pitch, (int)sub, ell, h->p16_fold, h->D, splits,
+                                         out, ell, (int64_t)sub * ell, h->tc_err, st);
+            });
+            if (e == cudaSuccess) {
+                done = true;
+                if (splits > 1)
+                    CU_TRY(timed(h, K_PROJECT_REDUCE, 1, st,
+                                 [&] { return launch_split_reduce(out, splits, (int64_t)sub * ell, (int)sub, ell, ell, Z, ell, st); }));
+            } else if (e != cudaErrorNotSupported) {
+                CU_TRY(e);
+            } else {
+                count(h, -1);
+            }
+        }
+        if (!done) {
+            const int tiles = (int)((sub + 63) / 64) * ((ell + 63) / 64);
+            const int splits = pick_splits(tiles, h->D, 1024);
+            ST_TRY(ensure(&h->zwork, &h->zwork_bytes, zred * (splits > 1 ? splits + 1 : 1)));
+            Z = h->zwork;
+            if (splits == 1) {
+                CU_TRY(timed(h, K_PROJECT, 1, st, [&] {
+                    return launch_gemm_nt(p + r0 * row_bytes, h->dtype, ld, S, h->pitch, (int)sub, ell, h->D, 1, Z, ell, 0, st);
+                }));
+            } else {
+                float* parts = h->zwork + (size_t)sub * ell;
+                CU_TRY(timed(h, K_PROJECT, 1, st, [&] {
+                    return launch_gemm_nt(p + r0 * row_bytes, h->dtype, ld, S, h->pitch, (int)sub, ell, h->D, splits, parts, ell,
+                                          (int64_t)sub * ell, st);
+                }));
+                CU_TRY(timed(h, K_PROJECT_REDUCE, 1, st,
+                             [&] { return launch_split_reduce(parts, splits, (int64_t)sub * ell, (int)sub, ell, ell, Z, ell, st); }));
+            }
         }
         const int64_t row = row_offset + r0;
         CU_TRY(timed(h, K_NORMALISE, 2, st, [&] {
@@ -606,7 +691,9 @@ sage_status_t sage_fd_stats(sage_fd_t* h, sage_stats_t* out) {
     out->last_sweeps = info.sweeps;
     out->max_sweeps = info.max_sweeps;
     out->last_rank = info.rank;
-    out->device_flags = info.flags;
+    int tc_err = 0;
+    CU_TRY(cudaMemcpy(&tc_err, h->tc_err, sizeof tc_err, cudaMemcpyDeviceToHost));
+    out->device_flags = info.flags | (tc_err ? 4u : 0u);
     out->kernel_launches = h->launches;
     return SAGE_OK;
 }

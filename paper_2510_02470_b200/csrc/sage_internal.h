@@ -35,6 +35,20 @@ cudaError_t launch_append(const void* rows, sage_dtype_t dt, int64_t n, int64_t 
 cudaError_t launch_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const float* Bm, int64_t ldb, int M, int N,
                            int64_t K, int splits, float* C, int64_t ldc, int64_t split_stride, cudaStream_t st);
 
+// Tensor-core version of launch_gemm_nt (tcgen05 + TMA). Both operands have element type dt (fp32 operands are
+// read as tf32) and must satisfy TMA's rules: 16-byte aligned base, pitch a multiple of 16 bytes.
+// Returns cudaErrorNotSupported when they do not, so that the caller can take launch_gemm_nt instead.
+// fold != 0: Bm holds two stacked operands, rows [0, N) and rows [n_pad, n_pad + N) with n_pad = N rounded up to
+// 16, and C receives the sum of both products (a two-term representation of a more precise B); needs 2 n_pad <= 256.
+// Without fold N <= 256. *err (device) is set to 1 if a bounded wait inside the kernel ran out.
+cudaError_t launch_tc_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const void* Bm, int64_t ldb, int M, int N, int fold,
+                              int64_t K, int splits, float* C, int64_t ldc, int64_t split_stride, int* err, cudaStream_t st);
+
+// hi[i][0:cols] = bf16(src[i][0:cols]) (round to nearest even) for i < rows; when lo != nullptr also
+// lo[i][:] = bf16(src - float(hi)), so that hi + lo carries 16 significant bits of src.
+cudaError_t launch_to_bf16(const float* src, int64_t lds, int rows, int64_t cols, __nv_bfloat16* hi, __nv_bfloat16* lo, int64_t ldd,
+                           cudaStream_t st);
+
 // out[i][j] = sum_z parts[z][i][j] in ascending z with fp64 accumulation. (M x N, pitches ldp / ldo.)
 cudaError_t launch_split_reduce(const float* parts, int splits, int64_t split_stride, int M, int N, int64_t ldp,
                                 float* out, int64_t ldo, cudaStream_t st);

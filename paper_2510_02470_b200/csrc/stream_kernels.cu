@@ -136,6 +136,19 @@ __global__ void __launch_bounds__(256) k_gemm_nt(const T* __restrict__ A, int64_
     }
 }
 
+__global__ void __launch_bounds__(256) k_to_bf16(const float* __restrict__ src, int64_t lds, int64_t cols, __nv_bfloat16* __restrict__ hi,
+                                                  __nv_bfloat16* __restrict__ lo, int64_t ldd) {
+    const float* s = src + (int64_t)blockIdx.y * lds;
+    __nv_bfloat16* dh = hi + (int64_t)blockIdx.y * ldd;
+    __nv_bfloat16* dl = lo ? lo + (int64_t)blockIdx.y * ldd : nullptr;
+    for (int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; c < cols; c += (int64_t)gridDim.x * blockDim.x) {
+        const float x = s[c];
+        const __nv_bfloat16 h = __float2bfloat16_rn(x);
+        dh[c] = h;
+        if (dl) dl[c] = __float2bfloat16_rn(x - __bfloat162float(h));
+    }
+}
+
 __global__ void __launch_bounds__(256) k_split_reduce(const float* __restrict__ parts, int splits, int64_t split_stride,
                                                       int M, int N, int64_t ldp, float* __restrict__ out, int64_t ldo) {
     const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -233,6 +246,15 @@ cudaError_t launch_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const fl
     else
         k_gemm_nt<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(A), lda, Bm, ldb, M, N, K, kps, C, ldc,
                                                        split_stride);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_to_bf16(const float* src, int64_t lds, int rows, int64_t cols, __nv_bfloat16* hi, __nv_bfloat16* lo, int64_t ldd,
+                           cudaStream_t st) {
+    if (rows <= 0 || cols <= 0) return cudaSuccess;
+    int64_t bx = (cols + 255) / 256;
+    if (bx > 1184) bx = 1184;
+    k_to_bf16<<<dim3((unsigned)bx, (unsigned)rows), 256, 0, st>>>(src, lds, cols, hi, lo, ldd);
     return cudaGetLastError();
 }
 

@@ -1,0 +1,223 @@
+// Tensor-core contraction C[z] = A_z * B_z^T over slices z of the contraction index, both operands
+// contiguous along that index ("K-major"): the pass-2 projection Z = G S^T (Method, "Two-pass scoring":
+// z_i = S g_i) with G streamed from HBM exactly once.
+//
+// One CTA owns a 128-row tile of A, all N rows of B and one K slice:
+//   warp 0   TMA producer: 128-byte-wide K tiles of A (128 rows) and B (N rows) into a ring of stages,
+//   warp 1   allocates TMEM and issues tcgen05.mma (M = 128, N, K = 32 bytes per instruction),
+//   warps 2-5 read the fp32 accumulator out of TMEM (one row per thread) and store the partial result.
+// Rows and K elements outside the matrices are zero-filled by TMA, so no tail code exists. Split-K
+// partials are summed by a separate kernel in a fixed order.
+#include "sage_internal.h"
+#include "tc05.cuh"
+
+namespace sage {
+namespace tc {
+
+bool make_tmap_2d(CUtensorMap* out, const void* base, int elem_bytes, uint64_t rows, uint64_t cols, uint64_t ld,
+                  uint32_t box_rows) {
+    using Fn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                            const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                            CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static Fn encode = [] {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            fn = nullptr;
+        return reinterpret_cast<Fn>(fn);
+    }();
+    if (!encode) return false;
+    if ((reinterpret_cast<uintptr_t>(base) & 15u) || ((ld * (uint64_t)elem_bytes) & 15u) || rows == 0 || cols == 0) return false;
+    if (box_rows == 0 || box_rows > 256 || cols >= (1ull << 32) || rows >= (1ull << 32)) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {ld * (uint64_t)elem_bytes};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(128 / elem_bytes), box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUtensorMapDataType dt = elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+    return encode(out, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int kTileM = 128;
+constexpr int kATileBytes = kTileM * 128;
+
+// kFmt: 1 = bf16 operands (64 elements per 128-byte K tile), 2 = fp32 operands read as tf32 (32 elements).
+template <int kFmt>
+__global__ void __launch_bounds__(kThreads, 1)
+k_tc_gemm_nt(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, int M, int N, int n_pad, int fold,
+             long long K, long long k_per_split, float* __restrict__ C, long long ldc, long long split_stride, int stages,
+             uint32_t tmem_cols, int* __restrict__ err) {
+    constexpr int BK = kFmt == 1 ? 64 : 32;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    const int n_mma = fold ? 2 * n_pad : n_pad;         // folded: B holds two stacked operands whose products are added
+    const int stage_bytes = kATileBytes + n_mma * 128;
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)stages * stage_bytes);
+    uint64_t* empty = full + stages;
+    uint64_t* tmem_full = empty + stages;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_full + 1);
+    volatile int* abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m0 = blockIdx.x * kTileM;
+    const long long k_begin = (long long)blockIdx.y * k_per_split;
+    const long long k_end = K < k_begin + k_per_split ? K : k_begin + k_per_split;
+    const int nkt = k_end > k_begin ? (int)((k_end - k_begin + BK - 1) / BK) : 0;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], 1);
+        }
+        mbar_init(tmem_full, 1);
+        *abort = 0;
+        mbar_fence_init();
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmB);
+    }
+    if (warp == 1) tmem_alloc(tmem_slot, tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            const uint32_t tx_bytes = (uint32_t)stage_bytes;
+            int issued = 0;
+            for (int kt = 0; kt < nkt; ++kt) {
+                const int s = kt % stages;
+                const uint32_t use = (uint32_t)(kt / stages);
+                if (!mbar_wait(&empty[s], (use & 1u) ^ 1u, abort)) break;
+                mbar_expect_tx(&full[s], tx_bytes);
+                const int x = (int)(k_begin + (long long)kt * BK);
+                tma_load_2d(smem + (size_t)s * stage_bytes, &tmA, &full[s], x, m0);
+                tma_load_2d(smem + (size_t)s * stage_bytes + kATileBytes, &tmB, &full[s], x, 0);
+                issued = kt + 1;
+            }
+            if (*abort) {   // give copies already in flight a bounded time to land before the block goes away
+                for (int kt = issued > stages ? issued - stages : 0; kt < issued; ++kt)
+                    mbar_wait_quiet(&full[kt % stages], (uint32_t)(kt / stages) & 1u, 20000000ll);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc(kFmt, kTileM, n_mma, 0, 0);
+            for (int kt = 0; kt < nkt; ++kt) {
+                const int s = kt % stages;
+                const uint32_t use = (uint32_t)(kt / stages);
+                if (!mbar_wait(&full[s], use & 1u, abort)) break;
+                tc_fence_after();
+                const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
+                const uint64_t adesc = smem_desc_k_sw128(a_addr);
+                const uint64_t bdesc = smem_desc_k_sw128(a_addr + kATileBytes);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {          // 4 x 32 bytes of K per 128-byte row
+                    if constexpr (kFmt == 1) mma_bf16(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, (kt | k) != 0);
+                    else mma_tf32(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, (kt | k) != 0);
+                }
+                mma_commit(&empty[s]);                 // the stage is free once these MMAs have read it
+            }
+            mma_commit(tmem_full);
+        }
+    } else {
+        const int quarter = warp & 3;                  // TMEM lanes this warp may read: 32 * (warp % 4) ...
+        bool ok = true;
+        if (nkt > 0) ok = mbar_wait(tmem_full, 0, abort);
+        ok = __all_sync(0xffffffffu, ok);
+        tc_fence_after();
+        const int row = m0 + quarter * 32 + lane;
+        float* crow = C + (long long)blockIdx.y * split_stride + (long long)row * ldc;
+        const bool vec = (ldc % 4 == 0) && ((reinterpret_cast<uintptr_t>(C) & 15u) == 0) && (split_stride % 4 == 0);
+        const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+        for (int c0 = 0; c0 < n_pad; c0 += 16) {
+            float v[16];
+            if (nkt > 0 && ok) {
+                tmem_ld16(lane_base + (uint32_t)c0, v);
+                if (fold) {
+                    float w[16];
+                    tmem_ld16(lane_base + (uint32_t)(n_pad + c0), w);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) v[j] += w[j];
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[j] = 0.f;
+            }
+            if (row < M) {
+                if (vec && c0 + 16 <= N) {
+#pragma unroll
+                    for (int j = 0; j < 16; j += 4) *reinterpret_cast<float4*>(crow + c0 + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        if (c0 + j < N) crow[c0 + j] = v[j];
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        if (nkt > 0) mbar_wait_quiet(tmem_full, 0, kWaitLimitCycles);   // no MMA in flight when TMEM is freed
+        tc_fence_after();
+        tmem_dealloc(tmem_base, tmem_cols);
+    }
+    if (threadIdx.x == 0 && *abort) atomicExch(err, 1);
+}
+
+}  // namespace
+}  // namespace tc
+
+namespace {
+int tc_gemm_pick_stages(int n_mma) {
+    const int stage_bytes = tc::kATileBytes + n_mma * 128;
+    int s = (200 * 1024) / stage_bytes;
+    if (s > 8) s = 8;
+    if (s < 2) s = 2;
+    return s;
+}
+}  // namespace
+
+cudaError_t launch_tc_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const void* Bm, int64_t ldb, int M, int N, int fold,
+                              int64_t K, int splits, float* C, int64_t ldc, int64_t split_stride, int* err, cudaStream_t st) {
+    if (M <= 0 || N <= 0 || K <= 0) return cudaSuccess;
+    const int es = dt == SAGE_F32 ? 4 : 2;
+    const int BK = 128 / es;
+    const int n_pad = ((N + 15) / 16) * 16;
+    const int n_mma = fold ? 2 * n_pad : n_pad;
+    if (n_mma > 256 || splits < 1 || splits > 65535) return cudaErrorNotSupported;
+    CUtensorMap tmA, tmB;
+    if (!tc::make_tmap_2d(&tmA, A, es, (uint64_t)M, (uint64_t)K, (uint64_t)lda, tc::kTileM)) return cudaErrorNotSupported;
+    if (!tc::make_tmap_2d(&tmB, Bm, es, (uint64_t)(fold ? n_pad + N : N), (uint64_t)K, (uint64_t)ldb, (uint32_t)n_mma))
+        return cudaErrorNotSupported;
+    int64_t kps = (K + splits - 1) / splits;
+    kps = ((kps + BK - 1) / BK) * BK;
+    if (splits > 1 && (int64_t)(splits - 1) * kps >= K) return cudaErrorInvalidValue;   // an empty slice: pick fewer splits
+    const int stages = tc_gemm_pick_stages(n_mma);
+    const int stage_bytes = tc::kATileBytes + n_mma * 128;
+    const size_t smem = (size_t)stages * stage_bytes + 1024 + (2 * stages + 1) * 8 + 16;
+    uint32_t tmem_cols = 32;
+    while (tmem_cols < (uint32_t)n_mma) tmem_cols <<= 1;
+    dim3 grid((unsigned)((M + tc::kTileM - 1) / tc::kTileM), (unsigned)splits);
+    cudaError_t e;
+    if (dt == SAGE_BF16) {
+        e = cudaFuncSetAttribute(tc::k_tc_gemm_nt<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        tc::k_tc_gemm_nt<1><<<grid, tc::kThreads, smem, st>>>(tmA, tmB, M, N, n_pad, fold, K, kps, C, ldc, split_stride, stages,
+                                                              tmem_cols, err);
+    } else {
+        e = cudaFuncSetAttribute(tc::k_tc_gemm_nt<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        tc::k_tc_gemm_nt<2><<<grid, tc::kThreads, smem, st>>>(tmA, tmB, M, N, n_pad, fold, K, kps, C, ldc, split_stride, stages,
+                                                              tmem_cols, err);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace sage
