@@ -44,6 +44,19 @@ cudaError_t launch_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const fl
 cudaError_t launch_tc_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const void* Bm, int64_t ldb, int M, int N, int fold,
                               int64_t K, int splits, float* C, int64_t ldc, int64_t split_stride, int* err, cudaStream_t st);
 
+// fp32-faithful tensor-core C[z] = A_z * Bm_z^T for fp32 operands (three tf32 MMAs on hi/lo halves split in shared
+// memory, accumulator drained into registers every few K tiles). Same alignment rules and return convention as
+// launch_tc_gemm_nt; any N. When A == Bm (a Gram matrix) the diagonal tiles load one operand only.
+cudaError_t launch_tc_gemm_nt_x3(const float* A, int64_t lda, const float* Bm, int64_t ldb, int M, int N, int64_t K, int splits,
+                                 float* C, int64_t ldc, int64_t split_stride, int* err, cudaStream_t st);
+
+// Tensor-core rebuild: Bdst[j][d] = sum_{i<r} W[j][i] * Bsrc[i][d] for j < keep, d < pitch (fp32-faithful, see
+// tc_rebuild.cu). Wsplit holds W already split for tf32: rows [0, j_pad) = W rounded to 11 significant bits, rows
+// [j_pad, 2 j_pad) = the remainder; row pitch ldw floats, columns i >= r and rows j >= keep zero. Needs j_pad a
+// multiple of 16 with keep <= j_pad <= 128 and r <= 256; returns cudaErrorNotSupported otherwise.
+cudaError_t launch_tc_rebuild(const float* Wsplit, int ldw, int j_pad, const float* Bsrc, float* Bdst, int64_t pitch, int64_t D, int r,
+                              int keep, int* err, cudaStream_t st);
+
 // hi[i][0:cols] = bf16(src[i][0:cols]) (round to nearest even) for i < rows; when lo != nullptr also
 // lo[i][:] = bf16(src - float(hi)), so that hi + lo carries 16 significant bits of src.
 cudaError_t launch_to_bf16(const float* src, int64_t lds, int rows, int64_t cols, __nv_bfloat16* hi, __nv_bfloat16* lo, int64_t ldd,

@@ -143,16 +143,18 @@ __device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t smem_addr_bytes) 
     d |= static_cast<uint64_t>(2) << 61;                              // 128-byte swizzle
     return d;
 }
-// Operand tile stored with the NON-contraction index contiguous (MN-major), 128-byte swizzle: one TMA
-// box of [k rows][128 bytes] per 128-byte span of that index; k rows are 128 bytes apart, groups of 8 k
-// rows 1024 bytes apart (stride offset), consecutive 128-byte spans `span_bytes` apart (leading offset).
-__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t smem_addr_bytes, uint32_t span_bytes) {
+// fp32 (tf32) operand tile stored with the NON-contraction index contiguous (MN-major). The tensor cores
+// accept such 32-bit operands only in the "128-byte swizzle with 32-byte atoms" layout: one TMA box of
+// [k rows][128 bytes] per 128-byte span of the contiguous index, k rows 128 bytes apart, the four 32-byte pieces of
+// a row permuted by (row mod 4), so the pattern repeats every 4 k rows = 512 bytes (stride offset); consecutive
+// 128-byte spans are `span_bytes` apart (leading offset). One MMA (8 k rows) covers two such groups.
+__device__ __forceinline__ uint64_t smem_desc_mn_sw128_atom32(uint32_t smem_addr_bytes, uint32_t span_bytes) {
     uint64_t d = 0;
     d |= static_cast<uint64_t>((smem_addr_bytes & 0x3ffffu) >> 4);
     d |= static_cast<uint64_t>((span_bytes >> 4) & 0x3fffu) << 16;
-    d |= static_cast<uint64_t>(1024 >> 4) << 32;
+    d |= static_cast<uint64_t>(512 >> 4) << 32;
     d |= static_cast<uint64_t>(1) << 46;
-    d |= static_cast<uint64_t>(2) << 61;
+    d |= static_cast<uint64_t>(1) << 61;                              // 128-byte swizzle, 32-byte atoms
     return d;
 }
 // Instruction descriptor: fp32 accumulate, A and B of one format (1 = bf16, 2 = tf32), M x N tile.
@@ -165,10 +167,11 @@ __host__ __device__ inline uint32_t instr_desc(int fmt, int M, int N, int a_mn, 
 
 // ---- host: tensor maps ---------------------------------------------------------------------------
 // 2-D row-major tensor (rows x cols elements, row pitch ld elements) -> tile loads of box_rows x 128 bytes
-// with the 128-byte swizzle. elem_bytes 2 (bf16) or 4 (fp32). Returns false when TMA's alignment rules do
-// not hold (base 16-byte aligned, pitch a multiple of 16 bytes) or the driver refuses.
+// with the 128-byte swizzle (atom32 != 0: its 32-byte-atom variant, for MN-major fp32 operands). elem_bytes 2
+// (bf16) or 4 (fp32). Returns false when TMA's alignment rules do not hold (base 16-byte aligned, pitch a
+// multiple of 16 bytes) or the driver refuses.
 bool make_tmap_2d(CUtensorMap* out, const void* base, int elem_bytes, uint64_t rows, uint64_t cols, uint64_t ld,
-                  uint32_t box_rows);
+                  uint32_t box_rows, int atom32 = 0);
 
 }  // namespace tc
 }  // namespace sage

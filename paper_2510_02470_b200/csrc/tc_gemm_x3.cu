@@ -1,0 +1,233 @@
+// fp32-faithful tensor-core contraction C[z] = A_z * B_z^T for fp32 operands (both contiguous along the
+// contraction index): the Gram matrix K = B B^T of the sketch buffer (Method, first paragraph: the SVD of
+// the buffer is taken through the eigen-decomposition of B B^T) and the pass-2 projection of fp32 rows.
+//
+// Two things keep fp32 fidelity on tensor cores:
+//   * tcgen05 kind::tf32 keeps 11 significant bits of each operand, so every fp32 value x is split in
+//     shared memory into hi = x rounded to 11 bits and lo = x - hi (exact), and three MMAs accumulate
+//     hi*hi + hi*lo + lo*hi; the dropped lo*lo term is below 2^-22 relative;
+//   * the TMEM accumulator rounds toward zero at every accumulation, which biases long sums of like-signed
+//     terms (measured about 0.45 * 2^-24 per MMA step), so the accumulator is drained every kChunk K
+//     tiles into fp32 registers with round-to-nearest additions and restarted from zero.
+//
+// One CTA owns a 128 x (<=128) output tile and one K slice:
+//   warp 0    TMA producer (raw fp32 tiles, 128-byte swizzle),
+//   warp 1    TMEM allocation and MMA issue into two ping-pong accumulators,
+//   warps 2-5 split each landed stage into hi (in place) and lo (second buffer),
+//   warps 6-9 drain finished accumulators into registers and store the tile at the end.
+// On the diagonal tiles of a Gram matrix only one operand tile is loaded and used on both sides.
+#include "sage_internal.h"
+#include "tc05.cuh"
+
+namespace sage {
+namespace tc {
+namespace {
+
+constexpr int kThreads = 320;
+constexpr int kSplitThreads = 128;
+constexpr int kDrainThreads = 128;
+constexpr int kTileM = 128;
+constexpr int kTileN = 128;
+constexpr int kTileBytes = 128 * 128;       // 128 rows of 128 bytes
+constexpr int BK = 32;                      // fp32 elements per 128-byte K tile
+constexpr int kChunk = 4;                   // K tiles accumulated in TMEM between drains
+
+__global__ void __launch_bounds__(kThreads, 1)
+k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, int M, int N, int gram,
+                int b_box_rows, long long K, long long k_per_split, float* __restrict__ C, long long ldc, long long split_stride,
+                int stages, int stage_bytes, int* __restrict__ err) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    const int m0 = blockIdx.x * kTileM, n0 = blockIdx.y * kTileN;
+    const bool diag = gram && m0 == n0;                   // A tile == B tile: load once
+    // stage layout: [hi: A | B][lo: A | B]; on diagonal tiles there is no separate B
+    const int half_bytes = diag ? kTileBytes : kTileBytes + b_box_rows * 128;
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)stages * stage_bytes);
+    uint64_t* split_done = full + stages;
+    uint64_t* empty = split_done + stages;
+    uint64_t* acc_full = empty + stages;                   // [2]
+    uint64_t* acc_empty = acc_full + 2;                    // [2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    volatile int* abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long k_begin = (long long)blockIdx.z * k_per_split;
+    const long long k_end = K < k_begin + k_per_split ? K : k_begin + k_per_split;
+    const int nkt = k_end > k_begin ? (int)((k_end - k_begin + BK - 1) / BK) : 0;
+    const int nchunks = (nkt + kChunk - 1) / kChunk;
+    int n_pad = N - n0 < kTileN ? N - n0 : kTileN;        // MMA width of this tile, a multiple of 16
+    n_pad = ((n_pad + 15) / 16) * 16;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&split_done[s], kSplitThreads);
+            mbar_init(&empty[s], 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&acc_full[b], 1);
+            mbar_init(&acc_empty[b], kDrainThreads);
+        }
+        *abort = 0;
+        mbar_fence_init();
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmB);
+    }
+    if (warp == 1) tmem_alloc(tmem_slot, 2 * kTileN);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int issued = 0;
+            for (int kt = 0; kt < nkt; ++kt) {
+                const int s = kt % stages;
+                const uint32_t use = (uint32_t)(kt / stages);
+                if (!mbar_wait(&empty[s], (use & 1u) ^ 1u, abort)) break;
+                mbar_expect_tx(&full[s], (uint32_t)half_bytes);
+                const int x = (int)(k_begin + (long long)kt * BK);
+                uint8_t* st = smem + (size_t)s * stage_bytes;
+                tma_load_2d(st, &tmA, &full[s], x, m0);
+                if (!diag) tma_load_2d(st + kTileBytes, &tmB, &full[s], x, n0);
+                issued = kt + 1;
+            }
+            if (*abort) {
+                for (int kt = issued > stages ? issued - stages : 0; kt < issued; ++kt)
+                    mbar_wait_quiet(&full[kt % stages], (uint32_t)(kt / stages) & 1u, 20000000ll);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc(2, kTileM, n_pad, 0, 0);
+            bool alive = true;
+            for (int kt = 0; kt < nkt && alive; ++kt) {
+                const int s = kt % stages;
+                const uint32_t use = (uint32_t)(kt / stages);
+                const int c = kt / kChunk, b = c & 1, in_chunk = kt - c * kChunk;
+                if (in_chunk == 0) alive = mbar_wait(&acc_empty[b], (((uint32_t)c >> 1) & 1u) ^ 1u, abort);
+                if (alive) alive = mbar_wait(&split_done[s], use & 1u, abort);
+                if (!alive) break;
+                tc_fence_after();
+                const uint32_t st = smem_u32(smem + (size_t)s * stage_bytes);
+                const uint32_t a_hi = st, a_lo = st + half_bytes;
+                const uint32_t b_hi = diag ? a_hi : st + kTileBytes, b_lo = b_hi + half_bytes;
+                const uint64_t d_ahi = smem_desc_k_sw128(a_hi), d_alo = smem_desc_k_sw128(a_lo);
+                const uint64_t d_bhi = smem_desc_k_sw128(b_hi), d_blo = smem_desc_k_sw128(b_lo);
+                const uint32_t acc = tmem_base + (uint32_t)(b * kTileN);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {          // 4 x 8 tf32 elements per 128-byte row
+                    mma_tf32(acc, d_ahi + 2 * k, d_bhi + 2 * k, idesc, (in_chunk | k) != 0);
+                    mma_tf32(acc, d_ahi + 2 * k, d_blo + 2 * k, idesc, 1);
+                    mma_tf32(acc, d_alo + 2 * k, d_bhi + 2 * k, idesc, 1);
+                }
+                mma_commit(&empty[s]);
+                if (in_chunk == kChunk - 1 || kt == nkt - 1) mma_commit(&acc_full[b]);
+            }
+        }
+    } else if (warp < 6) {
+        // ---- split landed stages into hi (in place) and lo ----
+        const int t = threadIdx.x - 64;                 // 0..127
+        const int chunks16 = half_bytes / 16;
+        for (int kt = 0; kt < nkt; ++kt) {
+            const int s = kt % stages;
+            const uint32_t use = (uint32_t)(kt / stages);
+            if (!mbar_wait(&full[s], use & 1u, abort)) break;
+            uint4* hi = reinterpret_cast<uint4*>(smem + (size_t)s * stage_bytes);
+            uint4* lo = reinterpret_cast<uint4*>(smem + (size_t)s * stage_bytes + half_bytes);
+            for (int c = t; c < chunks16; c += kSplitThreads) {
+                const uint4 v = hi[c];
+                uint4 h, l;
+                h.x = (v.x + 0x1000u) & 0xffffe000u; l.x = __float_as_uint(__uint_as_float(v.x) - __uint_as_float(h.x));
+                h.y = (v.y + 0x1000u) & 0xffffe000u; l.y = __float_as_uint(__uint_as_float(v.y) - __uint_as_float(h.y));
+                h.z = (v.z + 0x1000u) & 0xffffe000u; l.z = __float_as_uint(__uint_as_float(v.z) - __uint_as_float(h.z));
+                h.w = (v.w + 0x1000u) & 0xffffe000u; l.w = __float_as_uint(__uint_as_float(v.w) - __uint_as_float(h.w));
+                hi[c] = h;
+                lo[c] = l;
+            }
+            fence_proxy_async_smem();                   // the tensor cores read these writes
+            mbar_arrive(&split_done[s]);
+        }
+    } else {
+        // ---- drain accumulators into registers; store the tile ----
+        const int quarter = warp & 3;
+        const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+        float acc[kTileN];
+#pragma unroll
+        for (int j = 0; j < kTileN; ++j) acc[j] = 0.f;
+        bool ok = true;
+        for (int c = 0; c < nchunks; ++c) {
+            const int b = c & 1;
+            ok = mbar_wait(&acc_full[b], ((uint32_t)c >> 1) & 1u, abort);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll
+            for (int c0 = 0; c0 < kTileN; c0 += 16) {
+                if (c0 < n_pad) {
+                    float v[16];
+                    tmem_ld16(lane_base + (uint32_t)(b * kTileN + c0), v);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) acc[c0 + j] += v[j];
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(&acc_empty[b]);
+        }
+        const int row = m0 + quarter * 32 + lane;
+        if (row < M) {
+            float* crow = C + (long long)blockIdx.z * split_stride + (long long)row * ldc + n0;
+            const bool vec = (ldc % 4 == 0) && ((reinterpret_cast<uintptr_t>(C) & 15u) == 0) && (split_stride % 4 == 0);
+#pragma unroll
+            for (int c0 = 0; c0 < kTileN; c0 += 4) {
+                if (n0 + c0 + 4 <= N && vec) {
+                    *reinterpret_cast<float4*>(crow + c0) = make_float4(acc[c0], acc[c0 + 1], acc[c0 + 2], acc[c0 + 3]);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        if (n0 + c0 + j < N) crow[c0 + j] = acc[c0 + j];
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        // no MMA may be in flight when TMEM is freed: the last chunk's commit covers every MMA issued
+        if (nchunks > 0 && !*abort) mbar_wait_quiet(&acc_full[(nchunks - 1) & 1], ((uint32_t)(nchunks - 1) >> 1) & 1u, kWaitLimitCycles);
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 2 * kTileN);
+    }
+    if (threadIdx.x == 0 && *abort) atomicExch(err, 1);
+}
+
+}  // namespace
+}  // namespace tc
+
+cudaError_t launch_tc_gemm_nt_x3(const float* A, int64_t lda, const float* Bm, int64_t ldb, int M, int N, int64_t K, int splits,
+                                 float* C, int64_t ldc, int64_t split_stride, int* err, cudaStream_t st) {
+    if (M <= 0 || N <= 0 || K <= 0) return cudaSuccess;
+    if (splits < 1 || splits > 65535) return cudaErrorNotSupported;
+    const int gram = (A == Bm && lda == ldb && M == N) ? 1 : 0;
+    CUtensorMap tmA, tmB;
+    if (!tc::make_tmap_2d(&tmA, A, 4, (uint64_t)M, (uint64_t)K, (uint64_t)lda, tc::kTileM)) return cudaErrorNotSupported;
+    const int b_box_rows = N >= tc::kTileN ? tc::kTileN : ((N + 15) / 16) * 16;
+    if (!tc::make_tmap_2d(&tmB, Bm, 4, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, (uint32_t)b_box_rows)) return cudaErrorNotSupported;
+    int64_t kps = (K + splits - 1) / splits;
+    kps = ((kps + tc::BK - 1) / tc::BK) * tc::BK;
+    if (splits > 1 && (int64_t)(splits - 1) * kps >= K) return cudaErrorInvalidValue;
+    // a Gram matrix of at most 128 rows has diagonal tiles only: one operand per stage
+    const int stage_bytes = 2 * ((gram && M <= tc::kTileM) ? tc::kTileBytes : tc::kTileBytes + b_box_rows * 128);
+    int stages = (200 * 1024) / stage_bytes;
+    if (stages > 8) stages = 8;
+    const size_t smem = (size_t)stages * stage_bytes + 1024 + (3 * stages + 4) * 8 + 16;
+    dim3 grid((unsigned)((M + tc::kTileM - 1) / tc::kTileM), (unsigned)((N + tc::kTileN - 1) / tc::kTileN), (unsigned)splits);
+    cudaError_t e = cudaFuncSetAttribute(tc::k_tc_gemm_nt_x3, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    tc::k_tc_gemm_nt_x3<<<grid, tc::kThreads, smem, st>>>(tmA, tmB, M, N, gram, b_box_rows, K, kps, C, ldc, split_stride, stages,
+                                                                 stage_bytes, err);
+    return cudaGetLastError();
+}
+
+}  // namespace sage

@@ -1,0 +1,219 @@
+// Tensor-core rebuild of the sketch buffer (Method, first paragraph: "reconstruct S <- Sigma' V^T").
+// With B B^T = U Lambda U^T, Sigma' V^T = diag(sigma'_j / sigma_j) U^T B, i.e.
+//     out[j][d] = sum_i W[j][i] * B[i][d],   W[j][i] = U[i][j] * sqrt(max(1 - delta/lambda_j, 0)).
+// The buffer is the streamed operand: a CTA walks 128-column tiles of it, and for each tile accumulates over
+// chunks of 32 buffer rows   D[d][j] += B[i][d] * W[j][i]   with d on the 128 TMEM lanes (the buffer tile is the
+// "A" operand, stored with d contiguous = MN-major), so the epilogue writes out[j][d0..d0+127] as full lines.
+//
+// fp32 fidelity as in the Gram kernel: buffer values are split in shared memory into hi (11 significant
+// bits) and lo = x - hi; W arrives already split from global memory as two stacked operands [W_hi; W_lo],
+// so one MMA of width 2*j_pad gives hi*W_hi and hi*W_lo side by side and a second one adds lo*W_hi; the
+// epilogue adds the two halves. A tile accumulates at most 8 chunks (256 buffer rows) in TMEM.
+//
+//   warp 0    TMA producer: per chunk 4 boxes of [32 rows][32 columns] of the buffer (128-byte swizzle with
+//             32-byte atoms, the only layout the tensor cores take for 32-bit MN-major operands) and one box of W,
+//   warp 1    TMEM allocation, MMA issue into two ping-pong accumulators (one per column tile),
+//   warps 2-5 split the buffer part of each landed stage into hi / lo,
+//   warps 6-9 epilogue: TMEM -> registers -> out.
+#include "sage_internal.h"
+#include "tc05.cuh"
+
+namespace sage {
+namespace tc {
+namespace {
+
+constexpr int kThreads = 320;
+constexpr int kSplitThreads = 128;
+constexpr int kEpiThreads = 128;
+constexpr int kTileD = 128;                 // buffer columns per tile (MMA M)
+constexpr int kChunkRows = 32;              // buffer rows per stage (MMA K = 4 x 8)
+constexpr int kBufBytes = kChunkRows * kTileD * 4;   // 16 KB: 4 spans of [32 rows][128 bytes]
+constexpr int kSpanBytes = kChunkRows * 128;         // 4 KB
+
+__global__ void __launch_bounds__(kThreads, 1)
+k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ CUtensorMap tmW, int r, int keep, int j_pad,
+             long long pitch, long long num_tiles, float* __restrict__ out, int stages, int* __restrict__ err) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    // stage layout: [buffer hi 16 KB][buffer lo 16 KB][W_hi ; W_lo: 2*j_pad rows of 128 bytes]
+    const int w_bytes = 2 * j_pad * 128;
+    const int stage_bytes = 2 * kBufBytes + w_bytes;
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)stages * stage_bytes);
+    uint64_t* split_done = full + stages;
+    uint64_t* empty = split_done + stages;
+    uint64_t* acc_full = empty + stages;                   // [2]
+    uint64_t* acc_empty = acc_full + 2;                    // [2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    volatile int* abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nchunk = (r + kChunkRows - 1) / kChunkRows;
+    const int n_mma = 2 * j_pad;                           // <= 256
+    uint32_t tmem_cols = 32;
+    while (tmem_cols < (uint32_t)(2 * n_mma)) tmem_cols <<= 1;
+    // tiles of this CTA: blockIdx.x, blockIdx.x + gridDim.x, ...
+    const long long my_tiles = num_tiles > blockIdx.x ? (num_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&split_done[s], kSplitThreads);
+            mbar_init(&empty[s], 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&acc_full[b], 1);
+            mbar_init(&acc_empty[b], kEpiThreads);
+        }
+        *abort = 0;
+        mbar_fence_init();
+        tma_prefetch_desc(&tmBuf);
+        tma_prefetch_desc(&tmW);
+    }
+    if (warp == 1) tmem_alloc(tmem_slot, tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            long long q = 0, issued = 0;
+            bool alive = true;
+            for (long long lt = 0; lt < my_tiles && alive; ++lt) {
+                const long long d0 = (blockIdx.x + lt * gridDim.x) * kTileD;
+                for (int c = 0; c < nchunk; ++c, ++q) {
+                    const int s = (int)(q % stages);
+                    const uint32_t use = (uint32_t)(q / stages);
+                    if (!mbar_wait(&empty[s], (use & 1u) ^ 1u, abort)) { alive = false; break; }
+                    mbar_expect_tx(&full[s], (uint32_t)(kBufBytes + w_bytes));
+                    uint8_t* st = smem + (size_t)s * stage_bytes;
+#pragma unroll
+                    for (int sp = 0; sp < 4; ++sp) tma_load_2d(st + sp * kSpanBytes, &tmBuf, &full[s], (int)(d0 + 32 * sp), c * kChunkRows);
+                    tma_load_2d(st + 2 * kBufBytes, &tmW, &full[s], c * kChunkRows, 0);
+                    issued = q + 1;
+                }
+            }
+            if (*abort) {
+                for (long long k = issued > stages ? issued - stages : 0; k < issued; ++k)
+                    mbar_wait_quiet(&full[k % stages], (uint32_t)(k / stages) & 1u, 20000000ll);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc_fold = instr_desc(2, kTileD, n_mma, 1, 0);   // A (buffer) MN-major, B (W) K-major
+            const uint32_t idesc_half = instr_desc(2, kTileD, j_pad, 1, 0);
+            long long q = 0;
+            bool alive = true;
+            for (long long lt = 0; lt < my_tiles && alive; ++lt) {
+                const int b = (int)(lt & 1);
+                alive = mbar_wait(&acc_empty[b], (((uint32_t)(lt >> 1)) & 1u) ^ 1u, abort);
+                if (!alive) break;
+                const uint32_t acc = tmem_base + (uint32_t)(b * n_mma);
+                for (int c = 0; c < nchunk; ++c, ++q) {
+                    const int s = (int)(q % stages);
+                    const uint32_t use = (uint32_t)(q / stages);
+                    if (!mbar_wait(&split_done[s], use & 1u, abort)) { alive = false; break; }
+                    tc_fence_after();
+                    const uint32_t st = smem_u32(smem + (size_t)s * stage_bytes);
+                    const uint32_t w_addr = st + 2 * kBufBytes;
+                    const uint64_t d_w = smem_desc_k_sw128(w_addr);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {          // 8 buffer rows per MMA: one 1024-byte row group
+                        const uint64_t d_hi = smem_desc_mn_sw128_atom32(st + k * 1024, kSpanBytes);
+                        const uint64_t d_lo = smem_desc_mn_sw128_atom32(st + kBufBytes + k * 1024, kSpanBytes);
+                        mma_tf32(acc, d_hi, d_w + 2 * k, idesc_fold, (c | k) != 0);   // hi*W_hi | hi*W_lo
+                        mma_tf32(acc, d_lo, d_w + 2 * k, idesc_half, 1);              // + lo*W_hi
+                    }
+                    mma_commit(&empty[s]);
+                }
+                if (alive) mma_commit(&acc_full[b]);
+            }
+        }
+    } else if (warp < 6) {
+        const int t = threadIdx.x - 64;
+        const long long total = my_tiles * nchunk;
+        for (long long q = 0; q < total; ++q) {
+            const int s = (int)(q % stages);
+            const uint32_t use = (uint32_t)(q / stages);
+            if (!mbar_wait(&full[s], use & 1u, abort)) break;
+            uint4* hi = reinterpret_cast<uint4*>(smem + (size_t)s * stage_bytes);
+            uint4* lo = reinterpret_cast<uint4*>(smem + (size_t)s * stage_bytes + kBufBytes);
+#pragma unroll
+            for (int c = 0; c < kBufBytes / 16 / kSplitThreads; ++c) {
+                const int idx = t + c * kSplitThreads;
+                const uint4 v = hi[idx];
+                uint4 h, l;
+                h.x = (v.x + 0x1000u) & 0xffffe000u; l.x = __float_as_uint(__uint_as_float(v.x) - __uint_as_float(h.x));
+                h.y = (v.y + 0x1000u) & 0xffffe000u; l.y = __float_as_uint(__uint_as_float(v.y) - __uint_as_float(h.y));
+                h.z = (v.z + 0x1000u) & 0xffffe000u; l.z = __float_as_uint(__uint_as_float(v.z) - __uint_as_float(h.z));
+                h.w = (v.w + 0x1000u) & 0xffffe000u; l.w = __float_as_uint(__uint_as_float(v.w) - __uint_as_float(h.w));
+                hi[idx] = h;
+                lo[idx] = l;
+            }
+            fence_proxy_async_smem();
+            mbar_arrive(&split_done[s]);
+        }
+    } else {
+        const int quarter = warp & 3;
+        const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+        for (long long lt = 0; lt < my_tiles; ++lt) {
+            const int b = (int)(lt & 1);
+            bool ok = mbar_wait(&acc_full[b], ((uint32_t)(lt >> 1)) & 1u, abort);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const long long d = (blockIdx.x + lt * gridDim.x) * kTileD + quarter * 32 + lane;
+            const uint32_t acc = lane_base + (uint32_t)(b * n_mma);
+            for (int j0 = 0; j0 < j_pad; j0 += 16) {
+                float v[16], w[16];
+                tmem_ld16(acc + (uint32_t)j0, v);
+                tmem_ld16(acc + (uint32_t)(j_pad + j0), w);
+                if (d < pitch) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        if (j0 + j < keep) out[(long long)(j0 + j) * pitch + d] = v[j] + w[j];
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(&acc_empty[b]);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        if (my_tiles > 0 && !*abort) mbar_wait_quiet(&acc_full[(my_tiles - 1) & 1], ((uint32_t)((my_tiles - 1) >> 1)) & 1u, kWaitLimitCycles);
+        tc_fence_after();
+        tmem_dealloc(tmem_base, tmem_cols);
+    }
+    if (threadIdx.x == 0 && *abort) atomicExch(err, 1);
+}
+
+}  // namespace
+}  // namespace tc
+
+// See sage_internal.h.
+cudaError_t launch_tc_rebuild(const float* Wsplit, int ldw, int j_pad, const float* Bsrc, float* Bdst, int64_t pitch, int64_t D, int r,
+                              int keep, int* err, cudaStream_t st) {
+    if (keep <= 0 || r <= 0) return cudaSuccess;
+    if (j_pad < 16 || j_pad > 128 || (j_pad & 15) || keep > j_pad || r > 256) return cudaErrorNotSupported;
+    CUtensorMap tmBuf, tmW;
+    // buffer: columns beyond D up to the pitch are zero and are rebuilt as zero, so the map spans the pitch
+    if (!tc::make_tmap_2d(&tmBuf, Bsrc, 4, (uint64_t)r, (uint64_t)pitch, (uint64_t)pitch, tc::kChunkRows, 1)) return cudaErrorNotSupported;
+    const int kcols = ((r + tc::kChunkRows - 1) / tc::kChunkRows) * tc::kChunkRows;
+    if (kcols > ldw) return cudaErrorNotSupported;
+    if (!tc::make_tmap_2d(&tmW, Wsplit, 4, (uint64_t)(2 * j_pad), (uint64_t)kcols, (uint64_t)ldw, (uint32_t)(2 * j_pad)))
+        return cudaErrorNotSupported;
+    (void)D;
+    const int stage_bytes = 2 * tc::kBufBytes + 2 * j_pad * 128;
+    int stages = (200 * 1024) / stage_bytes;
+    if (stages > 8) stages = 8;
+    const size_t smem = (size_t)stages * stage_bytes + 1024 + (3 * stages + 4) * 8 + 16;
+    const long long num_tiles = (pitch + tc::kTileD - 1) / tc::kTileD;
+    const int grid = (int)(num_tiles < 148 ? num_tiles : 148);
+    cudaError_t e = cudaFuncSetAttribute(tc::k_tc_rebuild, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    tc::k_tc_rebuild<<<grid, tc::kThreads, smem, st>>>(tmBuf, tmW, r, keep, j_pad, pitch, num_tiles, Bdst, stages, err);
+    return cudaGetLastError();
+}
+
+}  // namespace sage
