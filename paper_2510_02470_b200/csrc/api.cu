@@ -89,7 +89,8 @@ struct sage_fd {
     State state = SKETCHING;
     int delta_rank = 0, max_sweeps = 30;
     // Gram / eigen workspaces
-    float* gram_parts = nullptr;   // 296 tiles of 64 x 64 floats
+    float* gram_parts = nullptr;   // split-K partials of the Gram matrix (kGramPartFloats floats)
+    float* Wsplit = nullptr;       // rebuild factors split for the tensor cores: 256 rows x kWsplitLd floats
     float* Kmat = nullptr;         // m x m
     float* Ur = nullptr;           // m x m
     float* eig_work = nullptr;     // m x m
@@ -140,6 +141,9 @@ cudaError_t timed(sage_fd* h, int cls, int nlaunch, cudaStream_t st, F&& f) {
     return e;
 }
 
+constexpr size_t kGramPartFloats = (size_t)148 * 128 * 128;   // >= 296 tiles of 64 x 64
+constexpr int kWsplitLd = 256;
+
 int gram_tiles(int r) {
     const int t = (r + 63) / 64;
     return t * t;
@@ -181,12 +185,36 @@ sage_status_t enqueue_freeze_aux(sage_fd* h, cudaStream_t st) {
 
 // Gram of the first r buffer rows -> Kmat (r x r, pitch m).
 sage_status_t enqueue_gram(sage_fd* h, int r, cudaStream_t st) {
+    float* Bc = h->B[h->cur];
+    if (h->use_tc) {
+        // tensor cores: 128 x 128 output tiles, as many K slices as fill the SMs (each at least 1024 columns)
+        const int t = (r + 127) / 128;
+        const int ldc = ((r + 3) / 4) * 4;
+        const int64_t stride = (int64_t)r * ldc;
+        int cap = (int)(kGramPartFloats / (size_t)stride);
+        if (cap > 148) cap = 148;
+        const int splits = pick_splits_waves(t * t, h->D, 1024, cap);
+        cudaError_t e;
+        if (splits == 1) {
+            e = timed(h, K_GRAM, 1, st, [&] { return launch_tc_gemm_nt_x3(Bc, h->pitch, Bc, h->pitch, r, r, h->D, 1, h->Kmat, h->m, 0, h->tc_err, st); });
+        } else {
+            e = timed(h, K_GRAM, 1, st, [&] {
+                return launch_tc_gemm_nt_x3(Bc, h->pitch, Bc, h->pitch, r, r, h->D, splits, h->gram_parts, ldc, stride, h->tc_err, st);
+            });
+        }
+        if (e == cudaSuccess) {
+            if (splits > 1)
+                CU_TRY(timed(h, K_GRAM_REDUCE, 1, st, [&] { return launch_split_reduce(h->gram_parts, splits, stride, r, r, ldc, h->Kmat, h->m, st); }));
+            return SAGE_OK;
+        }
+        if (e != cudaErrorNotSupported) CU_TRY(e);
+        count(h, -1);
+    }
     // splits * tiles <= 296, and the partials are stored compactly (pitch r_pad), so they always fit in
     // the 296 tiles of 64 x 64 floats allocated at create.
     const int splits = pick_splits(gram_tiles(r), h->D, 256);
     const int r_pad = ((r + 63) / 64) * 64;
     const int64_t stride = (int64_t)r_pad * r_pad;
-    float* Bc = h->B[h->cur];
     if (splits == 1) {
         CU_TRY(timed(h, K_GRAM, 1, st, [&] { return launch_gemm_nt(Bc, SAGE_F32, h->pitch, Bc, h->pitch, r, r, h->D, 1, h->Kmat, h->m, 0, st); }));
     } else {
@@ -201,14 +229,32 @@ sage_status_t enqueue_gram(sage_fd* h, int r, cudaStream_t st) {
 // Factor the first r rows and rebuild `keep` rows into the other buffer; rows keep..zero_to-1 are zeroed.
 sage_status_t enqueue_factor(sage_fd* h, int r, int do_shrink, int keep, int zero_to, cudaStream_t st) {
     ST_TRY(enqueue_gram(h, r, st));
+    const int j_pad = ((keep + 15) / 16) * 16;
+    const bool tc_rebuild = h->use_tc && h->Wsplit && keep > 0 && j_pad <= 128 && r <= 256;
     CU_TRY(timed(h, K_EIG, 1, st, [&] {
         return launch_eig_shrink(h->Kmat, h->m, r, do_shrink, h->delta_rank, keep, h->Ur, h->m, h->sigma, h->ell, h->eig_work,
-                                 h->max_sweeps, h->info, st);
+                                 h->max_sweeps, h->info, tc_rebuild ? h->Wsplit : nullptr, kWsplitLd, j_pad, st);
     }));
     const int m_total = zero_to > keep ? zero_to : keep;
-    CU_TRY(timed(h, K_REBUILD, 1, st, [&] {
-        return launch_rebuild(h->Ur, h->m, h->B[h->cur], h->B[1 - h->cur], h->pitch, h->D, r, keep, m_total, st);
-    }));
+    bool done = false;
+    if (tc_rebuild) {
+        cudaError_t e = timed(h, K_REBUILD, 1, st, [&] {
+            return launch_tc_rebuild(h->Wsplit, kWsplitLd, j_pad, h->B[h->cur], h->B[1 - h->cur], h->pitch, h->D, r, keep, h->tc_err, st);
+        });
+        if (e == cudaSuccess) {
+            done = true;
+            if (m_total > keep)
+                CU_TRY(cudaMemsetAsync(h->B[1 - h->cur] + (size_t)keep * h->pitch, 0, (size_t)(m_total - keep) * h->pitch * sizeof(float), st));
+        } else if (e != cudaErrorNotSupported) {
+            CU_TRY(e);
+        } else {
+            count(h, -1);
+        }
+    }
+    if (!done)
+        CU_TRY(timed(h, K_REBUILD, 1, st, [&] {
+            return launch_rebuild(h->Ur, h->m, h->B[h->cur], h->B[1 - h->cur], h->pitch, h->D, r, keep, m_total, st);
+        }));
     h->cur = 1 - h->cur;
     h->fill = keep;
     return SAGE_OK;
@@ -300,7 +346,9 @@ sage_status_t sage_fd_create(sage_fd_t** out, int64_t D, int32_t ell, sage_dtype
     cudaError_t e;
     for (int i = 0; i < 2; ++i)
         if ((e = cudaMalloc((void**)&h->B[i], bbytes)) != cudaSuccess) return fail(e, "cudaMalloc(buffer)");
-    if ((e = cudaMalloc((void**)&h->gram_parts, (size_t)296 * 64 * 64 * sizeof(float))) != cudaSuccess) return fail(e, "cudaMalloc(gram)");
+    if ((e = cudaMalloc((void**)&h->gram_parts, kGramPartFloats * sizeof(float))) != cudaSuccess) return fail(e, "cudaMalloc(gram)");
+    if (ell <= 128 && (e = cudaMalloc((void**)&h->Wsplit, (size_t)256 * kWsplitLd * sizeof(float))) != cudaSuccess)
+        return fail(e, "cudaMalloc(W)");
     if ((e = cudaMalloc((void**)&h->Kmat, mm)) != cudaSuccess) return fail(e, "cudaMalloc(K)");
     if ((e = cudaMalloc((void**)&h->Ur, mm)) != cudaSuccess) return fail(e, "cudaMalloc(U)");
     if ((e = cudaMalloc((void**)&h->eig_work, mm)) != cudaSuccess) return fail(e, "cudaMalloc(eig)");
@@ -333,6 +381,7 @@ void sage_fd_destroy(sage_fd_t* h) {
     cudaFree(h->B[0]);
     cudaFree(h->B[1]);
     cudaFree(h->gram_parts);
+    cudaFree(h->Wsplit);
     cudaFree(h->Kmat);
     cudaFree(h->Ur);
     cudaFree(h->eig_work);
@@ -544,9 +593,12 @@ sage_status_t sage_score_chunk(sage_fd_t* h, const void* rows, int64_t n, int64_
     const size_t row_bytes = (size_t)ld * elem_size(h->dtype);
     const float* S = h->B[h->cur];
     // Tensor-core path: bf16 rows against the bf16 copy of the sketch (a one-term bf16 sketch is only used for
-    // long rows, where its rounding errors average out). fp32 rows keep the CUDA-core kernel.
+    // long rows, where its rounding errors average out). 
     const bool tc_ok = h->use_tc && h->dtype == SAGE_BF16 && h->P16 && (h->p16_fold || h->D >= 16384) &&
                        (reinterpret_cast<uintptr_t>(rows) & 15u) == 0 && (row_bytes & 15u) == 0;
+    // fp32 rows: the fp32-faithful three-MMA kernel against the fp32 sketch itself (one 128-wide tile of S)
+    const bool tc32_ok = h->use_tc && h->dtype == SAGE_F32 && ell <= 128 && (reinterpret_cast<uintptr_t>(rows) & 15u) == 0 &&
+                         (row_bytes & 15u) == 0;
     for (int64_t r0 = 0; r0 < n; r0 += sub_max) {
         const int64_t sub = (n - r0 < sub_max) ? n - r0 : sub_max;
         const size_t nb = (size_t)((sub + 63) / 64);
@@ -554,6 +606,26 @@ sage_status_t sage_score_chunk(sage_fd_t* h, const void* rows, int64_t n, int64_
         const size_t zred = (size_t)sub * ell * sizeof(float);
         bool done = false;
         float* Z = nullptr;
+        if (tc32_ok) {
+            const int splits = pick_splits_waves((int)((sub + 127) / 128), h->D, 2048, 64);
+            ST_TRY(ensure(&h->zwork, &h->zwork_bytes, zred * (splits > 1 ? splits + 1 : 1)));
+            Z = h->zwork;
+            float* out = splits > 1 ? h->zwork + (size_t)sub * ell : Z;
+            cudaError_t e = timed(h, K_PROJECT, 1, st, [&] {
+                return launch_tc_gemm_nt_x3(reinterpret_cast<const float*>(p + r0 * row_bytes), ld, S, h->pitch, (int)sub, ell, h->D,
+                                            splits, out, ell, (int64_t)sub * ell, h->tc_err, st);
+            });
+            if (e == cudaSuccess) {
+                done = true;
+                if (splits > 1)
+                    CU_TRY(timed(h, K_PROJECT_REDUCE, 1, st,
+                                 [&] { return launch_split_reduce(out, splits, (int64_t)sub * ell, (int)sub, ell, ell, Z, ell, st); }));
+            } else if (e != cudaErrorNotSupported) {
+                CU_TRY(e);
+            } else {
+                count(h, -1);
+            }
+        }
         if (tc_ok) {
             const int splits = pick_splits_waves((int)((sub + 127) / 128), h->D, 4096, 64);
             ST_TRY(ensure(&h->zwork, &h->zwork_bytes, zred * (splits > 1 ? splits + 1 : 1)));

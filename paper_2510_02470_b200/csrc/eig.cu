@@ -66,7 +66,8 @@ constexpr int kMaxFast = 192;
 template <int T>
 __global__ void __launch_bounds__(kThreads, 1)
 k_eig_shrink_fast(const float* __restrict__ K, int ldk, int n, int do_shrink, int delta_rank, int keep, float* __restrict__ Ur,
-                  int ldu, float* __restrict__ sigma_out, int n_sigma, int max_sweeps, EigInfo* __restrict__ info) {
+                  int ldu, float* __restrict__ sigma_out, int n_sigma, int max_sweeps, EigInfo* __restrict__ info,
+                  float* __restrict__ Wsplit, int ldw, int j_pad) {
     constexpr int LD = 64 * T;
     constexpr int R = 2 * T;            // rows per lane when 32 lanes span a column
     constexpr int Q = 2 * T;            // float4 per lane when 8 lanes span a column
@@ -329,12 +330,25 @@ k_eig_shrink_fast(const float* __restrict__ K, int ldk, int n, int do_shrink, in
         }
         Ur[(size_t)i * ldu + j] = v;
     }
+    if (Wsplit) {   // the same factors transposed and split for the tensor-core rebuild: [W_hi ; W_lo], zero padded
+        for (int e = tid; e < j_pad * ldw; e += kThreads) {
+            const int j = e / ldw, i = e - j * ldw;
+            float v = 0.f;
+            if (j < keep && j < n && i < n) {
+                const int k = order[j];
+                if (k < rank) v = X[perm[k] * LD + i] * fac[j];
+            }
+            const float hi = __uint_as_float((__float_as_uint(v) + 0x1000u) & 0xffffe000u);
+            Wsplit[(size_t)j * ldw + i] = hi;
+            Wsplit[(size_t)(j_pad + j) * ldw + i] = v - hi;
+        }
+    }
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
 k_eig_shrink(const float* __restrict__ K, int ldk, int n, int do_shrink, int delta_rank, int keep, float* __restrict__ Ur,
              int ldu, float* __restrict__ sigma_out, int n_sigma, float* __restrict__ work, int use_smem, int max_sweeps,
-             EigInfo* __restrict__ info) {
+             EigInfo* __restrict__ info, float* __restrict__ Wsplit, int ldw, int j_pad) {
     extern __shared__ __align__(16) float smem[];
     float* lam = smem;                 // n   eigenvalues (unsorted), later reused
     float* fac = lam + 512;            // n   per sorted position: r_j / sigma_j
@@ -537,12 +551,29 @@ k_eig_shrink(const float* __restrict__ K, int ldk, int n, int do_shrink, int del
         if (j < n) v = X[(size_t)order[j] * ldx + i] * fac[j];
         Ur[(size_t)perm[i] * ldu + j] = v;
     }
+    if (Wsplit) {
+        for (int e = tid; e < j_pad * ldw; e += kThreads) {
+            const int j = e / ldw, c = e - j * ldw;
+            Wsplit[(size_t)j * ldw + c] = 0.f;
+            Wsplit[(size_t)(j_pad + j) * ldw + c] = 0.f;
+        }
+        __syncthreads();
+        for (int e = tid; e < n * keep; e += kThreads) {
+            const int j = e / n, i = e % n;
+            if (j >= n || j >= j_pad) continue;
+            const float v = X[(size_t)order[j] * ldx + i] * fac[j];
+            const float hi = __uint_as_float((__float_as_uint(v) + 0x1000u) & 0xffffe000u);
+            Wsplit[(size_t)j * ldw + perm[i]] = hi;
+            Wsplit[(size_t)(j_pad + j) * ldw + perm[i]] = v - hi;
+        }
+    }
 }
 
 }  // namespace
 
 cudaError_t launch_eig_shrink(const float* K, int ldk, int n, int do_shrink, int delta_rank, int keep, float* Ur, int ldu,
-                              float* sigma_out, int n_sigma, float* work, int max_sweeps, EigInfo* info, cudaStream_t st) {
+                              float* sigma_out, int n_sigma, float* work, int max_sweeps, EigInfo* info, float* Wsplit, int ldw,
+                              int j_pad, cudaStream_t st) {
     if (n <= 0 || n > 512) return cudaErrorInvalidValue;
     if (n <= kMaxFast) {
         const int T = (n + 63) / 64;
@@ -552,7 +583,7 @@ cudaError_t launch_eig_shrink(const float* K, int ldk, int n, int do_shrink, int
     e = cudaFuncSetAttribute(k_eig_shrink_fast<TT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);          \
     if (e != cudaSuccess) return e;                                                                                    \
     k_eig_shrink_fast<TT><<<1, kThreads, bytes, st>>>(K, ldk, n, do_shrink, delta_rank, keep, Ur, ldu, sigma_out, n_sigma, \
-                                                      max_sweeps, info);
+                                                      max_sweeps, info, Wsplit, ldw, j_pad);
         if (T == 1) { SAGE_EIG_FAST(1) } else if (T == 2) { SAGE_EIG_FAST(2) } else { SAGE_EIG_FAST(3) }
 #undef SAGE_EIG_FAST
         return cudaGetLastError();
@@ -570,7 +601,7 @@ cudaError_t launch_eig_shrink(const float* K, int ldk, int n, int do_shrink, int
     cudaError_t e = cudaFuncSetAttribute(k_eig_shrink, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     k_eig_shrink<<<1, kThreads, smem, st>>>(K, ldk, n, do_shrink, delta_rank, keep, Ur, ldu, sigma_out, n_sigma, work, use_smem,
-                                            max_sweeps, info);
+                                            max_sweeps, info, Wsplit, ldw, j_pad);
     return cudaGetLastError();
 }
 

@@ -76,9 +76,12 @@ cudaError_t launch_rebuild(const float* Ur, int ldu, const float* Bsrc, float* B
 // Writes Ur[i*ldu + j] = U[i][j] * sqrt(max(1 - delta/lambda_j, 0)) for j < keep (eigenvalues descending),
 // sigma_out[j] = sqrt(max(lambda_j - delta, 0)) for j < n_sigma, and updates *info.
 // `work` is scratch of at least n*n floats (used when the matrix does not fit in shared memory).
+// Wsplit != nullptr: also writes the factors transposed and split for launch_tc_rebuild, rows [0, j_pad) =
+// W rounded to 11 significant bits and rows [j_pad, 2 j_pad) = the remainders, W[j][i] = Ur[i][j], pitch ldw >= n,
+// zero outside j < keep, i < n.
 cudaError_t launch_eig_shrink(const float* K, int ldk, int n, int do_shrink, int delta_rank, int keep, float* Ur,
                               int ldu, float* sigma_out, int n_sigma, float* work, int max_sweeps, EigInfo* info,
-                              cudaStream_t st);
+                              float* Wsplit, int ldw, int j_pad, cudaStream_t st);
 
 // Z (n x ell, pitch ldz, already reduced over splits) -> zhat rows, ||z|| and per-block partial sums of zhat.
 // zsum (ell doubles) += the partial sums in ascending block order (done by a second, single-block kernel).

@@ -198,7 +198,7 @@ cudaError_t launch_tc_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const
         return cudaErrorNotSupported;
     int64_t kps = (K + splits - 1) / splits;
     kps = ((kps + BK - 1) / BK) * BK;
-    if (splits > 1 && (int64_t)(splits - 1) * kps >= K) return cudaErrorInvalidValue;   // an empty slice: pick fewer splits
+    // a trailing slice may be empty after rounding to whole K tiles: its CTAs store zeros
     const int stages = tc_gemm_pick_stages(n_mma);
     const int stage_bytes = tc::kATileBytes + n_mma * 128;
     const size_t smem = (size_t)stages * stage_bytes + 1024 + (2 * stages + 1) * 8 + 16;

@@ -216,7 +216,7 @@ cudaError_t launch_tc_gemm_nt_x3(const float* A, int64_t lda, const float* Bm, i
     if (!tc::make_tmap_2d(&tmB, Bm, 4, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, (uint32_t)b_box_rows)) return cudaErrorNotSupported;
     int64_t kps = (K + splits - 1) / splits;
     kps = ((kps + tc::BK - 1) / tc::BK) * tc::BK;
-    if (splits > 1 && (int64_t)(splits - 1) * kps >= K) return cudaErrorInvalidValue;
+    // a trailing slice may be empty after rounding to whole K tiles: its CTAs store zeros
     // a Gram matrix of at most 128 rows has diagonal tiles only: one operand per stage
     const int stage_bytes = 2 * ((gram && M <= tc::kTileM) ? tc::kTileBytes : tc::kTileBytes + b_box_rows * 128);
     int stages = (200 * 1024) / stage_bytes;
