@@ -187,13 +187,13 @@ sage_status_t enqueue_freeze_aux(sage_fd* h, cudaStream_t st) {
 sage_status_t enqueue_gram(sage_fd* h, int r, cudaStream_t st) {
     float* Bc = h->B[h->cur];
     if (h->use_tc) {
-        // tensor cores: 128 x 128 output tiles, as many K slices as fill the SMs (each at least 1024 columns)
+        // tensor cores: 128 x 128 output tiles, as many K slices as fill the SMs (each at least 256 columns)
         const int t = (r + 127) / 128;
         const int ldc = ((r + 3) / 4) * 4;
         const int64_t stride = (int64_t)r * ldc;
         int cap = (int)(kGramPartFloats / (size_t)stride);
         if (cap > 148) cap = 148;
-        const int splits = pick_splits_waves(t * t, h->D, 1024, cap);
+        const int splits = pick_splits_waves(t * t, h->D, 256, cap);
         cudaError_t e;
         if (splits == 1) {
             e = timed(h, K_GRAM, 1, st, [&] { return launch_tc_gemm_nt_x3(Bc, h->pitch, Bc, h->pitch, r, r, h->D, 1, h->Kmat, h->m, 0, h->tc_err, st); });
@@ -359,10 +359,10 @@ sage_status_t sage_fd_create(sage_fd_t** out, int64_t D, int32_t ell, sage_dtype
     if ((e = cudaMalloc((void**)&h->tc_err, sizeof(int))) != cudaSuccess) return fail(e, "cudaMalloc(err)");
     if ((e = cudaMemset(h->tc_err, 0, sizeof(int))) != cudaSuccess) return fail(e, "cudaMemset");
     if (row_dtype == SAGE_BF16) {
-        // Two-term bf16 sketch (16 significant bits) wherever the doubled tensor work stays well below the HBM
-        // time of the rows: ell <= 64, or short rows where rounding errors average over few terms.
+        // Two-term bf16 sketch (16 significant bits) for short rows, where the rounding errors of a one-term
+        // sketch would average over too few terms; long rows take the one-term sketch (half the operand traffic).
         h->p16_npad = ((ell + 15) / 16) * 16;
-        h->p16_fold = (2 * h->p16_npad <= 256 && (ell <= 64 || D < 16384)) ? 1 : 0;
+        h->p16_fold = (2 * h->p16_npad <= 256 && D < 16384) ? 1 : 0;
         const size_t prow = h->p16_fold ? 2 * (size_t)h->p16_npad : (size_t)ell;
         if ((e = cudaMalloc((void**)&h->P16, prow * h->pitch * sizeof(__nv_bfloat16))) != cudaSuccess) return fail(e, "cudaMalloc(P16)");
         if ((e = cudaMemset(h->P16, 0, prow * h->pitch * sizeof(__nv_bfloat16))) != cudaSuccess) return fail(e, "cudaMemset");
@@ -627,12 +627,18 @@ sage_status_t sage_score_chunk(sage_fd_t* h, const void* rows, int64_t n, int64_
             }
         }
         if (tc_ok) {
-            const int splits = pick_splits_waves((int)((sub + 127) / 128), h->D, 4096, 64);
+            // row tiles per CTA: as many as TMEM holds (512 columns), fewer when that would leave SMs without work
+            const int n_mma = (h->p16_fold ? 2 : 1) * h->p16_npad;
+            const int tiles = (int)((sub + 127) / 128);
+            int mt = 512 / n_mma >= 4 ? 4 : (512 / n_mma >= 2 ? 2 : 1);
+            if (tiles >= 148) mt = 1;        // a full wave of row tiles needs no K split, hence no partials
+            while (mt > 1 && (int64_t)((tiles + mt - 1) / mt) * (h->D / 4096 > 0 ? h->D / 4096 : 1) < 148) mt >>= 1;
+            const int splits = pick_splits_waves((tiles + mt - 1) / mt, h->D, 4096, 148);
             ST_TRY(ensure(&h->zwork, &h->zwork_bytes, zred * (splits > 1 ? splits + 1 : 1)));
             Z = h->zwork;
             float* out = splits > 1 ? h->zwork + (size_t)sub * ell : Z;
             cudaError_t e = timed(h, K_PROJECT, 1, st, [&] {
-                return launch_tc_gemm_nt(p + r0 * row_bytes, SAGE_BF16, ld, h->P16, h->pitch, (int)sub, ell, h->p16_fold, h->D, splits,
+                return launch_tc_gemm_nt(p + r0 * row_bytes, SAGE_BF16, ld, h->P16, h->pitch, (int)sub, ell, h->p16_fold, mt, h->D, splits,
                                          out, ell, (int64_t)sub * ell, h->tc_err, st);
             });
             if (e == cudaSuccess) {

@@ -41,8 +41,9 @@ cudaError_t launch_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const fl
 // fold != 0: Bm holds two stacked operands, rows [0, N) and rows [n_pad, n_pad + N) with n_pad = N rounded up to
 // 16, and C receives the sum of both products (a two-term representation of a more precise B); needs 2 n_pad <= 256.
 // Without fold N <= 256. *err (device) is set to 1 if a bounded wait inside the kernel ran out.
+// mt (1, 2 or 4) row tiles of 128 share each B tile inside one CTA; needs mt * (fold ? 2 n_pad : n_pad) <= 512.
 cudaError_t launch_tc_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const void* Bm, int64_t ldb, int M, int N, int fold,
-                              int64_t K, int splits, float* C, int64_t ldc, int64_t split_stride, int* err, cudaStream_t st);
+                              int mt, int64_t K, int splits, float* C, int64_t ldc, int64_t split_stride, int* err, cudaStream_t st);
 
 // fp32-faithful tensor-core C[z] = A_z * Bm_z^T for fp32 operands (three tf32 MMAs on hi/lo halves split in shared
 // memory, accumulator drained into registers every few K tiles). Same alignment rules and return convention as

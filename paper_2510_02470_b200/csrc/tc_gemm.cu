@@ -2,10 +2,11 @@
 // contiguous along that index ("K-major"): the pass-2 projection Z = G S^T (Method, "Two-pass scoring":
 // z_i = S g_i) with G streamed from HBM exactly once.
 //
-// One CTA owns a 128-row tile of A, all N rows of B and one K slice:
-//   warp 0   TMA producer: 128-byte-wide K tiles of A (128 rows) and B (N rows) into a ring of stages,
-//   warp 1   allocates TMEM and issues tcgen05.mma (M = 128, N, K = 32 bytes per instruction),
-//   warps 2-5 read the fp32 accumulator out of TMEM (one row per thread) and store the partial result.
+// One CTA owns mt (1, 2 or 4) consecutive 128-row tiles of A, all N rows of B and one K slice; the B tile of
+// a stage is shared by the mt row tiles, so B crosses L2 -> SM once per mt * 128 rows:
+//   warp 0   TMA producer: 128-byte-wide K tiles of A (mt x 128 rows) and B (N rows) into a ring of stages,
+//   warp 1   allocates TMEM and issues tcgen05.mma (M = 128, N, K = 32 bytes per instruction) into mt accumulators,
+//   warps 2-5 read the fp32 accumulators out of TMEM (one row per thread) and store the partial result.
 // Rows and K elements outside the matrices are zero-filled by TMA, so no tail code exists. Split-K
 // partials are summed by a separate kernel in a fixed order.
 #include "sage_internal.h"
@@ -50,13 +51,14 @@ constexpr int kATileBytes = kTileM * 128;
 template <int kFmt>
 __global__ void __launch_bounds__(kThreads, 1)
 k_tc_gemm_nt(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, int M, int N, int n_pad, int fold,
-             long long K, long long k_per_split, float* __restrict__ C, long long ldc, long long split_stride, int stages,
+             int mt, long long K, long long k_per_split, float* __restrict__ C, long long ldc, long long split_stride, int stages,
              uint32_t tmem_cols, int* __restrict__ err) {
     constexpr int BK = kFmt == 1 ? 64 : 32;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     const int n_mma = fold ? 2 * n_pad : n_pad;         // folded: B holds two stacked operands whose products are added
-    const int stage_bytes = kATileBytes + n_mma * 128;
+    const int a_bytes = mt * kATileBytes;
+    const int stage_bytes = a_bytes + n_mma * 128;
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)stages * stage_bytes);
     uint64_t* empty = full + stages;
     uint64_t* tmem_full = empty + stages;
@@ -64,7 +66,7 @@ k_tc_gemm_nt(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     volatile int* abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.x * kTileM;
+    const int m0 = blockIdx.x * kTileM * mt;
     const long long k_begin = (long long)blockIdx.y * k_per_split;
     const long long k_end = K < k_begin + k_per_split ? K : k_begin + k_per_split;
     const int nkt = k_end > k_begin ? (int)((k_end - k_begin + BK - 1) / BK) : 0;
@@ -96,8 +98,9 @@ k_tc_gemm_nt(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 if (!mbar_wait(&empty[s], (use & 1u) ^ 1u, abort)) break;
                 mbar_expect_tx(&full[s], tx_bytes);
                 const int x = (int)(k_begin + (long long)kt * BK);
-                tma_load_2d(smem + (size_t)s * stage_bytes, &tmA, &full[s], x, m0);
-                tma_load_2d(smem + (size_t)s * stage_bytes + kATileBytes, &tmB, &full[s], x, 0);
+                for (int t = 0; t < mt; ++t)     // row tiles past the end of A are zero-filled by TMA
+                    tma_load_2d(smem + (size_t)s * stage_bytes + (size_t)t * kATileBytes, &tmA, &full[s], x, m0 + t * kTileM);
+                tma_load_2d(smem + (size_t)s * stage_bytes + a_bytes, &tmB, &full[s], x, 0);
                 issued = kt + 1;
             }
             if (*abort) {   // give copies already in flight a bounded time to land before the block goes away
@@ -114,12 +117,15 @@ k_tc_gemm_nt(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 if (!mbar_wait(&full[s], use & 1u, abort)) break;
                 tc_fence_after();
                 const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
-                const uint64_t adesc = smem_desc_k_sw128(a_addr);
-                const uint64_t bdesc = smem_desc_k_sw128(a_addr + kATileBytes);
+                const uint64_t bdesc = smem_desc_k_sw128(a_addr + a_bytes);
+                for (int t = 0; t < mt; ++t) {
+                    const uint64_t adesc = smem_desc_k_sw128(a_addr + t * kATileBytes);
+                    const uint32_t acc = tmem_base + (uint32_t)(t * n_mma);
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {          // 4 x 32 bytes of K per 128-byte row
-                    if constexpr (kFmt == 1) mma_bf16(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, (kt | k) != 0);
-                    else mma_tf32(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, (kt | k) != 0);
+                    for (int k = 0; k < 4; ++k) {      // 4 x 32 bytes of K per 128-byte row
+                        if constexpr (kFmt == 1) mma_bf16(acc, adesc + 2 * k, bdesc + 2 * k, idesc, (kt | k) != 0);
+                        else mma_tf32(acc, adesc + 2 * k, bdesc + 2 * k, idesc, (kt | k) != 0);
+                    }
                 }
                 mma_commit(&empty[s]);                 // the stage is free once these MMAs have read it
             }
@@ -131,32 +137,34 @@ k_tc_gemm_nt(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         if (nkt > 0) ok = mbar_wait(tmem_full, 0, abort);
         ok = __all_sync(0xffffffffu, ok);
         tc_fence_after();
-        const int row = m0 + quarter * 32 + lane;
-        float* crow = C + (long long)blockIdx.y * split_stride + (long long)row * ldc;
         const bool vec = (ldc % 4 == 0) && ((reinterpret_cast<uintptr_t>(C) & 15u) == 0) && (split_stride % 4 == 0);
-        const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
-        for (int c0 = 0; c0 < n_pad; c0 += 16) {
-            float v[16];
-            if (nkt > 0 && ok) {
-                tmem_ld16(lane_base + (uint32_t)c0, v);
-                if (fold) {
-                    float w[16];
-                    tmem_ld16(lane_base + (uint32_t)(n_pad + c0), w);
+        for (int t = 0; t < mt; ++t) {
+            const int row = m0 + t * kTileM + quarter * 32 + lane;
+            float* crow = C + (long long)blockIdx.y * split_stride + (long long)row * ldc;
+            const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + (uint32_t)(t * n_mma);
+            for (int c0 = 0; c0 < n_pad; c0 += 16) {
+                float v[16];
+                if (nkt > 0 && ok) {
+                    tmem_ld16(lane_base + (uint32_t)c0, v);
+                    if (fold) {
+                        float w[16];
+                        tmem_ld16(lane_base + (uint32_t)(n_pad + c0), w);
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) v[j] += w[j];
-                }
-            } else {
-#pragma unroll
-                for (int j = 0; j < 16; ++j) v[j] = 0.f;
-            }
-            if (row < M) {
-                if (vec && c0 + 16 <= N) {
-#pragma unroll
-                    for (int j = 0; j < 16; j += 4) *reinterpret_cast<float4*>(crow + c0 + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                        for (int j = 0; j < 16; ++j) v[j] += w[j];
+                    }
                 } else {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j)
-                        if (c0 + j < N) crow[c0 + j] = v[j];
+                    for (int j = 0; j < 16; ++j) v[j] = 0.f;
+                }
+                if (row < M) {
+                    if (vec && c0 + 16 <= N) {
+#pragma unroll
+                        for (int j = 0; j < 16; j += 4) *reinterpret_cast<float4*>(crow + c0 + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (c0 + j < N) crow[c0 + j] = v[j];
+                    }
                 }
             }
         }
@@ -174,24 +182,15 @@ k_tc_gemm_nt(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 }  // namespace
 }  // namespace tc
 
-namespace {
-int tc_gemm_pick_stages(int n_mma) {
-    const int stage_bytes = tc::kATileBytes + n_mma * 128;
-    int s = (200 * 1024) / stage_bytes;
-    if (s > 8) s = 8;
-    if (s < 2) s = 2;
-    return s;
-}
-}  // namespace
-
 cudaError_t launch_tc_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const void* Bm, int64_t ldb, int M, int N, int fold,
-                              int64_t K, int splits, float* C, int64_t ldc, int64_t split_stride, int* err, cudaStream_t st) {
+                              int mt, int64_t K, int splits, float* C, int64_t ldc, int64_t split_stride, int* err, cudaStream_t st) {
     if (M <= 0 || N <= 0 || K <= 0) return cudaSuccess;
     const int es = dt == SAGE_F32 ? 4 : 2;
     const int BK = 128 / es;
     const int n_pad = ((N + 15) / 16) * 16;
     const int n_mma = fold ? 2 * n_pad : n_pad;
     if (n_mma > 256 || splits < 1 || splits > 65535) return cudaErrorNotSupported;
+    if ((mt != 1 && mt != 2 && mt != 4) || mt * n_mma > 512) return cudaErrorNotSupported;
     CUtensorMap tmA, tmB;
     if (!tc::make_tmap_2d(&tmA, A, es, (uint64_t)M, (uint64_t)K, (uint64_t)lda, tc::kTileM)) return cudaErrorNotSupported;
     if (!tc::make_tmap_2d(&tmB, Bm, es, (uint64_t)(fold ? n_pad + N : N), (uint64_t)K, (uint64_t)ldb, (uint32_t)n_mma))
@@ -199,22 +198,25 @@ cudaError_t launch_tc_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const
     int64_t kps = (K + splits - 1) / splits;
     kps = ((kps + BK - 1) / BK) * BK;
     // a trailing slice may be empty after rounding to whole K tiles: its CTAs store zeros
-    const int stages = tc_gemm_pick_stages(n_mma);
-    const int stage_bytes = tc::kATileBytes + n_mma * 128;
+    const int stage_bytes = mt * tc::kATileBytes + n_mma * 128;
+    int stages = (200 * 1024) / stage_bytes;
+    if (stages > 8) stages = 8;
+    if (stages < 2) return cudaErrorNotSupported;
     const size_t smem = (size_t)stages * stage_bytes + 1024 + (2 * stages + 1) * 8 + 16;
     uint32_t tmem_cols = 32;
-    while (tmem_cols < (uint32_t)n_mma) tmem_cols <<= 1;
-    dim3 grid((unsigned)((M + tc::kTileM - 1) / tc::kTileM), (unsigned)splits);
+    while (tmem_cols < (uint32_t)(mt * n_mma)) tmem_cols <<= 1;
+    const int tiles = (M + tc::kTileM - 1) / tc::kTileM;
+    dim3 grid((unsigned)((tiles + mt - 1) / mt), (unsigned)splits);
     cudaError_t e;
     if (dt == SAGE_BF16) {
         e = cudaFuncSetAttribute(tc::k_tc_gemm_nt<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        tc::k_tc_gemm_nt<1><<<grid, tc::kThreads, smem, st>>>(tmA, tmB, M, N, n_pad, fold, K, kps, C, ldc, split_stride, stages,
+        tc::k_tc_gemm_nt<1><<<grid, tc::kThreads, smem, st>>>(tmA, tmB, M, N, n_pad, fold, mt, K, kps, C, ldc, split_stride, stages,
                                                               tmem_cols, err);
     } else {
         e = cudaFuncSetAttribute(tc::k_tc_gemm_nt<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        tc::k_tc_gemm_nt<2><<<grid, tc::kThreads, smem, st>>>(tmA, tmB, M, N, n_pad, fold, K, kps, C, ldc, split_stride, stages,
+        tc::k_tc_gemm_nt<2><<<grid, tc::kThreads, smem, st>>>(tmA, tmB, M, N, n_pad, fold, mt, K, kps, C, ldc, split_stride, stages,
                                                               tmem_cols, err);
     }
     return cudaGetLastError();
