@@ -158,6 +158,7 @@ def main():
     ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c4", "c5"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--rows", type=int, default=0, help="use only the first ROWS rows of the workload (debugging)")
+    ap.add_argument("--dim", type=int, default=0, help="override the row dimension D (small cases for profiler captures)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--seed", type=int, default=0)
@@ -167,6 +168,8 @@ def main():
     w = wl.WORKLOADS[args.workload]
     if args.rows:
         w = wl.scaled(w, N=args.rows)
+    if args.dim:
+        w = wl.scaled(w, D=args.dim)
     if args.impl == "reference":
         run_reference(args, w)
         return

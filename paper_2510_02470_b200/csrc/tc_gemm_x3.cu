@@ -12,9 +12,11 @@
 //
 // One CTA owns a 128 x (<=128) output tile and one K slice:
 //   warp 0    TMA producer (raw fp32 tiles, 128-byte swizzle),
-//   warp 1    TMEM allocation and MMA issue into two ping-pong accumulators,
-//   warps 2-5 split each landed stage into hi (in place) and lo (second buffer),
-//   warps 6-9 drain finished accumulators into registers and store the tile at the end.
+//   warp 1    TMEM allocation and MMA issue into a ring of four accumulators,
+//   warps 2-9 split each landed stage into hi (in place) and lo (second buffer); every kChunk stages they also
+//             drain the accumulator that was finished two chunks earlier (its MMAs are long done, so the drain
+//             never waits) into registers, and store the tile at the end. Warp w drains TMEM lanes
+//             32 * (w % 4) and columns 64 * ((w - 2) / 4).
 // On the diagonal tiles of a Gram matrix only one operand tile is loaded and used on both sides.
 #include "sage_internal.h"
 #include "tc05.cuh"
@@ -24,13 +26,20 @@ namespace tc {
 namespace {
 
 constexpr int kThreads = 320;
-constexpr int kSplitThreads = 128;
-constexpr int kDrainThreads = 128;
+constexpr int kWorkers = 256;               // warps 2-9
 constexpr int kTileM = 128;
 constexpr int kTileN = 128;
 constexpr int kTileBytes = 128 * 128;       // 128 rows of 128 bytes
 constexpr int BK = 32;                      // fp32 elements per 128-byte K tile
 constexpr int kChunk = 4;                   // K tiles accumulated in TMEM between drains
+constexpr int kAccs = 4;                    // accumulators in TMEM (4 x 128 columns)
+
+__device__ __forceinline__ void split4(const uint4 v, uint4& h, uint4& l) {
+    h.x = (v.x + 0x1000u) & 0xffffe000u; l.x = __float_as_uint(__uint_as_float(v.x) - __uint_as_float(h.x));
+    h.y = (v.y + 0x1000u) & 0xffffe000u; l.y = __float_as_uint(__uint_as_float(v.y) - __uint_as_float(h.y));
+    h.z = (v.z + 0x1000u) & 0xffffe000u; l.z = __float_as_uint(__uint_as_float(v.z) - __uint_as_float(h.z));
+    h.w = (v.w + 0x1000u) & 0xffffe000u; l.w = __float_as_uint(__uint_as_float(v.w) - __uint_as_float(h.w));
+}
 
 __global__ void __launch_bounds__(kThreads, 1)
 k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, int M, int N, int gram,
@@ -45,9 +54,9 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)stages * stage_bytes);
     uint64_t* split_done = full + stages;
     uint64_t* empty = split_done + stages;
-    uint64_t* acc_full = empty + stages;                   // [2]
-    uint64_t* acc_empty = acc_full + 2;                    // [2]
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    uint64_t* acc_full = empty + stages;                   // [kAccs]
+    uint64_t* acc_empty = acc_full + kAccs;                // [kAccs]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + kAccs);
     volatile int* abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -61,19 +70,19 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
             mbar_init(&full[s], 1);
-            mbar_init(&split_done[s], kSplitThreads);
+            mbar_init(&split_done[s], kWorkers);
             mbar_init(&empty[s], 1);
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < kAccs; ++b) {
             mbar_init(&acc_full[b], 1);
-            mbar_init(&acc_empty[b], kDrainThreads);
+            mbar_init(&acc_empty[b], kWorkers);
         }
         *abort = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmA);
         tma_prefetch_desc(&tmB);
     }
-    if (warp == 1) tmem_alloc(tmem_slot, 2 * kTileN);
+    if (warp == 1) tmem_alloc(tmem_slot, kAccs * kTileN);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -105,8 +114,8 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             for (int kt = 0; kt < nkt && alive; ++kt) {
                 const int s = kt % stages;
                 const uint32_t use = (uint32_t)(kt / stages);
-                const int c = kt / kChunk, b = c & 1, in_chunk = kt - c * kChunk;
-                if (in_chunk == 0) alive = mbar_wait(&acc_empty[b], (((uint32_t)c >> 1) & 1u) ^ 1u, abort);
+                const int c = kt / kChunk, b = c & (kAccs - 1), in_chunk = kt - c * kChunk;
+                if (in_chunk == 0) alive = mbar_wait(&acc_empty[b], (((uint32_t)c / kAccs) & 1u) ^ 1u, abort);
                 if (alive) alive = mbar_wait(&split_done[s], use & 1u, abort);
                 if (!alive) break;
                 tc_fence_after();
@@ -126,46 +135,25 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 if (in_chunk == kChunk - 1 || kt == nkt - 1) mma_commit(&acc_full[b]);
             }
         }
-    } else if (warp < 6) {
-        // ---- split landed stages into hi (in place) and lo ----
-        const int t = threadIdx.x - 64;                 // 0..127
-        const int chunks16 = half_bytes / 16;
-        for (int kt = 0; kt < nkt; ++kt) {
-            const int s = kt % stages;
-            const uint32_t use = (uint32_t)(kt / stages);
-            if (!mbar_wait(&full[s], use & 1u, abort)) break;
-            uint4* hi = reinterpret_cast<uint4*>(smem + (size_t)s * stage_bytes);
-            uint4* lo = reinterpret_cast<uint4*>(smem + (size_t)s * stage_bytes + half_bytes);
-            for (int c = t; c < chunks16; c += kSplitThreads) {
-                const uint4 v = hi[c];
-                uint4 h, l;
-                h.x = (v.x + 0x1000u) & 0xffffe000u; l.x = __float_as_uint(__uint_as_float(v.x) - __uint_as_float(h.x));
-                h.y = (v.y + 0x1000u) & 0xffffe000u; l.y = __float_as_uint(__uint_as_float(v.y) - __uint_as_float(h.y));
-                h.z = (v.z + 0x1000u) & 0xffffe000u; l.z = __float_as_uint(__uint_as_float(v.z) - __uint_as_float(h.z));
-                h.w = (v.w + 0x1000u) & 0xffffe000u; l.w = __float_as_uint(__uint_as_float(v.w) - __uint_as_float(h.w));
-                hi[c] = h;
-                lo[c] = l;
-            }
-            fence_proxy_async_smem();                   // the tensor cores read these writes
-            mbar_arrive(&split_done[s]);
-        }
     } else {
-        // ---- drain accumulators into registers; store the tile ----
-        const int quarter = warp & 3;
-        const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
-        float acc[kTileN];
+        // ---- workers: split landed stages into hi (in place) and lo; drain finished accumulators ----
+        const int t = threadIdx.x - 64;                 // 0..255
+        const int chunks16 = half_bytes / 16;
+        const int quarter = warp & 3, chalf = (warp - 2) >> 2;
+        const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + (uint32_t)(chalf * 64);
+        float acc[64];
 #pragma unroll
-        for (int j = 0; j < kTileN; ++j) acc[j] = 0.f;
+        for (int j = 0; j < 64; ++j) acc[j] = 0.f;
         bool ok = true;
-        for (int c = 0; c < nchunks; ++c) {
-            const int b = c & 1;
-            ok = mbar_wait(&acc_full[b], ((uint32_t)c >> 1) & 1u, abort);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
+        auto drain = [&](int c) {
+            const int b = c & (kAccs - 1);
+            bool w = mbar_wait(&acc_full[b], ((uint32_t)c / kAccs) & 1u, abort);
+            w = __all_sync(0xffffffffu, w);
+            if (!w) { ok = false; return; }
             tc_fence_after();
 #pragma unroll
-            for (int c0 = 0; c0 < kTileN; c0 += 16) {
-                if (c0 < n_pad) {
+            for (int c0 = 0; c0 < 64; c0 += 16) {
+                if (chalf * 64 + c0 < n_pad) {
                     float v[16];
                     tmem_ld16(lane_base + (uint32_t)(b * kTileN + c0), v);
 #pragma unroll
@@ -174,19 +162,44 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             }
             tc_fence_before();
             mbar_arrive(&acc_empty[b]);
+        };
+        int drained = 0;                                // chunks drained so far
+        for (int kt = 0; kt < nkt && ok; ++kt) {
+            const int s = kt % stages;
+            const uint32_t use = (uint32_t)(kt / stages);
+            if (!mbar_wait(&full[s], use & 1u, abort)) { ok = false; break; }
+            uint4* hi = reinterpret_cast<uint4*>(smem + (size_t)s * stage_bytes);
+            uint4* lo = reinterpret_cast<uint4*>(smem + (size_t)s * stage_bytes + half_bytes);
+            for (int c = t; c < chunks16; c += 4 * kWorkers) {     // four independent 16-byte pieces in flight
+                uint4 v[4], h[4], l[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (c + u * kWorkers < chunks16) v[u] = hi[c + u * kWorkers];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) split4(v[u], h[u], l[u]);
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (c + u * kWorkers < chunks16) { hi[c + u * kWorkers] = h[u]; lo[c + u * kWorkers] = l[u]; }
+            }
+            fence_proxy_async_smem();                   // the tensor cores read these writes
+            mbar_arrive(&split_done[s]);
+            // the chunk that ended two chunks ago has certainly been multiplied: fold it into the registers
+            if ((kt + 1) % kChunk == 0 && kt / kChunk - 2 >= drained) drain(drained++);
         }
+        while (ok && drained < nchunks) drain(drained++);
         const int row = m0 + quarter * 32 + lane;
         if (row < M) {
-            float* crow = C + (long long)blockIdx.z * split_stride + (long long)row * ldc + n0;
+            float* crow = C + (long long)blockIdx.z * split_stride + (long long)row * ldc + n0 + chalf * 64;
             const bool vec = (ldc % 4 == 0) && ((reinterpret_cast<uintptr_t>(C) & 15u) == 0) && (split_stride % 4 == 0);
 #pragma unroll
-            for (int c0 = 0; c0 < kTileN; c0 += 4) {
-                if (n0 + c0 + 4 <= N && vec) {
+            for (int c0 = 0; c0 < 64; c0 += 4) {
+                const int col = n0 + chalf * 64 + c0;
+                if (col + 4 <= N && vec) {
                     *reinterpret_cast<float4*>(crow + c0) = make_float4(acc[c0], acc[c0 + 1], acc[c0 + 2], acc[c0 + 3]);
                 } else {
 #pragma unroll
                     for (int j = 0; j < 4; ++j)
-                        if (n0 + c0 + j < N) crow[c0 + j] = acc[c0 + j];
+                        if (col + j < N) crow[c0 + j] = acc[c0 + j];
                 }
             }
         }
@@ -195,9 +208,10 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     __syncthreads();
     if (warp == 1) {
         // no MMA may be in flight when TMEM is freed: the last chunk's commit covers every MMA issued
-        if (nchunks > 0 && !*abort) mbar_wait_quiet(&acc_full[(nchunks - 1) & 1], ((uint32_t)(nchunks - 1) >> 1) & 1u, kWaitLimitCycles);
+        if (nchunks > 0 && !*abort)
+            mbar_wait_quiet(&acc_full[(nchunks - 1) & (kAccs - 1)], ((uint32_t)(nchunks - 1) / kAccs) & 1u, kWaitLimitCycles);
         tc_fence_after();
-        tmem_dealloc(tmem_base, 2 * kTileN);
+        tmem_dealloc(tmem_base, kAccs * kTileN);
     }
     if (threadIdx.x == 0 && *abort) atomicExch(err, 1);
 }
@@ -221,7 +235,7 @@ cudaError_t launch_tc_gemm_nt_x3(const float* A, int64_t lda, const float* Bm, i
     const int stage_bytes = 2 * ((gram && M <= tc::kTileM) ? tc::kTileBytes : tc::kTileBytes + b_box_rows * 128);
     int stages = (200 * 1024) / stage_bytes;
     if (stages > 8) stages = 8;
-    const size_t smem = (size_t)stages * stage_bytes + 1024 + (3 * stages + 4) * 8 + 16;
+    const size_t smem = (size_t)stages * stage_bytes + 1024 + (3 * stages + 2 * tc::kAccs) * 8 + 16;
     dim3 grid((unsigned)((M + tc::kTileM - 1) / tc::kTileM), (unsigned)((N + tc::kTileN - 1) / tc::kTileN), (unsigned)splits);
     cudaError_t e = cudaFuncSetAttribute(tc::k_tc_gemm_nt_x3, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
