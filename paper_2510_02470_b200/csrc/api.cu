@@ -351,7 +351,8 @@ sage_status_t sage_fd_create(sage_fd_t** out, int64_t D, int32_t ell, sage_dtype
         return fail(e, "cudaMalloc(W)");
     if ((e = cudaMalloc((void**)&h->Kmat, mm)) != cudaSuccess) return fail(e, "cudaMalloc(K)");
     if ((e = cudaMalloc((void**)&h->Ur, mm)) != cudaSuccess) return fail(e, "cudaMalloc(U)");
-    if ((e = cudaMalloc((void**)&h->eig_work, mm)) != cudaSuccess) return fail(e, "cudaMalloc(eig)");
+    if ((e = cudaMalloc((void**)&h->eig_work, mm > 256 * 256 * sizeof(float) ? mm : 256 * 256 * sizeof(float))) != cudaSuccess)
+        return fail(e, "cudaMalloc(eig)");
     if ((e = cudaMalloc((void**)&h->sigma, ell * sizeof(float))) != cudaSuccess) return fail(e, "cudaMalloc(sigma)");
     if ((e = cudaMalloc((void**)&h->info, sizeof(EigInfo))) != cudaSuccess) return fail(e, "cudaMalloc(info)");
     if ((e = cudaMalloc((void**)&h->zsum, 256 * sizeof(double))) != cudaSuccess) return fail(e, "cudaMalloc(zsum)");

@@ -61,25 +61,27 @@ __device__ __forceinline__ void rr_pair(int n_even, int round, int slot, int& p,
 // X is column-major with a row pitch of LD = 64*T floats; column c of the factor stays at the physical
 // position of the c-th pivot, so the rows of U come out in the original buffer order.
 // ------------------------------------------------------------------------------------------------
-constexpr int kMaxFast = 192;
+constexpr int kMaxFast = 192;      // largest n whose matrix fits in shared memory
+constexpr int kMaxN = 256;         // largest n of this kernel (above kMaxFast the matrix stays in global memory, i.e. L2)
 
-template <int T>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int T, int NT, bool G>
+__global__ void __launch_bounds__(NT, 1)
 k_eig_shrink_fast(const float* __restrict__ K, int ldk, int n, int do_shrink, int delta_rank, int keep, float* __restrict__ Ur,
                   int ldu, float* __restrict__ sigma_out, int n_sigma, int max_sweeps, EigInfo* __restrict__ info,
-                  float* __restrict__ Wsplit, int ldw, int j_pad) {
+                  float* __restrict__ Wsplit, int ldw, int j_pad, float* __restrict__ gwork) {
     constexpr int LD = 64 * T;
+    constexpr int NW = NT / 32;
     constexpr int R = 2 * T;            // rows per lane when 32 lanes span a column
     constexpr int Q = 2 * T;            // float4 per lane when 8 lanes span a column
     extern __shared__ __align__(16) float smem[];
-    float* X = smem;                                    // LD x LD
-    float* lam = X + LD * LD;                           // kMaxFast each from here on
-    float* fac = lam + kMaxFast;
-    float* scl = fac + kMaxFast;
-    int* ord = reinterpret_cast<int*>(scl + kMaxFast);  // physical index -> pivot step (-1: never pivoted)
-    int* perm = ord + kMaxFast;                         // pivot step -> physical index
-    int* order = perm + kMaxFast;                       // sorted position -> pivot step
-    float* sh_f = reinterpret_cast<float*>(order + kMaxFast);
+    float* X = G ? gwork : smem;                        // LD x LD (global scratch when it does not fit on chip)
+    float* lam = G ? smem : smem + LD * LD;             // kMaxN each from here on
+    float* fac = lam + kMaxN;
+    float* scl = fac + kMaxN;
+    int* ord = reinterpret_cast<int*>(scl + kMaxN);     // physical index -> pivot step (-1: never pivoted)
+    int* perm = ord + kMaxN;                            // pivot step -> physical index
+    int* order = perm + kMaxN;                          // sorted position -> pivot step
+    float* sh_f = reinterpret_cast<float*>(order + kMaxN);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
@@ -101,21 +103,21 @@ k_eig_shrink_fast(const float* __restrict__ K, int ldk, int n, int do_shrink, in
     if (warp == 0 && bad) atomicOr(&info->flags, kFlagNonFinite);
     const bool empty = !(dmax >= 1e-30f);              // nothing to factor: rank 0
     const float kscale = empty ? 0.f : 1.f / dmax;
-    for (int e = tid; e < n * LD; e += kThreads) {
+    for (int e = tid; e < n * LD; e += NT) {
         const int c = e / LD, i = e - c * LD;
         X[e] = (i < n) ? K[(size_t)c * ldk + i] * kscale : 0.f;  // K is symmetric: row c serves as column c
     }
 #pragma unroll
     for (int t = 0; t < R; ++t) dg[t] *= kscale;
-    if (tid < kMaxFast) ord[tid] = -1;
+    for (int i = tid; i < kMaxN; i += NT) ord[i] = -1;
     __syncthreads();
 
     // ---- pivoted Cholesky without swaps (scaled matrix: diagonal <= 1) ----
-    constexpr int CW = (kMaxFast + kWarps - 1) / kWarps;       // columns a warp owns: warp + 32 u
+    constexpr int CW = (LD + NW - 1) / NW;                     // columns a warp owns: warp + NW u
     unsigned colmask = 0u;                                     // bit u: column warp + 32 u is still unpivoted
 #pragma unroll
     for (int u = 0; u < CW; ++u)
-        if (warp + kWarps * u < n) colmask |= 1u << u;
+        if (warp + NW * u < n) colmask |= 1u << u;
     const float tol = 1e-7f;
     int rank = empty ? 0 : n;
     for (int k = 0; k < rank; ++k) {
@@ -130,7 +132,7 @@ k_eig_shrink_fast(const float* __restrict__ K, int ldk, int n, int do_shrink, in
         const float d = Xp[p];
         if (!(d > tol)) { rank = k; break; }
         const float inv = rsqrtf(d);
-        if ((p & (kWarps - 1)) == warp) colmask &= ~(1u << (p / kWarps));
+        if ((p & (NW - 1)) == warp) colmask &= ~(1u << (p / NW));
         float li[R];
 #pragma unroll
         for (int t = 0; t < R; ++t) {
@@ -143,10 +145,10 @@ k_eig_shrink_fast(const float* __restrict__ K, int ldk, int n, int do_shrink, in
         for (int u0 = 0; u0 < CW; u0 += 2) {                      // two columns at a time: loads first, then stores
             const bool on0 = (colmask >> u0) & 1u, on1 = (u0 + 1 < CW) && ((colmask >> (u0 + 1)) & 1u);
             if (!on0 && !on1) continue;
-            float* c0 = X + (warp + kWarps * u0) * LD;
-            float* c1 = X + (warp + kWarps * (u0 + 1)) * LD;
-            const float l0 = on0 ? Xp[warp + kWarps * u0] * inv : 0.f;
-            const float l1 = on1 ? Xp[warp + kWarps * (u0 + 1)] * inv : 0.f;
+            float* c0 = X + (warp + NW * u0) * LD;
+            float* c1 = X + (warp + NW * (u0 + 1)) * LD;
+            const float l0 = on0 ? Xp[warp + NW * u0] * inv : 0.f;
+            const float l1 = on1 ? Xp[warp + NW * (u0 + 1)] * inv : 0.f;
             float v0[R], v1[R];
 #pragma unroll
             for (int t = 0; t < R; ++t) {
@@ -164,7 +166,7 @@ k_eig_shrink_fast(const float* __restrict__ K, int ldk, int n, int do_shrink, in
     }
     __syncthreads();
     // ---- scale the pivot columns into the factor L (zero above the pivot order, zero unpivoted columns) ----
-    for (int e = tid; e < n * LD; e += kThreads) {
+    for (int e = tid; e < n * LD; e += NT) {
         const int c = e / LD, i = e - c * LD;
         const int kc = ord[c];
         float v = 0.f;
@@ -188,9 +190,10 @@ k_eig_shrink_fast(const float* __restrict__ K, int ldk, int n, int do_shrink, in
     if (tid < 2) sh_flag[tid] = 0;
     __syncthreads();
     if (rank >= 2) {
-        const int nb = (rank + 3) >> 2, nbe = nb + (nb & 1), nbm1 = nbe - 1, nact = nbe >> 1;   // nact <= 24 warps
-        if (warp < nact) {
-            const int nthreads = nact * 32;
+        const int nb = (rank + 3) >> 2, nbe = nb + (nb & 1), nbm1 = nbe - 1, nact = nbe >> 1;   // block pairs per round
+        const int nwork = nact < NW ? nact : NW;                  // warps that take part; each owns slots w, w + nwork, ...
+        if (warp < nwork) {
+            const int nthreads = nwork * 32;
             auto pair_step = [&](int p, int q) {                  // p, q: pivot-order columns, q >= rank means no pair
                 const bool valid = p < rank && q < rank;
                 float4* xp = reinterpret_cast<float4*>(X + (valid ? perm[p] : 0) * LD) + l8;
@@ -236,11 +239,12 @@ k_eig_shrink_fast(const float* __restrict__ K, int ldk, int n, int do_shrink, in
             while (sweeps < max_sweeps) {
                 worst2 = 0.f;
                 for (int br = 0; br < nbm1; ++br) {
-                    int ba, bb;                                   // the two blocks of this warp in this block round
-                    if (warp == 0) { ba = nbm1; bb = br; }
+                  for (int slot = warp; slot < nact; slot += nwork) {
+                    int ba, bb;                                   // the two blocks of this slot in this block round
+                    if (slot == 0) { ba = nbm1; bb = br; }
                     else {
-                        ba = br + warp; if (ba >= nbm1) ba -= nbm1;
-                        bb = br + nbm1 - warp; if (bb >= nbm1) bb -= nbm1;
+                        ba = br + slot; if (ba >= nbm1) ba -= nbm1;
+                        bb = br + nbm1 - slot; if (bb >= nbm1) bb -= nbm1;
                     }
                     if (br == 0) {                                // pairs inside each block: quarters 0,1 -> ba, 2,3 -> bb
                         const int base = 4 * ((qd < 2) ? ba : bb), h = qd & 1;
@@ -249,8 +253,77 @@ k_eig_shrink_fast(const float* __restrict__ K, int ldk, int n, int do_shrink, in
                         pair_step(base + (h ? 1 : 0), base + (h ? 2 : 3));
                     }
                     const int lo = min(ba, bb), hi = max(ba, bb);
-#pragma unroll 1
-                    for (int r = 0; r < 4; ++r) pair_step(4 * lo + qd, 4 * hi + ((qd + r) & 3));
+                    {   // the 16 cross pairs, columns held in registers: quarter qd keeps column qd of block lo and
+                        // the columns of block hi travel from quarter to quarter by shuffles between the 4 rounds
+                        const int pa = 4 * lo + qd, pb = 4 * hi + qd;
+                        const bool va = pa < rank, vb0 = pb < rank;
+                        float4* xa = reinterpret_cast<float4*>(X + (va ? perm[pa] : 0) * LD) + l8;
+                        float4* xb = reinterpret_cast<float4*>(X + (vb0 ? perm[pb] : 0) * LD) + l8;
+                        float4 x[Q], y[Q];
+#pragma unroll
+                        for (int t = 0; t < Q; ++t) {
+                            x[t] = va ? xa[8 * t] : make_float4(0.f, 0.f, 0.f, 0.f);
+                            y[t] = vb0 ? xb[8 * t] : make_float4(0.f, 0.f, 0.f, 0.f);
+                        }
+#pragma unroll
+                        for (int r = 0; r < 4; ++r) {
+                            const bool valid = va && (4 * hi + ((qd + r) & 3) < rank);
+                            float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f, g0 = 0.f, g1 = 0.f;
+#pragma unroll
+                            for (int t = 0; t < Q; ++t) {
+                                a0 = fmaf(x[t].x, x[t].x, a0); a1 = fmaf(x[t].y, x[t].y, a1); a0 = fmaf(x[t].z, x[t].z, a0); a1 = fmaf(x[t].w, x[t].w, a1);
+                                b0 = fmaf(y[t].x, y[t].x, b0); b1 = fmaf(y[t].y, y[t].y, b1); b0 = fmaf(y[t].z, y[t].z, b0); b1 = fmaf(y[t].w, y[t].w, b1);
+                                g0 = fmaf(x[t].x, y[t].x, g0); g1 = fmaf(x[t].y, y[t].y, g1); g0 = fmaf(x[t].z, y[t].z, g0); g1 = fmaf(x[t].w, y[t].w, g1);
+                            }
+                            float a = a0 + a1, b = b0 + b1, g = g0 + g1;
+#pragma unroll
+                            for (int o = 4; o > 0; o >>= 1) {
+                                a += __shfl_xor_sync(0xffffffffu, a, o);
+                                b += __shfl_xor_sync(0xffffffffu, b, o);
+                                g += __shfl_xor_sync(0xffffffffu, g, o);
+                            }
+                            const float ab = a * b, g2 = g * g;
+                            if (valid && ab > 0.f && g2 > 1e-12f * ab) {
+                                worst2 = fmaxf(worst2, __fdividef(g2, ab));
+                                const float zeta = __fdividef(b - a, 2.f * g);
+                                const float tt = copysignf(__fdividef(1.f, fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.f))), zeta);
+                                const float c = rsqrtf(fmaf(tt, tt, 1.f));
+                                const float s = c * tt;
+#pragma unroll
+                                for (int t = 0; t < Q; ++t) {
+                                    float4 nx, ny;
+                                    nx.x = fmaf(-s, y[t].x, c * x[t].x); ny.x = fmaf(s, x[t].x, c * y[t].x);
+                                    nx.y = fmaf(-s, y[t].y, c * x[t].y); ny.y = fmaf(s, x[t].y, c * y[t].y);
+                                    nx.z = fmaf(-s, y[t].z, c * x[t].z); ny.z = fmaf(s, x[t].z, c * y[t].z);
+                                    nx.w = fmaf(-s, y[t].w, c * x[t].w); ny.w = fmaf(s, x[t].w, c * y[t].w);
+                                    x[t] = nx;
+                                    y[t] = ny;
+                                }
+                            }
+                            if (r < 3) {                          // quarter qd takes over the column quarter qd + 1 holds
+                                const int src = (lane + 8) & 31;
+#pragma unroll
+                                for (int t = 0; t < Q; ++t) {
+                                    y[t].x = __shfl_sync(0xffffffffu, y[t].x, src);
+                                    y[t].y = __shfl_sync(0xffffffffu, y[t].y, src);
+                                    y[t].z = __shfl_sync(0xffffffffu, y[t].z, src);
+                                    y[t].w = __shfl_sync(0xffffffffu, y[t].w, src);
+                                }
+                            }
+                        }
+                        const int pl = 4 * hi + ((qd + 3) & 3);   // the hi column this quarter ends up with
+                        if (va) {
+#pragma unroll
+                            for (int t = 0; t < Q; ++t) xa[8 * t] = x[t];
+                        }
+                        if (pl < rank) {
+                            float4* xl = reinterpret_cast<float4*>(X + perm[pl] * LD) + l8;
+#pragma unroll
+                            for (int t = 0; t < Q; ++t) xl[8 * t] = y[t];
+                        }
+                        __syncwarp();
+                    }
+                  }
                     asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
                 }
                 ++sweeps;
@@ -269,7 +342,7 @@ k_eig_shrink_fast(const float* __restrict__ K, int ldk, int n, int do_shrink, in
     const int not_converged = rank >= 2 && sh_f[4] != 0.f;     // stopped at the sweep limit while still rotating visibly
 
     // ---- eigenvalues = squared column norms (pivot-step order), scaled back; sort descending, stable ----
-    for (int k = warp; k < n; k += kWarps) {
+    for (int k = warp; k < n; k += NW) {
         float a = 0.f;
         if (k < rank) {
             const float* x = X + perm[k] * LD;
@@ -319,9 +392,9 @@ k_eig_shrink_fast(const float* __restrict__ K, int ldk, int n, int do_shrink, in
         fac[tid] = f;
         if (tid < n_sigma) sigma_out[tid] = sp;
     }
-    for (int j = n + tid; j < n_sigma; j += kThreads) sigma_out[j] = 0.f;
+    for (int j = n + tid; j < n_sigma; j += NT) sigma_out[j] = 0.f;
     __syncthreads();
-    for (int e = tid; e < n * keep; e += kThreads) {
+    for (int e = tid; e < n * keep; e += NT) {
         const int j = e / n, i = e - j * n;
         float v = 0.f;
         if (j < n) {
@@ -331,7 +404,7 @@ k_eig_shrink_fast(const float* __restrict__ K, int ldk, int n, int do_shrink, in
         Ur[(size_t)i * ldu + j] = v;
     }
     if (Wsplit) {   // the same factors transposed and split for the tensor-core rebuild: [W_hi ; W_lo], zero padded
-        for (int e = tid; e < j_pad * ldw; e += kThreads) {
+        for (int e = tid; e < j_pad * ldw; e += NT) {
             const int j = e / ldw, i = e - j * ldw;
             float v = 0.f;
             if (j < keep && j < n && i < n) {
@@ -575,16 +648,18 @@ cudaError_t launch_eig_shrink(const float* K, int ldk, int n, int do_shrink, int
                               float* sigma_out, int n_sigma, float* work, int max_sweeps, EigInfo* info, float* Wsplit, int ldw,
                               int j_pad, cudaStream_t st) {
     if (n <= 0 || n > 512) return cudaErrorInvalidValue;
-    if (n <= kMaxFast) {
+    if (n <= kMaxN) {
         const int T = (n + 63) / 64;
-        const size_t bytes = ((size_t)(64 * T) * (64 * T) + 3 * kMaxFast) * sizeof(float) + 3 * kMaxFast * sizeof(int) + 32;
+        const size_t aux_bytes = 3 * kMaxN * sizeof(float) + 3 * kMaxN * sizeof(int) + 32;
+        const size_t bytes = (T <= 3 ? (size_t)(64 * T) * (64 * T) * sizeof(float) : 0) + aux_bytes;
         cudaError_t e;
-#define SAGE_EIG_FAST(TT)                                                                                              \
-    e = cudaFuncSetAttribute(k_eig_shrink_fast<TT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);          \
+#define SAGE_EIG_FAST(TT, NTT, GG)                                                                                     \
+    e = cudaFuncSetAttribute(k_eig_shrink_fast<TT, NTT, GG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes); \
     if (e != cudaSuccess) return e;                                                                                    \
-    k_eig_shrink_fast<TT><<<1, kThreads, bytes, st>>>(K, ldk, n, do_shrink, delta_rank, keep, Ur, ldu, sigma_out, n_sigma, \
-                                                      max_sweeps, info, Wsplit, ldw, j_pad);
-        if (T == 1) { SAGE_EIG_FAST(1) } else if (T == 2) { SAGE_EIG_FAST(2) } else { SAGE_EIG_FAST(3) }
+    k_eig_shrink_fast<TT, NTT, GG><<<1, NTT, bytes, st>>>(K, ldk, n, do_shrink, delta_rank, keep, Ur, ldu, sigma_out, n_sigma, \
+                                                          max_sweeps, info, Wsplit, ldw, j_pad, work);
+        if (T == 1) { SAGE_EIG_FAST(1, 1024, false) } else if (T == 2) { SAGE_EIG_FAST(2, 1024, false) }
+        else if (T == 3) { SAGE_EIG_FAST(3, 1024, false) } else { SAGE_EIG_FAST(4, 512, true) }   // work: >= 256 x 256 floats
 #undef SAGE_EIG_FAST
         return cudaGetLastError();
     }
