@@ -166,6 +166,43 @@ def test_lemma_identity_on_gpu_outputs():
     assert np.linalg.norm(Z[T].mean(axis=0)) >= xi * zn[T].mean() * (1 - 1e-4)
 
 
+# ------------------------------------------------------------------ tensor-core kernels against the CUDA-core kernels
+
+def _run_with_option(rows, D, ell, use_tc):
+    dev = torch.device("cuda", 0)
+    g = rows.to(dev)
+    fd = sage.SageFD(D, ell, rows.dtype, 0)
+    fd.set_option(4, 1.0 if use_tc else 0.0)
+    fd.update(g)
+    fd.finalize()
+    S, _ = fd.sketch()
+    a = fd.score(g)
+    torch.cuda.synchronize()
+    st = fd.stats()
+    fd.close()
+    return S.double().cpu().numpy(), a.double().cpu().numpy(), st
+
+
+@pytest.mark.parametrize("dtype,N,D,ell", [(torch.float32, 900, 2052, 40), (torch.bfloat16, 700, 4104, 64),
+                                           (torch.bfloat16, 600, 20008, 24), (torch.float32, 500, 1000, 128)])
+def test_tensor_core_path_agrees_with_cuda_core_path(dtype, N, D, ell):
+    """Same rows through option 4 = 1 (tcgen05 Gram / rebuild / projection) and option 4 = 0 (fp32 FMA kernels):
+    both must match the oracle, and each other far more tightly than the tolerances."""
+    rows = lowrank_rows(N, D, 6, 0.4, N + ell, dtype)
+    S1, a1, st1 = _run_with_option(rows, D, ell, True)
+    S0, a0, st0 = _run_with_option(rows, D, ell, False)
+    assert st1["device_flags"] == 0 and st0["device_flags"] == 0 and st1["shrinks"] == st0["shrinks"]
+    A = metrics.rows_as_f64(rows, D)
+    F2 = float(np.linalg.norm(A) ** 2)
+    assert metrics.signed_gram_norm(S1, S0) / F2 <= 2e-5
+    # bf16 rows: the tensor-core path rounds the sketch to bf16 (one term for D >= 16384), the CUDA-core path does not
+    assert np.max(np.abs(a1 - a0)) <= (2e-5 if dtype == torch.float32 else TOL_SCORE[dtype])
+    ref = oracle.run(rows, D, ell, 0.1, route=1)
+    for S, a in ((S1, a1), (S0, a0)):
+        assert metrics.signed_gram_norm(S, ref["S"]) / F2 <= 1e-4
+        assert np.max(np.abs(a - ref["alpha"])) <= TOL_SCORE[dtype]
+
+
 # ------------------------------------------------------------------ the benchmark workloads
 
 def test_c1_full():
