@@ -191,19 +191,22 @@ sage_status_t enqueue_gram(sage_fd* h, int r, cudaStream_t st) {
         const int t = (r + 127) / 128;
         const int ldc = ((r + 3) / 4) * 4;
         const int64_t stride = (int64_t)r * ldc;
+        const int sym = r <= 128 ? 1 : 0;    // one diagonal tile: two MMAs per K step, transpose added in the reduction
         int cap = (int)(kGramPartFloats / (size_t)stride);
         if (cap > 148) cap = 148;
         const int splits = pick_splits_waves(t * t, h->D, 256, cap);
         cudaError_t e;
-        if (splits == 1) {
-            e = timed(h, K_GRAM, 1, st, [&] { return launch_tc_gemm_nt_x3(Bc, h->pitch, Bc, h->pitch, r, r, h->D, 1, h->Kmat, h->m, 0, h->tc_err, st); });
+        if (splits == 1 && !sym) {
+            e = timed(h, K_GRAM, 1, st, [&] { return launch_tc_gemm_nt_x3(Bc, h->pitch, Bc, h->pitch, r, r, h->D, 1, h->Kmat, h->m, 0, 0, h->tc_err, st); });
         } else {
             e = timed(h, K_GRAM, 1, st, [&] {
-                return launch_tc_gemm_nt_x3(Bc, h->pitch, Bc, h->pitch, r, r, h->D, splits, h->gram_parts, ldc, stride, h->tc_err, st);
+                return launch_tc_gemm_nt_x3(Bc, h->pitch, Bc, h->pitch, r, r, h->D, splits, h->gram_parts, ldc, stride, sym, h->tc_err, st);
             });
         }
         if (e == cudaSuccess) {
-            if (splits > 1)
+            if (sym)
+                CU_TRY(timed(h, K_GRAM_REDUCE, 1, st, [&] { return launch_gram_sym_reduce(h->gram_parts, splits, stride, r, ldc, h->Kmat, h->m, st); }));
+            else if (splits > 1)
                 CU_TRY(timed(h, K_GRAM_REDUCE, 1, st, [&] { return launch_split_reduce(h->gram_parts, splits, stride, r, r, ldc, h->Kmat, h->m, st); }));
             return SAGE_OK;
         }
@@ -614,7 +617,7 @@ sage_status_t sage_score_chunk(sage_fd_t* h, const void* rows, int64_t n, int64_
             float* out = splits > 1 ? h->zwork + (size_t)sub * ell : Z;
             cudaError_t e = timed(h, K_PROJECT, 1, st, [&] {
                 return launch_tc_gemm_nt_x3(reinterpret_cast<const float*>(p + r0 * row_bytes), ld, S, h->pitch, (int)sub, ell, h->D,
-                                            splits, out, ell, (int64_t)sub * ell, h->tc_err, st);
+                                            splits, out, ell, (int64_t)sub * ell, 0, h->tc_err, st);
             });
             if (e == cudaSuccess) {
                 done = true;

@@ -48,8 +48,12 @@ cudaError_t launch_tc_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const
 // fp32-faithful tensor-core C[z] = A_z * Bm_z^T for fp32 operands (three tf32 MMAs on hi/lo halves split in shared
 // memory, accumulator drained into registers every few K tiles). Same alignment rules and return convention as
 // launch_tc_gemm_nt; any N. When A == Bm (a Gram matrix) the diagonal tiles load one operand only.
+// sym != 0 (only for a Gram matrix of at most 128 rows): two MMAs per K step instead of three; slice z then stores
+// T_z = hi*hi^T + 2*hi*lo^T and the Gram matrix is sum_z (T_z + T_z^T)/2: see launch_gram_sym_reduce.
 cudaError_t launch_tc_gemm_nt_x3(const float* A, int64_t lda, const float* Bm, int64_t ldb, int M, int N, int64_t K, int splits,
-                                 float* C, int64_t ldc, int64_t split_stride, int* err, cudaStream_t st);
+                                 float* C, int64_t ldc, int64_t split_stride, int sym, int* err, cudaStream_t st);
+cudaError_t launch_gram_sym_reduce(const float* parts, int splits, int64_t stride, int r, int64_t ldp, float* out, int64_t ldo,
+                                   cudaStream_t st);
 
 // Tensor-core rebuild: Bdst[j][d] = sum_{i<r} W[j][i] * Bsrc[i][d] for j < keep, d < pitch (fp32-faithful, see
 // tc_rebuild.cu). Wsplit holds W already split for tf32: rows [0, j_pad) = W rounded to 11 significant bits, rows

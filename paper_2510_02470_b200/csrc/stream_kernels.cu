@@ -159,6 +159,20 @@ __global__ void __launch_bounds__(256) k_split_reduce(const float* __restrict__ 
     out[(int64_t)i * ldo + j] = (float)s;
 }
 
+// Split reduction of a Gram matrix computed in the two-MMA symmetric form: slice z left T_z = hi*hi^T + 2*hi*lo^T
+// at parts + z*stride; K = sum_z (T_z + T_z^T) / 2, ascending z, fp64.
+__global__ void __launch_bounds__(256) k_gram_sym_reduce(const float* __restrict__ parts, int splits, int64_t stride, int r,
+                                                         int64_t ldp, float* __restrict__ out, int64_t ldo) {
+    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= (int64_t)r * r) return;
+    const int i = (int)(e / r), j = (int)(e % r);
+    const float* a = parts + (int64_t)i * ldp + j;
+    const float* b = parts + (int64_t)j * ldp + i;
+    double s = 0.0;
+    for (int z = 0; z < splits; ++z) s += (double)a[(int64_t)z * stride] + (double)b[(int64_t)z * stride];
+    out[(int64_t)i * ldo + j] = (float)(0.5 * s);
+}
+
 // ------------------------------------------------------------------------------------------------
 // Rebuild (Method, first paragraph: "reconstruct S <- Sigma' V^T"): with B B^T = U Lambda U^T,
 // Sigma' V^T = diag(sigma'_j / sigma_j) U^T B, so out[j][:] = sum_i Ur[i][j] B[i][:] where Ur already
@@ -263,6 +277,13 @@ cudaError_t launch_split_reduce(const float* parts, int splits, int64_t split_st
     const int64_t total = (int64_t)M * N;
     if (total <= 0) return cudaSuccess;
     k_split_reduce<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(parts, splits, split_stride, M, N, ldp, out, ldo);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gram_sym_reduce(const float* parts, int splits, int64_t stride, int r, int64_t ldp, float* out, int64_t ldo,
+                                   cudaStream_t st) {
+    if (r <= 0) return cudaSuccess;
+    k_gram_sym_reduce<<<(unsigned)(((int64_t)r * r + 255) / 256), 256, 0, st>>>(parts, splits, stride, r, ldp, out, ldo);
     return cudaGetLastError();
 }
 

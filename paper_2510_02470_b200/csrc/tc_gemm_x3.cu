@@ -17,7 +17,12 @@
 //             drain the accumulator that was finished two chunks earlier (its MMAs are long done, so the drain
 //             never waits) into registers, and store the tile at the end. Warp w drains TMEM lanes
 //             32 * (w % 4) and columns 64 * ((w - 2) / 4).
-// On the diagonal tiles of a Gram matrix only one operand tile is loaded and used on both sides.
+// On the diagonal tiles of a Gram matrix only one operand tile is loaded and used on both sides. A Gram matrix
+// of at most 128 rows (sym mode) needs ONE 256-wide MMA per K step: the hi tile and the (doubled) lo tile lie
+// back to back in the stage and serve as one 256-row B operand, so the accumulator holds hi*hi^T | 2*hi*lo^T side
+// by side; their sum T satisfies (T + T^T)/2 = hi*hi^T + hi*lo^T + lo*hi^T, formed by the split reduction. (Issuing
+// a tf32 MMA costs the issuing thread about 110 cycles whatever its width, and a 128 x 128 x 8 one executes in
+// about 70: narrow MMAs leave the tensor pipe idle, wide ones do not.)
 #include "sage_internal.h"
 #include "tc05.cuh"
 
@@ -31,7 +36,7 @@ constexpr int kTileM = 128;
 constexpr int kTileN = 128;
 constexpr int kTileBytes = 128 * 128;       // 128 rows of 128 bytes
 constexpr int BK = 32;                      // fp32 elements per 128-byte K tile
-constexpr int kChunk = 4;                   // K tiles accumulated in TMEM between drains
+constexpr int kChunkTiles = 4;              // K tiles accumulated in TMEM between drains
 constexpr int kAccs = 4;                    // accumulators in TMEM (4 x 128 columns)
 
 __device__ __forceinline__ void split4(const uint4 v, uint4& h, uint4& l) {
@@ -43,7 +48,7 @@ __device__ __forceinline__ void split4(const uint4 v, uint4& h, uint4& l) {
 
 __global__ void __launch_bounds__(kThreads, 1)
 k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, int M, int N, int gram,
-                int b_box_rows, long long K, long long k_per_split, float* __restrict__ C, long long ldc, long long split_stride,
+                int b_box_rows, int sym, long long K, long long k_per_split, float* __restrict__ C, long long ldc, long long split_stride,
                 int stages, int stage_bytes, int* __restrict__ err) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -63,7 +68,10 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const long long k_begin = (long long)blockIdx.z * k_per_split;
     const long long k_end = K < k_begin + k_per_split ? K : k_begin + k_per_split;
     const int nkt = k_end > k_begin ? (int)((k_end - k_begin + BK - 1) / BK) : 0;
+    const int kChunk = kChunkTiles;
     const int nchunks = (nkt + kChunk - 1) / kChunk;
+    const int acc_cols = sym ? 2 * kTileN : kTileN;       // sym: P and 2Q side by side
+    const int ring = (kAccs * kTileN) / acc_cols;         // accumulators in flight: 4, or 2 in sym mode
     int n_pad = N - n0 < kTileN ? N - n0 : kTileN;        // MMA width of this tile, a multiple of 16
     n_pad = ((n_pad + 15) / 16) * 16;
 
@@ -109,13 +117,13 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            const uint32_t idesc = instr_desc(2, kTileM, n_pad, 0, 0);
+            const uint32_t idesc = instr_desc(2, kTileM, sym ? 2 * kTileN : n_pad, 0, 0);
             bool alive = true;
             for (int kt = 0; kt < nkt && alive; ++kt) {
                 const int s = kt % stages;
                 const uint32_t use = (uint32_t)(kt / stages);
-                const int c = kt / kChunk, b = c & (kAccs - 1), in_chunk = kt - c * kChunk;
-                if (in_chunk == 0) alive = mbar_wait(&acc_empty[b], (((uint32_t)c / kAccs) & 1u) ^ 1u, abort);
+                const int c = kt / kChunk, b = c % ring, in_chunk = kt - c * kChunk;
+                if (in_chunk == 0) alive = mbar_wait(&acc_empty[b], (((uint32_t)c / ring) & 1u) ^ 1u, abort);
                 if (alive) alive = mbar_wait(&split_done[s], use & 1u, abort);
                 if (!alive) break;
                 tc_fence_after();
@@ -124,12 +132,14 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 const uint32_t b_hi = diag ? a_hi : st + kTileBytes, b_lo = b_hi + half_bytes;
                 const uint64_t d_ahi = smem_desc_k_sw128(a_hi), d_alo = smem_desc_k_sw128(a_lo);
                 const uint64_t d_bhi = smem_desc_k_sw128(b_hi), d_blo = smem_desc_k_sw128(b_lo);
-                const uint32_t acc = tmem_base + (uint32_t)(b * kTileN);
+                const uint32_t acc = tmem_base + (uint32_t)(b * acc_cols);
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {          // 4 x 8 tf32 elements per 128-byte row
-                    mma_tf32(acc, d_ahi + 2 * k, d_bhi + 2 * k, idesc, (in_chunk | k) != 0);
-                    mma_tf32(acc, d_ahi + 2 * k, d_blo + 2 * k, idesc, 1);
-                    mma_tf32(acc, d_alo + 2 * k, d_bhi + 2 * k, idesc, 1);
+                    mma_tf32(acc, d_ahi + 2 * k, d_bhi + 2 * k, idesc, (in_chunk | k) != 0);   // sym: B = [hi ; 2 lo]
+                    if (!sym) {
+                        mma_tf32(acc, d_ahi + 2 * k, d_blo + 2 * k, idesc, 1);
+                        mma_tf32(acc, d_alo + 2 * k, d_bhi + 2 * k, idesc, 1);
+                    }
                 }
                 mma_commit(&empty[s]);
                 if (in_chunk == kChunk - 1 || kt == nkt - 1) mma_commit(&acc_full[b]);
@@ -146,8 +156,8 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         for (int j = 0; j < 64; ++j) acc[j] = 0.f;
         bool ok = true;
         auto drain = [&](int c) {
-            const int b = c & (kAccs - 1);
-            bool w = mbar_wait(&acc_full[b], ((uint32_t)c / kAccs) & 1u, abort);
+            const int b = c % ring;
+            bool w = mbar_wait(&acc_full[b], ((uint32_t)c / ring) & 1u, abort);
             w = __all_sync(0xffffffffu, w);
             if (!w) { ok = false; return; }
             tc_fence_after();
@@ -155,9 +165,14 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             for (int c0 = 0; c0 < 64; c0 += 16) {
                 if (chalf * 64 + c0 < n_pad) {
                     float v[16];
-                    tmem_ld16(lane_base + (uint32_t)(b * kTileN + c0), v);
+                    tmem_ld16(lane_base + (uint32_t)(b * acc_cols + c0), v);
 #pragma unroll
                     for (int j = 0; j < 16; ++j) acc[c0 + j] += v[j];
+                    if (sym) {
+                        tmem_ld16(lane_base + (uint32_t)(b * acc_cols + kTileN + c0), v);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) acc[c0 + j] += v[j];
+                    }
                 }
             }
             tc_fence_before();
@@ -176,7 +191,13 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 for (int u = 0; u < 4; ++u)
                     if (c + u * kWorkers < chunks16) v[u] = hi[c + u * kWorkers];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) split4(v[u], h[u], l[u]);
+                for (int u = 0; u < 4; ++u) {
+                    split4(v[u], h[u], l[u]);
+                    if (sym) {      // doubled remainder (exact): see the note on sym mode above
+                        l[u].x = __float_as_uint(2.f * __uint_as_float(l[u].x)); l[u].y = __float_as_uint(2.f * __uint_as_float(l[u].y));
+                        l[u].z = __float_as_uint(2.f * __uint_as_float(l[u].z)); l[u].w = __float_as_uint(2.f * __uint_as_float(l[u].w));
+                    }
+                }
 #pragma unroll
                 for (int u = 0; u < 4; ++u)
                     if (c + u * kWorkers < chunks16) { hi[c + u * kWorkers] = h[u]; lo[c + u * kWorkers] = l[u]; }
@@ -184,7 +205,7 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             fence_proxy_async_smem();                   // the tensor cores read these writes
             mbar_arrive(&split_done[s]);
             // the chunk that ended two chunks ago has certainly been multiplied: fold it into the registers
-            if ((kt + 1) % kChunk == 0 && kt / kChunk - 2 >= drained) drain(drained++);
+            if ((kt + 1) % kChunk == 0 && kt / kChunk - ring / 2 >= drained) drain(drained++);
         }
         while (ok && drained < nchunks) drain(drained++);
         const int row = m0 + quarter * 32 + lane;
@@ -209,7 +230,7 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     if (warp == 1) {
         // no MMA may be in flight when TMEM is freed: the last chunk's commit covers every MMA issued
         if (nchunks > 0 && !*abort)
-            mbar_wait_quiet(&acc_full[(nchunks - 1) & (kAccs - 1)], ((uint32_t)(nchunks - 1) / kAccs) & 1u, kWaitLimitCycles);
+            mbar_wait_quiet(&acc_full[(nchunks - 1) % ring], ((uint32_t)(nchunks - 1) / ring) & 1u, kWaitLimitCycles);
         tc_fence_after();
         tmem_dealloc(tmem_base, kAccs * kTileN);
     }
@@ -220,10 +241,11 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 }  // namespace tc
 
 cudaError_t launch_tc_gemm_nt_x3(const float* A, int64_t lda, const float* Bm, int64_t ldb, int M, int N, int64_t K, int splits,
-                                 float* C, int64_t ldc, int64_t split_stride, int* err, cudaStream_t st) {
+                                 float* C, int64_t ldc, int64_t split_stride, int sym, int* err, cudaStream_t st) {
     if (M <= 0 || N <= 0 || K <= 0) return cudaSuccess;
     if (splits < 1 || splits > 65535) return cudaErrorNotSupported;
     const int gram = (A == Bm && lda == ldb && M == N) ? 1 : 0;
+    if (sym && !(gram && M <= tc::kTileM)) return cudaErrorInvalidValue;
     CUtensorMap tmA, tmB;
     if (!tc::make_tmap_2d(&tmA, A, 4, (uint64_t)M, (uint64_t)K, (uint64_t)lda, tc::kTileM)) return cudaErrorNotSupported;
     const int b_box_rows = N >= tc::kTileN ? tc::kTileN : ((N + 15) / 16) * 16;
@@ -239,7 +261,7 @@ cudaError_t launch_tc_gemm_nt_x3(const float* A, int64_t lda, const float* Bm, i
     dim3 grid((unsigned)((M + tc::kTileM - 1) / tc::kTileM), (unsigned)((N + tc::kTileN - 1) / tc::kTileN), (unsigned)splits);
     cudaError_t e = cudaFuncSetAttribute(tc::k_tc_gemm_nt_x3, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    tc::k_tc_gemm_nt_x3<<<grid, tc::kThreads, smem, st>>>(tmA, tmB, M, N, gram, b_box_rows, K, kps, C, ldc, split_stride, stages,
+    tc::k_tc_gemm_nt_x3<<<grid, tc::kThreads, smem, st>>>(tmA, tmB, M, N, gram, b_box_rows, sym, K, kps, C, ldc, split_stride, stages,
                                                                  stage_bytes, err);
     return cudaGetLastError();
 }
