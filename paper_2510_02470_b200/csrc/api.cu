@@ -109,6 +109,8 @@ struct sage_fd {
     __nv_bfloat16* P16 = nullptr;  // frozen sketch in bf16 (bf16 handles: tensor-core projection operand); with p16_fold
                                    // rows [0, ell) hold bf16(S) and rows [n_pad, n_pad + ell) hold bf16(S - bf16(S))
     int p16_fold = 0, p16_npad = 0;
+    cudaStream_t side = nullptr;   // appends of the next shrink cycle run here, beside the eigen-solve of the current one
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     int* tc_err = nullptr;         // set by a tensor-core kernel whose bounded wait ran out
     bool use_tc = true;            // option 4: tensor-core kernels where their alignment rules hold
     int64_t launches = 0;
@@ -232,6 +234,7 @@ sage_status_t enqueue_gram(sage_fd* h, int r, cudaStream_t st) {
 // Factor the first r rows and rebuild `keep` rows into the other buffer; rows keep..zero_to-1 are zeroed.
 sage_status_t enqueue_factor(sage_fd* h, int r, int do_shrink, int keep, int zero_to, cudaStream_t st) {
     ST_TRY(enqueue_gram(h, r, st));
+    CU_TRY(cudaEventRecord(h->ev_fork, st));       // from here on HBM is idle until the rebuild: see sage_fd_update
     const int j_pad = ((keep + 15) / 16) * 16;
     const bool tc_rebuild = h->use_tc && h->Wsplit && keep > 0 && j_pad <= 128 && r <= 256;
     CU_TRY(timed(h, K_EIG, 1, st, [&] {
@@ -361,6 +364,9 @@ sage_status_t sage_fd_create(sage_fd_t** out, int64_t D, int32_t ell, sage_dtype
     if ((e = cudaMalloc((void**)&h->zsum, 256 * sizeof(double))) != cudaSuccess) return fail(e, "cudaMalloc(zsum)");
     if ((e = cudaMalloc((void**)&h->u, 256 * sizeof(float))) != cudaSuccess) return fail(e, "cudaMalloc(u)");
     if ((e = cudaMalloc((void**)&h->tc_err, sizeof(int))) != cudaSuccess) return fail(e, "cudaMalloc(err)");
+    if ((e = cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking)) != cudaSuccess) return fail(e, "cudaStreamCreate");
+    if ((e = cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
+    if ((e = cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
     if ((e = cudaMemset(h->tc_err, 0, sizeof(int))) != cudaSuccess) return fail(e, "cudaMemset");
     if (row_dtype == SAGE_BF16) {
         // Two-term bf16 sketch (16 significant bits) for short rows, where the rounding errors of a one-term
@@ -399,6 +405,9 @@ void sage_fd_destroy(sage_fd_t* h) {
     cudaFree(h->u);
     cudaFree(h->P16);
     cudaFree(h->tc_err);
+    if (h->side) cudaStreamDestroy(h->side);
+    if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+    if (h->ev_join) cudaEventDestroy(h->ev_join);
     for (auto& p : h->prof.pending) {
         cudaEventDestroy(p.a);
         cudaEventDestroy(p.b);
@@ -464,15 +473,36 @@ sage_status_t sage_fd_update(sage_fd_t* h, const void* rows, int64_t n, int64_t 
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const char* p = static_cast<const char*>(rows);
     const size_t row_bytes = (size_t)ld * elem_size(h->dtype);
+    // Appends that follow a shrink go to a side stream: they write rows [keep, m) of the buffer the rebuild is
+    // filling (rows [0, keep)) and touch nothing the eigen-solve / rebuild of that shrink read or write, so they run
+    // beside the eigen-solve, which leaves HBM idle. The side stream starts when the Gram kernel of the shrink has
+    // finished (running beside it only takes bandwidth from it) and is joined before the next Gram and before this
+    // call returns.
+    bool on_side = false, side_pending = false;
     while (n > 0) {
         const int64_t room = h->m - h->fill;
         const int64_t take = n < room ? n : room;
-        CU_TRY(timed(h, K_APPEND, 1, st, [&] { return launch_append(p, h->dtype, take, ld, h->D, h->B[h->cur], h->pitch, h->fill, st); }));
+        cudaStream_t as = on_side ? h->side : st;
+        CU_TRY(timed(h, K_APPEND, 1, as, [&] { return launch_append(p, h->dtype, take, ld, h->D, h->B[h->cur], h->pitch, h->fill, as); }));
+        if (on_side) side_pending = true;
         h->fill += (int)take;
         h->rows_seen += take;
         p += take * row_bytes;
         n -= take;
-        if (h->fill == h->m) ST_TRY(enqueue_factor(h, h->m, 1, h->delta_rank - 1, 0, st));
+        if (h->fill == h->m) {
+            if (side_pending) {
+                CU_TRY(cudaEventRecord(h->ev_join, h->side));
+                CU_TRY(cudaStreamWaitEvent(st, h->ev_join, 0));
+                side_pending = false;
+            }
+            ST_TRY(enqueue_factor(h, h->m, 1, h->delta_rank - 1, 0, st));
+            CU_TRY(cudaStreamWaitEvent(h->side, h->ev_fork, 0));
+            on_side = true;
+        }
+    }
+    if (side_pending) {
+        CU_TRY(cudaEventRecord(h->ev_join, h->side));
+        CU_TRY(cudaStreamWaitEvent(st, h->ev_join, 0));
     }
     return SAGE_OK;
 }
