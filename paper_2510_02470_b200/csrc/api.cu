@@ -357,7 +357,9 @@ sage_status_t sage_fd_create(sage_fd_t** out, int64_t D, int32_t ell, sage_dtype
         return fail(e, "cudaMalloc(W)");
     if ((e = cudaMalloc((void**)&h->Kmat, mm)) != cudaSuccess) return fail(e, "cudaMalloc(K)");
     if ((e = cudaMalloc((void**)&h->Ur, mm)) != cudaSuccess) return fail(e, "cudaMalloc(U)");
-    if ((e = cudaMalloc((void**)&h->eig_work, mm > 256 * 256 * sizeof(float) ? mm : 256 * 256 * sizeof(float))) != cudaSuccess)
+    // eigen workspace: the matrix padded to 256 or 512 rows/columns plus a few flag words
+    const size_t ew = h->m > 256 ? (size_t)512 * 512 : (size_t)256 * 256;
+    if ((e = cudaMalloc((void**)&h->eig_work, (ew + 64) * sizeof(float))) != cudaSuccess)
         return fail(e, "cudaMalloc(eig)");
     if ((e = cudaMalloc((void**)&h->sigma, ell * sizeof(float))) != cudaSuccess) return fail(e, "cudaMalloc(sigma)");
     if ((e = cudaMalloc((void**)&h->info, sizeof(EigInfo))) != cudaSuccess) return fail(e, "cudaMalloc(info)");

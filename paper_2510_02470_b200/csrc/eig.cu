@@ -10,10 +10,14 @@
 // keep their relative accuracy. One thread block does the whole solve; the matrix lives in shared
 // memory when it fits (n <= 232) and in global scratch (L2-resident) otherwise. All loops are bounded;
 // hitting the sweep limit sets a flag instead of spinning.
+#include <cooperative_groups.h>
+
 #include "sage_internal.h"
 
 namespace sage {
 namespace {
+
+namespace cg = cooperative_groups;
 
 constexpr int kThreads = 1024;
 constexpr int kWarps = kThreads / 32;
@@ -418,6 +422,378 @@ k_eig_shrink_fast(const float* __restrict__ K, int ldk, int n, int do_shrink, in
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Cluster solver for 192 < n <= 512: the same algorithm as k_eig_shrink_fast, run by a thread-block cluster
+// (8 CTAs of 256 threads on 8 SMs) with the matrix in global memory (L2-resident) and a hardware cluster
+// barrier where the one-CTA kernel has a block barrier. Every warp of the cluster owns Cholesky columns and one
+// Jacobi block pair, so a block round costs one L2 round trip for its 8 columns, 4 register-resident local rounds
+// and one cluster barrier, instead of several passes over 16 warps on one SM. Control flow is identical in
+// every CTA (pivot search and convergence flag are computed from identical data), so every thread of the cluster
+// reaches every barrier; the small tables (pivot order, eigenvalues, factors) are kept per CTA.
+// ------------------------------------------------------------------------------------------------
+template <int T>
+__global__ void __launch_bounds__(256, 1)
+k_eig_shrink_cluster(const float* __restrict__ K, int ldk, int n, int do_shrink, int delta_rank, int keep, float* __restrict__ Ur,
+                  int ldu, float* __restrict__ sigma_out, int n_sigma, int max_sweeps, EigInfo* __restrict__ info,
+                  float* __restrict__ Wsplit, int ldw, int j_pad, float* __restrict__ gwork) {
+    constexpr int LD = 64 * T;
+    constexpr int NT = 256;                              // threads per CTA
+    constexpr int kMaxN = 512;                           // shadows the namespace constant: this kernel serves n <= 512
+    cg::cluster_group cluster = cg::this_cluster();
+    const int csize = (int)cluster.num_blocks(), crank = (int)cluster.block_rank();
+    const int NW = 8 * csize;                            // warps of the whole cluster
+    const int GT = NT * csize;                           // threads of the whole cluster
+    constexpr int R = 2 * T;            // rows per lane when 32 lanes span a column
+    constexpr int Q = 2 * T;            // float4 per lane when 8 lanes span a column
+    extern __shared__ __align__(16) float smem[];
+    float* X = gwork;                                   // LD x LD in global memory (L2), shared by the cluster
+    int* gflag = reinterpret_cast<int*>(gwork + (size_t)LD * LD);   // two convergence words after the matrix
+    float* lam = smem;                                  // kMaxN each from here on (one copy per CTA)
+    float* fac = lam + kMaxN;
+    float* scl = fac + kMaxN;
+    int* ord = reinterpret_cast<int*>(scl + kMaxN);     // physical index -> pivot step (-1: never pivoted)
+    int* perm = ord + kMaxN;                            // pivot step -> physical index
+    int* order = perm + kMaxN;                          // sorted position -> pivot step
+    float* sh_f = reinterpret_cast<float*>(order + kMaxN);
+
+    const int tid = threadIdx.x, lane = tid & 31, lwarp = tid >> 5;
+    const int warp = crank * 8 + lwarp;                  // warp index within the cluster
+    const int gtid = crank * NT + tid;
+
+    // running diagonal and liveness of the rows this lane owns (rows lane + 32 t), one copy per warp
+    float dg[R];
+    bool alive[R];
+    bool bad = false;
+    float dmax = 0.f;
+#pragma unroll
+    for (int t = 0; t < R; ++t) {
+        const int i = lane + 32 * t;
+        dg[t] = (i < n) ? K[(size_t)i * ldk + i] : -1.f;
+        alive[t] = i < n;
+        if (alive[t] && !(fabsf(dg[t]) <= 3.0e38f)) { bad = true; alive[t] = false; }
+        if (alive[t]) dmax = fmaxf(dmax, dg[t]);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) dmax = fmaxf(dmax, __shfl_xor_sync(0xffffffffu, dmax, o));
+    if (warp == 0 && bad) atomicOr(&info->flags, kFlagNonFinite);
+    const bool empty = !(dmax >= 1e-30f);              // nothing to factor: rank 0
+    const float kscale = empty ? 0.f : 1.f / dmax;
+    for (int e = gtid; e < n * LD; e += GT) {
+        const int c = e / LD, i = e - c * LD;
+        X[e] = (i < n) ? K[(size_t)c * ldk + i] * kscale : 0.f;  // K is symmetric: row c serves as column c
+    }
+    if (gtid < 2) gflag[gtid] = 0;
+#pragma unroll
+    for (int t = 0; t < R; ++t) dg[t] *= kscale;
+    for (int i = tid; i < kMaxN; i += NT) ord[i] = -1;
+    cluster.sync();
+
+    // ---- pivoted Cholesky without swaps (scaled matrix: diagonal <= 1) ----
+    constexpr int CW = (LD + 63) / 64 * 2;                     // upper bound of columns a warp owns (warp + NW u) for NW >= 32
+    unsigned colmask = 0u;                                     // bit u: column warp + 32 u is still unpivoted
+#pragma unroll
+    for (int u = 0; u < CW; ++u)
+        if (warp + NW * u < n) colmask |= 1u << u;
+    const float tol = 1e-7f;
+    int rank = empty ? 0 : n;
+    for (int k = 0; k < rank; ++k) {
+        unsigned key = 0u;
+#pragma unroll
+        for (int t = 0; t < R; ++t)
+            if (alive[t]) key = max(key, (__float_as_uint(fmaxf(dg[t], 0.f)) & 0xfffffe00u) | (unsigned)(511 - (lane + 32 * t)));
+        key = __reduce_max_sync(0xffffffffu, key);                // largest diagonal (24 significant bits), smaller index on ties
+        const int p = 511 - (int)(key & 511u);
+        if (key == 0u || p >= n) { rank = k; break; }             // identical in every warp
+        const float* Xp = X + p * LD;
+        const float d = __ldcg(Xp + p);
+        if (!(d > tol)) { rank = k; break; }
+        const float inv = rsqrtf(d);
+        if ((p % NW) == warp) colmask &= ~(1u << (p / NW));
+        float li[R];
+#pragma unroll
+        for (int t = 0; t < R; ++t) {
+            const int i = lane + 32 * t;
+            if (i == p) alive[t] = false;
+            li[t] = alive[t] ? __ldcg(Xp + i) * inv : 0.f;
+            dg[t] = fmaf(-li[t], li[t], dg[t]);
+        }
+#pragma unroll
+        for (int u0 = 0; u0 < CW; u0 += 2) {                      // two columns at a time: loads first, then stores
+            const bool on0 = (colmask >> u0) & 1u, on1 = (u0 + 1 < CW) && ((colmask >> (u0 + 1)) & 1u);
+            if (!on0 && !on1) continue;
+            float* c0 = X + (warp + NW * u0) * LD;
+            float* c1 = X + (warp + NW * (u0 + 1)) * LD;
+            const float l0 = on0 ? __ldcg(Xp + warp + NW * u0) * inv : 0.f;
+            const float l1 = on1 ? __ldcg(Xp + warp + NW * (u0 + 1)) * inv : 0.f;
+            float v0[R], v1[R];
+#pragma unroll
+            for (int t = 0; t < R; ++t) {
+                v0[t] = on0 ? __ldcg(c0 + lane + 32 * t) : 0.f;
+                v1[t] = on1 ? __ldcg(c1 + lane + 32 * t) : 0.f;
+            }
+#pragma unroll
+            for (int t = 0; t < R; ++t) {
+                if (on0) c0[lane + 32 * t] = fmaf(-li[t], l0, v0[t]);
+                if (on1) c1[lane + 32 * t] = fmaf(-li[t], l1, v1[t]);
+            }
+        }
+        if (tid == 0) { ord[p] = k; perm[k] = p; scl[k] = inv; }   // every CTA keeps its own copy of the tables
+        cluster.sync();
+    }
+    cluster.sync();
+    // ---- scale the pivot columns into the factor L (zero above the pivot order, zero unpivoted columns) ----
+    for (int e = gtid; e < n * LD; e += GT) {
+        const int c = e / LD, i = e - c * LD;
+        const int kc = ord[c];
+        float v = 0.f;
+        if (kc >= 0 && i < n) {
+            const int ki = ord[i];
+            if (!(ki >= 0 && ki < kc)) v = __ldcg(X + e) * scl[kc];
+        }
+        X[e] = v;
+    }
+    cluster.sync();
+
+    // ---- one-sided cyclic Jacobi on the rank pivot columns ----
+    // Columns (in pivot order) form blocks of 4. A block round pairs the blocks round-robin, one block
+    // pair per warp; the warp rotates the 16 cross pairs of its two blocks in 4 local rounds (one pair per
+    // quarter-warp, synchronised inside the warp only), and in the first block round of a sweep also the
+    // pairs inside each block. Only the warps that own a block pair take part, on a named barrier.
+    const int l8 = tid & 7, qd = lane >> 3;
+    int sweeps = 0;
+    float worst2 = 0.f;                 // largest squared cosine met in the current sweep
+    if (rank >= 2) {
+        const int nb = (rank + 3) >> 2, nbe = nb + (nb & 1), nbm1 = nbe - 1, nact = nbe >> 1;   // block pairs per round
+        const int nwork = nact < NW ? nact : NW;                  // warps that take part; each owns slots w, w + nwork, ...
+        {
+            const bool active = warp < nwork;                     // the other warps only take part in the cluster barriers
+            auto pair_step = [&](int p, int q) {                  // p, q: pivot-order columns, q >= rank means no pair
+                const bool valid = p < rank && q < rank;
+                float4* xp = reinterpret_cast<float4*>(X + (valid ? perm[p] : 0) * LD) + l8;
+                float4* xq = reinterpret_cast<float4*>(X + (valid ? perm[q] : 0) * LD) + l8;
+                float4 x[Q], y[Q];
+                float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f, g0 = 0.f, g1 = 0.f;
+#pragma unroll
+                for (int t = 0; t < Q; ++t) {
+                    x[t] = __ldcg(xp + 8 * t);
+                    y[t] = __ldcg(xq + 8 * t);
+                    a0 = fmaf(x[t].x, x[t].x, a0); a1 = fmaf(x[t].y, x[t].y, a1); a0 = fmaf(x[t].z, x[t].z, a0); a1 = fmaf(x[t].w, x[t].w, a1);
+                    b0 = fmaf(y[t].x, y[t].x, b0); b1 = fmaf(y[t].y, y[t].y, b1); b0 = fmaf(y[t].z, y[t].z, b0); b1 = fmaf(y[t].w, y[t].w, b1);
+                    g0 = fmaf(x[t].x, y[t].x, g0); g1 = fmaf(x[t].y, y[t].y, g1); g0 = fmaf(x[t].z, y[t].z, g0); g1 = fmaf(x[t].w, y[t].w, g1);
+                }
+                float a = a0 + a1, b = b0 + b1, g = g0 + g1;
+#pragma unroll
+                for (int o = 4; o > 0; o >>= 1) {
+                    a += __shfl_xor_sync(0xffffffffu, a, o);
+                    b += __shfl_xor_sync(0xffffffffu, b, o);
+                    g += __shfl_xor_sync(0xffffffffu, g, o);
+                }
+                const float ab = a * b, g2 = g * g;
+                if (valid && ab > 0.f && g2 > 1e-12f * ab) {
+                    worst2 = fmaxf(worst2, __fdividef(g2, ab));
+                    const float zeta = __fdividef(b - a, 2.f * g);
+                    const float tt = copysignf(__fdividef(1.f, fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.f))), zeta);
+                    const float c = rsqrtf(fmaf(tt, tt, 1.f));
+                    const float s = c * tt;
+#pragma unroll
+                    for (int t = 0; t < Q; ++t) {
+                        float4 nx, ny;
+                        nx.x = fmaf(-s, y[t].x, c * x[t].x); ny.x = fmaf(s, x[t].x, c * y[t].x);
+                        nx.y = fmaf(-s, y[t].y, c * x[t].y); ny.y = fmaf(s, x[t].y, c * y[t].y);
+                        nx.z = fmaf(-s, y[t].z, c * x[t].z); ny.z = fmaf(s, x[t].z, c * y[t].z);
+                        nx.w = fmaf(-s, y[t].w, c * x[t].w); ny.w = fmaf(s, x[t].w, c * y[t].w);
+                        xp[8 * t] = nx;
+                        xq[8 * t] = ny;
+                    }
+                }
+                __syncwarp();
+            };
+            int more = 0;
+            while (sweeps < max_sweeps) {
+                worst2 = 0.f;
+                for (int br = 0; br < nbm1; ++br) {
+                  for (int slot = active ? warp : nact; slot < nact; slot += nwork) {
+                    int ba, bb;                                   // the two blocks of this slot in this block round
+                    if (slot == 0) { ba = nbm1; bb = br; }
+                    else {
+                        ba = br + slot; if (ba >= nbm1) ba -= nbm1;
+                        bb = br + nbm1 - slot; if (bb >= nbm1) bb -= nbm1;
+                    }
+                    if (br == 0) {                                // pairs inside each block: quarters 0,1 -> ba, 2,3 -> bb
+                        const int base = 4 * ((qd < 2) ? ba : bb), h = qd & 1;
+                        pair_step(base + (h ? 2 : 0), base + (h ? 3 : 1));
+                        pair_step(base + (h ? 1 : 0), base + (h ? 3 : 2));
+                        pair_step(base + (h ? 1 : 0), base + (h ? 2 : 3));
+                    }
+                    const int lo = min(ba, bb), hi = max(ba, bb);
+                    {   // the 16 cross pairs, columns held in registers: quarter qd keeps column qd of block lo and
+                        // the columns of block hi travel from quarter to quarter by shuffles between the 4 rounds
+                        const int pa = 4 * lo + qd, pb = 4 * hi + qd;
+                        const bool va = pa < rank, vb0 = pb < rank;
+                        float4* xa = reinterpret_cast<float4*>(X + (va ? perm[pa] : 0) * LD) + l8;
+                        float4* xb = reinterpret_cast<float4*>(X + (vb0 ? perm[pb] : 0) * LD) + l8;
+                        float4 x[Q], y[Q];
+#pragma unroll
+                        for (int t = 0; t < Q; ++t) {
+                            x[t] = va ? __ldcg(xa + 8 * t) : make_float4(0.f, 0.f, 0.f, 0.f);
+                            y[t] = vb0 ? __ldcg(xb + 8 * t) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        }
+#pragma unroll
+                        for (int r = 0; r < 4; ++r) {
+                            const bool valid = va && (4 * hi + ((qd + r) & 3) < rank);
+                            float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f, g0 = 0.f, g1 = 0.f;
+#pragma unroll
+                            for (int t = 0; t < Q; ++t) {
+                                a0 = fmaf(x[t].x, x[t].x, a0); a1 = fmaf(x[t].y, x[t].y, a1); a0 = fmaf(x[t].z, x[t].z, a0); a1 = fmaf(x[t].w, x[t].w, a1);
+                                b0 = fmaf(y[t].x, y[t].x, b0); b1 = fmaf(y[t].y, y[t].y, b1); b0 = fmaf(y[t].z, y[t].z, b0); b1 = fmaf(y[t].w, y[t].w, b1);
+                                g0 = fmaf(x[t].x, y[t].x, g0); g1 = fmaf(x[t].y, y[t].y, g1); g0 = fmaf(x[t].z, y[t].z, g0); g1 = fmaf(x[t].w, y[t].w, g1);
+                            }
+                            float a = a0 + a1, b = b0 + b1, g = g0 + g1;
+#pragma unroll
+                            for (int o = 4; o > 0; o >>= 1) {
+                                a += __shfl_xor_sync(0xffffffffu, a, o);
+                                b += __shfl_xor_sync(0xffffffffu, b, o);
+                                g += __shfl_xor_sync(0xffffffffu, g, o);
+                            }
+                            const float ab = a * b, g2 = g * g;
+                            if (valid && ab > 0.f && g2 > 1e-12f * ab) {
+                                worst2 = fmaxf(worst2, __fdividef(g2, ab));
+                                const float zeta = __fdividef(b - a, 2.f * g);
+                                const float tt = copysignf(__fdividef(1.f, fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.f))), zeta);
+                                const float c = rsqrtf(fmaf(tt, tt, 1.f));
+                                const float s = c * tt;
+#pragma unroll
+                                for (int t = 0; t < Q; ++t) {
+                                    float4 nx, ny;
+                                    nx.x = fmaf(-s, y[t].x, c * x[t].x); ny.x = fmaf(s, x[t].x, c * y[t].x);
+                                    nx.y = fmaf(-s, y[t].y, c * x[t].y); ny.y = fmaf(s, x[t].y, c * y[t].y);
+                                    nx.z = fmaf(-s, y[t].z, c * x[t].z); ny.z = fmaf(s, x[t].z, c * y[t].z);
+                                    nx.w = fmaf(-s, y[t].w, c * x[t].w); ny.w = fmaf(s, x[t].w, c * y[t].w);
+                                    x[t] = nx;
+                                    y[t] = ny;
+                                }
+                            }
+                            if (r < 3) {                          // quarter qd takes over the column quarter qd + 1 holds
+                                const int src = (lane + 8) & 31;
+#pragma unroll
+                                for (int t = 0; t < Q; ++t) {
+                                    y[t].x = __shfl_sync(0xffffffffu, y[t].x, src);
+                                    y[t].y = __shfl_sync(0xffffffffu, y[t].y, src);
+                                    y[t].z = __shfl_sync(0xffffffffu, y[t].z, src);
+                                    y[t].w = __shfl_sync(0xffffffffu, y[t].w, src);
+                                }
+                            }
+                        }
+                        const int pl = 4 * hi + ((qd + 3) & 3);   // the hi column this quarter ends up with
+                        if (va) {
+#pragma unroll
+                            for (int t = 0; t < Q; ++t) xa[8 * t] = x[t];
+                        }
+                        if (pl < rank) {
+                            float4* xl = reinterpret_cast<float4*>(X + perm[pl] * LD) + l8;
+#pragma unroll
+                            for (int t = 0; t < Q; ++t) xl[8 * t] = y[t];
+                        }
+                        __syncwarp();
+                    }
+                  }
+                    cluster.sync();
+                }
+                ++sweeps;
+                const int par = sweeps & 1;
+                if (__any_sync(0xffffffffu, worst2 > 9e-8f) && lane == 0) atomicOr(&gflag[par], 1);
+                if (gtid == 0) gflag[par ^ 1] = 0;
+                cluster.sync();
+                more = __ldcg(&gflag[par]);
+                if (!more) break;               // every cosine of this sweep was below 3e-4: converged after it
+            }
+            if (tid == 0) { sh_f[1] = (float)sweeps; sh_f[4] = more ? 1.f : 0.f; }
+        }
+    }
+    __syncthreads();
+    sweeps = rank >= 2 ? (int)sh_f[1] : 0;
+    const int not_converged = rank >= 2 && sh_f[4] != 0.f;     // stopped at the sweep limit while still rotating visibly
+
+    // ---- eigenvalues = squared column norms (pivot-step order), scaled back; sort descending, stable ----
+    for (int k = lwarp; k < n; k += 8) {                          // every CTA forms all eigenvalues for its own tables
+        float a = 0.f;
+        if (k < rank) {
+            const float* x = X + perm[k] * LD;
+#pragma unroll
+            for (int t = 0; t < R; ++t) { const float xv = __ldcg(x + lane + 32 * t); a = fmaf(xv, xv, a); }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+        }
+        if (lane == 0) lam[k] = a * dmax;
+    }
+    __syncthreads();
+    for (int t = tid; t < n; t += NT) {
+        const float mine = lam[t];
+        int pos = 0;
+        for (int i = 0; i < n; ++i) {
+            const float o = lam[i];
+            pos += (o > mine) || (o == mine && i < t);
+        }
+        order[pos] = t;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        float delta = 0.f;
+        if (do_shrink && delta_rank - 1 < n) delta = lam[order[delta_rank - 1]];
+        sh_f[0] = delta;
+        if (crank == 0) {
+            info->delta = delta;
+            info->sweeps = sweeps;
+            if (sweeps > info->max_sweeps) info->max_sweeps = sweeps;
+            info->rank = rank;
+            if (not_converged) info->flags |= kFlagNotConverged;
+            if (do_shrink) {
+                info->sum_delta += (double)delta;
+                info->shrinks += 1;
+            }
+        }
+    }
+    __syncthreads();
+    const float delta = sh_f[0];
+    const float back = sqrtf(dmax);     // columns of X are sigma_j u_j / sqrt(dmax)
+    for (int t = tid; t < n; t += NT) {
+        const float l = lam[order[t]];
+        float f = 0.f, sp = 0.f;
+        if (l > 0.f && t < keep) {
+            const float kept = fmaxf(l - delta, 0.f);
+            sp = sqrtf(kept);
+            f = sqrtf(kept / l) * rsqrtf(l) * back;   // (sigma'/sigma) / sigma, for the unscaled column
+        }
+        fac[t] = f;
+        if (t < n_sigma && crank == 0) sigma_out[t] = sp;
+    }
+    if (crank == 0)
+        for (int j = n + tid; j < n_sigma; j += NT) sigma_out[j] = 0.f;
+    __syncthreads();
+    for (int e = gtid; e < n * keep; e += GT) {
+        const int j = e / n, i = e - j * n;
+        float v = 0.f;
+        if (j < n) {
+            const int k = order[j];
+            if (k < rank) v = __ldcg(X + perm[k] * LD + i) * fac[j];
+        }
+        Ur[(size_t)i * ldu + j] = v;
+    }
+    if (Wsplit) {   // the same factors transposed and split for the tensor-core rebuild: [W_hi ; W_lo], zero padded
+        for (int e = gtid; e < j_pad * ldw; e += GT) {
+            const int j = e / ldw, i = e - j * ldw;
+            float v = 0.f;
+            if (j < keep && j < n && i < n) {
+                const int k = order[j];
+                if (k < rank) v = __ldcg(X + perm[k] * LD + i) * fac[j];
+            }
+            const float hi = __uint_as_float((__float_as_uint(v) + 0x1000u) & 0xffffe000u);
+            Wsplit[(size_t)j * ldw + i] = hi;
+            Wsplit[(size_t)(j_pad + j) * ldw + i] = v - hi;
+        }
+    }
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 k_eig_shrink(const float* __restrict__ K, int ldk, int n, int do_shrink, int delta_rank, int keep, float* __restrict__ Ur,
              int ldu, float* __restrict__ sigma_out, int n_sigma, float* __restrict__ work, int use_smem, int max_sweeps,
@@ -648,20 +1024,40 @@ cudaError_t launch_eig_shrink(const float* K, int ldk, int n, int do_shrink, int
                               float* sigma_out, int n_sigma, float* work, int max_sweeps, EigInfo* info, float* Wsplit, int ldw,
                               int j_pad, cudaStream_t st) {
     if (n <= 0 || n > 512) return cudaErrorInvalidValue;
-    if (n <= kMaxN) {
+    if (n <= kMaxFast) {
         const int T = (n + 63) / 64;
         const size_t aux_bytes = 3 * kMaxN * sizeof(float) + 3 * kMaxN * sizeof(int) + 32;
-        const size_t bytes = (T <= 3 ? (size_t)(64 * T) * (64 * T) * sizeof(float) : 0) + aux_bytes;
+        const size_t bytes = (size_t)(64 * T) * (64 * T) * sizeof(float) + aux_bytes;
         cudaError_t e;
-#define SAGE_EIG_FAST(TT, NTT, GG)                                                                                     \
-    e = cudaFuncSetAttribute(k_eig_shrink_fast<TT, NTT, GG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes); \
+#define SAGE_EIG_FAST(TT)                                                                                              \
+    e = cudaFuncSetAttribute(k_eig_shrink_fast<TT, 1024, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes); \
     if (e != cudaSuccess) return e;                                                                                    \
-    k_eig_shrink_fast<TT, NTT, GG><<<1, NTT, bytes, st>>>(K, ldk, n, do_shrink, delta_rank, keep, Ur, ldu, sigma_out, n_sigma, \
-                                                          max_sweeps, info, Wsplit, ldw, j_pad, work);
-        if (T == 1) { SAGE_EIG_FAST(1, 1024, false) } else if (T == 2) { SAGE_EIG_FAST(2, 1024, false) }
-        else if (T == 3) { SAGE_EIG_FAST(3, 1024, false) } else { SAGE_EIG_FAST(4, 512, true) }   // work: >= 256 x 256 floats
+    k_eig_shrink_fast<TT, 1024, false><<<1, 1024, bytes, st>>>(K, ldk, n, do_shrink, delta_rank, keep, Ur, ldu, sigma_out,  \
+                                                               n_sigma, max_sweeps, info, Wsplit, ldw, j_pad, work);
+        if (T == 1) { SAGE_EIG_FAST(1) } else if (T == 2) { SAGE_EIG_FAST(2) } else { SAGE_EIG_FAST(3) }
 #undef SAGE_EIG_FAST
         return cudaGetLastError();
+    }
+    {   // thread-block cluster, matrix in `work` (>= 512*512 + 64 floats when n > 256, else >= 256*256 + 64)
+        const size_t bytes = 3 * 512 * sizeof(float) + 3 * 512 * sizeof(int) + 32;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(8);
+        cfg.blockDim = dim3(256);
+        cfg.dynamicSmemBytes = bytes;
+        cfg.stream = st;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 8;
+        at[0].val.clusterDim.y = 1;
+        at[0].val.clusterDim.z = 1;
+        cfg.attrs = at;
+        cfg.numAttrs = 1;
+        cudaError_t e = n <= 256 ? cudaLaunchKernelEx(&cfg, k_eig_shrink_cluster<4>, K, ldk, n, do_shrink, delta_rank, keep, Ur, ldu,
+                                                      sigma_out, n_sigma, max_sweeps, info, Wsplit, ldw, j_pad, work)
+                                 : cudaLaunchKernelEx(&cfg, k_eig_shrink_cluster<8>, K, ldk, n, do_shrink, delta_rank, keep, Ur, ldu,
+                                                      sigma_out, n_sigma, max_sweeps, info, Wsplit, ldw, j_pad, work);
+        if (e == cudaSuccess) return cudaGetLastError();
+        (void)cudaGetLastError();          // no cluster launch on this device: the one-CTA kernel below serves n <= 512
     }
     const size_t aux = (4 * 512 + 2 * kWarps + 8) * sizeof(float);
     const size_t xbytes = (size_t)n * n * sizeof(float);

@@ -80,7 +80,8 @@ cudaError_t launch_rebuild(const float* Ur, int ldu, const float* Bsrc, float* B
 // matrix has fewer eigenvalues), keep = delta_rank-1 columns. do_shrink == 0: delta = 0, keep columns.
 // Writes Ur[i*ldu + j] = U[i][j] * sqrt(max(1 - delta/lambda_j, 0)) for j < keep (eigenvalues descending),
 // sigma_out[j] = sqrt(max(lambda_j - delta, 0)) for j < n_sigma, and updates *info.
-// `work` is scratch of at least max(n*n, 256*256) floats (used when the matrix does not fit in shared memory).
+// `work` is scratch of at least 256*256 + 64 floats (512*512 + 64 when n > 256), used when the matrix does not fit in
+// shared memory.
 // Wsplit != nullptr: also writes the factors transposed and split for launch_tc_rebuild, rows [0, j_pad) =
 // W rounded to 11 significant bits and rows [j_pad, 2 j_pad) = the remainders, W[j][i] = Ur[i][j], pitch ldw >= n,
 // zero outside j < keep, i < n.
