@@ -60,8 +60,8 @@ __device__ __forceinline__ void rr_pair(int n_even, int round, int slot, int& p,
 //   * one-sided Jacobi with one pair per QUARTER-warp: 8 lanes hold both columns in registers (float4
 //     accesses, conflict-free), reduce the three dot products with 3 shuffle steps and rotate; warps
 //     without a pair only take part in the barrier;
-//   * a sweep whose largest pre-rotation cosine is below 3e-4 ends the iteration (the next sweep
-//     would find cosines near 1e-7, below the rotation threshold).
+//   * a sweep whose largest pre-rotation cosine is below 1e-3 ends the iteration (the next sweep
+//     would find cosines near 1e-6, the rotation threshold).
 // X is column-major with a row pitch of LD = 64*T floats; column c of the factor stays at the physical
 // position of the c-th pivot, so the rows of U come out in the original buffer order.
 // ------------------------------------------------------------------------------------------------
@@ -332,11 +332,11 @@ k_eig_shrink_fast(const float* __restrict__ K, int ldk, int n, int do_shrink, in
                 }
                 ++sweeps;
                 const int par = sweeps & 1;
-                if (__any_sync(0xffffffffu, worst2 > 9e-8f) && lane == 0) atomicOr(&sh_flag[par], 1);
+                if (__any_sync(0xffffffffu, worst2 > 1e-6f) && lane == 0) atomicOr(&sh_flag[par], 1);
                 if (tid == 0) sh_flag[par ^ 1] = 0;
                 asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
                 more = sh_flag[par];
-                if (!more) break;               // every cosine of this sweep was below 3e-4: converged after it
+                if (!more) break;               // every cosine of this sweep was below 1e-3: converged after it
             }
             if (tid == 0) { sh_f[1] = (float)sweeps; sh_f[4] = more ? 1.f : 0.f; }
         }
@@ -701,11 +701,11 @@ k_eig_shrink_cluster(const float* __restrict__ K, int ldk, int n, int do_shrink,
                 }
                 ++sweeps;
                 const int par = sweeps & 1;
-                if (__any_sync(0xffffffffu, worst2 > 9e-8f) && lane == 0) atomicOr(&gflag[par], 1);
+                if (__any_sync(0xffffffffu, worst2 > 1e-6f) && lane == 0) atomicOr(&gflag[par], 1);
                 if (gtid == 0) gflag[par ^ 1] = 0;
                 cluster.sync();
                 more = __ldcg(&gflag[par]);
-                if (!more) break;               // every cosine of this sweep was below 3e-4: converged after it
+                if (!more) break;               // every cosine of this sweep was below 1e-3: converged after it
             }
             if (tid == 0) { sh_f[1] = (float)sweeps; sh_f[4] = more ? 1.f : 0.f; }
         }
