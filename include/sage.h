@@ -129,6 +129,32 @@ int64_t sage_select_count(int64_t N, double keep_rate);
 sage_status_t sage_select(const float* scores, int64_t N, double keep_rate, int64_t* idx, int64_t* k_out,
                           void* cuda_stream);
 
+/* Class-balanced variant (Algorithm 1, branch "class balance required"; "Agreement Scoring and Selection"): after a
+ * finished scoring pass on this handle (sage_score or sage_score_end over N rows), replace the consensus u by the
+ * per-class unit centroids u_c = zbar_c / ||zbar_c||, zbar_c the mean of zhat_i over the examples of class c (u_c = 0
+ * when that mean is zero), and score every example against the centroid of its own class.
+ *   labels       device, N int32 class ids of the rows of that pass, in the same order; ids outside
+ *                [0, num_classes) take no part: such examples score 0.
+ *   num_classes  1 .. 65535.
+ *   scores       device, N floats.
+ * Asynchronous on the stream (the first call with a larger num_classes allocates and synchronises). */
+sage_status_t sage_score_classes(sage_fd_t* h, const int32_t* labels, int32_t num_classes, float* scores, void* cuda_stream);
+
+/* Borrowed device pointers to the result of the last sage_score_classes: U num_classes x ell fp32 unit centroids,
+ * counts num_classes int32 class sizes. Any out-pointer may be NULL. */
+sage_status_t sage_score_class_centroids(const sage_fd_t* h, const float** U, const int32_t** counts, int32_t* num_classes);
+
+/* Algorithm 1, "Select top-k_c per class (sum_c k_c = k)". The paper fixes only the sum; here
+ * k = sage_select_count(N_valid, keep_rate) with N_valid the number of examples whose label lies in [0, num_classes),
+ * and k_c is proportional to the class size n_c with largest-remainder rounding: k_c = floor(k n_c / N_valid), the
+ * k - sum floor(.) classes with the largest remainders (ties: smaller class id) get one more. Inside a class the order
+ * is (score descending, index ascending); idx lists the picks of class 0, then class 1, ...
+ *   scores, labels  device, N floats / N int32.      idx  device, capacity >= k int64.
+ *   k_per_class     host, num_classes values (may be NULL).      k_out  host (may be NULL).
+ * Synchronises the stream (class sizes are read back to derive k_c); allocates O(N) scratch from the stream-ordered pool. */
+sage_status_t sage_select_classes(const float* scores, const int32_t* labels, int64_t N, int32_t num_classes, double keep_rate,
+                                  int64_t* idx, int64_t* k_per_class, int64_t* k_out, void* cuda_stream);
+
 /* Selection without any allocation (the paper has no counterpart; this is a packaging variant of
  * sage_select with identical results). For callers that cannot allocate device memory at call time:
  * code running inside a loop whose memory was handed out once at start-up by a pool it does not own,

@@ -39,6 +39,9 @@ SIGNATURES = {
     "sage_score_intermediates": (_i32, [_vp, _vp, _vp, _vp]),
     "sage_select_count": (_i64, [_i64, _f64]),
     "sage_select": (_i32, [_vp, _i64, _f64, _vp, _vp, _vp]),
+    "sage_score_classes": (_i32, [_vp, _vp, _i32, _vp, _vp]),
+    "sage_score_class_centroids": (_i32, [_vp, _vp, _vp, _vp]),
+    "sage_select_classes": (_i32, [_vp, _vp, _i64, _i32, _f64, _vp, _vp, _vp, _vp]),
     "sage_select_static": (_i32, [_vp, _i64, _f64, _vp, _vp, _vp]),
     "sage_select_from_host": (_i32, [_vp, _i64, _i64, _i64, _i32, _i32, _f64, _i64, _i32, _vp, _vp, _vp]),
     "sage_fd_stats": (_i32, [_vp, _vp]),
@@ -190,6 +193,33 @@ def sage_select(scores: torch.Tensor, keep_rate: float, idx: Optional[torch.Tens
     return idx[: k_out.value]
 
 
+def sage_score_classes(h: int, labels: torch.Tensor, num_classes: int, scores: torch.Tensor) -> None:
+    assert labels.dtype == torch.int32 and labels.is_contiguous() and scores.dtype == torch.float32 and scores.is_contiguous()
+    assert labels.numel() == scores.numel()
+    _check(lib().sage_score_classes(h, labels.data_ptr(), num_classes, scores.data_ptr(), _stream(scores.device)))
+
+
+def sage_score_class_centroids(h: int, ell: int, device) -> Tuple[torch.Tensor, torch.Tensor]:
+    U, cnt, C_ = _vp(), _vp(), _i32(0)
+    _check(lib().sage_score_class_centroids(h, C.byref(U), C.byref(cnt), C.byref(C_)))
+    nc = C_.value
+    Ut = _borrow(U.value, (nc, ell), (ell * 4, 4), device).clone()
+    ct = torch.as_tensor(_DevArray(cnt.value, (nc,), (4,), "<i4"), device=device).clone()
+    return Ut, ct
+
+
+def sage_select_classes(scores: torch.Tensor, labels: torch.Tensor, num_classes: int, keep_rate: float):
+    """Returns (idx on the device, list of k_c)."""
+    assert scores.dtype == torch.float32 and scores.is_contiguous() and labels.dtype == torch.int32 and labels.is_contiguous()
+    N = scores.numel()
+    idx = torch.empty((max(sage_select_count(N, keep_rate), 1),), dtype=torch.int64, device=scores.device)
+    kc = (C.c_int64 * num_classes)()
+    k_out = _i64(0)
+    _check(lib().sage_select_classes(scores.data_ptr(), labels.data_ptr(), N, num_classes, keep_rate, idx.data_ptr(), kc,
+                                     C.byref(k_out), _stream(scores.device)))
+    return idx[: k_out.value], [int(v) for v in kc]
+
+
 def sage_select_static(scores: torch.Tensor, keep_rate: float, idx: torch.Tensor) -> torch.Tensor:
     """sage_select for callers that cannot allocate: the caller passes ``idx`` (capacity >= k) and the
     library uses its built-in scratch (N <= 262,144). Runs on the current device, current stream."""
@@ -292,6 +322,15 @@ class SageFD:
 
     def score_end(self, scores: torch.Tensor) -> None:
         sage_score_end(self._h, scores)
+
+    def score_classes(self, labels: torch.Tensor, num_classes: int, scores: Optional[torch.Tensor] = None) -> torch.Tensor:
+        if scores is None:
+            scores = torch.empty((labels.numel(),), dtype=torch.float32, device=labels.device)
+        sage_score_classes(self._h, labels, num_classes, scores)
+        return scores
+
+    def class_centroids(self):
+        return sage_score_class_centroids(self._h, self.ell, torch.device("cuda", self.device))
 
     def intermediates(self, N: int):
         return sage_score_intermediates(self._h, N, self.ell, torch.device("cuda", self.device))

@@ -1,6 +1,7 @@
 // Host orchestration behind the C ABI: state machine, buffer management and the launch sequences of
 // pass 1 (append -> Gram -> eigen/shrink -> rebuild), freeze, pass 2 (project -> normalise -> consensus
 // -> score) and selection. No device->host synchronisation happens inside sage_fd_update.
+#include <algorithm>
 #include <atomic>
 #include <cmath>
 #include <cstdarg>
@@ -106,6 +107,10 @@ struct sage_fd {
     size_t partials_bytes = 0;
     double* zsum = nullptr;
     float* u = nullptr;
+    bool scored = false;           // a scoring pass over N_total rows has finished: zhat holds their normalised projections
+    float* class_U = nullptr;      // class-balanced variant: unit centroids (class_cap x ell) and class sizes
+    int* class_counts = nullptr;
+    int class_cap = 0, class_num = 0;
     __nv_bfloat16* P16 = nullptr;  // frozen sketch in bf16 (bf16 handles: tensor-core projection operand); with p16_fold
                                    // rows [0, ell) hold bf16(S) and rows [n_pad, n_pad + ell) hold bf16(S - bf16(S))
     int p16_fold = 0, p16_npad = 0;
@@ -405,6 +410,8 @@ void sage_fd_destroy(sage_fd_t* h) {
     cudaFree(h->partials);
     cudaFree(h->zsum);
     cudaFree(h->u);
+    cudaFree(h->class_U);
+    cudaFree(h->class_counts);
     cudaFree(h->P16);
     cudaFree(h->tc_err);
     if (h->side) cudaStreamDestroy(h->side);
@@ -428,6 +435,7 @@ sage_status_t sage_fd_reset(sage_fd_t* h) {
     h->fill = 0;
     h->rows_seen = 0;
     h->cur = 0;
+    h->scored = false;
     h->state = SKETCHING;
     h->launches = 0;
     return SAGE_OK;
@@ -576,6 +584,7 @@ sage_status_t sage_fd_load_sketch(sage_fd_t* h, const float* S, int64_t ld, void
     CU_TRY(cudaMemsetAsync(h->sigma, 0, h->ell * sizeof(float), st));
     ST_TRY(enqueue_freeze_aux(h, st));
     h->fill = h->ell;
+    h->scored = false;
     h->state = FROZEN;
     return SAGE_OK;
 }
@@ -605,6 +614,7 @@ sage_status_t sage_score_begin(sage_fd_t* h, int64_t N_total, void* cuda_stream)
     CU_TRY(cudaMemsetAsync(h->zsum, 0, 256 * sizeof(double), st));
     h->N_total = N_total;
     h->next_row = 0;
+    h->scored = false;
     h->state = SCORING;
     return SAGE_OK;
 }
@@ -733,6 +743,7 @@ sage_status_t sage_score_end(sage_fd_t* h, float* scores, void* cuda_stream) {
     DeviceGuard g(h->device);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     CU_TRY(timed(h, K_SCORE, 1, st, [&] { return launch_consensus_score(h->zsum, h->zhat, h->N_total, h->ell, h->u, scores, st); }));
+    h->scored = true;
     h->state = FROZEN;
     return SAGE_OK;
 }
@@ -785,6 +796,121 @@ sage_status_t sage_select(const float* scores, int64_t N, double keep_rate, int6
         while (idx_bits < 32 && (1ll << idx_bits) < N) ++idx_bits;
         count(nullptr, 2 + 3 * (4 + (idx_bits + 7) / 8));
     }
+    if (k_out) *k_out = k;
+    return SAGE_OK;
+}
+
+sage_status_t sage_score_classes(sage_fd_t* h, const int32_t* labels, int32_t num_classes, float* scores, void* cuda_stream) {
+    ST_TRY(check_handle(h));
+    if (h->state != FROZEN || !h->scored) {
+        set_err("sage_score_classes: needs a finished scoring pass (sage_score or sage_score_end) on this handle");
+        return SAGE_ERR_BAD_STATE;
+    }
+    if (num_classes < 1 || num_classes > 65535 || (h->N_total > 0 && (!labels || !scores))) {
+        set_err("sage_score_classes: bad argument (num_classes=%d labels=%p scores=%p)", (int)num_classes, (const void*)labels, (void*)scores);
+        return SAGE_ERR_INVALID_ARG;
+    }
+    DeviceGuard g(h->device);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (num_classes > h->class_cap) {
+        CU_TRY(cudaStreamSynchronize(st));
+        if (h->class_U) CU_TRY(cudaFree(h->class_U));
+        if (h->class_counts) CU_TRY(cudaFree(h->class_counts));
+        h->class_U = nullptr;
+        h->class_counts = nullptr;
+        h->class_cap = 0;
+        CU_TRY(cudaMalloc((void**)&h->class_U, (size_t)num_classes * h->ell * sizeof(float)));
+        CU_TRY(cudaMalloc((void**)&h->class_counts, (size_t)num_classes * sizeof(int)));
+        h->class_cap = num_classes;
+    }
+    h->class_num = num_classes;
+    CU_TRY(launch_class_scores(h->zhat, labels, h->N_total, h->ell, num_classes, h->class_U, h->class_counts, scores, st));
+    count(h, h->N_total > 0 ? 2 : 1);
+    return SAGE_OK;
+}
+
+sage_status_t sage_score_class_centroids(const sage_fd_t* h, const float** U, const int32_t** counts, int32_t* num_classes) {
+    ST_TRY(check_handle(h));
+    if (!h->class_U || h->class_num == 0) {
+        set_err("sage_score_class_centroids: sage_score_classes has not run on this handle");
+        return SAGE_ERR_BAD_STATE;
+    }
+    if (U) *U = h->class_U;
+    if (counts) *counts = h->class_counts;
+    if (num_classes) *num_classes = h->class_num;
+    return SAGE_OK;
+}
+
+sage_status_t sage_select_classes(const float* scores, const int32_t* labels, int64_t N, int32_t num_classes, double keep_rate,
+                                  int64_t* idx, int64_t* k_per_class, int64_t* k_out, void* cuda_stream) {
+    if (N < 0 || N >= (1ll << 31) || !(keep_rate == keep_rate) || num_classes < 1 || num_classes > 65535 || (N > 0 && (!scores || !labels))) {
+        set_err("sage_select_classes: bad argument (N=%lld num_classes=%d keep_rate=%g)", (long long)N, (int)num_classes, keep_rate);
+        return SAGE_ERR_INVALID_ARG;
+    }
+    const int C = num_classes;
+    std::vector<long long> kc(C, 0), offs(C, 0);
+    long long k = 0;
+    if (N > 0) {
+        cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+        size_t sel_bytes = 0;
+        select_scratch_bytes(N, &sel_bytes);
+        const size_t a256 = 255;
+        const size_t sorted_off = (sel_bytes + a256) & ~a256;
+        const size_t counts_off = (sorted_off + (size_t)N * 8 + a256) & ~a256;
+        const size_t kc_off = (counts_off + (size_t)C * 4 + a256) & ~a256;
+        const size_t offs_off = (kc_off + (size_t)C * 8 + a256) & ~a256;
+        const size_t total = offs_off + (size_t)C * 8;
+        char* scratch = nullptr;
+        CU_TRY(cudaMallocAsync((void**)&scratch, total, st));
+        auto body = [&]() -> sage_status_t {
+            int* d_counts = reinterpret_cast<int*>(scratch + counts_off);
+            CU_TRY(launch_class_count(labels, N, C, d_counts, st));
+            std::vector<int> counts(C);
+            CU_TRY(cudaMemcpyAsync(counts.data(), d_counts, (size_t)C * sizeof(int), cudaMemcpyDeviceToHost, st));
+            CU_TRY(cudaStreamSynchronize(st));
+            long long n_valid = 0;
+            for (int c = 0; c < C; ++c) n_valid += counts[c];
+            k = sage_select_count(n_valid, keep_rate);
+            // k_c proportional to the class sizes, largest remainder, ties to the smaller class (exact integers)
+            std::vector<long long> rem(C, 0);
+            long long given = 0;
+            if (n_valid > 0)
+                for (int c = 0; c < C; ++c) {
+                    const long long num = (long long)counts[c] * k;
+                    kc[c] = num / n_valid;
+                    rem[c] = num - kc[c] * n_valid;
+                    given += kc[c];
+                }
+            std::vector<int> order(C);
+            for (int c = 0; c < C; ++c) order[c] = c;
+            std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return rem[a] > rem[b]; });
+            for (long long t = 0; t < k - given; ++t) kc[order[(size_t)t]] += 1;
+            long long run = 0;
+            for (int c = 0; c < C; ++c) { offs[c] = run; run += kc[c]; }
+            if (k > 0 && !idx) {
+                set_err("sage_select_classes: null idx");
+                return SAGE_ERR_INVALID_ARG;
+            }
+            if (k > 0) {
+                CU_TRY(cudaMemcpyAsync(scratch + kc_off, kc.data(), (size_t)C * 8, cudaMemcpyHostToDevice, st));
+                CU_TRY(cudaMemcpyAsync(scratch + offs_off, offs.data(), (size_t)C * 8, cudaMemcpyHostToDevice, st));
+                int64_t* sorted = reinterpret_cast<int64_t*>(scratch + sorted_off);
+                CU_TRY(launch_select(scores, N, N, sorted, scratch, st));
+                CU_TRY(launch_class_pick(sorted, labels, N, C, reinterpret_cast<const long long*>(scratch + kc_off),
+                                         reinterpret_cast<const long long*>(scratch + offs_off), idx, st));
+                CU_TRY(cudaStreamSynchronize(st));        // kc / offs are host vectors of this call
+                int idx_bits = 1;
+                while (idx_bits < 32 && (1ll << idx_bits) < N) ++idx_bits;
+                count(nullptr, 3 + 3 * (4 + (idx_bits + 7) / 8) + 2);
+            }
+            return SAGE_OK;
+        };
+        const sage_status_t rc = body();
+        cudaFreeAsync(scratch, st);
+        if (rc != SAGE_OK) return rc;
+    }
+    if (k_per_class)
+        for (int c = 0; c < C; ++c) k_per_class[c] = kc[c];
     if (k_out) *k_out = k;
     return SAGE_OK;
 }

@@ -98,6 +98,15 @@ cudaError_t launch_normalise(const float* Z, int64_t ldz, int64_t n, int ell, fl
 cudaError_t launch_consensus_score(const double* zsum, const float* zhat, int64_t N, int ell, float* u, float* scores,
                                    cudaStream_t st);
 
+// Class-balanced variant. U (C x ell) receives the unit centroids, counts (C) the class sizes, scores (N) the
+// per-class agreement scores; labels outside [0, C) score 0.
+cudaError_t launch_class_scores(const float* zhat, const int* labels, int64_t N, int ell, int C, float* U, int* counts, float* scores,
+                                cudaStream_t st);
+cudaError_t launch_class_count(const int* labels, int64_t N, int C, int* counts, cudaStream_t st);
+// out[offs[c] + r] = the r-th example of class c in the order of `sorted` (all N examples, best first), r < kc[c].
+cudaError_t launch_class_pick(const int64_t* sorted, const int* labels, int64_t N, int C, const long long* kc, const long long* offs,
+                              int64_t* out, cudaStream_t st);
+
 // Top-k by (score desc, index asc). keys/vals scratch: see select.cu. Returns through idx (device).
 cudaError_t select_scratch_bytes(int64_t N, size_t* bytes);
 cudaError_t launch_select(const float* scores, int64_t N, int64_t k, int64_t* idx, void* scratch, cudaStream_t st);
