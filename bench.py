@@ -317,10 +317,11 @@ def main():
     dom_launches_per_step = prof_dom["launches"] / args.steps
     if dominant == "eig_shrink":
         achieved = eig_flops / (dom_ms_per_step * 1e-3) / 1e12
-        roof = {"kernel": "k_eig_shrink", "bound": "alu", "achieved": achieved, "peak": FP32_ALU_PEAK_TFLOPS, "unit": "TFLOP/s",
+        roof = {"kernel": "k_eig_shrink_fast" if 2 * ell <= 192 else "k_eig_shrink_cluster", "bound": "alu", "achieved": achieved, "peak": FP32_ALU_PEAK_TFLOPS, "unit": "TFLOP/s",
                 "frac": achieved / FP32_ALU_PEAK_TFLOPS, "traffic": None,
                 "peak_source": "derived: 148 SMs x 128 fp32 FMA lanes x 2 flop x 1.965 GHz",
-                "algorithmic": "9*n^3 flop per n x n symmetric eigen-solve (textbook count)"}
+                "algorithmic": "9*n^3 flop per n x n symmetric eigen-solve (textbook count)",
+                "frac_of_the_sms_it_runs_on": achieved / (FP32_ALU_PEAK_TFLOPS * (1 if 2 * ell <= 192 else 8) / 148.0)}
     else:
         gbs = per_step_bytes.get(dominant, 0) / (dom_ms_per_step * 1e-3) / 1e9
         roof = {"kernel": dominant, "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -340,6 +341,28 @@ def main():
     roof_pass2_s = max(N * D * e / (peaks["hbm_gbs"] * 1e9), 2.0 * N * ell * D / (peaks["bf16_tflops_sustained"] * 1e12))
     p1_bytes = per_step_bytes["append"] + per_step_bytes["gram"] + per_step_bytes["rebuild"]
     roof_pass1_s = p1_bytes / (peaks["hbm_gbs"] * 1e9)
+
+    # ---- class-balanced variant on the scores of the last step (reported beside the step, not part of it) ----
+    cb_info = None
+    try:
+        C_cls = {"c1": 16, "c2": 10, "c3": 100, "c4": 64, "c5": 10}[w.name]
+        gcb = torch.Generator(device=dev)
+        gcb.manual_seed(1234)
+        labels = torch.randint(0, C_cls, (N,), generator=gcb, device=dev, dtype=torch.int32)
+        cb_scores = torch.empty((N,), dtype=torch.float32, device=dev)
+        c0, c1 = ev(), ev()
+        fd.score_classes(labels, C_cls, cb_scores)
+        sage.sage_select_classes(cb_scores, labels, C_cls, w.keep_rates[0])
+        torch.cuda.synchronize()
+        c0.record()
+        for _ in range(3):
+            fd.score_classes(labels, C_cls, cb_scores)
+            sage.sage_select_classes(cb_scores, labels, C_cls, w.keep_rates[0])
+        c1.record()
+        torch.cuda.synchronize()
+        cb_info = {"classes": C_cls, "labels": "uniform random (synthetic)", "ms_score_and_select": c0.elapsed_time(c1) / 3}
+    except Exception as exc:       # the variant needs a finished scoring pass on the handle
+        cb_info = {"error": str(exc)}
 
     # ---- end to end through the host-pointer entry point ------------------------------------------------
     e2e = None
@@ -390,7 +413,7 @@ def main():
                        "pass1_stream_frac_of_hbm_roofline": (roof_pass1_s * 1e3) / max(1e-9, sum(prof_all[k]["ms"] for k in ("append", "gram", "gram_reduce", "rebuild"))),
                        "note": "generator time of streamed workloads is excluded from the pass times; *_stream_* figures are "
                                "CUDA-event sums over the streaming kernels of the profiled warm-up step (eigen-solves apart)"},
-            "roofline": roof, "kernels_profiled_step": kernels,
+            "roofline": roof, "kernels_profiled_step": kernels, "class_balanced": cb_info,
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
             "clocks": clocks, "fd_stats": {k: stats[k] for k in ("shrinks", "max_sweeps", "last_rank", "device_flags")},
         }

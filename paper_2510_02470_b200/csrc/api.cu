@@ -7,6 +7,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -74,6 +75,36 @@ struct Prof {
 };
 
 size_t elem_size(sage_dtype_t dt) { return dt == SAGE_F32 ? 4 : 2; }
+
+// Stream-ordered scratch of the selection entry points comes from a pool of the library's own whose memory stays
+// cached across synchronisations (the device's default pool gives its memory back at every synchronisation, and
+// getting it again costs milliseconds). One pool per device, created on first use, kept until the process exits.
+cudaError_t scratch_alloc(void** p, size_t bytes, cudaStream_t st) {
+    static cudaMemPool_t pools[64] = {};
+    static std::mutex mu;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaMallocAsync(p, bytes, st);
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (!pools[dev]) {
+            cudaMemPoolProps props = {};
+            props.allocType = cudaMemAllocationTypePinned;
+            props.handleTypes = cudaMemHandleTypeNone;
+            props.location.type = cudaMemLocationTypeDevice;
+            props.location.id = dev;
+            cudaMemPool_t pool = nullptr;
+            e = cudaMemPoolCreate(&pool, &props);
+            if (e != cudaSuccess) return e;
+            unsigned long long keep = ~0ull;
+            e = cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
+            if (e != cudaSuccess) return e;
+            pools[dev] = pool;
+        }
+    }
+    return cudaMallocFromPoolAsync(p, bytes, pools[dev], st);
+}
 
 }  // namespace
 
@@ -787,7 +818,7 @@ sage_status_t sage_select(const float* scores, int64_t N, double keep_rate, int6
         size_t bytes = 0;
         select_scratch_bytes(N, &bytes);
         void* scratch = nullptr;
-        CU_TRY(cudaMallocAsync(&scratch, bytes, st));
+        CU_TRY(scratch_alloc(&scratch, bytes, st));
         cudaError_t e = launch_select(scores, N, k, idx, scratch, st);
         cudaError_t e2 = cudaFreeAsync(scratch, st);
         CU_TRY(e);
@@ -861,7 +892,7 @@ sage_status_t sage_select_classes(const float* scores, const int32_t* labels, in
         const size_t offs_off = (kc_off + (size_t)C * 8 + a256) & ~a256;
         const size_t total = offs_off + (size_t)C * 8;
         char* scratch = nullptr;
-        CU_TRY(cudaMallocAsync((void**)&scratch, total, st));
+        CU_TRY(scratch_alloc((void**)&scratch, total, st));
         auto body = [&]() -> sage_status_t {
             int* d_counts = reinterpret_cast<int*>(scratch + counts_off);
             CU_TRY(launch_class_count(labels, N, C, d_counts, st));
