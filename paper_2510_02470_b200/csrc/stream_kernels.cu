@@ -159,18 +159,26 @@ __global__ void __launch_bounds__(256) k_split_reduce(const float* __restrict__ 
     out[(int64_t)i * ldo + j] = (float)s;
 }
 
-// Split reduction of a Gram matrix computed in the two-MMA symmetric form: slice z left T_z = hi*hi^T + 2*hi*lo^T
-// at parts + z*stride; K = sum_z (T_z + T_z^T) / 2, ascending z, fp64.
-__global__ void __launch_bounds__(256) k_gram_sym_reduce(const float* __restrict__ parts, int splits, int64_t stride, int r,
-                                                         int64_t ldp, float* __restrict__ out, int64_t ldo) {
-    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= (int64_t)r * r) return;
-    const int i = (int)(e / r), j = (int)(e % r);
-    const float* a = parts + (int64_t)i * ldp + j;
-    const float* b = parts + (int64_t)j * ldp + i;
-    double s = 0.0;
-    for (int z = 0; z < splits; ++z) s += (double)a[(int64_t)z * stride] + (double)b[(int64_t)z * stride];
-    out[(int64_t)i * ldo + j] = (float)(0.5 * s);
+// Split reduction of a Gram matrix computed in the symmetric form: slice z left T_z = hi*hi^T + 2*hi*lo^T at
+// parts + z*stride; K = sum_z (T_z + T_z^T) / 2, ascending z, fp64. One block per 32 x 32 tile (I, J): thread
+// (ty, tx) sums T[I+ty][J+tx] and T[J+ty][I+tx] (both read along rows), the second is transposed through shared memory.
+__global__ void __launch_bounds__(1024) k_gram_sym_reduce(const float* __restrict__ parts, int splits, int64_t stride, int r,
+                                                          int64_t ldp, float* __restrict__ out, int64_t ldo) {
+    __shared__ double tr[32][33];
+    const int tx = threadIdx.x, ty = threadIdx.y;
+    const int i = blockIdx.y * 32 + ty, j = blockIdx.x * 32 + tx;          // direct element (i, j)
+    const int ti = blockIdx.x * 32 + ty, tj = blockIdx.y * 32 + tx;        // element (ti, tj) of the mirrored tile
+    double a = 0.0, b = 0.0;
+    const bool in_a = i < r && j < r, in_b = ti < r && tj < r;
+    const float* pa = parts + (int64_t)i * ldp + j;
+    const float* pb = parts + (int64_t)ti * ldp + tj;
+    for (int z = 0; z < splits; ++z) {
+        if (in_a) a += (double)pa[(int64_t)z * stride];
+        if (in_b) b += (double)pb[(int64_t)z * stride];
+    }
+    tr[ty][tx] = b;                                                        // b belongs to out[tj][ti] = out[i'][j'] with i' = I + tx
+    __syncthreads();
+    if (in_a) out[(int64_t)i * ldo + j] = (float)(0.5 * (a + tr[tx][ty]));
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -283,7 +291,8 @@ cudaError_t launch_split_reduce(const float* parts, int splits, int64_t split_st
 cudaError_t launch_gram_sym_reduce(const float* parts, int splits, int64_t stride, int r, int64_t ldp, float* out, int64_t ldo,
                                    cudaStream_t st) {
     if (r <= 0) return cudaSuccess;
-    k_gram_sym_reduce<<<(unsigned)(((int64_t)r * r + 255) / 256), 256, 0, st>>>(parts, splits, stride, r, ldp, out, ldo);
+    const unsigned t = (unsigned)((r + 31) / 32);
+    k_gram_sym_reduce<<<dim3(t, t), dim3(32, 32), 0, st>>>(parts, splits, stride, r, ldp, out, ldo);
     return cudaGetLastError();
 }
 
