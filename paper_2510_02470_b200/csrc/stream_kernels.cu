@@ -164,21 +164,30 @@ __global__ void __launch_bounds__(256) k_split_reduce(const float* __restrict__ 
 // (ty, tx) sums T[I+ty][J+tx] and T[J+ty][I+tx] (both read along rows), the second is transposed through shared memory.
 __global__ void __launch_bounds__(1024) k_gram_sym_reduce(const float* __restrict__ parts, int splits, int64_t stride, int r,
                                                           int64_t ldp, float* __restrict__ out, int64_t ldo) {
-    __shared__ double tr[32][33];
-    const int tx = threadIdx.x, ty = threadIdx.y;
-    const int i = blockIdx.y * 32 + ty, j = blockIdx.x * 32 + tx;          // direct element (i, j)
-    const int ti = blockIdx.x * 32 + ty, tj = blockIdx.y * 32 + tx;        // element (ti, tj) of the mirrored tile
+    // 16 x 16 outputs per block; the four z-layers of the block each sum a quarter of the partial matrices
+    // (several loads in flight per thread: the kernel is bound by load latency, not by bytes).
+    __shared__ double sa[4][16][17], sb[4][16][17];
+    const int tx = threadIdx.x, ty = threadIdx.y, tz = threadIdx.z;
+    const int i = blockIdx.y * 16 + ty, j = blockIdx.x * 16 + tx;          // direct element (i, j)
+    const int ti = blockIdx.x * 16 + ty, tj = blockIdx.y * 16 + tx;        // element (ti, tj) of the mirrored tile
     double a = 0.0, b = 0.0;
     const bool in_a = i < r && j < r, in_b = ti < r && tj < r;
-    const float* pa = parts + (int64_t)i * ldp + j;
-    const float* pb = parts + (int64_t)ti * ldp + tj;
-    for (int z = 0; z < splits; ++z) {
-        if (in_a) a += (double)pa[(int64_t)z * stride];
-        if (in_b) b += (double)pb[(int64_t)z * stride];
+    const float* pa = parts + (in_a ? (int64_t)i * ldp + j : 0);
+    const float* pb = parts + (in_b ? (int64_t)ti * ldp + tj : 0);
+#pragma unroll 4
+    for (int z = tz; z < splits; z += 4) {
+        const float va = pa[(int64_t)z * stride], vb = pb[(int64_t)z * stride];
+        a += (double)va;
+        b += (double)vb;
     }
-    tr[ty][tx] = b;                                                        // b belongs to out[tj][ti] = out[i'][j'] with i' = I + tx
+    sa[tz][ty][tx] = a;
+    sb[tz][ty][tx] = b;                                                    // belongs to out[I + tx'][J + ty'] after the transpose
     __syncthreads();
-    if (in_a) out[(int64_t)i * ldo + j] = (float)(0.5 * (a + tr[tx][ty]));
+    if (tz == 0 && in_a) {
+        const double sum_a = (sa[0][ty][tx] + sa[1][ty][tx]) + (sa[2][ty][tx] + sa[3][ty][tx]);
+        const double sum_b = (sb[0][tx][ty] + sb[1][tx][ty]) + (sb[2][tx][ty] + sb[3][tx][ty]);
+        out[(int64_t)i * ldo + j] = (float)(0.5 * (sum_a + sum_b));
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -291,8 +300,8 @@ cudaError_t launch_split_reduce(const float* parts, int splits, int64_t split_st
 cudaError_t launch_gram_sym_reduce(const float* parts, int splits, int64_t stride, int r, int64_t ldp, float* out, int64_t ldo,
                                    cudaStream_t st) {
     if (r <= 0) return cudaSuccess;
-    const unsigned t = (unsigned)((r + 31) / 32);
-    k_gram_sym_reduce<<<dim3(t, t), dim3(32, 32), 0, st>>>(parts, splits, stride, r, ldp, out, ldo);
+    const unsigned t = (unsigned)((r + 15) / 16);
+    k_gram_sym_reduce<<<dim3(t, t), dim3(16, 16, 4), 0, st>>>(parts, splits, stride, r, ldp, out, ldo);
     return cudaGetLastError();
 }
 
