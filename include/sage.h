@@ -198,7 +198,10 @@ sage_status_t sage_fd_stats(sage_fd_t* h, sage_stats_t* out);
  * delta; default ell), key 2 = maximum Jacobi sweeps (default 30). At any time: key 3 = bit mask of
  * kernel classes to time with CUDA events on the launching stream (see sage_fd_profile; default 0); key 4 =
  * 1 (default) to use the tensor-core kernels wherever the operands meet their alignment rules (16-byte
- * aligned base, row pitch a multiple of 16 bytes), 0 to use the CUDA-core kernels everywhere. */
+ * aligned base, row pitch a multiple of 16 bytes), 0 to use the CUDA-core kernels everywhere; key 5 = which
+ * kernels run the eigen-solve: 0 (default) a cluster of 8 thread blocks with the Jacobi columns in distributed
+ * shared memory, 1 the single-block kernel (buffers of up to 192 rows) or the cluster kernel that keeps the
+ * matrix in L2. Same algorithm either way; results agree up to rounding order. */
 sage_status_t sage_fd_set_option(sage_fd_t* h, int key, double value);
 
 /* Per-kernel device time of this handle's launches since the previous call, for the classes selected

@@ -149,6 +149,7 @@ struct sage_fd {
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     int* tc_err = nullptr;         // set by a tensor-core kernel whose bounded wait ran out
     bool use_tc = true;            // option 4: tensor-core kernels where their alignment rules hold
+    int eig_variant = 0;           // option 5: 0 cluster eigen-solve in distributed shared memory, 1 the one-CTA / L2 kernels
     int64_t launches = 0;
     Prof prof;
 };
@@ -275,7 +276,7 @@ sage_status_t enqueue_factor(sage_fd* h, int r, int do_shrink, int keep, int zer
     const bool tc_rebuild = h->use_tc && h->Wsplit && keep > 0 && j_pad <= 128 && r <= 256;
     CU_TRY(timed(h, K_EIG, 1, st, [&] {
         return launch_eig_shrink(h->Kmat, h->m, r, do_shrink, h->delta_rank, keep, h->Ur, h->m, h->sigma, h->ell, h->eig_work,
-                                 h->max_sweeps, h->info, tc_rebuild ? h->Wsplit : nullptr, kWsplitLd, j_pad, st);
+                                 h->max_sweeps, h->info, tc_rebuild ? h->Wsplit : nullptr, kWsplitLd, j_pad, h->eig_variant, st);
     }));
     const int m_total = zero_to > keep ? zero_to : keep;
     bool done = false;
@@ -480,6 +481,10 @@ sage_status_t sage_fd_set_option(sage_fd_t* h, int key, double value) {
     }
     if (key == 4) {                          // 0: CUDA-core kernels only, 1: tensor-core kernels where possible
         h->use_tc = value != 0.0;
+        return SAGE_OK;
+    }
+    if (key == 5) {                          // eigen-solve kernel family (same algorithm, same results up to rounding order)
+        h->eig_variant = value != 0.0 ? 1 : 0;
         return SAGE_OK;
     }
     if (h->rows_seen != 0 || h->state != SKETCHING) {

@@ -794,6 +794,517 @@ k_eig_shrink_cluster(const float* __restrict__ K, int ldk, int n, int do_shrink,
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Distributed-shared-memory solver, all n <= 512: the same algorithm again, with the Jacobi phase spread over a
+// thread-block cluster of 8 CTAs and its columns kept ON CHIP. The one-CTA kernel is bound by instruction issue
+// (16 block pairs share four schedulers); here every block pair has a warp of its own on one of 8 SMs, so a local
+// round costs its dependent-latency chain only.
+//   * Round-robin slots are dealt to the CTAs in runs (slot s -> CTA s / SPC, warp s % SPC). Each warp owns a slot
+//     buffer of 2 blocks x 4 columns in its CTA's shared memory. A block round: load the 8 columns into registers,
+//     rotate the 16 cross pairs in 4 local rounds (as in the one-CTA kernel), then store every column straight
+//     into the slot buffer of the warp that needs it next (a remote shared-memory store when that warp sits in
+//     another CTA; the tournament moves a block to a neighbouring slot, so most stores stay local).
+//   * Two cluster barriers per block round: "everyone has loaded" (its wait is hidden behind the local rounds)
+//     before the stores, "everyone has stored" before the next loads. All threads of the cluster execute the same
+//     number of barriers: trip counts depend only on the rank, the sweep limit and a convergence word that all
+//     read from global memory after a barrier.
+//   * Cholesky: for n <= 192 CTA 0 factors the matrix alone in its shared memory (a cluster barrier per pivot
+//     step would cost more than it saves) and hands factor, pivot order and rank over through global memory;
+//     for larger n the cluster factors it in global memory (L2) as k_eig_shrink_cluster does.
+// `gwork`: LD*LD floats (factor), then 2 convergence words, the rank, and from +64 on the pivot order (512 ints).
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void cl_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cl_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+
+// The two blocks slot `slot` holds in block round `br` (half 0: ba, half 1: bb).
+__device__ __forceinline__ void rr_blocks(int slot, int br, int nbm1, int& ba, int& bb) {
+    if (slot == 0) { ba = nbm1; bb = br; }
+    else {
+        ba = br + slot; if (ba >= nbm1) ba -= nbm1;
+        bb = br + nbm1 - slot; if (bb >= nbm1) bb -= nbm1;
+    }
+}
+// Inverse: slot and half that hold block b in block round br.
+__device__ __forceinline__ void rr_slot_of(int b, int br, int nbm1, int nact, int& slot, int& half) {
+    if (b == nbm1) { slot = 0; half = 0; return; }
+    int d = b - br;
+    if (d < 0) d += nbm1;
+    if (d == 0) { slot = 0; half = 1; }
+    else if (d < nact) { slot = d; half = 0; }
+    else { slot = nbm1 - d; half = 1; }
+}
+
+template <int T, int NT>
+__global__ void __launch_bounds__(NT, 1)
+k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int delta_rank, int keep, float* __restrict__ Ur,
+                 int ldu, float* __restrict__ sigma_out, int n_sigma, int max_sweeps, EigInfo* __restrict__ info,
+                 float* __restrict__ Wsplit, int ldw, int j_pad, float* __restrict__ gwork) {
+    constexpr int LD = 64 * T;
+    constexpr int kMaxN = 512;                           // shadows the namespace constant
+    constexpr int WPC = NT / 32;                         // warps per CTA
+    constexpr bool kLocalChol = T <= 3;                  // CTA 0 factors alone in shared memory
+    constexpr int R = 2 * T;            // rows per lane when 32 lanes span a column
+    constexpr int Q = 2 * T;            // float4 per lane when 8 lanes span a column
+    cg::cluster_group cluster = cg::this_cluster();
+    const int csize = (int)cluster.num_blocks(), crank = (int)cluster.block_rank();
+    const int GT = NT * csize;
+    extern __shared__ __align__(16) float smem[];
+    float* X = gwork;                                   // LD x LD factor in global memory (L2)
+    int* gflag = reinterpret_cast<int*>(gwork + (size_t)LD * LD);   // [0],[1] convergence words, [2] rank
+    int* gperm = gflag + 64;                            // pivot step -> physical index (kLocalChol hand-over)
+    float* lam = smem;                                  // kMaxN each from here on (one copy per CTA)
+    float* fac = lam + kMaxN;
+    float* scl = fac + kMaxN;
+    int* ord = reinterpret_cast<int*>(scl + kMaxN);     // physical index -> pivot step (-1: never pivoted)
+    int* perm = ord + kMaxN;                            // pivot step -> physical index
+    int* order = perm + kMaxN;                          // sorted position -> pivot step
+    float* sh_f = reinterpret_cast<float*>(order + kMaxN);
+    float* sbuf = sh_f + 8;                             // slot buffers: [T slots][2 halves][4 columns][LD]
+    float* Xl = sbuf + T * 8 * LD;                      // LD x LD, kLocalChol only
+
+    const int tid = threadIdx.x, lane = tid & 31, lwarp = tid >> 5;
+    const int gtid = crank * NT + tid;
+
+    // running diagonal and liveness of the rows this lane owns (rows lane + 32 t), one copy per warp
+    float dg[R];
+    bool alive[R];
+    bool bad = false;
+    float dmax = 0.f;
+#pragma unroll
+    for (int t = 0; t < R; ++t) {
+        const int i = lane + 32 * t;
+        dg[t] = (i < n) ? K[(size_t)i * ldk + i] : -1.f;
+        alive[t] = i < n;
+        if (alive[t] && !(fabsf(dg[t]) <= 3.0e38f)) { bad = true; alive[t] = false; }
+        if (alive[t]) dmax = fmaxf(dmax, dg[t]);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) dmax = fmaxf(dmax, __shfl_xor_sync(0xffffffffu, dmax, o));
+    if (gtid < 32 && bad) atomicOr(&info->flags, kFlagNonFinite);
+    const bool empty = !(dmax >= 1e-30f);              // nothing to factor: rank 0
+    const float kscale = empty ? 0.f : 1.f / dmax;
+#pragma unroll
+    for (int t = 0; t < R; ++t) dg[t] *= kscale;
+    for (int i = tid; i < kMaxN; i += NT) { ord[i] = -1; perm[i] = 0; }
+    if (gtid < 2) gflag[gtid] = 0;
+    const float tol = 1e-7f;
+    int rank = empty ? 0 : n;
+
+    if constexpr (kLocalChol) {
+        if (crank == 0) {
+            for (int e = tid; e < n * LD; e += NT) {
+                const int c = e / LD, i = e - c * LD;
+                Xl[e] = (i < n) ? K[(size_t)c * ldk + i] * kscale : 0.f;  // K is symmetric: row c serves as column c
+            }
+            __syncthreads();
+            // ---- pivoted Cholesky without swaps, one CTA (see k_eig_shrink_fast) ----
+            constexpr int CW = (LD + WPC - 1) / WPC;                   // columns a warp owns: lwarp + WPC u
+            unsigned colmask = 0u;
+#pragma unroll
+            for (int u = 0; u < CW; ++u)
+                if (lwarp + WPC * u < n) colmask |= 1u << u;
+            for (int k = 0; k < rank; ++k) {
+                unsigned key = 0u;
+#pragma unroll
+                for (int t = 0; t < R; ++t)
+                    if (alive[t]) key = max(key, (__float_as_uint(fmaxf(dg[t], 0.f)) & 0xffffff00u) | (unsigned)(255 - (lane + 32 * t)));
+                key = __reduce_max_sync(0xffffffffu, key);
+                const int p = 255 - (int)(key & 255u);
+                if (key == 0u || p >= n) { rank = k; break; }             // identical in every warp
+                const float* Xp = Xl + p * LD;
+                const float d = Xp[p];
+                if (!(d > tol)) { rank = k; break; }
+                const float inv = rsqrtf(d);
+                if ((p % WPC) == lwarp) colmask &= ~(1u << (p / WPC));
+                float li[R];
+#pragma unroll
+                for (int t = 0; t < R; ++t) {
+                    const int i = lane + 32 * t;
+                    if (i == p) alive[t] = false;
+                    li[t] = alive[t] ? Xp[i] * inv : 0.f;
+                    dg[t] = fmaf(-li[t], li[t], dg[t]);
+                }
+#pragma unroll
+                for (int u0 = 0; u0 < CW; u0 += 2) {                      // two columns at a time: loads first, then stores
+                    const bool on0 = (colmask >> u0) & 1u, on1 = (u0 + 1 < CW) && ((colmask >> (u0 + 1)) & 1u);
+                    if (!on0 && !on1) continue;
+                    float* c0 = Xl + (lwarp + WPC * u0) * LD;
+                    float* c1 = Xl + (lwarp + WPC * (u0 + 1)) * LD;
+                    const float l0 = on0 ? Xp[lwarp + WPC * u0] * inv : 0.f;
+                    const float l1 = on1 ? Xp[lwarp + WPC * (u0 + 1)] * inv : 0.f;
+                    float v0[R], v1[R];
+#pragma unroll
+                    for (int t = 0; t < R; ++t) {
+                        v0[t] = on0 ? c0[lane + 32 * t] : 0.f;
+                        v1[t] = on1 ? c1[lane + 32 * t] : 0.f;
+                    }
+#pragma unroll
+                    for (int t = 0; t < R; ++t) {
+                        if (on0) c0[lane + 32 * t] = fmaf(-li[t], l0, v0[t]);
+                        if (on1) c1[lane + 32 * t] = fmaf(-li[t], l1, v1[t]);
+                    }
+                }
+                if (tid == 0) { ord[p] = k; perm[k] = p; scl[k] = inv; }
+                __syncthreads();
+            }
+            __syncthreads();
+            // factor L into global memory (zero above the pivot order, zero unpivoted columns) + the hand-over words
+            for (int e = tid; e < n * LD; e += NT) {
+                const int c = e / LD, i = e - c * LD;
+                const int kc = ord[c];
+                float v = 0.f;
+                if (kc >= 0 && i < n) {
+                    const int ki = ord[i];
+                    if (!(ki >= 0 && ki < kc)) v = Xl[e] * scl[kc];
+                }
+                X[e] = v;
+            }
+            for (int i = tid; i < n; i += NT) gperm[i] = perm[i];
+            if (tid == 0) gflag[2] = rank;
+        }
+        cluster.sync();
+        rank = __ldcg(&gflag[2]);
+        if (crank != 0)
+            for (int i = tid; i < n; i += NT) perm[i] = __ldcg(&gperm[i]);
+        __syncthreads();
+    } else {
+        const int NW = WPC * csize;                          // warps of the whole cluster
+        const int warp = crank * WPC + lwarp;
+        for (int e = gtid; e < n * LD; e += GT) {
+            const int c = e / LD, i = e - c * LD;
+            X[e] = (i < n) ? K[(size_t)c * ldk + i] * kscale : 0.f;
+        }
+        cluster.sync();
+        // ---- pivoted Cholesky without swaps, whole cluster, matrix in L2 (see k_eig_shrink_cluster) ----
+        constexpr int CW = (LD + 63) / 64 * 2;                     // upper bound of columns a warp owns for NW >= 32
+        unsigned colmask = 0u;
+#pragma unroll
+        for (int u = 0; u < CW; ++u)
+            if (warp + NW * u < n) colmask |= 1u << u;
+        for (int k = 0; k < rank; ++k) {
+            unsigned key = 0u;
+#pragma unroll
+            for (int t = 0; t < R; ++t)
+                if (alive[t]) key = max(key, (__float_as_uint(fmaxf(dg[t], 0.f)) & 0xfffffe00u) | (unsigned)(511 - (lane + 32 * t)));
+            key = __reduce_max_sync(0xffffffffu, key);
+            const int p = 511 - (int)(key & 511u);
+            if (key == 0u || p >= n) { rank = k; break; }             // identical in every warp of the cluster
+            const float* Xp = X + p * LD;
+            const float d = __ldcg(Xp + p);
+            if (!(d > tol)) { rank = k; break; }
+            const float inv = rsqrtf(d);
+            if ((p % NW) == warp) colmask &= ~(1u << (p / NW));
+            float li[R];
+#pragma unroll
+            for (int t = 0; t < R; ++t) {
+                const int i = lane + 32 * t;
+                if (i == p) alive[t] = false;
+                li[t] = alive[t] ? __ldcg(Xp + i) * inv : 0.f;
+                dg[t] = fmaf(-li[t], li[t], dg[t]);
+            }
+#pragma unroll
+            for (int u0 = 0; u0 < CW; u0 += 2) {
+                const bool on0 = (colmask >> u0) & 1u, on1 = (u0 + 1 < CW) && ((colmask >> (u0 + 1)) & 1u);
+                if (!on0 && !on1) continue;
+                float* c0 = X + (warp + NW * u0) * LD;
+                float* c1 = X + (warp + NW * (u0 + 1)) * LD;
+                const float l0 = on0 ? __ldcg(Xp + warp + NW * u0) * inv : 0.f;
+                const float l1 = on1 ? __ldcg(Xp + warp + NW * (u0 + 1)) * inv : 0.f;
+                float v0[R], v1[R];
+#pragma unroll
+                for (int t = 0; t < R; ++t) {
+                    v0[t] = on0 ? __ldcg(c0 + lane + 32 * t) : 0.f;
+                    v1[t] = on1 ? __ldcg(c1 + lane + 32 * t) : 0.f;
+                }
+#pragma unroll
+                for (int t = 0; t < R; ++t) {
+                    if (on0) c0[lane + 32 * t] = fmaf(-li[t], l0, v0[t]);
+                    if (on1) c1[lane + 32 * t] = fmaf(-li[t], l1, v1[t]);
+                }
+            }
+            if (tid == 0) { ord[p] = k; perm[k] = p; scl[k] = inv; }   // every CTA keeps its own copy of the tables
+            cluster.sync();
+        }
+        cluster.sync();
+        for (int e = gtid; e < n * LD; e += GT) {
+            const int c = e / LD, i = e - c * LD;
+            const int kc = ord[c];
+            float v = 0.f;
+            if (kc >= 0 && i < n) {
+                const int ki = ord[i];
+                if (!(ki >= 0 && ki < kc)) v = __ldcg(X + e) * scl[kc];
+            }
+            X[e] = v;
+        }
+        cluster.sync();
+    }
+
+    // ---- one-sided cyclic Jacobi on the rank pivot columns, columns in distributed shared memory ----
+    const int l8 = lane & 7, qd = lane >> 3;
+    int sweeps = 0, more = 0;
+    float worst2 = 0.f;                 // largest squared cosine met in the current sweep
+    if (rank >= 2) {
+        const int nb = (rank + 3) >> 2, nbe = nb + (nb & 1), nbm1 = nbe - 1, nact = nbe >> 1;   // block pairs per round
+        const int SPC = (nact + csize - 1) / csize;               // slots per CTA
+        const int slot = crank * SPC + lwarp;
+        const bool fits = SPC <= T && SPC <= WPC;                 // holds for a cluster of 8; otherwise report, do not run
+        const bool active = fits && lwarp < SPC && slot < nact;   // the other warps only take part in the barriers
+        float* mybuf = sbuf + (size_t)(lwarp < T ? lwarp : 0) * 8 * LD;
+        if (active) {                                             // columns of block round 0 from the factor in L2
+            int ba, bb;
+            rr_blocks(slot, 0, nbm1, ba, bb);
+            for (int hc = 0; hc < 8; ++hc) {
+                const int p = 4 * (hc < 4 ? ba : bb) + (hc & 3);
+                const float* src = X + (size_t)perm[p < rank ? p : 0] * LD;
+#pragma unroll
+                for (int t = 0; t < R; ++t) mybuf[hc * LD + lane + 32 * t] = (p < rank) ? __ldcg(src + lane + 32 * t) : 0.f;
+            }
+        }
+        __syncwarp();
+        auto pair_step = [&](float* cp, float* cq, bool valid) {   // one column pair of the warp's own buffer
+            float4* xp = reinterpret_cast<float4*>(cp) + l8;
+            float4* xq = reinterpret_cast<float4*>(cq) + l8;
+            float4 x[Q], y[Q];
+            float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f, g0 = 0.f, g1 = 0.f;
+#pragma unroll
+            for (int t = 0; t < Q; ++t) {
+                x[t] = xp[8 * t];
+                y[t] = xq[8 * t];
+                a0 = fmaf(x[t].x, x[t].x, a0); a1 = fmaf(x[t].y, x[t].y, a1); a0 = fmaf(x[t].z, x[t].z, a0); a1 = fmaf(x[t].w, x[t].w, a1);
+                b0 = fmaf(y[t].x, y[t].x, b0); b1 = fmaf(y[t].y, y[t].y, b1); b0 = fmaf(y[t].z, y[t].z, b0); b1 = fmaf(y[t].w, y[t].w, b1);
+                g0 = fmaf(x[t].x, y[t].x, g0); g1 = fmaf(x[t].y, y[t].y, g1); g0 = fmaf(x[t].z, y[t].z, g0); g1 = fmaf(x[t].w, y[t].w, g1);
+            }
+            float a = a0 + a1, b = b0 + b1, g = g0 + g1;
+#pragma unroll
+            for (int o = 4; o > 0; o >>= 1) {
+                a += __shfl_xor_sync(0xffffffffu, a, o);
+                b += __shfl_xor_sync(0xffffffffu, b, o);
+                g += __shfl_xor_sync(0xffffffffu, g, o);
+            }
+            const float ab = a * b, g2 = g * g;
+            if (valid && ab > 0.f && g2 > 1e-12f * ab) {
+                worst2 = fmaxf(worst2, __fdividef(g2, ab));
+                const float zeta = __fdividef(b - a, 2.f * g);
+                const float tt = copysignf(__fdividef(1.f, fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.f))), zeta);
+                const float c = rsqrtf(fmaf(tt, tt, 1.f));
+                const float s = c * tt;
+#pragma unroll
+                for (int t = 0; t < Q; ++t) {
+                    float4 nx, ny;
+                    nx.x = fmaf(-s, y[t].x, c * x[t].x); ny.x = fmaf(s, x[t].x, c * y[t].x);
+                    nx.y = fmaf(-s, y[t].y, c * x[t].y); ny.y = fmaf(s, x[t].y, c * y[t].y);
+                    nx.z = fmaf(-s, y[t].z, c * x[t].z); ny.z = fmaf(s, x[t].z, c * y[t].z);
+                    nx.w = fmaf(-s, y[t].w, c * x[t].w); ny.w = fmaf(s, x[t].w, c * y[t].w);
+                    xp[8 * t] = nx;
+                    xq[8 * t] = ny;
+                }
+            }
+            __syncwarp();
+        };
+        while (sweeps < max_sweeps) {
+            worst2 = 0.f;
+            for (int br = 0; br < nbm1; ++br) {
+                float4 x[Q], y[Q];
+                int lo = 0, hi = 0;
+                bool va = false;
+                if (active) {
+                    int ba, bb;
+                    rr_blocks(slot, br, nbm1, ba, bb);
+                    if (br == 0) {                                // pairs inside each block: quarters 0,1 -> ba, 2,3 -> bb
+                        const int half = (qd < 2) ? 0 : 1, base = 4 * (half ? bb : ba), h = qd & 1;
+                        float* blk = mybuf + half * 4 * LD;
+                        const int c0 = h ? 2 : 0, c1 = h ? 3 : 1, c2 = h ? 1 : 0, c3 = h ? 3 : 2, c4 = h ? 1 : 0, c5 = h ? 2 : 3;
+                        pair_step(blk + c0 * LD, blk + c1 * LD, base + c0 < rank && base + c1 < rank);
+                        pair_step(blk + c2 * LD, blk + c3 * LD, base + c2 < rank && base + c3 < rank);
+                        pair_step(blk + c4 * LD, blk + c5 * LD, base + c4 < rank && base + c5 < rank);
+                    }
+                    lo = min(ba, bb);
+                    hi = max(ba, bb);
+                    const int half_lo = (ba < bb) ? 0 : 1;
+                    // quarter qd keeps column qd of block lo; the columns of block hi travel between quarters
+                    const float4* xa = reinterpret_cast<const float4*>(mybuf + (half_lo * 4 + qd) * LD) + l8;
+                    const float4* xb = reinterpret_cast<const float4*>(mybuf + ((1 - half_lo) * 4 + qd) * LD) + l8;
+                    va = 4 * lo + qd < rank;
+#pragma unroll
+                    for (int t = 0; t < Q; ++t) {
+                        x[t] = xa[8 * t];
+                        y[t] = xb[8 * t];
+                    }
+                }
+                cl_arrive();                                       // "loaded": completes while the local rounds run
+                if (active) {
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) {
+                        const bool valid = va && (4 * hi + ((qd + r) & 3) < rank);
+                        float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f, g0 = 0.f, g1 = 0.f;
+#pragma unroll
+                        for (int t = 0; t < Q; ++t) {
+                            a0 = fmaf(x[t].x, x[t].x, a0); a1 = fmaf(x[t].y, x[t].y, a1); a0 = fmaf(x[t].z, x[t].z, a0); a1 = fmaf(x[t].w, x[t].w, a1);
+                            b0 = fmaf(y[t].x, y[t].x, b0); b1 = fmaf(y[t].y, y[t].y, b1); b0 = fmaf(y[t].z, y[t].z, b0); b1 = fmaf(y[t].w, y[t].w, b1);
+                            g0 = fmaf(x[t].x, y[t].x, g0); g1 = fmaf(x[t].y, y[t].y, g1); g0 = fmaf(x[t].z, y[t].z, g0); g1 = fmaf(x[t].w, y[t].w, g1);
+                        }
+                        float a = a0 + a1, b = b0 + b1, g = g0 + g1;
+#pragma unroll
+                        for (int o = 4; o > 0; o >>= 1) {
+                            a += __shfl_xor_sync(0xffffffffu, a, o);
+                            b += __shfl_xor_sync(0xffffffffu, b, o);
+                            g += __shfl_xor_sync(0xffffffffu, g, o);
+                        }
+                        const float ab = a * b, g2 = g * g;
+                        if (valid && ab > 0.f && g2 > 1e-12f * ab) {
+                            worst2 = fmaxf(worst2, __fdividef(g2, ab));
+                            const float zeta = __fdividef(b - a, 2.f * g);
+                            const float tt = copysignf(__fdividef(1.f, fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.f))), zeta);
+                            const float c = rsqrtf(fmaf(tt, tt, 1.f));
+                            const float s = c * tt;
+#pragma unroll
+                            for (int t = 0; t < Q; ++t) {
+                                float4 nx, ny;
+                                nx.x = fmaf(-s, y[t].x, c * x[t].x); ny.x = fmaf(s, x[t].x, c * y[t].x);
+                                nx.y = fmaf(-s, y[t].y, c * x[t].y); ny.y = fmaf(s, x[t].y, c * y[t].y);
+                                nx.z = fmaf(-s, y[t].z, c * x[t].z); ny.z = fmaf(s, x[t].z, c * y[t].z);
+                                nx.w = fmaf(-s, y[t].w, c * x[t].w); ny.w = fmaf(s, x[t].w, c * y[t].w);
+                                x[t] = nx;
+                                y[t] = ny;
+                            }
+                        }
+                        if (r < 3) {                              // quarter qd takes over the column quarter qd + 1 holds
+                            const int src = (lane + 8) & 31;
+#pragma unroll
+                            for (int t = 0; t < Q; ++t) {
+                                y[t].x = __shfl_sync(0xffffffffu, y[t].x, src);
+                                y[t].y = __shfl_sync(0xffffffffu, y[t].y, src);
+                                y[t].z = __shfl_sync(0xffffffffu, y[t].z, src);
+                                y[t].w = __shfl_sync(0xffffffffu, y[t].w, src);
+                            }
+                        }
+                    }
+                }
+                cl_wait();                                         // every warp of the cluster holds its columns in registers
+                if (active) {                                      // store each column where the next block round reads it
+                    const int brn = (br + 1 == nbm1) ? 0 : br + 1;
+                    int s_lo, h_lo, s_hi, h_hi;
+                    rr_slot_of(lo, brn, nbm1, nact, s_lo, h_lo);
+                    rr_slot_of(hi, brn, nbm1, nact, s_hi, h_hi);
+                    const int c_lo = s_lo / SPC, c_hi = s_hi / SPC;
+                    float* d_lo = cluster.map_shared_rank(sbuf, c_lo) + ((size_t)(s_lo - c_lo * SPC) * 8 + h_lo * 4 + qd) * LD;
+                    float* d_hi = cluster.map_shared_rank(sbuf, c_hi) + ((size_t)(s_hi - c_hi * SPC) * 8 + h_hi * 4 + ((qd + 3) & 3)) * LD;
+                    float4* o_lo = reinterpret_cast<float4*>(d_lo) + l8;
+                    float4* o_hi = reinterpret_cast<float4*>(d_hi) + l8;
+#pragma unroll
+                    for (int t = 0; t < Q; ++t) {
+                        o_lo[8 * t] = x[t];
+                        o_hi[8 * t] = y[t];
+                    }
+                }
+                if (br == nbm1 - 1) {                              // end of a sweep: publish whether anything still rotated
+                    const int par = (sweeps + 1) & 1;
+                    if (__any_sync(0xffffffffu, worst2 > 1e-6f) && lane == 0) atomicOr(&gflag[par], 1);
+                    if (gtid == 0) gflag[par ^ 1] = 0;
+                }
+                cl_arrive();
+                cl_wait();                                         // "stored": the next block round may load
+            }
+            ++sweeps;
+            more = fits ? __ldcg(&gflag[sweeps & 1]) : 1;
+            if (!more) break;               // every cosine of this sweep was below 1e-3: converged after it
+            if (!fits) break;
+        }
+        if (active) {                                             // back to the factor in L2, for the final phase
+            int ba, bb;
+            rr_blocks(slot, 0, nbm1, ba, bb);
+            for (int hc = 0; hc < 8; ++hc) {
+                const int p = 4 * (hc < 4 ? ba : bb) + (hc & 3);
+                if (p < rank) {
+                    float* dst = X + (size_t)perm[p] * LD;
+#pragma unroll
+                    for (int t = 0; t < R; ++t) dst[lane + 32 * t] = mybuf[hc * LD + lane + 32 * t];
+                }
+            }
+        }
+    }
+    cluster.sync();
+    const int not_converged = rank >= 2 && more != 0;          // stopped at the sweep limit while still rotating visibly
+    // ---- eigenvalues = squared column norms (pivot-step order), scaled back; sort descending, stable ----
+    for (int k = lwarp; k < n; k += WPC) {                          // every CTA forms all eigenvalues for its own tables
+        float a = 0.f;
+        if (k < rank) {
+            const float* x = X + perm[k] * LD;
+#pragma unroll
+            for (int t = 0; t < R; ++t) { const float xv = __ldcg(x + lane + 32 * t); a = fmaf(xv, xv, a); }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+        }
+        if (lane == 0) lam[k] = a * dmax;
+    }
+    __syncthreads();
+    for (int t = tid; t < n; t += NT) {
+        const float mine = lam[t];
+        int pos = 0;
+        for (int i = 0; i < n; ++i) {
+            const float o = lam[i];
+            pos += (o > mine) || (o == mine && i < t);
+        }
+        order[pos] = t;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        float delta = 0.f;
+        if (do_shrink && delta_rank - 1 < n) delta = lam[order[delta_rank - 1]];
+        sh_f[0] = delta;
+        if (crank == 0) {
+            info->delta = delta;
+            info->sweeps = sweeps;
+            if (sweeps > info->max_sweeps) info->max_sweeps = sweeps;
+            info->rank = rank;
+            if (not_converged) info->flags |= kFlagNotConverged;
+            if (do_shrink) {
+                info->sum_delta += (double)delta;
+                info->shrinks += 1;
+            }
+        }
+    }
+    __syncthreads();
+    const float delta = sh_f[0];
+    const float back = sqrtf(dmax);     // columns of X are sigma_j u_j / sqrt(dmax)
+    for (int t = tid; t < n; t += NT) {
+        const float l = lam[order[t]];
+        float f = 0.f, sp = 0.f;
+        if (l > 0.f && t < keep) {
+            const float kept = fmaxf(l - delta, 0.f);
+            sp = sqrtf(kept);
+            f = sqrtf(kept / l) * rsqrtf(l) * back;   // (sigma'/sigma) / sigma, for the unscaled column
+        }
+        fac[t] = f;
+        if (t < n_sigma && crank == 0) sigma_out[t] = sp;
+    }
+    if (crank == 0)
+        for (int j = n + tid; j < n_sigma; j += NT) sigma_out[j] = 0.f;
+    __syncthreads();
+    for (int e = gtid; e < n * keep; e += GT) {
+        const int j = e / n, i = e - j * n;
+        float v = 0.f;
+        if (j < n) {
+            const int k = order[j];
+            if (k < rank) v = __ldcg(X + perm[k] * LD + i) * fac[j];
+        }
+        Ur[(size_t)i * ldu + j] = v;
+    }
+    if (Wsplit) {   // the same factors transposed and split for the tensor-core rebuild: [W_hi ; W_lo], zero padded
+        for (int e = gtid; e < j_pad * ldw; e += GT) {
+            const int j = e / ldw, i = e - j * ldw;
+            float v = 0.f;
+            if (j < keep && j < n && i < n) {
+                const int k = order[j];
+                if (k < rank) v = __ldcg(X + perm[k] * LD + i) * fac[j];
+            }
+            const float hi = __uint_as_float((__float_as_uint(v) + 0x1000u) & 0xffffe000u);
+            Wsplit[(size_t)j * ldw + i] = hi;
+            Wsplit[(size_t)(j_pad + j) * ldw + i] = v - hi;
+        }
+    }
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 k_eig_shrink(const float* __restrict__ K, int ldk, int n, int do_shrink, int delta_rank, int keep, float* __restrict__ Ur,
              int ldu, float* __restrict__ sigma_out, int n_sigma, float* __restrict__ work, int use_smem, int max_sweeps,
@@ -1022,8 +1533,37 @@ k_eig_shrink(const float* __restrict__ K, int ldk, int n, int do_shrink, int del
 
 cudaError_t launch_eig_shrink(const float* K, int ldk, int n, int do_shrink, int delta_rank, int keep, float* Ur, int ldu,
                               float* sigma_out, int n_sigma, float* work, int max_sweeps, EigInfo* info, float* Wsplit, int ldw,
-                              int j_pad, cudaStream_t st) {
+                              int j_pad, int variant, cudaStream_t st) {
     if (n <= 0 || n > 512) return cudaErrorInvalidValue;
+    if (variant == 0) {   // cluster of 8 CTAs, Jacobi columns in distributed shared memory
+        const int T = n <= 64 ? 1 : n <= 128 ? 2 : n <= 192 ? 3 : n <= 256 ? 4 : 8;
+        const int LD = 64 * T;
+        const size_t bytes = 3 * 512 * sizeof(float) + 3 * 512 * sizeof(int) + 32 + (size_t)T * 8 * LD * sizeof(float) +
+                             (T <= 3 ? (size_t)LD * LD * sizeof(float) : 0);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(8);
+        cfg.blockDim = dim3(T <= 3 ? 512 : 256);
+        cfg.dynamicSmemBytes = bytes;
+        cfg.stream = st;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 8;
+        at[0].val.clusterDim.y = 1;
+        at[0].val.clusterDim.z = 1;
+        cfg.attrs = at;
+        cfg.numAttrs = 1;
+        cudaError_t e = cudaSuccess;
+#define SAGE_EIG_DSM(TT, NTT)                                                                                                 \
+    e = cudaFuncSetAttribute(k_eig_shrink_dsm<TT, NTT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);              \
+    if (e == cudaSuccess)                                                                                                      \
+        e = cudaLaunchKernelEx(&cfg, k_eig_shrink_dsm<TT, NTT>, K, ldk, n, do_shrink, delta_rank, keep, Ur, ldu, sigma_out, n_sigma, \
+                               max_sweeps, info, Wsplit, ldw, j_pad, work);
+        if (T == 1) { SAGE_EIG_DSM(1, 512) } else if (T == 2) { SAGE_EIG_DSM(2, 512) } else if (T == 3) { SAGE_EIG_DSM(3, 512) }
+        else if (T == 4) { SAGE_EIG_DSM(4, 256) } else { SAGE_EIG_DSM(8, 256) }
+#undef SAGE_EIG_DSM
+        if (e == cudaSuccess) return cudaGetLastError();
+        (void)cudaGetLastError();          // no cluster launch on this device: the kernels below serve every n <= 512
+    }
     if (n <= kMaxFast) {
         const int T = (n + 63) / 64;
         const size_t aux_bytes = 3 * kMaxN * sizeof(float) + 3 * kMaxN * sizeof(int) + 32;

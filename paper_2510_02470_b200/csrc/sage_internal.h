@@ -87,7 +87,7 @@ cudaError_t launch_rebuild(const float* Ur, int ldu, const float* Bsrc, float* B
 // zero outside j < keep, i < n.
 cudaError_t launch_eig_shrink(const float* K, int ldk, int n, int do_shrink, int delta_rank, int keep, float* Ur,
                               int ldu, float* sigma_out, int n_sigma, float* work, int max_sweeps, EigInfo* info,
-                              float* Wsplit, int ldw, int j_pad, cudaStream_t st);
+                              float* Wsplit, int ldw, int j_pad, int variant, cudaStream_t st);
 
 // Z (n x ell, pitch ldz, already reduced over splits) -> zhat rows, ||z|| and per-block partial sums of zhat.
 // zsum (ell doubles) += the partial sums in ascending block order (done by a second, single-block kernel).

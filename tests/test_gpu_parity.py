@@ -203,6 +203,43 @@ def test_tensor_core_path_agrees_with_cuda_core_path(dtype, N, D, ell):
         assert np.max(np.abs(a - ref["alpha"])) <= TOL_SCORE[dtype]
 
 
+# ------------------------------------------------------------------ the two eigen-solve kernel families
+
+def _run_with_eig_variant(rows, D, ell, variant):
+    dev = torch.device("cuda", 0)
+    g = rows.to(dev)
+    fd = sage.SageFD(D, ell, rows.dtype, 0)
+    fd.set_option(5, float(variant))
+    fd.update(g)
+    fd.finalize()
+    S, sigma = fd.sketch()
+    a = fd.score(g)
+    torch.cuda.synchronize()
+    st = fd.stats()
+    fd.close()
+    return S.double().cpu().numpy(), sigma.double().cpu().numpy(), a.double().cpu().numpy(), st
+
+
+@pytest.mark.parametrize("N,D,ell,rank", [(300, 520, 8, 3), (700, 1028, 32, 6), (900, 1028, 64, 40), (900, 772, 96, 200),
+                                          (1200, 1028, 128, 12), (1500, 516, 256, 300), (150, 260, 64, 200)])
+def test_cluster_eigen_solve_agrees_with_one_cta_solve(N, D, ell, rank):
+    """Option 5 = 0 (cluster of 8 CTAs, Jacobi columns in distributed shared memory; buffers of 16 to 512 rows cover
+    every instantiation) against option 5 = 1 (one-CTA / L2 kernels): same algorithm, so the sketches agree to
+    rounding, and both match the oracle."""
+    rows = lowrank_rows(N, D, rank, 0.3, 7 * N + ell)
+    S0, sg0, a0, st0 = _run_with_eig_variant(rows, D, ell, 0)
+    S1, sg1, a1, st1 = _run_with_eig_variant(rows, D, ell, 1)
+    assert st0["device_flags"] == 0 and st1["device_flags"] == 0 and st0["shrinks"] == st1["shrinks"]
+    A = metrics.rows_as_f64(rows, D)
+    F2 = float(np.linalg.norm(A) ** 2)
+    assert metrics.signed_gram_norm(S0, S1) / F2 <= 2e-5
+    assert np.allclose(sg0, sg1, rtol=0, atol=2e-4 * max(sg1.max(), 1e-30))
+    assert np.max(np.abs(a0 - a1)) <= 5e-5
+    ref = oracle.run(rows, D, ell, 0.1, route=1)
+    assert metrics.signed_gram_norm(S0, ref["S"]) / F2 <= 1e-4
+    assert np.max(np.abs(a0 - ref["alpha"])) <= 1e-4
+
+
 # ------------------------------------------------------------------ the benchmark workloads
 
 def test_c1_full():
