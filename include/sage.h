@@ -187,7 +187,8 @@ typedef struct {
     int32_t max_sweeps;     /* largest sweep count seen */
     int32_t last_rank;      /* numerical rank found by the most recent factorisation */
     uint32_t device_flags;  /* bit 0: eigen-solver not converged, bit 1: non-finite input seen,
-                               bit 2: a tensor-core kernel gave up a bounded wait (results invalid) */
+                               bit 2: a tensor-core kernel gave up a bounded wait (results invalid),
+                               bit 3: the cluster eigen-solve gave up a bounded wait (results invalid) */
     int64_t kernel_launches;/* kernels this handle has launched since create/reset */
 } sage_stats_t;
 

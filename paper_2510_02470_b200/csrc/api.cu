@@ -581,6 +581,10 @@ sage_status_t sage_fd_finalize(sage_fd_t* h, void* cuda_stream) {
         set_err("sage_fd_finalize: a tensor-core kernel gave up waiting on its pipeline (results are not valid)");
         return SAGE_ERR_CUDA;
     }
+    if (info.flags & kFlagExchangeTimeout) {
+        set_err("sage_fd_finalize: an eigen-solve gave up waiting for another thread block of its cluster (results are not valid)");
+        return SAGE_ERR_CUDA;
+    }
     if (info.flags & kFlagNotConverged) {
         set_err("sage_fd_finalize: an eigen-solve reached the sweep limit (%d)", h->max_sweeps);
         return SAGE_ERR_NOT_CONVERGED;

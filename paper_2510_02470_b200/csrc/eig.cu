@@ -48,6 +48,24 @@ __device__ __forceinline__ void rr_pair(int n_even, int round, int slot, int& p,
     q = max(a, b);
 }
 
+// Rotation that orthogonalises two columns with squared norms a, b and inner product g:
+// tan 2theta = 2g / (b - a), cos 2theta = |b - a| / r, c = sqrt((1 + cos 2theta) / 2), s = sin 2theta / (2c), from two
+// approximate reciprocal square roots, followed by one Newton step towards c^2 + s^2 = 1 taken from the residual
+// itself: scaling by 1.5 - 0.5 (c^2 + s^2) would be lost to the coarser float grid above 1 whenever c^2 + s^2 < 1,
+// a one-sided correction that shrinks every column a little at every rotation (measured 1e-5 relative on the
+// singular values after a few thousand rotations; with the residual form they agree with fp64 to 1e-7).
+__device__ __forceinline__ void jacobi_rotation(float a, float b, float g, float& c, float& s) {
+    const float tau = b - a, gam = 2.f * g;
+    const float inv_r = rsqrtf(fmaf(tau, tau, gam * gam));
+    const float c2 = fmaf(0.5f * fabsf(tau), inv_r, 0.5f);
+    const float invc = rsqrtf(c2);
+    c = c2 * invc;
+    s = copysignf(0.5f, tau) * gam * inv_r * invc;
+    const float half_res = 0.5f * fmaf(-s, s, fmaf(-c, c, 1.f));
+    c = fmaf(c, half_res, c);
+    s = fmaf(s, half_res, s);
+}
+
 // ------------------------------------------------------------------------------------------------
 // Shared-memory solver for n <= 192 (the common case: n = 2*ell <= 128, and partly filled buffers at
 // the freeze). Same mathematics as k_eig_shrink below, restructured for instruction count and latency:
@@ -222,10 +240,8 @@ k_eig_shrink_fast(const float* __restrict__ K, int ldk, int n, int do_shrink, in
                 const float ab = a * b, g2 = g * g;
                 if (valid && ab > 0.f && g2 > 1e-12f * ab) {
                     worst2 = fmaxf(worst2, __fdividef(g2, ab));
-                    const float zeta = __fdividef(b - a, 2.f * g);
-                    const float tt = copysignf(__fdividef(1.f, fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.f))), zeta);
-                    const float c = rsqrtf(fmaf(tt, tt, 1.f));
-                    const float s = c * tt;
+                    float c, s;
+                    jacobi_rotation(a, b, g, c, s);
 #pragma unroll
                     for (int t = 0; t < Q; ++t) {
                         float4 nx, ny;
@@ -289,10 +305,8 @@ k_eig_shrink_fast(const float* __restrict__ K, int ldk, int n, int do_shrink, in
                             const float ab = a * b, g2 = g * g;
                             if (valid && ab > 0.f && g2 > 1e-12f * ab) {
                                 worst2 = fmaxf(worst2, __fdividef(g2, ab));
-                                const float zeta = __fdividef(b - a, 2.f * g);
-                                const float tt = copysignf(__fdividef(1.f, fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.f))), zeta);
-                                const float c = rsqrtf(fmaf(tt, tt, 1.f));
-                                const float s = c * tt;
+                                float c, s;
+                                jacobi_rotation(a, b, g, c, s);
 #pragma unroll
                                 for (int t = 0; t < Q; ++t) {
                                     float4 nx, ny;
@@ -591,10 +605,8 @@ k_eig_shrink_cluster(const float* __restrict__ K, int ldk, int n, int do_shrink,
                 const float ab = a * b, g2 = g * g;
                 if (valid && ab > 0.f && g2 > 1e-12f * ab) {
                     worst2 = fmaxf(worst2, __fdividef(g2, ab));
-                    const float zeta = __fdividef(b - a, 2.f * g);
-                    const float tt = copysignf(__fdividef(1.f, fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.f))), zeta);
-                    const float c = rsqrtf(fmaf(tt, tt, 1.f));
-                    const float s = c * tt;
+                    float c, s;
+                    jacobi_rotation(a, b, g, c, s);
 #pragma unroll
                     for (int t = 0; t < Q; ++t) {
                         float4 nx, ny;
@@ -658,10 +670,8 @@ k_eig_shrink_cluster(const float* __restrict__ K, int ldk, int n, int do_shrink,
                             const float ab = a * b, g2 = g * g;
                             if (valid && ab > 0.f && g2 > 1e-12f * ab) {
                                 worst2 = fmaxf(worst2, __fdividef(g2, ab));
-                                const float zeta = __fdividef(b - a, 2.f * g);
-                                const float tt = copysignf(__fdividef(1.f, fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.f))), zeta);
-                                const float c = rsqrtf(fmaf(tt, tt, 1.f));
-                                const float s = c * tt;
+                                float c, s;
+                                jacobi_rotation(a, b, g, c, s);
 #pragma unroll
                                 for (int t = 0; t < Q; ++t) {
                                     float4 nx, ny;
@@ -804,14 +814,24 @@ k_eig_shrink_cluster(const float* __restrict__ K, int ldk, int n, int do_shrink,
 //     rotate the 16 cross pairs in 4 local rounds (as in the one-CTA kernel), then store every column straight
 //     into the slot buffer of the warp that needs it next (a remote shared-memory store when that warp sits in
 //     another CTA; the tournament moves a block to a neighbouring slot, so most stores stay local).
-//   * Two cluster barriers per block round: "everyone has loaded" (its wait is hidden behind the local rounds)
-//     before the stores, "everyone has stored" before the next loads. All threads of the cluster execute the same
-//     number of barriers: trip counts depend only on the rank, the sweep limit and a convergence word that all
-//     read from global memory after a barrier.
+//   * Exchange, n <= 256: two buffer sets per slot, used by alternate block rounds, and one mbarrier per slot and
+//     set. A warp sends its columns into the reader's other set with asynchronous stores (st.async) that count
+//     their bytes on the reader's barrier as they land: one-way latency, no fence or round trip on the writer's
+//     side (a plain remote store followed by a releasing arrival, or by a cluster barrier, cost the writer about
+//     900 cycles per block round); the reader announces the 8 columns it expects and waits for the phase. A set
+//     is overwritten two rounds after it was read: the writer could only finish the round in between after the
+//     reader had finished the round before that (the tournament makes every slot's readers also its suppliers), so
+//     no write overtakes a read. Waits are bounded; one that runs out raises a cluster-wide word, every warp stops
+//     exchanging and the solve ends with an error flag. One cluster barrier per sweep, for the convergence word.
+//   * Exchange, n > 256 (only one set fits): two cluster barriers per block round, "everyone has loaded" (its wait
+//     is hidden behind the local rounds) before the stores, "everyone has stored" before the next loads.
+//   * All threads of the cluster execute the same number of cluster barriers: trip counts depend only on the rank,
+//     the sweep limit and words that all read from global memory after a barrier.
 //   * Cholesky: for n <= 192 CTA 0 factors the matrix alone in its shared memory (a cluster barrier per pivot
 //     step would cost more than it saves) and hands factor, pivot order and rank over through global memory;
 //     for larger n the cluster factors it in global memory (L2) as k_eig_shrink_cluster does.
-// `gwork`: LD*LD floats (factor), then 2 convergence words, the rank, and from +64 on the pivot order (512 ints).
+// `gwork`: LD*LD floats (factor), then 2 convergence words, the rank, the give-up word, and from +64 on the pivot
+// order (512 ints).
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ void cl_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cl_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
@@ -834,6 +854,142 @@ __device__ __forceinline__ void rr_slot_of(int b, int br, int nbm1, int nact, in
     else { slot = nbm1 - d; half = 1; }
 }
 
+// ---- pieces of the cluster exchange: cluster-scope shared-memory addresses, mbarrier operations, async stores ----
+__device__ __forceinline__ uint32_t smem_addr_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t local_addr, uint32_t cta_rank) {   // same offset in another CTA of the cluster
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(cta_rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_init_cluster(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr_u32(bar)), "r"(count) : "memory");
+}
+// The reader's own arrival for the current phase, announcing how many bytes asynchronous stores will deliver.
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr_u32(bar)), "r"(bytes) : "memory");
+}
+// 16 bytes into the shared memory of a CTA of the cluster; the store itself counts its bytes on the barrier (same
+// CTA as the data) when it has landed, so the writer needs neither a fence nor a round trip.
+__device__ __forceinline__ void st_async_v4(uint32_t cluster_addr, const float4& v, uint32_t cluster_bar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(cluster_addr),
+                 "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "r"(cluster_bar)
+                 : "memory");
+}
+constexpr long long kExchangeWaitCycles = 400000000ll;   // about 0.2 s
+// Waits for the phase with the given parity of a barrier in this CTA's shared memory. Bounded: gives up (false) after
+// kExchangeWaitCycles or as soon as another warp of the cluster has given up (*gabort != 0).
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, const int* gabort) {
+    const uint32_t a = smem_addr_u32(bar);
+    const long long t0 = clock64();
+    for (int it = 0;; ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n"
+            ".reg .pred p;\n"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+            "selp.u32 %0, 1, 0, p;\n"
+            "}\n"
+            : "=r"(ok)
+            : "r"(a), "r"(parity)
+            : "memory");
+        if (ok) return true;
+        if ((it & 63) == 63 && (clock64() - t0 > kExchangeWaitCycles || __ldcg(gabort) != 0)) return false;
+    }
+}
+
+// One column pair held in shared memory, 8 lanes per pair (Q float4 per lane and column).
+template <int Q>
+__device__ __forceinline__ void jacobi_pair_in_smem(float* cp, float* cq, bool valid, int l8, float& worst2) {
+    float4* xp = reinterpret_cast<float4*>(cp) + l8;
+    float4* xq = reinterpret_cast<float4*>(cq) + l8;
+    float4 x[Q], y[Q];
+    float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f, g0 = 0.f, g1 = 0.f;
+#pragma unroll
+    for (int t = 0; t < Q; ++t) {
+        x[t] = xp[8 * t];
+        y[t] = xq[8 * t];
+        a0 = fmaf(x[t].x, x[t].x, a0); a1 = fmaf(x[t].y, x[t].y, a1); a0 = fmaf(x[t].z, x[t].z, a0); a1 = fmaf(x[t].w, x[t].w, a1);
+        b0 = fmaf(y[t].x, y[t].x, b0); b1 = fmaf(y[t].y, y[t].y, b1); b0 = fmaf(y[t].z, y[t].z, b0); b1 = fmaf(y[t].w, y[t].w, b1);
+        g0 = fmaf(x[t].x, y[t].x, g0); g1 = fmaf(x[t].y, y[t].y, g1); g0 = fmaf(x[t].z, y[t].z, g0); g1 = fmaf(x[t].w, y[t].w, g1);
+    }
+    float a = a0 + a1, b = b0 + b1, g = g0 + g1;
+#pragma unroll
+    for (int o = 4; o > 0; o >>= 1) {
+        a += __shfl_xor_sync(0xffffffffu, a, o);
+        b += __shfl_xor_sync(0xffffffffu, b, o);
+        g += __shfl_xor_sync(0xffffffffu, g, o);
+    }
+    const float ab = a * b, g2 = g * g;
+    if (valid && ab > 0.f && g2 > 1e-12f * ab) {
+        worst2 = fmaxf(worst2, __fdividef(g2, ab));
+        float c, s;
+        jacobi_rotation(a, b, g, c, s);
+#pragma unroll
+        for (int t = 0; t < Q; ++t) {
+            float4 nx, ny;
+            nx.x = fmaf(-s, y[t].x, c * x[t].x); ny.x = fmaf(s, x[t].x, c * y[t].x);
+            nx.y = fmaf(-s, y[t].y, c * x[t].y); ny.y = fmaf(s, x[t].y, c * y[t].y);
+            nx.z = fmaf(-s, y[t].z, c * x[t].z); ny.z = fmaf(s, x[t].z, c * y[t].z);
+            nx.w = fmaf(-s, y[t].w, c * x[t].w); ny.w = fmaf(s, x[t].w, c * y[t].w);
+            xp[8 * t] = nx;
+            xq[8 * t] = ny;
+        }
+    }
+    __syncwarp();
+}
+
+// The 16 cross pairs of two blocks of 4 columns, columns in registers: quarter qd of the warp keeps column qd of the
+// lower block (x) and meets the 4 columns of the higher block (y) in 4 rounds; between rounds the y columns move to
+// the next quarter by shuffles. Afterwards quarter qd holds column (qd + 3) % 4 of the higher block.
+template <int Q>
+__device__ __forceinline__ void jacobi_cross_rounds(float4 (&x)[Q], float4 (&y)[Q], bool va, int hi, int rank, int qd, int lane,
+                                                    float& worst2) {
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        const bool valid = va && (4 * hi + ((qd + r) & 3) < rank);
+        float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f, g0 = 0.f, g1 = 0.f;
+#pragma unroll
+        for (int t = 0; t < Q; ++t) {
+            a0 = fmaf(x[t].x, x[t].x, a0); a1 = fmaf(x[t].y, x[t].y, a1); a0 = fmaf(x[t].z, x[t].z, a0); a1 = fmaf(x[t].w, x[t].w, a1);
+            b0 = fmaf(y[t].x, y[t].x, b0); b1 = fmaf(y[t].y, y[t].y, b1); b0 = fmaf(y[t].z, y[t].z, b0); b1 = fmaf(y[t].w, y[t].w, b1);
+            g0 = fmaf(x[t].x, y[t].x, g0); g1 = fmaf(x[t].y, y[t].y, g1); g0 = fmaf(x[t].z, y[t].z, g0); g1 = fmaf(x[t].w, y[t].w, g1);
+        }
+        float a = a0 + a1, b = b0 + b1, g = g0 + g1;
+#pragma unroll
+        for (int o = 4; o > 0; o >>= 1) {
+            a += __shfl_xor_sync(0xffffffffu, a, o);
+            b += __shfl_xor_sync(0xffffffffu, b, o);
+            g += __shfl_xor_sync(0xffffffffu, g, o);
+        }
+        const float ab = a * b, g2 = g * g;
+        if (valid && ab > 0.f && g2 > 1e-12f * ab) {
+            worst2 = fmaxf(worst2, __fdividef(g2, ab));
+            float c, s;
+            jacobi_rotation(a, b, g, c, s);
+#pragma unroll
+            for (int t = 0; t < Q; ++t) {
+                float4 nx, ny;
+                nx.x = fmaf(-s, y[t].x, c * x[t].x); ny.x = fmaf(s, x[t].x, c * y[t].x);
+                nx.y = fmaf(-s, y[t].y, c * x[t].y); ny.y = fmaf(s, x[t].y, c * y[t].y);
+                nx.z = fmaf(-s, y[t].z, c * x[t].z); ny.z = fmaf(s, x[t].z, c * y[t].z);
+                nx.w = fmaf(-s, y[t].w, c * x[t].w); ny.w = fmaf(s, x[t].w, c * y[t].w);
+                x[t] = nx;
+                y[t] = ny;
+            }
+        }
+        if (r < 3) {                              // quarter qd takes over the column quarter qd + 1 holds
+            const int src = (lane + 8) & 31;
+#pragma unroll
+            for (int t = 0; t < Q; ++t) {
+                y[t].x = __shfl_sync(0xffffffffu, y[t].x, src);
+                y[t].y = __shfl_sync(0xffffffffu, y[t].y, src);
+                y[t].z = __shfl_sync(0xffffffffu, y[t].z, src);
+                y[t].w = __shfl_sync(0xffffffffu, y[t].w, src);
+            }
+        }
+    }
+}
+
 template <int T, int NT>
 __global__ void __launch_bounds__(NT, 1)
 k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int delta_rank, int keep, float* __restrict__ Ur,
@@ -843,6 +999,8 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
     constexpr int kMaxN = 512;                           // shadows the namespace constant
     constexpr int WPC = NT / 32;                         // warps per CTA
     constexpr bool kLocalChol = T <= 3;                  // CTA 0 factors alone in shared memory
+    constexpr bool kP2P = T <= 4;                        // exchange by asynchronous stores, per-slot barriers and two buffer sets
+    constexpr int kSets = kP2P ? 2 : 1;
     constexpr int R = 2 * T;            // rows per lane when 32 lanes span a column
     constexpr int Q = 2 * T;            // float4 per lane when 8 lanes span a column
     cg::cluster_group cluster = cg::this_cluster();
@@ -859,8 +1017,9 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
     int* perm = ord + kMaxN;                            // pivot step -> physical index
     int* order = perm + kMaxN;                          // sorted position -> pivot step
     float* sh_f = reinterpret_cast<float*>(order + kMaxN);
-    float* sbuf = sh_f + 8;                             // slot buffers: [T slots][2 halves][4 columns][LD]
-    float* Xl = sbuf + T * 8 * LD;                      // LD x LD, kLocalChol only
+    uint64_t* mbar = reinterpret_cast<uint64_t*>(sh_f + 8);   // [2 sets][8 slots] exchange barriers (kP2P)
+    float* sbuf = reinterpret_cast<float*>(mbar + 16);  // slot buffers: [kSets][T slots][2 halves][4 columns][LD]
+    float* Xl = sbuf + kSets * T * 8 * LD;              // LD x LD, kLocalChol only
 
     const int tid = threadIdx.x, lane = tid & 31, lwarp = tid >> 5;
     const int gtid = crank * NT + tid;
@@ -886,7 +1045,9 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
 #pragma unroll
     for (int t = 0; t < R; ++t) dg[t] *= kscale;
     for (int i = tid; i < kMaxN; i += NT) { ord[i] = -1; perm[i] = 0; }
-    if (gtid < 2) gflag[gtid] = 0;
+    if (gtid < 4) gflag[gtid] = 0;
+    if (tid < 16) mbar_init_cluster(&mbar[tid], 1);     // the reader's own arrival; the stores count bytes
+    if (tid == 0) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     const float tol = 1e-7f;
     int rank = empty ? 0 : n;
 
@@ -1046,10 +1207,12 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
     if (rank >= 2) {
         const int nb = (rank + 3) >> 2, nbe = nb + (nb & 1), nbm1 = nbe - 1, nact = nbe >> 1;   // block pairs per round
         const int SPC = (nact + csize - 1) / csize;               // slots per CTA
+        const unsigned spc_inv = (65536u + (unsigned)SPC - 1u) / (unsigned)SPC;   // s / SPC = (s * spc_inv) >> 16 for s < 64
         const int slot = crank * SPC + lwarp;
         const bool fits = SPC <= T && SPC <= WPC;                 // holds for a cluster of 8; otherwise report, do not run
         const bool active = fits && lwarp < SPC && slot < nact;   // the other warps only take part in the barriers
-        float* mybuf = sbuf + (size_t)(lwarp < T ? lwarp : 0) * 8 * LD;
+        const int myslot = lwarp < T ? lwarp : 0;
+        float* mybuf = sbuf + (size_t)myslot * 8 * LD;            // set 0
         if (active) {                                             // columns of block round 0 from the factor in L2
             int ba, bb;
             rr_blocks(slot, 0, nbm1, ba, bb);
@@ -1061,140 +1224,91 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
             }
         }
         __syncwarp();
-        auto pair_step = [&](float* cp, float* cq, bool valid) {   // one column pair of the warp's own buffer
-            float4* xp = reinterpret_cast<float4*>(cp) + l8;
-            float4* xq = reinterpret_cast<float4*>(cq) + l8;
-            float4 x[Q], y[Q];
-            float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f, g0 = 0.f, g1 = 0.f;
-#pragma unroll
-            for (int t = 0; t < Q; ++t) {
-                x[t] = xp[8 * t];
-                y[t] = xq[8 * t];
-                a0 = fmaf(x[t].x, x[t].x, a0); a1 = fmaf(x[t].y, x[t].y, a1); a0 = fmaf(x[t].z, x[t].z, a0); a1 = fmaf(x[t].w, x[t].w, a1);
-                b0 = fmaf(y[t].x, y[t].x, b0); b1 = fmaf(y[t].y, y[t].y, b1); b0 = fmaf(y[t].z, y[t].z, b0); b1 = fmaf(y[t].w, y[t].w, b1);
-                g0 = fmaf(x[t].x, y[t].x, g0); g1 = fmaf(x[t].y, y[t].y, g1); g0 = fmaf(x[t].z, y[t].z, g0); g1 = fmaf(x[t].w, y[t].w, g1);
-            }
-            float a = a0 + a1, b = b0 + b1, g = g0 + g1;
-#pragma unroll
-            for (int o = 4; o > 0; o >>= 1) {
-                a += __shfl_xor_sync(0xffffffffu, a, o);
-                b += __shfl_xor_sync(0xffffffffu, b, o);
-                g += __shfl_xor_sync(0xffffffffu, g, o);
-            }
-            const float ab = a * b, g2 = g * g;
-            if (valid && ab > 0.f && g2 > 1e-12f * ab) {
-                worst2 = fmaxf(worst2, __fdividef(g2, ab));
-                const float zeta = __fdividef(b - a, 2.f * g);
-                const float tt = copysignf(__fdividef(1.f, fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.f))), zeta);
-                const float c = rsqrtf(fmaf(tt, tt, 1.f));
-                const float s = c * tt;
-#pragma unroll
-                for (int t = 0; t < Q; ++t) {
-                    float4 nx, ny;
-                    nx.x = fmaf(-s, y[t].x, c * x[t].x); ny.x = fmaf(s, x[t].x, c * y[t].x);
-                    nx.y = fmaf(-s, y[t].y, c * x[t].y); ny.y = fmaf(s, x[t].y, c * y[t].y);
-                    nx.z = fmaf(-s, y[t].z, c * x[t].z); ny.z = fmaf(s, x[t].z, c * y[t].z);
-                    nx.w = fmaf(-s, y[t].w, c * x[t].w); ny.w = fmaf(s, x[t].w, c * y[t].w);
-                    xp[8 * t] = nx;
-                    xq[8 * t] = ny;
-                }
-            }
-            __syncwarp();
-        };
+        int g = 0;                                                // block rounds done so far, over all sweeps
+        bool failed = false;                                      // an exchange wait ran out (kP2P only)
         while (sweeps < max_sweeps) {
             worst2 = 0.f;
-            for (int br = 0; br < nbm1; ++br) {
+            for (int br = 0; br < nbm1; ++br, ++g) {
                 float4 x[Q], y[Q];
-                int lo = 0, hi = 0;
+                int hi = 0;
                 bool va = false;
-                if (active) {
-                    int ba, bb;
-                    rr_blocks(slot, br, nbm1, ba, bb);
-                    if (br == 0) {                                // pairs inside each block: quarters 0,1 -> ba, 2,3 -> bb
-                        const int half = (qd < 2) ? 0 : 1, base = 4 * (half ? bb : ba), h = qd & 1;
-                        float* blk = mybuf + half * 4 * LD;
-                        const int c0 = h ? 2 : 0, c1 = h ? 3 : 1, c2 = h ? 1 : 0, c3 = h ? 3 : 2, c4 = h ? 1 : 0, c5 = h ? 2 : 3;
-                        pair_step(blk + c0 * LD, blk + c1 * LD, base + c0 < rank && base + c1 < rank);
-                        pair_step(blk + c2 * LD, blk + c3 * LD, base + c2 < rank && base + c3 < rank);
-                        pair_step(blk + c4 * LD, blk + c5 * LD, base + c4 < rank && base + c5 < rank);
+                float4 *o_lo = nullptr, *o_hi = nullptr;                // !kP2P: generic pointers into the readers' buffers
+                uint32_t a_lo = 0, a_hi = 0, bar_lo = 0, bar_hi = 0;   // kP2P: cluster addresses of data and barriers
+                const bool work = active && !failed;
+                bool loaded = false;
+                if (work) {
+                    float* cur = kP2P ? sbuf + (size_t)((g & 1) * T + myslot) * 8 * LD : mybuf;
+                    bool ok = true;
+                    if (kP2P && g > 0) {                          // both blocks of this round have landed in this set
+                        if (lane == 0) mbar_arrive_expect_tx(&mbar[(g & 1) * 8 + myslot], 8u * LD * sizeof(float));
+                        ok = mbar_wait_cluster(&mbar[(g & 1) * 8 + myslot], (uint32_t)((g - 1) >> 1) & 1u, &gflag[3]);
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (!ok) {
+                            failed = true;
+                            if (lane == 0) atomicOr(&gflag[3], 1);
+                        }
                     }
-                    lo = min(ba, bb);
-                    hi = max(ba, bb);
-                    const int half_lo = (ba < bb) ? 0 : 1;
-                    // quarter qd keeps column qd of block lo; the columns of block hi travel between quarters
-                    const float4* xa = reinterpret_cast<const float4*>(mybuf + (half_lo * 4 + qd) * LD) + l8;
-                    const float4* xb = reinterpret_cast<const float4*>(mybuf + ((1 - half_lo) * 4 + qd) * LD) + l8;
-                    va = 4 * lo + qd < rank;
-#pragma unroll
-                    for (int t = 0; t < Q; ++t) {
-                        x[t] = xa[8 * t];
-                        y[t] = xb[8 * t];
-                    }
-                }
-                cl_arrive();                                       // "loaded": completes while the local rounds run
-                if (active) {
-#pragma unroll
-                    for (int r = 0; r < 4; ++r) {
-                        const bool valid = va && (4 * hi + ((qd + r) & 3) < rank);
-                        float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f, g0 = 0.f, g1 = 0.f;
+                    if (ok) {
+                        loaded = true;
+                        int ba, bb;
+                        rr_blocks(slot, br, nbm1, ba, bb);
+                        if (br == 0) {                            // pairs inside each block: quarters 0,1 -> ba, 2,3 -> bb
+                            const int half = (qd < 2) ? 0 : 1, base = 4 * (half ? bb : ba), h = qd & 1;
+                            float* blk = cur + half * 4 * LD;
+                            const int c0 = h ? 2 : 0, c1 = h ? 3 : 1, c2 = h ? 1 : 0, c3 = h ? 3 : 2, c4 = h ? 1 : 0, c5 = h ? 2 : 3;
+                            jacobi_pair_in_smem<Q>(blk + c0 * LD, blk + c1 * LD, base + c0 < rank && base + c1 < rank, l8, worst2);
+                            jacobi_pair_in_smem<Q>(blk + c2 * LD, blk + c3 * LD, base + c2 < rank && base + c3 < rank, l8, worst2);
+                            jacobi_pair_in_smem<Q>(blk + c4 * LD, blk + c5 * LD, base + c4 < rank && base + c5 < rank, l8, worst2);
+                        }
+                        const int lo = min(ba, bb);
+                        hi = max(ba, bb);
+                        const int half_lo = (ba < bb) ? 0 : 1;
+                        // quarter qd keeps column qd of block lo; the columns of block hi travel between quarters
+                        const float4* xa = reinterpret_cast<const float4*>(cur + (half_lo * 4 + qd) * LD) + l8;
+                        const float4* xb = reinterpret_cast<const float4*>(cur + ((1 - half_lo) * 4 + qd) * LD) + l8;
+                        va = 4 * lo + qd < rank;
 #pragma unroll
                         for (int t = 0; t < Q; ++t) {
-                            a0 = fmaf(x[t].x, x[t].x, a0); a1 = fmaf(x[t].y, x[t].y, a1); a0 = fmaf(x[t].z, x[t].z, a0); a1 = fmaf(x[t].w, x[t].w, a1);
-                            b0 = fmaf(y[t].x, y[t].x, b0); b1 = fmaf(y[t].y, y[t].y, b1); b0 = fmaf(y[t].z, y[t].z, b0); b1 = fmaf(y[t].w, y[t].w, b1);
-                            g0 = fmaf(x[t].x, y[t].x, g0); g1 = fmaf(x[t].y, y[t].y, g1); g0 = fmaf(x[t].z, y[t].z, g0); g1 = fmaf(x[t].w, y[t].w, g1);
+                            x[t] = xa[8 * t];
+                            y[t] = xb[8 * t];
                         }
-                        float a = a0 + a1, b = b0 + b1, g = g0 + g1;
-#pragma unroll
-                        for (int o = 4; o > 0; o >>= 1) {
-                            a += __shfl_xor_sync(0xffffffffu, a, o);
-                            b += __shfl_xor_sync(0xffffffffu, b, o);
-                            g += __shfl_xor_sync(0xffffffffu, g, o);
-                        }
-                        const float ab = a * b, g2 = g * g;
-                        if (valid && ab > 0.f && g2 > 1e-12f * ab) {
-                            worst2 = fmaxf(worst2, __fdividef(g2, ab));
-                            const float zeta = __fdividef(b - a, 2.f * g);
-                            const float tt = copysignf(__fdividef(1.f, fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.f))), zeta);
-                            const float c = rsqrtf(fmaf(tt, tt, 1.f));
-                            const float s = c * tt;
-#pragma unroll
-                            for (int t = 0; t < Q; ++t) {
-                                float4 nx, ny;
-                                nx.x = fmaf(-s, y[t].x, c * x[t].x); ny.x = fmaf(s, x[t].x, c * y[t].x);
-                                nx.y = fmaf(-s, y[t].y, c * x[t].y); ny.y = fmaf(s, x[t].y, c * y[t].y);
-                                nx.z = fmaf(-s, y[t].z, c * x[t].z); ny.z = fmaf(s, x[t].z, c * y[t].z);
-                                nx.w = fmaf(-s, y[t].w, c * x[t].w); ny.w = fmaf(s, x[t].w, c * y[t].w);
-                                x[t] = nx;
-                                y[t] = ny;
-                            }
-                        }
-                        if (r < 3) {                              // quarter qd takes over the column quarter qd + 1 holds
-                            const int src = (lane + 8) & 31;
-#pragma unroll
-                            for (int t = 0; t < Q; ++t) {
-                                y[t].x = __shfl_sync(0xffffffffu, y[t].x, src);
-                                y[t].y = __shfl_sync(0xffffffffu, y[t].y, src);
-                                y[t].z = __shfl_sync(0xffffffffu, y[t].z, src);
-                                y[t].w = __shfl_sync(0xffffffffu, y[t].w, src);
-                            }
+                        // where the next block round reads the two columns this quarter ends up with
+                        const int brn = (br + 1 == nbm1) ? 0 : br + 1;
+                        int s_lo, h_lo, s_hi, h_hi;
+                        rr_slot_of(lo, brn, nbm1, nact, s_lo, h_lo);
+                        rr_slot_of(hi, brn, nbm1, nact, s_hi, h_hi);
+                        const int c_lo = (int)(((unsigned)s_lo * spc_inv) >> 16), c_hi = (int)(((unsigned)s_hi * spc_inv) >> 16);
+                        const int l_lo = s_lo - c_lo * SPC, l_hi = s_hi - c_hi * SPC;
+                        const int nset = kP2P ? ((g + 1) & 1) : 0;
+                        float* d_lo = sbuf + ((size_t)(nset * T + l_lo) * 8 + h_lo * 4 + qd) * LD + 4 * l8;                // in CTA c_lo
+                        float* d_hi = sbuf + ((size_t)(nset * T + l_hi) * 8 + h_hi * 4 + ((qd + 3) & 3)) * LD + 4 * l8;    // in CTA c_hi
+                        if (kP2P) {
+                            a_lo = mapa_u32(smem_addr_u32(d_lo), (uint32_t)c_lo);
+                            a_hi = mapa_u32(smem_addr_u32(d_hi), (uint32_t)c_hi);
+                            bar_lo = mapa_u32(smem_addr_u32(&mbar[nset * 8 + l_lo]), (uint32_t)c_lo);
+                            bar_hi = mapa_u32(smem_addr_u32(&mbar[nset * 8 + l_hi]), (uint32_t)c_hi);
+                        } else {
+                            o_lo = reinterpret_cast<float4*>(cluster.map_shared_rank(d_lo, c_lo));
+                            o_hi = reinterpret_cast<float4*>(cluster.map_shared_rank(d_hi, c_hi));
                         }
                     }
                 }
-                cl_wait();                                         // every warp of the cluster holds its columns in registers
-                if (active) {                                      // store each column where the next block round reads it
-                    const int brn = (br + 1 == nbm1) ? 0 : br + 1;
-                    int s_lo, h_lo, s_hi, h_hi;
-                    rr_slot_of(lo, brn, nbm1, nact, s_lo, h_lo);
-                    rr_slot_of(hi, brn, nbm1, nact, s_hi, h_hi);
-                    const int c_lo = s_lo / SPC, c_hi = s_hi / SPC;
-                    float* d_lo = cluster.map_shared_rank(sbuf, c_lo) + ((size_t)(s_lo - c_lo * SPC) * 8 + h_lo * 4 + qd) * LD;
-                    float* d_hi = cluster.map_shared_rank(sbuf, c_hi) + ((size_t)(s_hi - c_hi * SPC) * 8 + h_hi * 4 + ((qd + 3) & 3)) * LD;
-                    float4* o_lo = reinterpret_cast<float4*>(d_lo) + l8;
-                    float4* o_hi = reinterpret_cast<float4*>(d_hi) + l8;
+                if (!kP2P) cl_arrive();                            // "loaded": completes while the local rounds run
+                if (loaded) jacobi_cross_rounds<Q>(x, y, va, hi, rank, qd, lane, worst2);
+                if (!kP2P) cl_wait();                              // every warp of the cluster holds its columns in registers
+                if (loaded) {                                      // send each column to where the next block round reads it
+                    if (kP2P) {                                    // asynchronous stores that count their bytes on the reader's barrier
 #pragma unroll
-                    for (int t = 0; t < Q; ++t) {
-                        o_lo[8 * t] = x[t];
-                        o_hi[8 * t] = y[t];
+                        for (int t = 0; t < Q; ++t) {
+                            st_async_v4(a_lo + 128u * t, x[t], bar_lo);
+                            st_async_v4(a_hi + 128u * t, y[t], bar_hi);
+                        }
+                    } else {
+#pragma unroll
+                        for (int t = 0; t < Q; ++t) {
+                            o_lo[8 * t] = x[t];
+                            o_hi[8 * t] = y[t];
+                        }
                     }
                 }
                 if (br == nbm1 - 1) {                              // end of a sweep: publish whether anything still rotated
@@ -1202,15 +1316,28 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
                     if (__any_sync(0xffffffffu, worst2 > 1e-6f) && lane == 0) atomicOr(&gflag[par], 1);
                     if (gtid == 0) gflag[par ^ 1] = 0;
                 }
-                cl_arrive();
-                cl_wait();                                         // "stored": the next block round may load
+                if (!kP2P || br == nbm1 - 1) {
+                    cl_arrive();
+                    cl_wait();                                     // "stored" (kP2P: once per sweep, for the convergence word)
+                }
             }
             ++sweeps;
             more = fits ? __ldcg(&gflag[sweeps & 1]) : 1;
+            if (kP2P && __ldcg(&gflag[3])) { more = 2; break; }    // an exchange wait ran out somewhere: stop everywhere
             if (!more) break;               // every cosine of this sweep was below 1e-3: converged after it
             if (!fits) break;
         }
-        if (active) {                                             // back to the factor in L2, for the final phase
+        if (kP2P && active && more != 2 && g > 0) {               // the last round's columns: wait for them like any round's
+            if (lane == 0) mbar_arrive_expect_tx(&mbar[(g & 1) * 8 + myslot], 8u * LD * sizeof(float));
+            bool ok = mbar_wait_cluster(&mbar[(g & 1) * 8 + myslot], (uint32_t)((g - 1) >> 1) & 1u, &gflag[3]);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) {
+                failed = true;
+                if (lane == 0) atomicOr(&gflag[3], 1);
+            }
+        }
+        if (active && more != 2 && !failed) {                     // back to the factor in L2, for the final phase
+            const float* cur = kP2P ? sbuf + (size_t)((g & 1) * T + myslot) * 8 * LD : mybuf;
             int ba, bb;
             rr_blocks(slot, 0, nbm1, ba, bb);
             for (int hc = 0; hc < 8; ++hc) {
@@ -1218,12 +1345,14 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
                 if (p < rank) {
                     float* dst = X + (size_t)perm[p] * LD;
 #pragma unroll
-                    for (int t = 0; t < R; ++t) dst[lane + 32 * t] = mybuf[hc * LD + lane + 32 * t];
+                    for (int t = 0; t < R; ++t) dst[lane + 32 * t] = cur[hc * LD + lane + 32 * t];
                 }
             }
         }
     }
     cluster.sync();
+    if (kP2P && __ldcg(&gflag[3])) more = 2;
+    if (more == 2 && gtid == 0) atomicOr(&info->flags, kFlagExchangeTimeout);
     const int not_converged = rank >= 2 && more != 0;          // stopped at the sweep limit while still rotating visibly
     // ---- eigenvalues = squared column norms (pivot-step order), scaled back; sort descending, stable ----
     for (int k = lwarp; k < n; k += WPC) {                          // every CTA forms all eigenvalues for its own tables
@@ -1535,11 +1664,11 @@ cudaError_t launch_eig_shrink(const float* K, int ldk, int n, int do_shrink, int
                               float* sigma_out, int n_sigma, float* work, int max_sweeps, EigInfo* info, float* Wsplit, int ldw,
                               int j_pad, int variant, cudaStream_t st) {
     if (n <= 0 || n > 512) return cudaErrorInvalidValue;
-    if (variant == 0) {   // cluster of 8 CTAs, Jacobi columns in distributed shared memory
+    if (variant == 0 && n > 64) {   // cluster of 8 CTAs, Jacobi columns in distributed shared memory (n <= 64: one CTA is as fast)
         const int T = n <= 64 ? 1 : n <= 128 ? 2 : n <= 192 ? 3 : n <= 256 ? 4 : 8;
         const int LD = 64 * T;
-        const size_t bytes = 3 * 512 * sizeof(float) + 3 * 512 * sizeof(int) + 32 + (size_t)T * 8 * LD * sizeof(float) +
-                             (T <= 3 ? (size_t)LD * LD * sizeof(float) : 0);
+        const size_t bytes = 3 * 512 * sizeof(float) + 3 * 512 * sizeof(int) + 32 + 16 * sizeof(uint64_t) +
+                             (size_t)(T <= 4 ? 2 : 1) * T * 8 * LD * sizeof(float) + (T <= 3 ? (size_t)LD * LD * sizeof(float) : 0);
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(8);
         cfg.blockDim = dim3(T <= 3 ? 512 : 256);

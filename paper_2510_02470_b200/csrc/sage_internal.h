@@ -12,6 +12,7 @@ namespace sage {
 // Device-side flags accumulated in the handle's status word.
 constexpr uint32_t kFlagNotConverged = 1u;
 constexpr uint32_t kFlagNonFinite = 2u;
+constexpr uint32_t kFlagExchangeTimeout = 8u;   // a bounded wait between thread blocks of the eigen-solve ran out (4: tensor-core waits)
 
 // Results of one eigen-solve, written by the eigen kernel and read by later kernels / stats.
 struct EigInfo {
