@@ -814,7 +814,7 @@ k_eig_shrink_cluster(const float* __restrict__ K, int ldk, int n, int do_shrink,
 //     rotate the 16 cross pairs in 4 local rounds (as in the one-CTA kernel), then store every column straight
 //     into the slot buffer of the warp that needs it next (a remote shared-memory store when that warp sits in
 //     another CTA; the tournament moves a block to a neighbouring slot, so most stores stay local).
-//   * Exchange, n <= 256: two buffer sets per slot, used by alternate block rounds, and one mbarrier per slot and
+//   * Exchange, n <= 192: two buffer sets per slot, used by alternate block rounds, and one mbarrier per slot and
 //     set. A warp sends its columns into the reader's other set with asynchronous stores (st.async) that count
 //     their bytes on the reader's barrier as they land: one-way latency, no fence or round trip on the writer's
 //     side (a plain remote store followed by a releasing arrival, or by a cluster barrier, cost the writer about
@@ -823,7 +823,8 @@ k_eig_shrink_cluster(const float* __restrict__ K, int ldk, int n, int do_shrink,
 //     reader had finished the round before that (the tournament makes every slot's readers also its suppliers), so
 //     no write overtakes a read. Waits are bounded; one that runs out raises a cluster-wide word, every warp stops
 //     exchanging and the solve ends with an error flag. One cluster barrier per sweep, for the convergence word.
-//   * Exchange, n > 256 (only one set fits): two cluster barriers per block round, "everyone has loaded" (its wait
+//   * Exchange, n > 192 (asynchronous stores of 16 bytes become the bottleneck: 16 and more per lane and round
+//     measured slower than plain remote stores; above 256 only one set fits anyway): two cluster barriers per block round, "everyone has loaded" (its wait
 //     is hidden behind the local rounds) before the stores, "everyone has stored" before the next loads.
 //   * All threads of the cluster execute the same number of cluster barriers: trip counts depend only on the rank,
 //     the sweep limit and words that all read from global memory after a barrier.
@@ -999,7 +1000,7 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
     constexpr int kMaxN = 512;                           // shadows the namespace constant
     constexpr int WPC = NT / 32;                         // warps per CTA
     constexpr bool kLocalChol = T <= 3;                  // CTA 0 factors alone in shared memory
-    constexpr bool kP2P = T <= 4;                        // exchange by asynchronous stores, per-slot barriers and two buffer sets
+    constexpr bool kP2P = T <= 3;                        // exchange by asynchronous stores, per-slot barriers and two buffer sets
     constexpr int kSets = kP2P ? 2 : 1;
     constexpr int R = 2 * T;            // rows per lane when 32 lanes span a column
     constexpr int Q = 2 * T;            // float4 per lane when 8 lanes span a column
@@ -1668,7 +1669,7 @@ cudaError_t launch_eig_shrink(const float* K, int ldk, int n, int do_shrink, int
         const int T = n <= 64 ? 1 : n <= 128 ? 2 : n <= 192 ? 3 : n <= 256 ? 4 : 8;
         const int LD = 64 * T;
         const size_t bytes = 3 * 512 * sizeof(float) + 3 * 512 * sizeof(int) + 32 + 16 * sizeof(uint64_t) +
-                             (size_t)(T <= 4 ? 2 : 1) * T * 8 * LD * sizeof(float) + (T <= 3 ? (size_t)LD * LD * sizeof(float) : 0);
+                             (size_t)(T <= 3 ? 2 : 1) * T * 8 * LD * sizeof(float) + (T <= 3 ? (size_t)LD * LD * sizeof(float) : 0);
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(8);
         cfg.blockDim = dim3(T <= 3 ? 512 : 256);
