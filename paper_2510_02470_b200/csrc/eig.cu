@@ -828,11 +828,10 @@ k_eig_shrink_cluster(const float* __restrict__ K, int ldk, int n, int do_shrink,
 //     is hidden behind the local rounds) before the stores, "everyone has stored" before the next loads.
 //   * All threads of the cluster execute the same number of cluster barriers: trip counts depend only on the rank,
 //     the sweep limit and words that all read from global memory after a barrier.
-//   * Cholesky: for n <= 192 CTA 0 factors the matrix alone in its shared memory (a cluster barrier per pivot
-//     step would cost more than it saves) and hands factor, pivot order and rank over through global memory;
-//     for larger n the cluster factors it in global memory (L2) as k_eig_shrink_cluster does.
-// `gwork`: LD*LD floats (factor), then 2 convergence words, the rank, the give-up word, and from +64 on the pivot
-// order (512 ints).
+//   * Cholesky: the columns are dealt to the 8 CTAs and stay in their shared memory; the pivot column of a step
+//     reaches every CTA by asynchronous stores (see the comment at the loop). The factor is handed to the Jacobi
+//     phase through global memory (L2), so both phases can use the same shared memory.
+// `gwork`: LD*LD floats (factor), then 2 convergence words, a spare word and the give-up word.
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ void cl_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cl_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
@@ -864,6 +863,12 @@ __device__ __forceinline__ uint32_t mapa_u32(uint32_t local_addr, uint32_t cta_r
 }
 __device__ __forceinline__ void mbar_init_cluster(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_local(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {   // a barrier of any CTA of the cluster
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // The reader's own arrival for the current phase, announcing how many bytes asynchronous stores will deliver.
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
@@ -999,9 +1004,7 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
     constexpr int LD = 64 * T;
     constexpr int kMaxN = 512;                           // shadows the namespace constant
     constexpr int WPC = NT / 32;                         // warps per CTA
-    constexpr bool kLocalChol = T <= 3;                  // CTA 0 factors alone in shared memory
     constexpr bool kP2P = T <= 3;                        // exchange by asynchronous stores, per-slot barriers and two buffer sets
-    constexpr int kSets = kP2P ? 2 : 1;
     constexpr int R = 2 * T;            // rows per lane when 32 lanes span a column
     constexpr int Q = 2 * T;            // float4 per lane when 8 lanes span a column
     cg::cluster_group cluster = cg::this_cluster();
@@ -1010,7 +1013,6 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
     extern __shared__ __align__(16) float smem[];
     float* X = gwork;                                   // LD x LD factor in global memory (L2)
     int* gflag = reinterpret_cast<int*>(gwork + (size_t)LD * LD);   // [0],[1] convergence words, [2] rank
-    int* gperm = gflag + 64;                            // pivot step -> physical index (kLocalChol hand-over)
     float* lam = smem;                                  // kMaxN each from here on (one copy per CTA)
     float* fac = lam + kMaxN;
     float* scl = fac + kMaxN;
@@ -1019,8 +1021,12 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
     int* order = perm + kMaxN;                          // sorted position -> pivot step
     float* sh_f = reinterpret_cast<float*>(order + kMaxN);
     uint64_t* mbar = reinterpret_cast<uint64_t*>(sh_f + 8);   // [2 sets][8 slots] exchange barriers (kP2P)
-    float* sbuf = reinterpret_cast<float*>(mbar + 16);  // slot buffers: [kSets][T slots][2 halves][4 columns][LD]
-    float* Xl = sbuf + kSets * T * 8 * LD;              // LD x LD, kLocalChol only
+    uint64_t* pbar = mbar + 16;                         // Cholesky phase: [2] pivot column landed (bytes), then
+    uint64_t* cdone = mbar + 18;                        // [2] every warp of this CTA has finished the step, and
+    uint64_t* alldone = mbar + 20;                      // [2] every CTA of the cluster has
+    uint32_t* sched = reinterpret_cast<uint32_t*>(mbar + 24);   // [T slots][128 block rounds] packed exchange schedule
+    float* pbuf = reinterpret_cast<float*>(sched + T * 128);    // [2][LD] pivot columns of the Cholesky phase
+    float* sbuf = pbuf + 2 * LD;                        // slot buffers: [kSets][T slots][2 halves][4 columns][LD]
 
     const int tid = threadIdx.x, lane = tid & 31, lwarp = tid >> 5;
     const int gtid = crank * NT + tid;
@@ -1047,159 +1053,144 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
     for (int t = 0; t < R; ++t) dg[t] *= kscale;
     for (int i = tid; i < kMaxN; i += NT) { ord[i] = -1; perm[i] = 0; }
     if (gtid < 4) gflag[gtid] = 0;
-    if (tid < 16) mbar_init_cluster(&mbar[tid], 1);     // the reader's own arrival; the stores count bytes
+    if (tid < 18) mbar_init_cluster(&mbar[tid], 1);     // the reader's own arrival; the stores count bytes
+    if (tid >= 18 && tid < 20) mbar_init_cluster(&mbar[tid], WPC);
+    if (tid >= 20 && tid < 22) mbar_init_cluster(&mbar[tid], 8);
     if (tid == 0) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     const float tol = 1e-7f;
     int rank = empty ? 0 : n;
 
-    if constexpr (kLocalChol) {
-        if (crank == 0) {
-            for (int e = tid; e < n * LD; e += NT) {
-                const int c = e / LD, i = e - c * LD;
-                Xl[e] = (i < n) ? K[(size_t)c * ldk + i] * kscale : 0.f;  // K is symmetric: row c serves as column c
-            }
-            __syncthreads();
-            // ---- pivoted Cholesky without swaps, one CTA (see k_eig_shrink_fast) ----
-            constexpr int CW = (LD + WPC - 1) / WPC;                   // columns a warp owns: lwarp + WPC u
-            unsigned colmask = 0u;
+    // ---- pivoted Cholesky without swaps, columns dealt to the 8 CTAs (physical column j lives in CTA j % 8) ----
+    // Every warp of the cluster finds the pivot from its own copy of the running diagonal (identical everywhere).
+    // The warp that owns the pivot column sends it to all 8 CTAs with asynchronous stores that count their bytes
+    // on a barrier in each CTA; every warp waits for that, refreshes its diagonal and updates the columns it owns
+    // in its CTA's shared memory: a step costs one one-way trip instead of a cluster barrier plus L2 round trips,
+    // and the trailing update has the shared-memory bandwidth of 8 SMs. The two pivot buffers alternate; before a
+    // warp overwrites the buffer of step k - 2 it waits until every CTA has reported that step finished (each warp
+    // arrives on its CTA's `cdone` barrier at the end of a step; warp 0 of each CTA waits for that and arrives on
+    // the `alldone` barrier of all 8 CTAs: a whole step of slack, so the sender rarely waits). Every wait is bounded;
+    // one that runs out raises the cluster-wide give-up word, which ends all other waits, and every warp leaves the
+    // loop for the same barriers below.
+    constexpr int CPC = LD / 8;                          // local columns per CTA
+    constexpr int CW = (CPC + WPC - 1) / WPC;            // local columns a warp owns: lwarp + WPC u
+    float* Xc = sbuf;                                    // [CPC][LD], reuses the slot buffers (the hand-over goes through L2)
+    const bool geometry_ok = csize == 8;                 // the layout above assumes the cluster this kernel is launched with
+    if (!geometry_ok) rank = 0;
+    unsigned colmask = 0u;                               // bit u: local column lwarp + WPC u is still unpivoted
 #pragma unroll
-            for (int u = 0; u < CW; ++u)
-                if (lwarp + WPC * u < n) colmask |= 1u << u;
-            for (int k = 0; k < rank; ++k) {
-                unsigned key = 0u;
-#pragma unroll
-                for (int t = 0; t < R; ++t)
-                    if (alive[t]) key = max(key, (__float_as_uint(fmaxf(dg[t], 0.f)) & 0xffffff00u) | (unsigned)(255 - (lane + 32 * t)));
-                key = __reduce_max_sync(0xffffffffu, key);
-                const int p = 255 - (int)(key & 255u);
-                if (key == 0u || p >= n) { rank = k; break; }             // identical in every warp
-                const float* Xp = Xl + p * LD;
-                const float d = Xp[p];
-                if (!(d > tol)) { rank = k; break; }
-                const float inv = rsqrtf(d);
-                if ((p % WPC) == lwarp) colmask &= ~(1u << (p / WPC));
-                float li[R];
-#pragma unroll
-                for (int t = 0; t < R; ++t) {
-                    const int i = lane + 32 * t;
-                    if (i == p) alive[t] = false;
-                    li[t] = alive[t] ? Xp[i] * inv : 0.f;
-                    dg[t] = fmaf(-li[t], li[t], dg[t]);
-                }
-#pragma unroll
-                for (int u0 = 0; u0 < CW; u0 += 2) {                      // two columns at a time: loads first, then stores
-                    const bool on0 = (colmask >> u0) & 1u, on1 = (u0 + 1 < CW) && ((colmask >> (u0 + 1)) & 1u);
-                    if (!on0 && !on1) continue;
-                    float* c0 = Xl + (lwarp + WPC * u0) * LD;
-                    float* c1 = Xl + (lwarp + WPC * (u0 + 1)) * LD;
-                    const float l0 = on0 ? Xp[lwarp + WPC * u0] * inv : 0.f;
-                    const float l1 = on1 ? Xp[lwarp + WPC * (u0 + 1)] * inv : 0.f;
-                    float v0[R], v1[R];
-#pragma unroll
-                    for (int t = 0; t < R; ++t) {
-                        v0[t] = on0 ? c0[lane + 32 * t] : 0.f;
-                        v1[t] = on1 ? c1[lane + 32 * t] : 0.f;
-                    }
-#pragma unroll
-                    for (int t = 0; t < R; ++t) {
-                        if (on0) c0[lane + 32 * t] = fmaf(-li[t], l0, v0[t]);
-                        if (on1) c1[lane + 32 * t] = fmaf(-li[t], l1, v1[t]);
-                    }
-                }
-                if (tid == 0) { ord[p] = k; perm[k] = p; scl[k] = inv; }
-                __syncthreads();
-            }
-            __syncthreads();
-            // factor L into global memory (zero above the pivot order, zero unpivoted columns) + the hand-over words
-            for (int e = tid; e < n * LD; e += NT) {
-                const int c = e / LD, i = e - c * LD;
-                const int kc = ord[c];
-                float v = 0.f;
-                if (kc >= 0 && i < n) {
-                    const int ki = ord[i];
-                    if (!(ki >= 0 && ki < kc)) v = Xl[e] * scl[kc];
-                }
-                X[e] = v;
-            }
-            for (int i = tid; i < n; i += NT) gperm[i] = perm[i];
-            if (tid == 0) gflag[2] = rank;
-        }
-        cluster.sync();
-        rank = __ldcg(&gflag[2]);
-        if (crank != 0)
-            for (int i = tid; i < n; i += NT) perm[i] = __ldcg(&gperm[i]);
-        __syncthreads();
-    } else {
-        const int NW = WPC * csize;                          // warps of the whole cluster
-        const int warp = crank * WPC + lwarp;
-        for (int e = gtid; e < n * LD; e += GT) {
-            const int c = e / LD, i = e - c * LD;
-            X[e] = (i < n) ? K[(size_t)c * ldk + i] * kscale : 0.f;
-        }
-        cluster.sync();
-        // ---- pivoted Cholesky without swaps, whole cluster, matrix in L2 (see k_eig_shrink_cluster) ----
-        constexpr int CW = (LD + 63) / 64 * 2;                     // upper bound of columns a warp owns for NW >= 32
-        unsigned colmask = 0u;
-#pragma unroll
-        for (int u = 0; u < CW; ++u)
-            if (warp + NW * u < n) colmask |= 1u << u;
-        for (int k = 0; k < rank; ++k) {
-            unsigned key = 0u;
-#pragma unroll
-            for (int t = 0; t < R; ++t)
-                if (alive[t]) key = max(key, (__float_as_uint(fmaxf(dg[t], 0.f)) & 0xfffffe00u) | (unsigned)(511 - (lane + 32 * t)));
-            key = __reduce_max_sync(0xffffffffu, key);
-            const int p = 511 - (int)(key & 511u);
-            if (key == 0u || p >= n) { rank = k; break; }             // identical in every warp of the cluster
-            const float* Xp = X + p * LD;
-            const float d = __ldcg(Xp + p);
-            if (!(d > tol)) { rank = k; break; }
-            const float inv = rsqrtf(d);
-            if ((p % NW) == warp) colmask &= ~(1u << (p / NW));
-            float li[R];
+    for (int u = 0; u < CW; ++u) {
+        const int jl = lwarp + WPC * u, j = jl * 8 + crank;
+        if (jl < CPC && j < n && geometry_ok) {
+            colmask |= 1u << u;
 #pragma unroll
             for (int t = 0; t < R; ++t) {
                 const int i = lane + 32 * t;
-                if (i == p) alive[t] = false;
-                li[t] = alive[t] ? __ldcg(Xp + i) * inv : 0.f;
-                dg[t] = fmaf(-li[t], li[t], dg[t]);
+                Xc[jl * LD + i] = (i < n) ? K[(size_t)j * ldk + i] * kscale : 0.f;   // K is symmetric: row j serves as column j
             }
-#pragma unroll
-            for (int u0 = 0; u0 < CW; u0 += 2) {
-                const bool on0 = (colmask >> u0) & 1u, on1 = (u0 + 1 < CW) && ((colmask >> (u0 + 1)) & 1u);
-                if (!on0 && !on1) continue;
-                float* c0 = X + (warp + NW * u0) * LD;
-                float* c1 = X + (warp + NW * (u0 + 1)) * LD;
-                const float l0 = on0 ? __ldcg(Xp + warp + NW * u0) * inv : 0.f;
-                const float l1 = on1 ? __ldcg(Xp + warp + NW * (u0 + 1)) * inv : 0.f;
-                float v0[R], v1[R];
-#pragma unroll
-                for (int t = 0; t < R; ++t) {
-                    v0[t] = on0 ? __ldcg(c0 + lane + 32 * t) : 0.f;
-                    v1[t] = on1 ? __ldcg(c1 + lane + 32 * t) : 0.f;
-                }
-#pragma unroll
-                for (int t = 0; t < R; ++t) {
-                    if (on0) c0[lane + 32 * t] = fmaf(-li[t], l0, v0[t]);
-                    if (on1) c1[lane + 32 * t] = fmaf(-li[t], l1, v1[t]);
-                }
-            }
-            if (tid == 0) { ord[p] = k; perm[k] = p; scl[k] = inv; }   // every CTA keeps its own copy of the tables
-            cluster.sync();
         }
-        cluster.sync();
-        for (int e = gtid; e < n * LD; e += GT) {
-            const int c = e / LD, i = e - c * LD;
-            const int kc = ord[c];
-            float v = 0.f;
-            if (kc >= 0 && i < n) {
-                const int ki = ord[i];
-                if (!(ki >= 0 && ki < kc)) v = __ldcg(X + e) * scl[kc];
-            }
-            X[e] = v;
-        }
-        cluster.sync();
     }
+    __syncwarp();
+    cluster.sync();                                      // barriers initialised everywhere before the first remote store
+    bool chol_failed = false;
+    for (int k = 0; k < rank; ++k) {
+        unsigned key = 0u;
+#pragma unroll
+        for (int t = 0; t < R; ++t)
+            if (alive[t]) key = max(key, (__float_as_uint(fmaxf(dg[t], 0.f)) & 0xfffffe00u) | (unsigned)(511 - (lane + 32 * t)));
+        key = __reduce_max_sync(0xffffffffu, key);                // largest diagonal (23 significant bits), smaller index on ties
+        const int p = 511 - (int)(key & 511u);
+        if (key == 0u || p >= n) { rank = k; break; }             // identical in every warp of the cluster
+        const int set = k & 1;
+        float* pb = pbuf + set * LD;
+        {
+            const int ojl = p >> 3;
+            if ((p & 7) == crank && (ojl % WPC) == lwarp) {       // this warp owns the pivot column: send it to all 8 CTAs
+                if (k >= 2) {                                     // ... once nobody reads the step before last any more
+                    bool free_ = mbar_wait_cluster(&alldone[set], (uint32_t)((k >> 1) - 1) & 1u, &gflag[3]);
+                    free_ = __all_sync(0xffffffffu, free_);
+                    if (!free_) {
+                        if (lane == 0) atomicOr(&gflag[3], 1);
+                        chol_failed = true;
+                        break;
+                    }
+                }
+                const float4* src = reinterpret_cast<const float4*>(Xc + ojl * LD);
+                const uint32_t dst0 = smem_addr_u32(pb), bar0 = smem_addr_u32(&pbar[set]);
+                for (int q = lane; q < LD / 4; q += 32) {
+                    const float4 v = src[q];
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) st_async_v4(mapa_u32(dst0 + 16u * q, (uint32_t)c), v, mapa_u32(bar0, (uint32_t)c));
+                }
+                colmask &= ~(1u << (ojl / WPC));
+            }
+        }
+        if (tid == 0) mbar_arrive_expect_tx(&pbar[set], (uint32_t)(LD * sizeof(float)));
+        bool ok = mbar_wait_cluster(&pbar[set], (uint32_t)(k >> 1) & 1u, &gflag[3]);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) {
+            if (lane == 0) atomicOr(&gflag[3], 1);
+            chol_failed = true;
+            break;
+        }
+        const float d = pb[p];
+        if (!(d > tol)) { rank = k; break; }                      // identical everywhere: all read the same column
+        const float inv = rsqrtf(d);
+        float li[R];
+#pragma unroll
+        for (int t = 0; t < R; ++t) {
+            const int i = lane + 32 * t;
+            if (i == p) alive[t] = false;
+            li[t] = alive[t] ? pb[i] * inv : 0.f;
+            dg[t] = fmaf(-li[t], li[t], dg[t]);
+        }
+#pragma unroll
+        for (int u = 0; u < CW; ++u) {
+            if ((colmask >> u) & 1u) {
+                const int jl = lwarp + WPC * u;
+                float* col = Xc + jl * LD;
+                const float l = pb[jl * 8 + crank] * inv;
+#pragma unroll
+                for (int t = 0; t < R; ++t) col[lane + 32 * t] = fmaf(-li[t], l, col[lane + 32 * t]);
+            }
+        }
+        if (tid == 0) { ord[p] = k; perm[k] = p; scl[k] = inv; }   // every CTA keeps its own copy of the tables
+        __syncwarp();                                             // the sender reads whole float4s of what the lanes updated
+        if (lane == 0) mbar_arrive_local(&cdone[set]);            // this warp has finished step k
+        if (lwarp == 0) {                                         // warp 0 reports the whole CTA to all 8 CTAs
+            bool fin = mbar_wait_cluster(&cdone[set], (uint32_t)(k >> 1) & 1u, &gflag[3]);
+            fin = __all_sync(0xffffffffu, fin);
+            if (!fin) {
+                if (lane == 0) atomicOr(&gflag[3], 1);
+                chol_failed = true;
+                break;
+            }
+            if (lane < 8) mbar_arrive_remote(mapa_u32(smem_addr_u32(&alldone[set]), (uint32_t)lane));
+        }
+    }
+    __syncthreads();
+    // ---- scale the pivot columns into the factor L (zero above the pivot order, zero unpivoted columns), into L2 ----
+    if (!chol_failed) {
+#pragma unroll
+        for (int u = 0; u < CW; ++u) {
+            const int jl = lwarp + WPC * u, j = jl * 8 + crank;
+            if (jl < CPC && j < n && geometry_ok) {
+                const int kc = ord[j];
+#pragma unroll
+                for (int t = 0; t < R; ++t) {
+                    const int i = lane + 32 * t;
+                    float v = 0.f;
+                    if (kc >= 0 && i < n) {
+                        const int ki = ord[i];
+                        if (!(ki >= 0 && ki < kc)) v = Xc[jl * LD + i] * scl[kc];
+                    }
+                    X[(size_t)j * LD + i] = v;
+                }
+            }
+        }
+    }
+    cluster.sync();
+    if (__ldcg(&gflag[3]) != 0 || !geometry_ok) rank = 0;         // a wait ran out somewhere: no Jacobi, flagged below
+    __syncthreads();
 
     // ---- one-sided cyclic Jacobi on the rank pivot columns, columns in distributed shared memory ----
     const int l8 = lane & 7, qd = lane >> 3;
@@ -1222,6 +1213,25 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
                 const float* src = X + (size_t)perm[p < rank ? p : 0] * LD;
 #pragma unroll
                 for (int t = 0; t < R; ++t) mybuf[hc * LD + lane + 32 * t] = (p < rank) ? __ldcg(src + lane + 32 * t) : 0.f;
+            }
+        }
+        // The tournament repeats every sweep: block pair and destinations of every block round, packed into one word
+        // per round (a warp alone on its scheduler pays full latency for every dependent index instruction, so the
+        // schedule is worked out once, a round per lane, instead of in every round).
+        uint32_t* mysched = sched + myslot * 128;
+        if (active) {
+            for (int br = lane; br < nbm1; br += 32) {
+                int ba, bb;
+                rr_blocks(slot, br, nbm1, ba, bb);
+                const int lo = min(ba, bb), hi = max(ba, bb);
+                const int brn = (br + 1 == nbm1) ? 0 : br + 1;
+                int s_lo, h_lo, s_hi, h_hi;
+                rr_slot_of(lo, brn, nbm1, nact, s_lo, h_lo);
+                rr_slot_of(hi, brn, nbm1, nact, s_hi, h_hi);
+                const int c_lo = (int)(((unsigned)s_lo * spc_inv) >> 16), c_hi = (int)(((unsigned)s_hi * spc_inv) >> 16);
+                const int l_lo = s_lo - c_lo * SPC, l_hi = s_hi - c_hi * SPC;
+                mysched[br] = (uint32_t)ba | ((uint32_t)bb << 8) | ((uint32_t)c_lo << 16) | ((uint32_t)l_lo << 19) | ((uint32_t)h_lo << 22) |
+                              ((uint32_t)c_hi << 23) | ((uint32_t)l_hi << 26) | ((uint32_t)h_hi << 29);
             }
         }
         __syncwarp();
@@ -1251,8 +1261,8 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
                     }
                     if (ok) {
                         loaded = true;
-                        int ba, bb;
-                        rr_blocks(slot, br, nbm1, ba, bb);
+                        const uint32_t sc = mysched[br];
+                        const int ba = (int)(sc & 255u), bb = (int)((sc >> 8) & 255u);
                         if (br == 0) {                            // pairs inside each block: quarters 0,1 -> ba, 2,3 -> bb
                             const int half = (qd < 2) ? 0 : 1, base = 4 * (half ? bb : ba), h = qd & 1;
                             float* blk = cur + half * 4 * LD;
@@ -1274,12 +1284,8 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
                             y[t] = xb[8 * t];
                         }
                         // where the next block round reads the two columns this quarter ends up with
-                        const int brn = (br + 1 == nbm1) ? 0 : br + 1;
-                        int s_lo, h_lo, s_hi, h_hi;
-                        rr_slot_of(lo, brn, nbm1, nact, s_lo, h_lo);
-                        rr_slot_of(hi, brn, nbm1, nact, s_hi, h_hi);
-                        const int c_lo = (int)(((unsigned)s_lo * spc_inv) >> 16), c_hi = (int)(((unsigned)s_hi * spc_inv) >> 16);
-                        const int l_lo = s_lo - c_lo * SPC, l_hi = s_hi - c_hi * SPC;
+                        const int c_lo = (int)((sc >> 16) & 7u), l_lo = (int)((sc >> 19) & 7u), h_lo = (int)((sc >> 22) & 1u);
+                        const int c_hi = (int)((sc >> 23) & 7u), l_hi = (int)((sc >> 26) & 7u), h_hi = (int)((sc >> 29) & 1u);
                         const int nset = kP2P ? ((g + 1) & 1) : 0;
                         float* d_lo = sbuf + ((size_t)(nset * T + l_lo) * 8 + h_lo * 4 + qd) * LD + 4 * l8;                // in CTA c_lo
                         float* d_hi = sbuf + ((size_t)(nset * T + l_hi) * 8 + h_hi * 4 + ((qd + 3) & 3)) * LD + 4 * l8;    // in CTA c_hi
@@ -1352,7 +1358,7 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
         }
     }
     cluster.sync();
-    if (kP2P && __ldcg(&gflag[3])) more = 2;
+    if (__ldcg(&gflag[3])) more = 2;                           // a bounded wait ran out in either phase
     if (more == 2 && gtid == 0) atomicOr(&info->flags, kFlagExchangeTimeout);
     const int not_converged = rank >= 2 && more != 0;          // stopped at the sweep limit while still rotating visibly
     // ---- eigenvalues = squared column norms (pivot-step order), scaled back; sort descending, stable ----
@@ -1668,8 +1674,8 @@ cudaError_t launch_eig_shrink(const float* K, int ldk, int n, int do_shrink, int
     if (variant == 0 && n > 64) {   // cluster of 8 CTAs, Jacobi columns in distributed shared memory (n <= 64: one CTA is as fast)
         const int T = n <= 64 ? 1 : n <= 128 ? 2 : n <= 192 ? 3 : n <= 256 ? 4 : 8;
         const int LD = 64 * T;
-        const size_t bytes = 3 * 512 * sizeof(float) + 3 * 512 * sizeof(int) + 32 + 16 * sizeof(uint64_t) +
-                             (size_t)(T <= 3 ? 2 : 1) * T * 8 * LD * sizeof(float) + (T <= 3 ? (size_t)LD * LD * sizeof(float) : 0);
+        const size_t bytes = 3 * 512 * sizeof(float) + 3 * 512 * sizeof(int) + 32 + 24 * sizeof(uint64_t) + (size_t)T * 128 * sizeof(uint32_t) +
+                             2 * (size_t)LD * sizeof(float) + (size_t)(T <= 3 ? 2 : 1) * T * 8 * LD * sizeof(float);
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(8);
         cfg.blockDim = dim3(T <= 3 ? 512 : 256);
