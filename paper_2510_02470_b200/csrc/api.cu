@@ -145,6 +145,7 @@ struct sage_fd {
     __nv_bfloat16* P16 = nullptr;  // frozen sketch in bf16 (bf16 handles: tensor-core projection operand); with p16_fold
                                    // rows [0, ell) hold bf16(S) and rows [n_pad, n_pad + ell) hold bf16(S - bf16(S))
     int p16_fold = 0, p16_npad = 0;
+    float* S32split = nullptr;     // frozen sketch split into tf32 hi / lo rows (fp32 handles with ell <= 64): 128 x pitch
     cudaStream_t side = nullptr;   // appends of the next shrink cycle run here, beside the eigen-solve of the current one
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     int* tc_err = nullptr;         // set by a tensor-core kernel whose bounded wait ran out
@@ -214,6 +215,8 @@ int pick_splits_waves(int tiles, int64_t K, int64_t min_k, int max_splits) {
 
 // After the sketch is frozen: the bf16 copy the tensor-core projection reads (bf16 handles only).
 sage_status_t enqueue_freeze_aux(sage_fd* h, cudaStream_t st) {
+    if (h->dtype == SAGE_F32 && h->S32split)
+        CU_TRY(timed(h, K_APPEND, 1, st, [&] { return launch_split_tf32(h->B[h->cur], h->pitch, h->ell, h->pitch, h->S32split, h->pitch, st); }));
     if (h->dtype == SAGE_BF16 && h->P16)
         CU_TRY(timed(h, K_APPEND, 1, st, [&] {
             return launch_to_bf16(h->B[h->cur], h->pitch, h->ell, h->pitch, h->P16,
@@ -416,6 +419,11 @@ sage_status_t sage_fd_create(sage_fd_t** out, int64_t D, int32_t ell, sage_dtype
         if ((e = cudaMalloc((void**)&h->P16, prow * h->pitch * sizeof(__nv_bfloat16))) != cudaSuccess) return fail(e, "cudaMalloc(P16)");
         if ((e = cudaMemset(h->P16, 0, prow * h->pitch * sizeof(__nv_bfloat16))) != cudaSuccess) return fail(e, "cudaMemset");
     }
+    if (row_dtype == SAGE_F32 && ell <= 64) {
+        // fp32 rows, small sketch: the projection multiplies the rows against the sketch pre-split into tf32 hi / lo rows
+        if ((e = cudaMalloc((void**)&h->S32split, (size_t)128 * h->pitch * sizeof(float))) != cudaSuccess) return fail(e, "cudaMalloc(S split)");
+        if ((e = cudaMemset(h->S32split, 0, (size_t)128 * h->pitch * sizeof(float))) != cudaSuccess) return fail(e, "cudaMemset");
+    }
     if ((e = cudaMemset(h->info, 0, sizeof(EigInfo))) != cudaSuccess) return fail(e, "cudaMemset");
     if ((e = cudaMemset(h->sigma, 0, ell * sizeof(float))) != cudaSuccess) return fail(e, "cudaMemset");
     if ((e = cudaDeviceSynchronize()) != cudaSuccess) return fail(e, "cudaDeviceSynchronize");
@@ -445,6 +453,7 @@ void sage_fd_destroy(sage_fd_t* h) {
     cudaFree(h->class_U);
     cudaFree(h->class_counts);
     cudaFree(h->P16);
+    cudaFree(h->S32split);
     cudaFree(h->tc_err);
     if (h->side) cudaStreamDestroy(h->side);
     if (h->ev_fork) cudaEventDestroy(h->ev_fork);
@@ -694,18 +703,21 @@ sage_status_t sage_score_chunk(sage_fd_t* h, const void* rows, int64_t n, int64_
         float* Z = nullptr;
         if (tc32_ok) {
             const int splits = pick_splits_waves((int)((sub + 127) / 128), h->D, 2048, 64);
-            ST_TRY(ensure(&h->zwork, &h->zwork_bytes, zred * (splits > 1 ? splits + 1 : 1)));
+            // sketches of at most 64 rows: one wide MMA per K step against the pre-split sketch, two partial planes per K slice
+            const bool wide = h->S32split != nullptr;
+            const int planes = wide ? 2 * splits : splits;
+            ST_TRY(ensure(&h->zwork, &h->zwork_bytes, zred * (planes > 1 ? planes + 1 : 1)));
             Z = h->zwork;
-            float* out = splits > 1 ? h->zwork + (size_t)sub * ell : Z;
+            float* out = planes > 1 ? h->zwork + (size_t)sub * ell : Z;
             cudaError_t e = timed(h, K_PROJECT, 1, st, [&] {
-                return launch_tc_gemm_nt_x3(reinterpret_cast<const float*>(p + r0 * row_bytes), ld, S, h->pitch, (int)sub, ell, h->D,
-                                            splits, out, ell, (int64_t)sub * ell, 0, h->tc_err, st);
+                return launch_tc_gemm_nt_x3(reinterpret_cast<const float*>(p + r0 * row_bytes), ld, wide ? h->S32split : S, h->pitch, (int)sub,
+                                            ell, h->D, splits, out, ell, (int64_t)sub * ell, wide ? 2 : 0, h->tc_err, st);
             });
             if (e == cudaSuccess) {
                 done = true;
-                if (splits > 1)
+                if (planes > 1)
                     CU_TRY(timed(h, K_PROJECT_REDUCE, 1, st,
-                                 [&] { return launch_split_reduce(out, splits, (int64_t)sub * ell, (int)sub, ell, ell, Z, ell, st); }));
+                                 [&] { return launch_split_reduce(out, planes, (int64_t)sub * ell, (int)sub, ell, ell, Z, ell, st); }));
             } else if (e != cudaErrorNotSupported) {
                 CU_TRY(e);
             } else {

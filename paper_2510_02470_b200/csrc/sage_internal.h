@@ -51,6 +51,8 @@ cudaError_t launch_tc_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const
 // launch_tc_gemm_nt; any N. When A == Bm (a Gram matrix) the diagonal tiles load one operand only.
 // sym != 0 (only for a Gram matrix of at most 128 rows): two MMAs per K step instead of three; slice z then stores
 // T_z = hi*hi^T + 2*hi*lo^T and the Gram matrix is sum_z (T_z + T_z^T)/2: see launch_gram_sym_reduce.
+// sym == 2 (projection onto at most 64 sketch rows): Bm is the sketch already split by launch_split_tf32 (128 rows);
+// one MMA per K step; C receives 2 * splits partial planes (split_stride apart) whose sum is A * S^T (M x N).
 cudaError_t launch_tc_gemm_nt_x3(const float* A, int64_t lda, const float* Bm, int64_t ldb, int M, int N, int64_t K, int splits,
                                  float* C, int64_t ldc, int64_t split_stride, int sym, int* err, cudaStream_t st);
 cudaError_t launch_gram_sym_reduce(const float* parts, int splits, int64_t stride, int r, int64_t ldp, float* out, int64_t ldo,
@@ -69,6 +71,10 @@ cudaError_t launch_to_bf16(const float* src, int64_t lds, int rows, int64_t cols
                            cudaStream_t st);
 
 // out[i][j] = sum_z parts[z][i][j] in ascending z with fp64 accumulation. (M x N, pitches ldp / ldo.)
+// out (128 rows, pitch ldo): row j = src row j rounded to 11 significant bits, row 64 + j = the remainder, for
+// j < rows <= 64; the other rows are left as they are (zero from allocation).
+cudaError_t launch_split_tf32(const float* src, int64_t lds, int rows, int64_t cols, float* out, int64_t ldo, cudaStream_t st);
+
 cudaError_t launch_split_reduce(const float* parts, int splits, int64_t split_stride, int M, int N, int64_t ldp,
                                 float* out, int64_t ldo, cudaStream_t st);
 

@@ -149,6 +149,20 @@ __global__ void __launch_bounds__(256) k_to_bf16(const float* __restrict__ src, 
     }
 }
 
+// The frozen sketch split once for the tf32 tensor cores: hi = 11 significant bits, lo = the exact remainder.
+__global__ void __launch_bounds__(256) k_split_tf32(const float* __restrict__ src, int64_t lds, int64_t cols, float* __restrict__ out,
+                                                     int64_t ldo) {
+    const float* s = src + (int64_t)blockIdx.y * lds;
+    float* dh = out + (int64_t)blockIdx.y * ldo;
+    float* dl = out + (int64_t)(64 + blockIdx.y) * ldo;
+    for (int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; c < cols; c += (int64_t)gridDim.x * blockDim.x) {
+        const float x = s[c];
+        const float h = __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xffffe000u);
+        dh[c] = h;
+        dl[c] = x - h;
+    }
+}
+
 __global__ void __launch_bounds__(256) k_split_reduce(const float* __restrict__ parts, int splits, int64_t split_stride,
                                                       int M, int N, int64_t ldp, float* __restrict__ out, int64_t ldo) {
     const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -286,6 +300,15 @@ cudaError_t launch_to_bf16(const float* src, int64_t lds, int rows, int64_t cols
     int64_t bx = (cols + 255) / 256;
     if (bx > 1184) bx = 1184;
     k_to_bf16<<<dim3((unsigned)bx, (unsigned)rows), 256, 0, st>>>(src, lds, cols, hi, lo, ldd);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_split_tf32(const float* src, int64_t lds, int rows, int64_t cols, float* out, int64_t ldo, cudaStream_t st) {
+    if (rows <= 0 || cols <= 0) return cudaSuccess;
+    if (rows > 64) return cudaErrorInvalidValue;
+    int64_t bx = (cols + 255) / 256;
+    if (bx > 1184) bx = 1184;
+    k_split_tf32<<<dim3((unsigned)bx, (unsigned)rows), 256, 0, st>>>(src, lds, cols, out, ldo);
     return cudaGetLastError();
 }
 

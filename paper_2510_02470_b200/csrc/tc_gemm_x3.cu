@@ -3,9 +3,11 @@
 // the buffer is taken through the eigen-decomposition of B B^T) and the pass-2 projection of fp32 rows.
 //
 // Two things keep fp32 fidelity on tensor cores:
-//   * tcgen05 kind::tf32 keeps 11 significant bits of each operand, so every fp32 value x is split in
-//     shared memory into hi = x rounded to 11 bits and lo = x - hi (exact), and three MMAs accumulate
-//     hi*hi + hi*lo + lo*hi; the dropped lo*lo term is below 2^-22 relative;
+//   * tcgen05 kind::tf32 reads an fp32 word by ignoring its low 13 bits (11 significant bits), so every value x
+//     counts as hi = x with those bits cleared, and the workers write the remainder lo = x - hi (exact, then rounded
+//     to 11 bits) into a second buffer; the MMAs accumulate hi*hi + hi*lo + lo*hi. The dropped lo*lo term is below
+//     2^-20 relative (3e-7 on average on a Gram diagonal). The raw tile itself is the hi operand: nothing is written
+//     back over it, which saves a third of the workers' shared-memory stores;
 //   * the TMEM accumulator rounds toward zero at every accumulation, which biases long sums of like-signed
 //     terms (measured about 0.45 * 2^-24 per MMA step), so the accumulator is drained every kChunk K
 //     tiles into fp32 registers with round-to-nearest additions and restarted from zero.
@@ -13,7 +15,7 @@
 // One CTA owns a 128 x (<=128) output tile and one K slice:
 //   warp 0    TMA producer (raw fp32 tiles, 128-byte swizzle),
 //   warp 1    TMEM allocation and MMA issue into a ring of four accumulators,
-//   warps 2-9 split each landed stage into hi (in place) and lo (second buffer); every kChunk stages they also
+//   warps 2-9 write the lo part of each landed stage into its second buffer; every kChunk stages they also
 //             drain the accumulator that was finished two chunks earlier (its MMAs are long done, so the drain
 //             never waits) into registers, and store the tile at the end. Warp w drains TMEM lanes
 //             32 * (w % 4) and columns 64 * ((w - 2) / 4).
@@ -23,6 +25,12 @@
 // by side; their sum T satisfies (T + T^T)/2 = hi*hi^T + hi*lo^T + lo*hi^T, formed by the split reduction. (Issuing
 // a tf32 MMA costs the issuing thread about 110 cycles whatever its width, and a 128 x 128 x 8 one executes in
 // about 70: narrow MMAs leave the tensor pipe idle, wide ones do not.)
+// The projection of fp32 rows onto a sketch of at most 64 rows (proj mode, sym = 2) uses the same wide form with the
+// operands' roles exchanged: the sketch, split once into [hi (64 rows) ; lo (64 rows)] when it was frozen, is the
+// 128-row A operand and needs no work per stage; the tile of 128 data rows is split by the workers into hi | lo and
+// serves as one 256-row B operand. One MMA per K step leaves S_hi (G_hi | G_lo) on TMEM lanes 0-63 and
+// S_lo (G_hi | G_lo) on lanes 64-127; the drain adds the two column halves, and the lane halves are stored as two
+// partial planes of the (transposed) output, which the split reduction sums with the K slices.
 #include "sage_internal.h"
 #include "tc05.cuh"
 
@@ -39,11 +47,16 @@ constexpr int BK = 32;                      // fp32 elements per 128-byte K tile
 constexpr int kChunkTiles = 4;              // K tiles accumulated in TMEM between drains
 constexpr int kAccs = 4;                    // accumulators in TMEM (4 x 128 columns)
 
-__device__ __forceinline__ void split4(const uint4 v, uint4& h, uint4& l) {
-    h.x = (v.x + 0x1000u) & 0xffffe000u; l.x = __float_as_uint(__uint_as_float(v.x) - __uint_as_float(h.x));
-    h.y = (v.y + 0x1000u) & 0xffffe000u; l.y = __float_as_uint(__uint_as_float(v.y) - __uint_as_float(h.y));
-    h.z = (v.z + 0x1000u) & 0xffffe000u; l.z = __float_as_uint(__uint_as_float(v.z) - __uint_as_float(h.z));
-    h.w = (v.w + 0x1000u) & 0xffffe000u; l.w = __float_as_uint(__uint_as_float(v.w) - __uint_as_float(h.w));
+// The tensor cores read an fp32 word as tf32 by ignoring its low 13 bits, so the raw tile already is the hi operand
+// (hi = x with those bits cleared) and only the remainder has to be written: lo = x - hi, exact, then rounded to 11
+// significant bits so that the hardware's truncation of lo finds nothing to cut (a truncated lo would bias sums of
+// like-signed products). `scale` is 1 or, for the doubled remainder of sym mode, 2.
+__device__ __forceinline__ uint32_t lo_of(uint32_t x, float scale) {
+    const float l = scale * (__uint_as_float(x) - __uint_as_float(x & 0xffffe000u));
+    return (__float_as_uint(l) + 0x1000u) & 0xffffe000u;
+}
+__device__ __forceinline__ uint4 lo4(const uint4 v, float scale) {
+    return make_uint4(lo_of(v.x, scale), lo_of(v.y, scale), lo_of(v.z, scale), lo_of(v.w, scale));
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -53,9 +66,11 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     const int m0 = blockIdx.x * kTileM, n0 = blockIdx.y * kTileN;
+    const bool proj = sym == 2;
+    const bool wide = sym != 0;                           // one 256-wide MMA per K step
     const bool diag = gram && m0 == n0;                   // A tile == B tile: load once
-    // stage layout: [hi: A | B][lo: A | B]; on diagonal tiles there is no separate B
-    const int half_bytes = diag ? kTileBytes : kTileBytes + b_box_rows * 128;
+    // stage layout: [hi: A | B][lo: A | B]; on diagonal tiles there is no separate B; proj: [hi: rows][lo: rows][sketch]
+    const int half_bytes = (diag || proj) ? kTileBytes : kTileBytes + b_box_rows * 128;
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)stages * stage_bytes);
     uint64_t* split_done = full + stages;
     uint64_t* empty = split_done + stages;
@@ -70,20 +85,21 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const int nkt = k_end > k_begin ? (int)((k_end - k_begin + BK - 1) / BK) : 0;
     const int kChunk = kChunkTiles;
     const int nchunks = (nkt + kChunk - 1) / kChunk;
-    const int acc_cols = sym ? 2 * kTileN : kTileN;       // sym: P and 2Q side by side
+    const int acc_cols = wide ? 2 * kTileN : kTileN;      // sym: P and 2Q side by side; proj: hi and lo columns of the rows
     const int ring = (kAccs * kTileN) / acc_cols;         // accumulators in flight: 4, or 2 in sym mode
     int n_pad = N - n0 < kTileN ? N - n0 : kTileN;        // MMA width of this tile, a multiple of 16
     n_pad = ((n_pad + 15) / 16) * 16;
+    if (proj) n_pad = kTileN;                             // accumulator columns are the 128 data rows of the tile
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
             mbar_init(&full[s], 1);
-            mbar_init(&split_done[s], kWorkers);
+            mbar_init(&split_done[s], kWorkers / 32);   // one arrival per worker warp
             mbar_init(&empty[s], 1);
         }
         for (int b = 0; b < kAccs; ++b) {
             mbar_init(&acc_full[b], 1);
-            mbar_init(&acc_empty[b], kWorkers);
+            mbar_init(&acc_empty[b], kWorkers / 32);
         }
         *abort = 0;
         mbar_fence_init();
@@ -103,11 +119,12 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 const int s = kt % stages;
                 const uint32_t use = (uint32_t)(kt / stages);
                 if (!mbar_wait(&empty[s], (use & 1u) ^ 1u, abort)) break;
-                mbar_expect_tx(&full[s], (uint32_t)half_bytes);
+                mbar_expect_tx(&full[s], (uint32_t)(proj ? 2 * kTileBytes : half_bytes));
                 const int x = (int)(k_begin + (long long)kt * BK);
                 uint8_t* st = smem + (size_t)s * stage_bytes;
                 tma_load_2d(st, &tmA, &full[s], x, m0);
-                if (!diag) tma_load_2d(st + kTileBytes, &tmB, &full[s], x, n0);
+                if (proj) tma_load_2d(st + 2 * kTileBytes, &tmB, &full[s], x, 0);
+                else if (!diag) tma_load_2d(st + kTileBytes, &tmB, &full[s], x, n0);
                 issued = kt + 1;
             }
             if (*abort) {
@@ -117,7 +134,7 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            const uint32_t idesc = instr_desc(2, kTileM, sym ? 2 * kTileN : n_pad, 0, 0);
+            const uint32_t idesc = instr_desc(2, kTileM, wide ? 2 * kTileN : n_pad, 0, 0);
             bool alive = true;
             for (int kt = 0; kt < nkt && alive; ++kt) {
                 const int s = kt % stages;
@@ -128,15 +145,15 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 if (!alive) break;
                 tc_fence_after();
                 const uint32_t st = smem_u32(smem + (size_t)s * stage_bytes);
-                const uint32_t a_hi = st, a_lo = st + half_bytes;
-                const uint32_t b_hi = diag ? a_hi : st + kTileBytes, b_lo = b_hi + half_bytes;
+                const uint32_t a_hi = proj ? st + 2 * kTileBytes : st, a_lo = st + half_bytes;   // proj: A = the split sketch
+                const uint32_t b_hi = (diag || proj) ? st : st + kTileBytes, b_lo = b_hi + half_bytes;
                 const uint64_t d_ahi = smem_desc_k_sw128(a_hi), d_alo = smem_desc_k_sw128(a_lo);
                 const uint64_t d_bhi = smem_desc_k_sw128(b_hi), d_blo = smem_desc_k_sw128(b_lo);
                 const uint32_t acc = tmem_base + (uint32_t)(b * acc_cols);
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {          // 4 x 8 tf32 elements per 128-byte row
-                    mma_tf32(acc, d_ahi + 2 * k, d_bhi + 2 * k, idesc, (in_chunk | k) != 0);   // sym: B = [hi ; 2 lo]
-                    if (!sym) {
+                    mma_tf32(acc, d_ahi + 2 * k, d_bhi + 2 * k, idesc, (in_chunk | k) != 0);   // sym: B = [hi ; 2 lo], proj: [hi ; lo]
+                    if (!wide) {
                         mma_tf32(acc, d_ahi + 2 * k, d_blo + 2 * k, idesc, 1);
                         mma_tf32(acc, d_alo + 2 * k, d_bhi + 2 * k, idesc, 1);
                     }
@@ -146,9 +163,10 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             }
         }
     } else {
-        // ---- workers: split landed stages into hi (in place) and lo; drain finished accumulators ----
+        // ---- workers: write the lo part of landed stages; drain finished accumulators ----
         const int t = threadIdx.x - 64;                 // 0..255
         const int chunks16 = half_bytes / 16;
+        const float lo_scale = sym == 1 ? 2.f : 1.f;
         const int quarter = warp & 3, chalf = (warp - 2) >> 2;
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + (uint32_t)(chalf * 64);
         float acc[64];
@@ -161,55 +179,84 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             w = __all_sync(0xffffffffu, w);
             if (!w) { ok = false; return; }
             tc_fence_after();
+            // two TMEM loads in flight per wait (a wait after every load made the drain a third of the workers' time)
+            if (wide) {                                      // columns c and kTileN + c belong together
 #pragma unroll
-            for (int c0 = 0; c0 < 64; c0 += 16) {
-                if (chalf * 64 + c0 < n_pad) {
-                    float v[16];
-                    tmem_ld16(lane_base + (uint32_t)(b * acc_cols + c0), v);
+                for (int q = 0; q < 4; ++q) {
+                    if (chalf * 64 + 16 * q < n_pad) {
+                        uint32_t v0[16], v1[16];
+                        tmem_ld16_issue(lane_base + (uint32_t)(b * acc_cols + 16 * q), v0);
+                        tmem_ld16_issue(lane_base + (uint32_t)(b * acc_cols + kTileN + 16 * q), v1);
+                        tmem_ld_wait();
+                        tmem_ld_use(v0);
+                        tmem_ld_use(v1);
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) acc[c0 + j] += v[j];
-                    if (sym) {
-                        tmem_ld16(lane_base + (uint32_t)(b * acc_cols + kTileN + c0), v);
+                        for (int j = 0; j < 16; ++j) acc[16 * q + j] += __uint_as_float(v0[j]) + __uint_as_float(v1[j]);
+                    }
+                }
+            } else {
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) acc[c0 + j] += v[j];
+                for (int q = 0; q < 4; q += 2) {
+                    const bool on0 = chalf * 64 + 16 * q < n_pad, on1 = chalf * 64 + 16 * (q + 1) < n_pad;
+                    uint32_t v0[16], v1[16];
+                    if (on0) tmem_ld16_issue(lane_base + (uint32_t)(b * acc_cols + 16 * q), v0);
+                    if (on1) tmem_ld16_issue(lane_base + (uint32_t)(b * acc_cols + 16 * (q + 1)), v1);
+                    tmem_ld_wait();
+                    if (on0) {
+                        tmem_ld_use(v0);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) acc[16 * q + j] += __uint_as_float(v0[j]);
+                    }
+                    if (on1) {
+                        tmem_ld_use(v1);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) acc[16 * (q + 1) + j] += __uint_as_float(v1[j]);
                     }
                 }
             }
             tc_fence_before();
-            mbar_arrive(&acc_empty[b]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[b]);
         };
         int drained = 0;                                // chunks drained so far
         for (int kt = 0; kt < nkt && ok; ++kt) {
             const int s = kt % stages;
             const uint32_t use = (uint32_t)(kt / stages);
-            if (!mbar_wait(&full[s], use & 1u, abort)) { ok = false; break; }
+            bool landed = mbar_wait(&full[s], use & 1u, abort);
+            landed = __all_sync(0xffffffffu, landed);
+            if (!landed) { ok = false; break; }
             uint4* hi = reinterpret_cast<uint4*>(smem + (size_t)s * stage_bytes);
             uint4* lo = reinterpret_cast<uint4*>(smem + (size_t)s * stage_bytes + half_bytes);
             for (int c = t; c < chunks16; c += 4 * kWorkers) {     // four independent 16-byte pieces in flight
-                uint4 v[4], h[4], l[4];
+                uint4 v[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u)
                     if (c + u * kWorkers < chunks16) v[u] = hi[c + u * kWorkers];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    split4(v[u], h[u], l[u]);
-                    if (sym) {      // doubled remainder (exact): see the note on sym mode above
-                        l[u].x = __float_as_uint(2.f * __uint_as_float(l[u].x)); l[u].y = __float_as_uint(2.f * __uint_as_float(l[u].y));
-                        l[u].z = __float_as_uint(2.f * __uint_as_float(l[u].z)); l[u].w = __float_as_uint(2.f * __uint_as_float(l[u].w));
-                    }
-                }
-#pragma unroll
                 for (int u = 0; u < 4; ++u)
-                    if (c + u * kWorkers < chunks16) { hi[c + u * kWorkers] = h[u]; lo[c + u * kWorkers] = l[u]; }
+                    if (c + u * kWorkers < chunks16) lo[c + u * kWorkers] = lo4(v[u], lo_scale);   // sym: doubled remainder
             }
             fence_proxy_async_smem();                   // the tensor cores read these writes
-            mbar_arrive(&split_done[s]);
+            __syncwarp();                               // 256 arrivals on one barrier serialise: one per warp instead
+            if (lane == 0) mbar_arrive(&split_done[s]);
             // the chunk that ended two chunks ago has certainly been multiplied: fold it into the registers
             if ((kt + 1) % kChunk == 0 && kt / kChunk - ring / 2 >= drained) drain(drained++);
         }
         while (ok && drained < nchunks) drain(drained++);
         const int row = m0 + quarter * 32 + lane;
-        if (row < M) {
+        if (proj) {
+            // lane = sketch row (0-63: hi part, 64-127: lo part), register c = data row chalf * 64 + c of the tile:
+            // the output is stored transposed, 32 consecutive sketch rows of one data row per warp instruction
+            const int mrow = quarter * 32 + lane, plane = mrow >> 6, j = mrow & 63;
+            float* cbase = C + (2ll * blockIdx.z + plane) * split_stride + j;
+            if (j < N) {
+#pragma unroll
+                for (int c = 0; c < 64; ++c) {
+                    const int r = m0 + chalf * 64 + c;
+                    if (r < M) cbase[(long long)r * ldc] = acc[c];
+                }
+            }
+        } else if (row < M) {
             float* crow = C + (long long)blockIdx.z * split_stride + (long long)row * ldc + n0 + chalf * 64;
             const bool vec = (ldc % 4 == 0) && ((reinterpret_cast<uintptr_t>(C) & 15u) == 0) && (split_stride % 4 == 0);
 #pragma unroll
@@ -245,20 +292,22 @@ cudaError_t launch_tc_gemm_nt_x3(const float* A, int64_t lda, const float* Bm, i
     if (M <= 0 || N <= 0 || K <= 0) return cudaSuccess;
     if (splits < 1 || splits > 65535) return cudaErrorNotSupported;
     const int gram = (A == Bm && lda == ldb && M == N) ? 1 : 0;
-    if (sym && !(gram && M <= tc::kTileM)) return cudaErrorInvalidValue;
+    const bool proj = sym == 2;       // Bm: the sketch split into [hi (64 rows) ; lo (64 rows)], 128 rows of pitch ldb; N <= 64
+    if (sym == 1 && !(gram && M <= tc::kTileM)) return cudaErrorInvalidValue;
+    if (proj && (N > 64 || gram)) return cudaErrorInvalidValue;
     CUtensorMap tmA, tmB;
     if (!tc::make_tmap_2d(&tmA, A, 4, (uint64_t)M, (uint64_t)K, (uint64_t)lda, tc::kTileM)) return cudaErrorNotSupported;
-    const int b_box_rows = N >= tc::kTileN ? tc::kTileN : ((N + 15) / 16) * 16;
-    if (!tc::make_tmap_2d(&tmB, Bm, 4, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, (uint32_t)b_box_rows)) return cudaErrorNotSupported;
+    const int b_box_rows = proj ? tc::kTileN : (N >= tc::kTileN ? tc::kTileN : ((N + 15) / 16) * 16);
+    if (!tc::make_tmap_2d(&tmB, Bm, 4, (uint64_t)(proj ? 128 : N), (uint64_t)K, (uint64_t)ldb, (uint32_t)b_box_rows)) return cudaErrorNotSupported;
     int64_t kps = (K + splits - 1) / splits;
     kps = ((kps + tc::BK - 1) / tc::BK) * tc::BK;
     // a trailing slice may be empty after rounding to whole K tiles: its CTAs store zeros
     // a Gram matrix of at most 128 rows has diagonal tiles only: one operand per stage
-    const int stage_bytes = 2 * ((gram && M <= tc::kTileM) ? tc::kTileBytes : tc::kTileBytes + b_box_rows * 128);
+    const int stage_bytes = proj ? 3 * tc::kTileBytes : 2 * ((gram && M <= tc::kTileM) ? tc::kTileBytes : tc::kTileBytes + b_box_rows * 128);
     int stages = (200 * 1024) / stage_bytes;
     if (stages > 8) stages = 8;
     const size_t smem = (size_t)stages * stage_bytes + 1024 + (3 * stages + 2 * tc::kAccs) * 8 + 16;
-    dim3 grid((unsigned)((M + tc::kTileM - 1) / tc::kTileM), (unsigned)((N + tc::kTileN - 1) / tc::kTileN), (unsigned)splits);
+    dim3 grid((unsigned)((M + tc::kTileM - 1) / tc::kTileM), proj ? 1u : (unsigned)((N + tc::kTileN - 1) / tc::kTileN), (unsigned)splits);
     cudaError_t e = cudaFuncSetAttribute(tc::k_tc_gemm_nt_x3, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     tc::k_tc_gemm_nt_x3<<<grid, tc::kThreads, smem, st>>>(tmA, tmB, M, N, gram, b_box_rows, sym, K, kps, C, ldc, split_stride, stages,

@@ -5,15 +5,15 @@
 // chunks of 32 buffer rows   D[d][j] += B[i][d] * W[j][i]   with d on the 128 TMEM lanes (the buffer tile is the
 // "A" operand, stored with d contiguous = MN-major), so the epilogue writes out[j][d0..d0+127] as full lines.
 //
-// fp32 fidelity as in the Gram kernel: buffer values are split in shared memory into hi (11 significant
-// bits) and lo = x - hi; W arrives already split from global memory as two stacked operands [W_hi; W_lo],
+// fp32 fidelity as in the Gram kernel: the tensor cores read a buffer value as hi (its low 13 bits ignored),
+// the split warps write lo = x - hi into a second buffer; W arrives already split from global memory as two stacked operands [W_hi; W_lo],
 // so one MMA of width 2*j_pad gives hi*W_hi and hi*W_lo side by side and a second one adds lo*W_hi; the
 // epilogue adds the two halves. A tile accumulates at most 8 chunks (256 buffer rows) in TMEM.
 //
 //   warp 0    TMA producer: per chunk 4 boxes of [32 rows][32 columns] of the buffer (128-byte swizzle with
 //             32-byte atoms, the only layout the tensor cores take for 32-bit MN-major operands) and one box of W,
 //   warp 1    TMEM allocation, MMA issue into two ping-pong accumulators (one per column tile),
-//   warps 2-5 split the buffer part of each landed stage into hi / lo,
+//   warps 2-5 write the lo part of the buffer tile of each landed stage,
 //   warps 6-9 epilogue: TMEM -> registers -> out.
 #include "sage_internal.h"
 #include "tc05.cuh"
@@ -141,13 +141,14 @@ k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ 
 #pragma unroll
             for (int c = 0; c < kBufBytes / 16 / kSplitThreads; ++c) {
                 const int idx = t + c * kSplitThreads;
+                // the tensor cores ignore the low 13 bits of an fp32 word, so the raw tile is the hi operand as it stands;
+                // lo = x - hi (exact), rounded to 11 significant bits so that the same truncation cuts nothing from it
                 const uint4 v = hi[idx];
-                uint4 h, l;
-                h.x = (v.x + 0x1000u) & 0xffffe000u; l.x = __float_as_uint(__uint_as_float(v.x) - __uint_as_float(h.x));
-                h.y = (v.y + 0x1000u) & 0xffffe000u; l.y = __float_as_uint(__uint_as_float(v.y) - __uint_as_float(h.y));
-                h.z = (v.z + 0x1000u) & 0xffffe000u; l.z = __float_as_uint(__uint_as_float(v.z) - __uint_as_float(h.z));
-                h.w = (v.w + 0x1000u) & 0xffffe000u; l.w = __float_as_uint(__uint_as_float(v.w) - __uint_as_float(h.w));
-                hi[idx] = h;
+                uint4 l;
+                l.x = (__float_as_uint(__uint_as_float(v.x) - __uint_as_float(v.x & 0xffffe000u)) + 0x1000u) & 0xffffe000u;
+                l.y = (__float_as_uint(__uint_as_float(v.y) - __uint_as_float(v.y & 0xffffe000u)) + 0x1000u) & 0xffffe000u;
+                l.z = (__float_as_uint(__uint_as_float(v.z) - __uint_as_float(v.z & 0xffffe000u)) + 0x1000u) & 0xffffe000u;
+                l.w = (__float_as_uint(__uint_as_float(v.w) - __uint_as_float(v.w & 0xffffe000u)) + 0x1000u) & 0xffffe000u;
                 lo[idx] = l;
             }
             fence_proxy_async_smem();
