@@ -122,7 +122,8 @@ struct sage_fd {
     int delta_rank = 0, max_sweeps = 30;
     // Gram / eigen workspaces
     float* gram_parts = nullptr;   // split-K partials of the Gram matrix (kGramPartFloats floats)
-    float* Wsplit = nullptr;       // rebuild factors split for the tensor cores: 256 rows x kWsplitLd floats
+    float* Wsplit = nullptr;       // rebuild factors split for the tensor cores: wsplit_ld rows x wsplit_ld floats
+    int wsplit_ld = 256;           // 256 (buffers of up to 256 rows) or 512
     float* Kmat = nullptr;         // m x m
     float* Ur = nullptr;           // m x m
     float* eig_work = nullptr;     // m x m
@@ -182,7 +183,6 @@ cudaError_t timed(sage_fd* h, int cls, int nlaunch, cudaStream_t st, F&& f) {
 }
 
 constexpr size_t kGramPartFloats = (size_t)148 * 128 * 128;   // >= 296 tiles of 64 x 64
-constexpr int kWsplitLd = 256;
 
 int gram_tiles(int r) {
     const int t = (r + 63) / 64;
@@ -276,16 +276,17 @@ sage_status_t enqueue_factor(sage_fd* h, int r, int do_shrink, int keep, int zer
     ST_TRY(enqueue_gram(h, r, st));
     CU_TRY(cudaEventRecord(h->ev_fork, st));       // from here on HBM is idle until the rebuild: see sage_fd_update
     const int j_pad = ((keep + 15) / 16) * 16;
-    const bool tc_rebuild = h->use_tc && h->Wsplit && keep > 0 && j_pad <= 128 && r <= 256;
+    const bool tc_rebuild = h->use_tc && h->Wsplit && keep > 0 && j_pad <= h->wsplit_ld / 2 && r <= h->wsplit_ld;
     CU_TRY(timed(h, K_EIG, 1, st, [&] {
         return launch_eig_shrink(h->Kmat, h->m, r, do_shrink, h->delta_rank, keep, h->Ur, h->m, h->sigma, h->ell, h->eig_work,
-                                 h->max_sweeps, h->info, tc_rebuild ? h->Wsplit : nullptr, kWsplitLd, j_pad, h->eig_variant, st);
+                                 h->max_sweeps, h->info, tc_rebuild ? h->Wsplit : nullptr, h->wsplit_ld, j_pad, h->eig_variant, st);
     }));
     const int m_total = zero_to > keep ? zero_to : keep;
     bool done = false;
     if (tc_rebuild) {
-        cudaError_t e = timed(h, K_REBUILD, 1, st, [&] {
-            return launch_tc_rebuild(h->Wsplit, kWsplitLd, j_pad, h->B[h->cur], h->B[1 - h->cur], h->pitch, h->D, r, keep, h->tc_err, st);
+        const int parts = (j_pad > 128 ? 2 : 1) * (r > 256 ? 2 : 1);     // launches: 128 output rows x 256 buffer rows each
+        cudaError_t e = timed(h, K_REBUILD, parts, st, [&] {
+            return launch_tc_rebuild(h->Wsplit, h->wsplit_ld, j_pad, h->B[h->cur], h->B[1 - h->cur], h->pitch, h->D, r, keep, h->tc_err, st);
         });
         if (e == cudaSuccess) {
             done = true;
@@ -393,7 +394,8 @@ sage_status_t sage_fd_create(sage_fd_t** out, int64_t D, int32_t ell, sage_dtype
     for (int i = 0; i < 2; ++i)
         if ((e = cudaMalloc((void**)&h->B[i], bbytes)) != cudaSuccess) return fail(e, "cudaMalloc(buffer)");
     if ((e = cudaMalloc((void**)&h->gram_parts, kGramPartFloats * sizeof(float))) != cudaSuccess) return fail(e, "cudaMalloc(gram)");
-    if (ell <= 128 && (e = cudaMalloc((void**)&h->Wsplit, (size_t)256 * kWsplitLd * sizeof(float))) != cudaSuccess)
+    h->wsplit_ld = h->m <= 256 ? 256 : 512;
+    if ((e = cudaMalloc((void**)&h->Wsplit, (size_t)h->wsplit_ld * h->wsplit_ld * sizeof(float))) != cudaSuccess)
         return fail(e, "cudaMalloc(W)");
     if ((e = cudaMalloc((void**)&h->Kmat, mm)) != cudaSuccess) return fail(e, "cudaMalloc(K)");
     if ((e = cudaMalloc((void**)&h->Ur, mm)) != cudaSuccess) return fail(e, "cudaMalloc(U)");

@@ -33,6 +33,13 @@ __device__ __forceinline__ ArgMax better(ArgMax a, ArgMax b) {
     return a;
 }
 
+// Row of the split rebuild factors [W_hi ; W_lo] that holds output row j: stacked as two blocks of j_pad rows, or, when
+// more than 128 output rows are kept, as one such pair per 128 output rows (the rebuild kernel takes 128 at a time).
+__device__ __forceinline__ size_t wsplit_row(int j, int j_pad, bool lo) {
+    if (j_pad <= 128) return (size_t)(lo ? j_pad + j : j);
+    return (size_t)(j >> 7) * 256 + (size_t)(j & 127) + (lo ? 128 : 0);
+}
+
 // Round-robin pairing: n_even players, rounds 0..n_even-2, slots 0..n_even/2-1 give disjoint pairs.
 __device__ __forceinline__ void rr_pair(int n_even, int round, int slot, int& p, int& q) {
     const int nm1 = n_even - 1;
@@ -430,8 +437,8 @@ k_eig_shrink_fast(const float* __restrict__ K, int ldk, int n, int do_shrink, in
                 if (k < rank) v = X[perm[k] * LD + i] * fac[j];
             }
             const float hi = __uint_as_float((__float_as_uint(v) + 0x1000u) & 0xffffe000u);
-            Wsplit[(size_t)j * ldw + i] = hi;
-            Wsplit[(size_t)(j_pad + j) * ldw + i] = v - hi;
+            Wsplit[wsplit_row(j, j_pad, false) * ldw + i] = hi;
+            Wsplit[wsplit_row(j, j_pad, true) * ldw + i] = v - hi;
         }
     }
 }
@@ -798,8 +805,8 @@ k_eig_shrink_cluster(const float* __restrict__ K, int ldk, int n, int do_shrink,
                 if (k < rank) v = __ldcg(X + perm[k] * LD + i) * fac[j];
             }
             const float hi = __uint_as_float((__float_as_uint(v) + 0x1000u) & 0xffffe000u);
-            Wsplit[(size_t)j * ldw + i] = hi;
-            Wsplit[(size_t)(j_pad + j) * ldw + i] = v - hi;
+            Wsplit[wsplit_row(j, j_pad, false) * ldw + i] = hi;
+            Wsplit[wsplit_row(j, j_pad, true) * ldw + i] = v - hi;
         }
     }
 }
@@ -1435,8 +1442,8 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
                 if (k < rank) v = __ldcg(X + perm[k] * LD + i) * fac[j];
             }
             const float hi = __uint_as_float((__float_as_uint(v) + 0x1000u) & 0xffffe000u);
-            Wsplit[(size_t)j * ldw + i] = hi;
-            Wsplit[(size_t)(j_pad + j) * ldw + i] = v - hi;
+            Wsplit[wsplit_row(j, j_pad, false) * ldw + i] = hi;
+            Wsplit[wsplit_row(j, j_pad, true) * ldw + i] = v - hi;
         }
     }
 }
@@ -1650,8 +1657,8 @@ k_eig_shrink(const float* __restrict__ K, int ldk, int n, int do_shrink, int del
     if (Wsplit) {
         for (int e = tid; e < j_pad * ldw; e += kThreads) {
             const int j = e / ldw, c = e - j * ldw;
-            Wsplit[(size_t)j * ldw + c] = 0.f;
-            Wsplit[(size_t)(j_pad + j) * ldw + c] = 0.f;
+            Wsplit[wsplit_row(j, j_pad, false) * ldw + c] = 0.f;
+            Wsplit[wsplit_row(j, j_pad, true) * ldw + c] = 0.f;
         }
         __syncthreads();
         for (int e = tid; e < n * keep; e += kThreads) {
@@ -1659,8 +1666,8 @@ k_eig_shrink(const float* __restrict__ K, int ldk, int n, int do_shrink, int del
             if (j >= n || j >= j_pad) continue;
             const float v = X[(size_t)order[j] * ldx + i] * fac[j];
             const float hi = __uint_as_float((__float_as_uint(v) + 0x1000u) & 0xffffe000u);
-            Wsplit[(size_t)j * ldw + perm[i]] = hi;
-            Wsplit[(size_t)(j_pad + j) * ldw + perm[i]] = v - hi;
+            Wsplit[wsplit_row(j, j_pad, false) * ldw + perm[i]] = hi;
+            Wsplit[wsplit_row(j, j_pad, true) * ldw + perm[i]] = v - hi;
         }
     }
 }

@@ -32,7 +32,7 @@ constexpr int kSpanBytes = kChunkRows * 128;         // 4 KB
 
 __global__ void __launch_bounds__(kThreads, 1)
 k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ CUtensorMap tmW, int r, int keep, int j_pad,
-             long long pitch, long long num_tiles, float* __restrict__ out, int stages, int* __restrict__ err) {
+             long long pitch, long long num_tiles, float* __restrict__ out, int stages, int accumulate, int* __restrict__ err) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     // stage layout: [buffer hi 16 KB][buffer lo 16 KB][W_hi ; W_lo: 2*j_pad rows of 128 bytes]
@@ -172,7 +172,10 @@ k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ 
                 if (d < pitch) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
-                        if (j0 + j < keep) out[(long long)(j0 + j) * pitch + d] = v[j] + w[j];
+                        if (j0 + j < keep) {
+                            float* o = out + (long long)(j0 + j) * pitch + d;
+                            *o = accumulate ? *o + (v[j] + w[j]) : v[j] + w[j];   // second half of the buffer rows adds to the first
+                        }
                 }
             }
             tc_fence_before();
@@ -193,8 +196,8 @@ k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ 
 }  // namespace tc
 
 // See sage_internal.h.
-cudaError_t launch_tc_rebuild(const float* Wsplit, int ldw, int j_pad, const float* Bsrc, float* Bdst, int64_t pitch, int64_t D, int r,
-                              int keep, int* err, cudaStream_t st) {
+static cudaError_t launch_tc_rebuild_part(const float* Wsplit, int ldw, int j_pad, const float* Bsrc, float* Bdst, int64_t pitch, int r,
+                                          int keep, int accumulate, int* err, cudaStream_t st) {
     if (keep <= 0 || r <= 0) return cudaSuccess;
     if (j_pad < 16 || j_pad > 128 || (j_pad & 15) || keep > j_pad || r > 256) return cudaErrorNotSupported;
     CUtensorMap tmBuf, tmW;
@@ -204,7 +207,6 @@ cudaError_t launch_tc_rebuild(const float* Wsplit, int ldw, int j_pad, const flo
     if (kcols > ldw) return cudaErrorNotSupported;
     if (!tc::make_tmap_2d(&tmW, Wsplit, 4, (uint64_t)(2 * j_pad), (uint64_t)kcols, (uint64_t)ldw, (uint32_t)(2 * j_pad)))
         return cudaErrorNotSupported;
-    (void)D;
     const int stage_bytes = 2 * tc::kBufBytes + 2 * j_pad * 128;
     int stages = (200 * 1024) / stage_bytes;
     if (stages > 8) stages = 8;
@@ -213,8 +215,34 @@ cudaError_t launch_tc_rebuild(const float* Wsplit, int ldw, int j_pad, const flo
     const int grid = (int)(num_tiles < 148 ? num_tiles : 148);
     cudaError_t e = cudaFuncSetAttribute(tc::k_tc_rebuild, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    tc::k_tc_rebuild<<<grid, tc::kThreads, smem, st>>>(tmBuf, tmW, r, keep, j_pad, pitch, num_tiles, Bdst, stages, err);
+    tc::k_tc_rebuild<<<grid, tc::kThreads, smem, st>>>(tmBuf, tmW, r, keep, j_pad, pitch, num_tiles, Bdst, stages, accumulate, err);
     return cudaGetLastError();
+}
+
+// See sage_internal.h. One launch takes at most 128 output rows and 256 buffer rows (accumulator width and the number
+// of accumulations one TMEM accumulator should take); larger problems (ell = 256: 255 rows out of 512) run as up to
+// 2 x 2 launches, the second half of the buffer rows adding to what the first half stored.
+cudaError_t launch_tc_rebuild(const float* Wsplit, int ldw, int j_pad, const float* Bsrc, float* Bdst, int64_t pitch, int64_t D, int r,
+                              int keep, int* err, cudaStream_t st) {
+    (void)D;
+    if (keep <= 0 || r <= 0) return cudaSuccess;
+    if (j_pad < 16 || j_pad > 256 || (j_pad & 15) || keep > j_pad || r > 512) return cudaErrorNotSupported;
+    if (((reinterpret_cast<uintptr_t>(Bsrc) | reinterpret_cast<uintptr_t>(Wsplit)) & 15u) || (pitch & 3) || (ldw & 3)) return cudaErrorNotSupported;
+    const int jparts = j_pad > 128 ? 2 : 1, rparts = r > 256 ? 2 : 1;
+    if (rparts == 2 && ldw < 512) return cudaErrorNotSupported;
+    for (int jh = 0; jh < jparts; ++jh) {
+        const int jp = jparts == 2 ? 128 : j_pad;
+        const int keep_h = keep - jh * 128 < jp ? keep - jh * 128 : jp;
+        if (keep_h <= 0) continue;
+        const float* Wb = Wsplit + (size_t)(jparts == 2 ? jh * 256 : 0) * ldw;
+        for (int rh = 0; rh < rparts; ++rh) {
+            const int r_h = r - rh * 256 < 256 ? r - rh * 256 : 256;
+            cudaError_t e = launch_tc_rebuild_part(Wb + rh * 256, ldw, jp, Bsrc + (size_t)rh * 256 * pitch, Bdst + (size_t)jh * 128 * pitch, pitch,
+                                                   r_h, keep_h, rh > 0 ? 1 : 0, err, st);
+            if (e != cudaSuccess) return e;
+        }
+    }
+    return cudaSuccess;
 }
 
 }  // namespace sage

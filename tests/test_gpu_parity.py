@@ -269,6 +269,18 @@ def test_c2_prefix_three_keep_rates():
     compare(out2, ref, dense, w.D, 0.1, label="c2 dense pitch")
 
 
+def test_c2_full_size():
+    """The default benchmark workload at its full size (50,000 rows, 769 shrinks) against the oracle: errors of the
+    tensor-core Gram / rebuild accumulate over the shrinks, so the prefix test above does not bound them."""
+    w = wl.WORKLOADS["c2"]
+    rows = wl.host_rows(w, 0)
+    ref = oracle.run(rows, w.D, w.ell, 0.1, route=1)
+    out = gpu_run(rows, w.D, w.ell, 0.1)
+    rep = compare(out, ref, rows, w.D, 0.1, label="c2 full")
+    assert out["stats"]["shrinks"] == 769 and len(out["idx"]) == 5000
+    print(rep, out["stats"])
+
+
 def test_c3_prefix_bf16():
     w = wl.scaled(wl.WORKLOADS["c3"], N=1500)
     rows = wl.host_rows(w, 0)
