@@ -124,7 +124,7 @@ def cpu_oracle_sample(w, seed, sample_rows):
             "seconds": dt}
 
 
-CPU_SAMPLE_ROWS = {"c1": 4096, "c2": 6000, "c3": 1200, "c4": 768, "c5": 256}
+CPU_SAMPLE_ROWS = {"c1": 4096, "c2": 20000, "c3": 2000, "c4": 768, "c5": 256}
 
 
 def run_reference(args, w):
@@ -317,11 +317,11 @@ def main():
     dom_launches_per_step = prof_dom["launches"] / args.steps
     if dominant == "eig_shrink":
         achieved = eig_flops / (dom_ms_per_step * 1e-3) / 1e12
-        roof = {"kernel": "k_eig_shrink_fast" if 2 * ell <= 192 else "k_eig_shrink_cluster", "bound": "alu", "achieved": achieved, "peak": FP32_ALU_PEAK_TFLOPS, "unit": "TFLOP/s",
+        roof = {"kernel": "k_eig_shrink_fast" if 2 * ell <= 64 else "k_eig_shrink_dsm", "bound": "alu", "achieved": achieved, "peak": FP32_ALU_PEAK_TFLOPS, "unit": "TFLOP/s",
                 "frac": achieved / FP32_ALU_PEAK_TFLOPS, "traffic": None,
                 "peak_source": "derived: 148 SMs x 128 fp32 FMA lanes x 2 flop x 1.965 GHz",
                 "algorithmic": "9*n^3 flop per n x n symmetric eigen-solve (textbook count)",
-                "frac_of_the_sms_it_runs_on": achieved / (FP32_ALU_PEAK_TFLOPS * (1 if 2 * ell <= 192 else 8) / 148.0)}
+                "frac_of_the_sms_it_runs_on": achieved / (FP32_ALU_PEAK_TFLOPS * (1 if 2 * ell <= 64 else 8) / 148.0)}
     else:
         gbs = per_step_bytes.get(dominant, 0) / (dom_ms_per_step * 1e-3) / 1e9
         roof = {"kernel": dominant, "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
