@@ -15,10 +15,10 @@
 // One CTA owns a 128 x (<=128) output tile and one K slice:
 //   warp 0    TMA producer (raw fp32 tiles, 128-byte swizzle),
 //   warp 1    TMEM allocation and MMA issue into a ring of four accumulators,
-//   warps 2-9 write the lo part of each landed stage into its second buffer; every kChunk stages they also
-//             drain the accumulator that was finished two chunks earlier (its MMAs are long done, so the drain
-//             never waits) into registers, and store the tile at the end. Warp w drains TMEM lanes
-//             32 * (w % 4) and columns 64 * ((w - 2) / 4).
+//   warps 2-9 write the lo part of each landed stage into its second buffer, as two groups of four warps that take
+//             alternate stages; every kChunk stages each warp also drains its lanes and columns of the accumulator
+//             that was finished ring / 2 chunks earlier (its MMAs are long done, so the drain hardly waits) into
+//             registers, and stores them at the end. Warp w drains TMEM lanes 32 * (w % 4), columns 64 * ((w - 2) / 4).
 // On the diagonal tiles of a Gram matrix only one operand tile is loaded and used on both sides. A Gram matrix
 // of at most 128 rows (sym mode) needs ONE 256-wide MMA per K step: the hi tile and the (doubled) lo tile lie
 // back to back in the stage and serve as one 256-row B operand, so the accumulator holds hi*hi^T | 2*hi*lo^T side
@@ -94,7 +94,7 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
             mbar_init(&full[s], 1);
-            mbar_init(&split_done[s], kWorkers / 32);   // one arrival per worker warp
+            mbar_init(&split_done[s], kWorkers / 64);   // one arrival per warp of the group that handles the stage
             mbar_init(&empty[s], 1);
         }
         for (int b = 0; b < kAccs; ++b) {
@@ -218,8 +218,12 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[b]);
         };
+        // The eight warps work as two groups of four (warps 2-5 and 6-9) that take alternate stages: a stage's
+        // load -> remainder -> store -> fence -> arrive chain is latency, and two chains in flight hide half of it.
         int drained = 0;                                // chunks drained so far
-        for (int kt = 0; kt < nkt && ok; ++kt) {
+        const int grp = chalf, tg = t - 128 * grp;      // group and thread index within it
+        constexpr int kGroup = kWorkers / 2;
+        for (int kt = grp; kt < nkt && ok; kt += 2) {
             const int s = kt % stages;
             const uint32_t use = (uint32_t)(kt / stages);
             bool landed = mbar_wait(&full[s], use & 1u, abort);
@@ -227,20 +231,21 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             if (!landed) { ok = false; break; }
             uint4* hi = reinterpret_cast<uint4*>(smem + (size_t)s * stage_bytes);
             uint4* lo = reinterpret_cast<uint4*>(smem + (size_t)s * stage_bytes + half_bytes);
-            for (int c = t; c < chunks16; c += 4 * kWorkers) {     // four independent 16-byte pieces in flight
+            for (int c = tg; c < chunks16; c += 4 * kGroup) {      // four independent 16-byte pieces in flight
                 uint4 v[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u)
-                    if (c + u * kWorkers < chunks16) v[u] = hi[c + u * kWorkers];
+                    if (c + u * kGroup < chunks16) v[u] = hi[c + u * kGroup];
 #pragma unroll
                 for (int u = 0; u < 4; ++u)
-                    if (c + u * kWorkers < chunks16) lo[c + u * kWorkers] = lo4(v[u], lo_scale);   // sym: doubled remainder
+                    if (c + u * kGroup < chunks16) lo[c + u * kGroup] = lo4(v[u], lo_scale);   // sym: doubled remainder
             }
             fence_proxy_async_smem();                   // the tensor cores read these writes
-            __syncwarp();                               // 256 arrivals on one barrier serialise: one per warp instead
+            __syncwarp();                               // one arrival per warp
             if (lane == 0) mbar_arrive(&split_done[s]);
-            // the chunk that ended two chunks ago has certainly been multiplied: fold it into the registers
-            if ((kt + 1) % kChunk == 0 && kt / kChunk - ring / 2 >= drained) drain(drained++);
+            // a chunk is folded into the registers once the stages of the following ring / 2 chunks have been handled
+            // (its MMAs are long done by then); every warp drains its own lanes and columns of every chunk
+            while (ok && drained < nchunks && (drained + 1 + ring / 2) * kChunk - 2 <= kt) drain(drained++);
         }
         while (ok && drained < nchunks) drain(drained++);
         const int row = m0 + quarter * 32 + lane;
