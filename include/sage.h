@@ -4,10 +4,10 @@
  * The path (paper: Method section and Algorithm 1):
  *   pass 1  stream per-example gradient rows into a Frequent-Directions sketch
  *           (Algorithm 1, Phase I; Method, first paragraph),
- *   freeze  the ell x D sketch S (Algorithm 1, "Freeze S for scoring"),
+ *   freeze  the ell x D sketch S (Algorithm 1, the freeze step),
  *   pass 2  z_i = S g_i, zhat_i = z_i/||z_i||, consensus u, agreement score alpha_i = <zhat_i, u>
- *           (Method, "Two-pass scoring"; Algorithm 1, Phase II),
- *   select  the top-k examples by alpha (Algorithm 1, "Select top-k by alpha_i").
+ *           (Method, paragraph on two-pass scoring; Algorithm 1, Phase II),
+ *   select  the top-k examples by alpha (Algorithm 1, the top-k step).
  *
  * Conventions shared by every entry point
  *   - Every function returns a sage_status_t; nothing throws or aborts. Out-parameters are written only
@@ -82,7 +82,7 @@ sage_status_t sage_fd_reset(sage_fd_t* h);
  * synchronisation happens here. Device-side problems are reported by sage_fd_finalize. */
 sage_status_t sage_fd_update(sage_fd_t* h, const void* rows, int64_t n, int64_t ld, void* cuda_stream);
 
-/* Algorithm 1, "Freeze S for scoring": orthogonalise what the buffer holds, apply the shrink only if
+/* Algorithm 1, the freeze step: orthogonalise what the buffer holds, apply the shrink only if
  * more than ell rows are in use (so N <= ell is exact), keep the first ell rows as S.
  * Synchronises the stream once and returns SAGE_ERR_NOT_CONVERGED / SAGE_ERR_NONFINITE if the device
  * recorded such an event during pass 1 (the sketch is still usable). */
@@ -120,7 +120,7 @@ sage_status_t sage_score_intermediates(const sage_fd_t* h, const float** zhat, c
 /* Number of indices sage_select returns for N scores: floor(keep_rate*N + 0.5) clamped to [0, N]. */
 int64_t sage_select_count(int64_t N, double keep_rate);
 
-/* Algorithm 1, "Select top-k by alpha_i": the k = sage_select_count(N, keep_rate) largest scores,
+/* Algorithm 1, the top-k step: the k = sage_select_count(N, keep_rate) largest scores,
  * ordered by (score descending, index ascending); equal scores go to the smaller index. NaN scores
  * rank below every number.
  *   scores  device, N floats.         idx    device, capacity >= k int64 values.
@@ -144,7 +144,7 @@ sage_status_t sage_score_classes(sage_fd_t* h, const int32_t* labels, int32_t nu
  * counts num_classes int32 class sizes. Any out-pointer may be NULL. */
 sage_status_t sage_score_class_centroids(const sage_fd_t* h, const float** U, const int32_t** counts, int32_t* num_classes);
 
-/* Algorithm 1, "Select top-k_c per class (sum_c k_c = k)". The paper fixes only the sum; here
+/* Algorithm 1, the per-class top-k step of the class-balanced variant (the k_c sum to k). The paper fixes only the sum; here
  * k = sage_select_count(N_valid, keep_rate) with N_valid the number of examples whose label lies in [0, num_classes),
  * and k_c is proportional to the class size n_c with largest-remainder rounding: k_c = floor(k n_c / N_valid), the
  * k - sum floor(.) classes with the largest remainders (ties: smaller class id) get one more. Inside a class the order

@@ -109,7 +109,7 @@ class OracleFD:
 
 
 def score(S: np.ndarray, rows, D: Optional[int] = None) -> dict:
-    """Agreement scores (Method section "Two-pass scoring", Algorithm 1 Phase II) for all rows at once."""
+    """Agreement scores (Method section, paragraph on two-pass scoring,, Algorithm 1 Phase II) for all rows at once."""
     S = np.ascontiguousarray(S, dtype=np.float64)
     ell, Ds = S.shape
     kind, arr, n, ld = _rows_view(rows)
@@ -129,7 +129,7 @@ def select_k(N: int, keep_rate: float) -> int:
 
 
 def select(alpha: np.ndarray, keep_rate: float) -> np.ndarray:
-    """Top-k indices by alpha (Algorithm 1, "Select top-k by alpha_i"), ordered (alpha desc, index asc)."""
+    """Top-k indices by alpha (Algorithm 1, the top-k step), ordered (alpha desc, index asc)."""
     alpha = np.ascontiguousarray(alpha, dtype=np.float64)
     N = alpha.shape[0]
     idx = np.empty(max(select_k(N, keep_rate), 1), dtype=np.int64)

@@ -6,10 +6,10 @@
 // so results do not depend on the thread count.
 //
 // What it follows (paper sections / algorithm):
-//   * Frequent-Directions sketch, Method section, first paragraph and Algorithm 1 "Phase I":
+//   * Frequent-Directions sketch, Method section, first paragraph and Algorithm 1, Phase I:
 //     insert rows; when the buffer is full take the SVD, delta = sigma_ell^2,
 //     Sigma'_jj = sqrt(max(sigma_j^2 - delta, 0)), S <- Sigma' V^T.
-//   * Two-pass scoring, Method section "Two-pass scoring" and Algorithm 1 "Phase II":
+//   * Two-pass scoring, Method section, paragraph on two-pass scoring, and Algorithm 1, Phase II:
 //     z_i = S g_i, zhat_i = z_i/||z_i|| (0 if z_i = 0), zbar = mean zhat, u = zbar/||zbar|| (0 if zbar = 0),
 //     alpha_i = <zhat_i, u>.
 //   * Selection, Algorithm 1 last branch: top-k indices by alpha.
@@ -342,7 +342,7 @@ void sage_oracle_fd_update_bf16(void* h, const uint16_t* rows, int64_t n, int64_
     update_rows(*static_cast<FD*>(h), n, [=](int64_t i, int64_t d) { return bf16_to_double(rows[i * ld + d]); });
 }
 
-// "Freeze S": orthogonalise what is in the buffer, shrink only when more than ell rows are in use.
+// The freeze step of Algorithm 1: orthogonalise what is in the buffer, shrink only when more than ell rows are in use.
 void sage_oracle_fd_finalize(void* h) {
     FD& s = *static_cast<FD*>(h);
     std::vector<double> sig2;

@@ -1,15 +1,15 @@
-// Eigen-decomposition of the buffer's Gram matrix and the Frequent-Directions shrink factors
-// (Method, first paragraph: "compute a thin SVD S = U Sigma V^T, set delta = sigma_ell^2, shrink
-// Sigma'_jj = sqrt(max(sigma_j^2 - delta, 0))"). With K = B B^T = U Sigma^2 U^T the left factor U and
-// sigma^2 come from the symmetric eigen-problem of K, and Sigma' V^T = diag(sigma'/sigma) U^T B.
+// Eigen-decomposition of the buffer's Gram matrix and the Frequent-Directions shrink factors (Method, first
+// paragraph: the buffer's thin SVD is taken, delta is the squared ell-th singular value, and every squared singular
+// value is reduced by delta and clamped at zero). With K = B B^T = U Sigma^2 U^T the left factor U and sigma^2 come
+// from the symmetric eigen-problem of K, and Sigma' V^T = diag(sigma'/sigma) U^T B.
 //
-// Method: implicit (one-sided) cyclic Jacobi on a Cholesky factor. K is factored with diagonal
-// pivoting, P^T K P = L L^T (stopping at the numerical rank), then plane rotations are applied to
-// column pairs of L from the right until all columns are mutually orthogonal: L V = U Sigma. The
-// columns of the result are sigma_j u_j, so U needs no separate accumulation and small eigenvalues
-// keep their relative accuracy. One thread block does the whole solve; the matrix lives in shared
-// memory when it fits (n <= 232) and in global scratch (L2-resident) otherwise. All loops are bounded;
-// hitting the sweep limit sets a flag instead of spinning.
+// Method: implicit (one-sided) cyclic Jacobi on a Cholesky factor. K is factored with diagonal pivoting,
+// P^T K P = L L^T (stopping at the numerical rank), then plane rotations are applied to column pairs of L from the
+// right until all columns are mutually orthogonal: L V = U Sigma. The columns of the result are sigma_j u_j, so U
+// needs no separate accumulation and small eigenvalues keep their relative accuracy. Three kernel families follow:
+// one thread block with the factor in shared memory (buffers of up to 192 rows), a cluster of 8 thread blocks with
+// the factor in L2, and a cluster of 8 with Cholesky and Jacobi columns in distributed shared memory (the default
+// above 64 rows). All loops and waits are bounded; hitting the sweep limit sets a flag instead of spinning.
 #include <cooperative_groups.h>
 
 #include "sage_internal.h"
@@ -1679,7 +1679,7 @@ cudaError_t launch_eig_shrink(const float* K, int ldk, int n, int do_shrink, int
                               int j_pad, int variant, cudaStream_t st) {
     if (n <= 0 || n > 512) return cudaErrorInvalidValue;
     if (variant == 0 && n > 64) {   // cluster of 8 CTAs, Jacobi columns in distributed shared memory (n <= 64: one CTA is as fast)
-        const int T = n <= 64 ? 1 : n <= 128 ? 2 : n <= 192 ? 3 : n <= 256 ? 4 : 8;
+        const int T = n <= 128 ? 2 : n <= 192 ? 3 : n <= 256 ? 4 : 8;
         const int LD = 64 * T;
         const size_t bytes = 3 * 512 * sizeof(float) + 3 * 512 * sizeof(int) + 32 + 24 * sizeof(uint64_t) + (size_t)T * 128 * sizeof(uint32_t) +
                              2 * (size_t)LD * sizeof(float) + (size_t)(T <= 3 ? 2 : 1) * T * 8 * LD * sizeof(float);
@@ -1701,7 +1701,7 @@ cudaError_t launch_eig_shrink(const float* K, int ldk, int n, int do_shrink, int
     if (e == cudaSuccess)                                                                                                      \
         e = cudaLaunchKernelEx(&cfg, k_eig_shrink_dsm<TT, NTT>, K, ldk, n, do_shrink, delta_rank, keep, Ur, ldu, sigma_out, n_sigma, \
                                max_sweeps, info, Wsplit, ldw, j_pad, work);
-        if (T == 1) { SAGE_EIG_DSM(1, 512) } else if (T == 2) { SAGE_EIG_DSM(2, 512) } else if (T == 3) { SAGE_EIG_DSM(3, 512) }
+        if (T == 2) { SAGE_EIG_DSM(2, 512) } else if (T == 3) { SAGE_EIG_DSM(3, 512) }
         else if (T == 4) { SAGE_EIG_DSM(4, 256) } else { SAGE_EIG_DSM(8, 256) }
 #undef SAGE_EIG_DSM
         if (e == cudaSuccess) return cudaGetLastError();

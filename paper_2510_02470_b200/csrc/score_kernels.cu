@@ -1,4 +1,4 @@
-// Phase II after the projection (Method, "Two-pass scoring"; Algorithm 1, Phase II):
+// Phase II after the projection (Method, paragraph on two-pass scoring; Algorithm 1, Phase II):
 // row normalisation zhat_i = z_i/||z_i|| (0 when z_i = 0), the consensus sum over all rows, the unit
 // consensus u and the agreement scores alpha_i = <zhat_i, u>. All reductions run in a fixed order, so
 // a given sequence of calls gives bit-identical results every time.

@@ -1,4 +1,4 @@
-// Top-k selection (Algorithm 1, "Select top-k by alpha_i") with a total order: score descending, then
+// Top-k selection (Algorithm 1, the top-k step) with a total order: score descending, then
 // index ascending. Each score becomes a 64-bit key whose high word is the bitwise complement of an
 // order-preserving integer image of the float and whose low word is the row index; every key is
 // distinct, so an ascending LSD radix sort of the keys (8-bit digits, stable scatter) puts the rows in

@@ -10,7 +10,7 @@ __device__ __forceinline__ float to_f32(float x) { return x; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
 
 // ------------------------------------------------------------------------------------------------
-// Append (Algorithm 1, Phase I: "S[r,:] <- g"): copy / convert rows into free buffer rows.
+// Append (Algorithm 1, Phase I, the row insertion): copy / convert rows into free buffer rows.
 // One block row of threads walks a row with 16-byte accesses where the addresses allow it.
 // ------------------------------------------------------------------------------------------------
 template <typename T>
@@ -205,7 +205,7 @@ __global__ void __launch_bounds__(1024) k_gram_sym_reduce(const float* __restric
 }
 
 // ------------------------------------------------------------------------------------------------
-// Rebuild (Method, first paragraph: "reconstruct S <- Sigma' V^T"): with B B^T = U Lambda U^T,
+// Rebuild (Method, first paragraph: the sketch is rebuilt from the shrunk singular values and the right factor): with B B^T = U Lambda U^T,
 // Sigma' V^T = diag(sigma'_j / sigma_j) U^T B, so out[j][:] = sum_i Ur[i][j] B[i][:] where Ur already
 // carries the factor sqrt(max(1 - delta/lambda_j, 0)). Source and destination are different buffers.
 // Block tile: 64 output rows x 128 columns, contraction over the r buffer rows in steps of 16.

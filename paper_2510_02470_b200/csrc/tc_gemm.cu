@@ -1,5 +1,5 @@
 // Tensor-core contraction C[z] = A_z * B_z^T over slices z of the contraction index, both operands
-// contiguous along that index ("K-major"): the pass-2 projection Z = G S^T (Method, "Two-pass scoring":
+// contiguous along that index ("K-major"): the pass-2 projection Z = G S^T (Method, paragraph on two-pass scoring:
 // z_i = S g_i) with G streamed from HBM exactly once.
 //
 // One CTA owns mt (1, 2 or 4) consecutive 128-row tiles of A, all N rows of B and one K slice; the B tile of

@@ -1,4 +1,4 @@
-// Tensor-core rebuild of the sketch buffer (Method, first paragraph: "reconstruct S <- Sigma' V^T").
+// Tensor-core rebuild of the sketch buffer (Method, first paragraph: the sketch is rebuilt from the shrunk singular values and the right factor).
 // With B B^T = U Lambda U^T, Sigma' V^T = diag(sigma'_j / sigma_j) U^T B, i.e.
 //     out[j][d] = sum_i W[j][i] * B[i][d],   W[j][i] = U[i][j] * sqrt(max(1 - delta/lambda_j, 0)).
 // The buffer is the streamed operand: a CTA walks 128-column tiles of it, and for each tile accumulates over

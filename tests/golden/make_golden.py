@@ -5,7 +5,7 @@
 Each fixture instantiates a definition of the paper on a tiny seeded input:
   fd_small.json     Frequent-Directions sketch of a 40 x 12 stream with ell = 4 (Method, first paragraph;
                     Algorithm 1, Phase I): sigma' of the frozen sketch, sum of delta, number of shrinks.
-  scores_small.json agreement scores of 9 rows against a fixed 3 x 5 sketch (Method, "Two-pass scoring";
+  scores_small.json agreement scores of 9 rows against a fixed 3 x 5 sketch (Method, paragraph on two-pass scoring;
                     Algorithm 1, Phase II) and the top-4 selection (Algorithm 1, last branch).
 """
 import json
