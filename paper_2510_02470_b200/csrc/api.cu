@@ -685,7 +685,7 @@ sage_status_t sage_score_chunk(sage_fd_t* h, const void* rows, int64_t n, int64_
     DeviceGuard g(h->device);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const int ell = h->ell;
-    const int64_t sub_max = 148 * 128;       // one full wave of 128-row tiles
+    int64_t sub_max = 148 * 128;             // one full wave of 128-row tiles
     const char* p = static_cast<const char*>(rows);
     const size_t row_bytes = (size_t)ld * elem_size(h->dtype);
     const float* S = h->B[h->cur];
@@ -696,6 +696,9 @@ sage_status_t sage_score_chunk(sage_fd_t* h, const void* rows, int64_t n, int64_
     // fp32 rows: the fp32-faithful three-MMA kernel against the fp32 sketch itself (one 128-wide tile of S)
     const bool tc32_ok = h->use_tc && h->dtype == SAGE_F32 && ell <= 128 && (reinterpret_cast<uintptr_t>(rows) & 15u) == 0 &&
                          (row_bytes & 15u) == 0;
+    // fp32 rows against a small sketch: the projections of a sub-chunk are small (ell <= 64 floats per row and plane), so
+    // up to 8 waves go into one launch (fewer launch-scale overheads per pass)
+    if (tc32_ok && h->S32split) sub_max *= 8;
     for (int64_t r0 = 0; r0 < n; r0 += sub_max) {
         const int64_t sub = (n - r0 < sub_max) ? n - r0 : sub_max;
         const size_t nb = (size_t)((sub + 63) / 64);
