@@ -289,6 +289,66 @@ def test_c3_prefix_bf16():
     print(compare(out, ref, rows, w.D, 0.1, label="c3[:1500]"), out["stats"])
 
 
+def test_c3_full_size_properties():
+    """c3 at its full size (50,000 x 51,300 bf16, 387 shrinks), where the oracle would take an hour: checks that need no
+    oracle run. The Frequent-Directions bounds on A^T A - S^T S (largest eigenvalue by power iteration, at most the sum
+    of the deltas; smallest not below zero), the loss of squared Frobenius norm (at least ell times that sum), scores
+    of sampled rows recomputed in fp64 from the library's own S and u, the identity sum(alpha) = |sum(zhat)|, and the
+    selection redone by the oracle's sort on the library's scores."""
+    w = wl.WORKLOADS["c3"]
+    rows = wl.host_rows(w, 0)
+    g = rows.to(DEV)
+    N, D, ell = w.N, w.D, w.ell
+    fd = sage.SageFD(D, ell, rows.dtype, 0)
+    fd.update(g)
+    fd.finalize()
+    S, _ = fd.sketch()
+    scores = fd.score(g)
+    zhat, znorm, u = fd.intermediates(N)
+    idx = sage.sage_select(scores, 0.1)
+    torch.cuda.synchronize()
+    st = fd.stats()
+    assert st["shrinks"] == 387 and st["device_flags"] == 0
+    S64 = S[:, :D].double()
+
+    def op(x):                                     # x -> A^T (A x) - S^T (S x), fp64, rows converted chunk by chunk
+        y = torch.zeros_like(x)
+        for r0 in range(0, N, 2500):
+            a = g[r0:r0 + 2500, :D].double()
+            y += a.T @ (a @ x)
+        return y - S64.T @ (S64 @ x)
+
+    gen = torch.Generator(device=DEV).manual_seed(3)
+    fro_a = sum(float((g[r0:r0 + 5000, :D].double() ** 2).sum()) for r0 in range(0, N, 5000))
+    x = torch.randn(D, dtype=torch.float64, device=DEV, generator=gen)
+    lam_max = 0.0
+    for _ in range(25):
+        x = x / x.norm()
+        y = op(x)
+        lam_max = float(x @ y)
+        x = y
+    assert lam_max <= st["sum_delta"] * (1 + 1e-3), (lam_max, st["sum_delta"])
+    x = torch.randn(D, dtype=torch.float64, device=DEV, generator=gen)     # smallest eigenvalue: iterate on lam_max I - M
+    lam_min = 0.0
+    for _ in range(25):
+        x = x / x.norm()
+        y = lam_max * x - op(x)
+        lam_min = lam_max - float(x @ y)
+        x = y
+    assert lam_min >= -1e-5 * fro_a, (lam_min, fro_a)
+    assert fro_a - float((S64 ** 2).sum()) >= ell * st["sum_delta"] * (1 - 1e-3)
+    # scores of sampled rows from the library's own sketch and consensus, in fp64
+    pick = np.random.default_rng(5).choice(N, 256, replace=False)
+    z = g[torch.from_numpy(pick).to(DEV), :D].double() @ S64.T
+    zn = z.norm(dim=1, keepdim=True)
+    a64 = ((z / zn.clamp_min(1e-300)) @ u[:ell].double()).cpu().numpy()
+    a_gpu = scores.double().cpu().numpy()
+    assert np.max(np.abs(a64 - a_gpu[pick])) <= TOL_SCORE[torch.bfloat16]
+    assert abs(a_gpu.sum() - float(zhat.double().sum(dim=0).norm())) <= 1e-3 * N ** 0.5
+    assert np.array_equal(idx.cpu().numpy(), oracle.select(a_gpu, 0.1))
+    fd.close()
+
+
 def test_c4_shape_small_prefix():
     """c4's generator and ell=256 on a reduced D and row count (the full D is covered by bench checks)."""
     w = wl.scaled(wl.WORKLOADS["c4"], N=1300, D=8192, chunk_rows=650)
@@ -309,6 +369,82 @@ def test_c5_shape_small_prefix():
 
 
 # ------------------------------------------------------------------ host pipeline and state machine
+
+def _streamed_properties(w, sample_rows=192):
+    """Both passes streamed chunk by chunk, as the benchmark does for c4 and c5; returns what the checks need."""
+    stream = wl.DeviceStream(w, seed=0, device=DEV)
+    N, D, ell = w.N, w.D, w.ell
+    fd = sage.SageFD(D, ell, w.dtype, 0)
+    fro_a = 0.0
+    for j in range(w.num_chunks):
+        c = stream.chunk(j)
+        fro_a += float((c[:, :D].float() ** 2).sum(dtype=torch.float64))
+        fd.update(c)
+    fd.finalize()
+    S, _ = fd.sketch()
+    fd.score_begin(N)
+    pick = np.sort(np.random.default_rng(7).choice(N, min(sample_rows, N), replace=False))
+    kept = []
+    r0 = 0
+    for j in range(w.num_chunks):
+        c = stream.chunk(j)
+        fd.score_chunk(c, r0)
+        local = pick[(pick >= r0) & (pick < r0 + c.shape[0])] - r0
+        if local.size:
+            kept.append(c[torch.from_numpy(local).to(DEV), :D].clone())
+        r0 += c.shape[0]
+    scores = torch.empty((N,), dtype=torch.float32, device=DEV)
+    fd.score_end(scores)
+    zhat, znorm, u = fd.intermediates(N)
+    idx = sage.sage_select(scores, 0.1)
+    torch.cuda.synchronize()
+    st = fd.stats()
+    a_gpu = scores.double().cpu().numpy()
+    # sampled rows re-scored in fp64 from the library's own S and u, a block of sketch columns at a time
+    G = torch.cat(kept)
+    z = torch.zeros((G.shape[0], ell), dtype=torch.float64, device=DEV)
+    for c0 in range(0, D, 1 << 20):
+        z += G[:, c0:c0 + (1 << 20)].double() @ S[:, c0:min(D, c0 + (1 << 20))].double().T
+    a64 = ((z / z.norm(dim=1, keepdim=True).clamp_min(1e-300)) @ u[:ell].double()).cpu().numpy()
+    fro_s = float((S[:, :D] ** 2).sum(dtype=torch.float64))
+    out = {"stats": st, "fro_a": fro_a, "fro_s": fro_s, "a_gpu": a_gpu, "a64": a64, "pick": pick,
+           "sum_zhat_norm": float(zhat.double().sum(dim=0).norm()), "idx": idx.cpu().numpy()}
+    fd.close()
+    return out
+
+
+def _expected_shrinks(N, ell):
+    """Shrinks of a 2 ell-row buffer over N rows: one whenever the buffer fills up (ell - 1 rows survive), and one at
+    the freeze if more than ell rows are in use."""
+    fill = shrinks = 0
+    for _ in range(N):
+        fill += 1
+        if fill == 2 * ell:
+            shrinks += 1
+            fill = ell - 1
+    return shrinks + (1 if fill > ell else 0)
+
+
+def _check_streamed(o, w, shrinks):
+    st = o["stats"]
+    assert st["shrinks"] == shrinks and st["device_flags"] == 0
+    assert o["fro_a"] - o["fro_s"] >= w.ell * st["sum_delta"] * (1 - 1e-3)          # every shrink removes at least ell * delta
+    assert np.max(np.abs(o["a64"] - o["a_gpu"][o["pick"]])) <= TOL_SCORE[torch.bfloat16]
+    assert abs(o["a_gpu"].sum() - o["sum_zhat_norm"]) <= 1e-3 * w.N ** 0.5
+    assert np.array_equal(o["idx"], oracle.select(o["a_gpu"], 0.1))
+
+
+def test_c4_full_size_properties():
+    """c4 at its full size (200,000 x 262,144 bf16 in 25 chunks, ell = 256): the checks that need no oracle run."""
+    w = wl.WORKLOADS["c4"]
+    _check_streamed(_streamed_properties(w), w, _expected_shrinks(w.N, w.ell))
+
+
+def test_c5_full_size_properties():
+    """c5 at its full size (50,000 x 11,173,962 bf16 in 98 chunks, ell = 64)."""
+    w = wl.WORKLOADS["c5"]
+    _check_streamed(_streamed_properties(w, sample_rows=96), w, _expected_shrinks(w.N, w.ell))
+
 
 def test_select_from_host_matches_device_path():
     N, D, ell = 3000, 515, 16
