@@ -1028,12 +1028,12 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
     int* order = perm + kMaxN;                          // sorted position -> pivot step
     float* sh_f = reinterpret_cast<float*>(order + kMaxN);
     uint64_t* mbar = reinterpret_cast<uint64_t*>(sh_f + 8);   // [2 sets][8 slots] exchange barriers (kP2P)
-    uint64_t* pbar = mbar + 16;                         // Cholesky phase: [2] pivot column landed (bytes), then
-    uint64_t* cdone = mbar + 18;                        // [2] every warp of this CTA has finished the step, and
-    uint64_t* alldone = mbar + 20;                      // [2] every CTA of the cluster has
-    uint32_t* sched = reinterpret_cast<uint32_t*>(mbar + 24);   // [T slots][128 block rounds] packed exchange schedule
-    float* pbuf = reinterpret_cast<float*>(sched + T * 128);    // [2][LD] pivot columns of the Cholesky phase
-    float* sbuf = pbuf + 2 * LD;                        // slot buffers: [kSets][T slots][2 halves][4 columns][LD]
+    uint64_t* pbar = mbar + 16;                         // Cholesky phase: [3] pivot column landed (bytes), then
+    uint64_t* cdone = mbar + 19;                        // [3] every warp of this CTA has finished the step, and
+    uint64_t* alldone = mbar + 22;                      // [3] every CTA of the cluster has
+    uint32_t* sched = reinterpret_cast<uint32_t*>(mbar + 32);   // [T slots][128 block rounds] packed exchange schedule
+    float* pbuf = reinterpret_cast<float*>(sched + T * 128);    // [3][LD] pivot columns of the Cholesky phase
+    float* sbuf = pbuf + 3 * LD;                        // slot buffers: [kSets][T slots][2 halves][4 columns][LD]
 
     const int tid = threadIdx.x, lane = tid & 31, lwarp = tid >> 5;
     const int gtid = crank * NT + tid;
@@ -1060,9 +1060,9 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
     for (int t = 0; t < R; ++t) dg[t] *= kscale;
     for (int i = tid; i < kMaxN; i += NT) { ord[i] = -1; perm[i] = 0; }
     if (gtid < 4) gflag[gtid] = 0;
-    if (tid < 18) mbar_init_cluster(&mbar[tid], 1);     // the reader's own arrival; the stores count bytes
-    if (tid >= 18 && tid < 20) mbar_init_cluster(&mbar[tid], WPC);
-    if (tid >= 20 && tid < 22) mbar_init_cluster(&mbar[tid], 8);
+    if (tid < 19) mbar_init_cluster(&mbar[tid], 1);     // the reader's own arrival; the stores count bytes
+    if (tid >= 19 && tid < 22) mbar_init_cluster(&mbar[tid], WPC);
+    if (tid >= 22 && tid < 25) mbar_init_cluster(&mbar[tid], 8);
     if (tid == 0) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     const float tol = 1e-7f;
     int rank = empty ? 0 : n;
@@ -1072,8 +1072,10 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
     // The warp that owns the pivot column sends it to all 8 CTAs with asynchronous stores that count their bytes
     // on a barrier in each CTA; every warp waits for that, refreshes its diagonal and updates the columns it owns
     // in its CTA's shared memory: a step costs one one-way trip instead of a cluster barrier plus L2 round trips,
-    // and the trailing update has the shared-memory bandwidth of 8 SMs. The two pivot buffers alternate; before a
-    // warp overwrites the buffer of step k - 2 it waits until every CTA has reported that step finished (each warp
+    // and the trailing update has the shared-memory bandwidth of 8 SMs. The owner of the NEXT pivot column (known as
+    // soon as the diagonal is refreshed) updates that column first and sends it at once, so the trip overlaps the rest
+    // of the step. Three pivot buffers rotate; before a warp overwrites the buffer of step k - 3 it waits until every
+    // CTA has reported that step finished (each warp
     // arrives on its CTA's `cdone` barrier at the end of a step; warp 0 of each CTA waits for that and arrives on
     // the `alldone` barrier of all 8 CTAs: a whole step of slack, so the sender rarely waits). Every wait is bounded;
     // one that runs out raises the cluster-wide give-up word, which ends all other waits, and every warp leaves the
@@ -1099,46 +1101,55 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
     __syncwarp();
     cluster.sync();                                      // barriers initialised everywhere before the first remote store
     bool chol_failed = false;
-    for (int k = 0; k < rank; ++k) {
+    auto find_pivot = [&]() -> int {                              // largest remaining diagonal entry; -1: none left
         unsigned key = 0u;
 #pragma unroll
         for (int t = 0; t < R; ++t)
             if (alive[t]) key = max(key, (__float_as_uint(fmaxf(dg[t], 0.f)) & 0xfffffe00u) | (unsigned)(511 - (lane + 32 * t)));
-        key = __reduce_max_sync(0xffffffffu, key);                // largest diagonal (23 significant bits), smaller index on ties
+        key = __reduce_max_sync(0xffffffffu, key);                // 23 significant bits, smaller index on ties
         const int p = 511 - (int)(key & 511u);
-        if (key == 0u || p >= n) { rank = k; break; }             // identical in every warp of the cluster
-        const int set = k & 1;
-        float* pb = pbuf + set * LD;
-        {
-            const int ojl = p >> 3;
-            if ((p & 7) == crank && (ojl % WPC) == lwarp) {       // this warp owns the pivot column: send it to all 8 CTAs
-                if (k >= 2) {                                     // ... once nobody reads the step before last any more
-                    bool free_ = mbar_wait_cluster(&alldone[set], (uint32_t)((k >> 1) - 1) & 1u, &gflag[3]);
-                    free_ = __all_sync(0xffffffffu, free_);
-                    if (!free_) {
-                        if (lane == 0) atomicOr(&gflag[3], 1);
-                        chol_failed = true;
-                        break;
-                    }
-                }
-                const float4* src = reinterpret_cast<const float4*>(Xc + ojl * LD);
-                const uint32_t dst0 = smem_addr_u32(pb), bar0 = smem_addr_u32(&pbar[set]);
-                for (int q = lane; q < LD / 4; q += 32) {
-                    const float4 v = src[q];
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) st_async_v4(mapa_u32(dst0 + 16u * q, (uint32_t)c), v, mapa_u32(bar0, (uint32_t)c));
-                }
-                colmask &= ~(1u << (ojl / WPC));
+        return (key == 0u || p >= n) ? -1 : p;                    // identical in every warp of the cluster
+    };
+    // The warp that owns column p sends it to all 8 CTAs as the pivot column of step k (buffer and barrier k % 3), once
+    // every CTA has reported step k - 3 finished. Returns false if that wait ran out.
+    auto send_pivot = [&](int p, int k) -> bool {
+        const int ojl = p >> 3, set = k % 3;
+        if ((p & 7) != crank || (ojl % WPC) != lwarp) return true;
+        if (k >= 3) {
+            bool free_ = mbar_wait_cluster(&alldone[set], (uint32_t)(k / 3 - 1) & 1u, &gflag[3]);
+            free_ = __all_sync(0xffffffffu, free_);
+            if (!free_) {
+                if (lane == 0) atomicOr(&gflag[3], 1);
+                return false;
             }
         }
-        if (tid == 0) mbar_arrive_expect_tx(&pbar[set], (uint32_t)(LD * sizeof(float)));
-        bool ok = mbar_wait_cluster(&pbar[set], (uint32_t)(k >> 1) & 1u, &gflag[3]);
+        const float4* src = reinterpret_cast<const float4*>(Xc + ojl * LD);
+        const uint32_t dst0 = smem_addr_u32(pbuf + set * LD), bar0 = smem_addr_u32(&pbar[set]);
+        for (int q = lane; q < LD / 4; q += 32) {
+            const float4 v = src[q];
+#pragma unroll
+            for (int c = 0; c < 8; ++c) st_async_v4(mapa_u32(dst0 + 16u * q, (uint32_t)c), v, mapa_u32(bar0, (uint32_t)c));
+        }
+        colmask &= ~(1u << (ojl / WPC));
+        return true;
+    };
+    int p = rank > 0 ? find_pivot() : -1;
+    if (p >= 0 && !send_pivot(p, 0)) chol_failed = true;
+    if (tid == 0) mbar_arrive_expect_tx(&pbar[0], (uint32_t)(LD * sizeof(float)));   // this CTA expects the column of step 0
+    for (int k = 0; k < rank && !chol_failed; ++k) {
+        if (p < 0) { rank = k; break; }                           // identical in every warp of the cluster
+        const int set = k % 3;
+        const float* pb = pbuf + set * LD;
+        bool ok = mbar_wait_cluster(&pbar[set], (uint32_t)(k / 3) & 1u, &gflag[3]);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) {
             if (lane == 0) atomicOr(&gflag[3], 1);
             chol_failed = true;
             break;
         }
+        // announce the next step's column now (its barrier finished its previous use three steps ago), so that the
+        // other warps of this CTA never wait for warp 0, which has the reporting below to do
+        if (tid == 0) mbar_arrive_expect_tx(&pbar[(k + 1) % 3], (uint32_t)(LD * sizeof(float)));
         const float d = pb[p];
         if (!(d > tol)) { rank = k; break; }                      // identical everywhere: all read the same column
         const float inv = rsqrtf(d);
@@ -1150,21 +1161,28 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
             li[t] = alive[t] ? pb[i] * inv : 0.f;
             dg[t] = fmaf(-li[t], li[t], dg[t]);
         }
+        // Look-ahead: the refreshed diagonal already names the next pivot; its owner brings that column up to date first
+        // and sends it, so that its trip to the other CTAs overlaps the rest of this step's update.
+        const int p_next = (k + 1 < rank) ? find_pivot() : -1;
+        auto update_column = [&](int u) {
+            const int jl = lwarp + WPC * u;
+            float* col = Xc + jl * LD;
+            const float l = pb[jl * 8 + crank] * inv;
 #pragma unroll
-        for (int u = 0; u < CW; ++u) {
-            if ((colmask >> u) & 1u) {
-                const int jl = lwarp + WPC * u;
-                float* col = Xc + jl * LD;
-                const float l = pb[jl * 8 + crank] * inv;
-#pragma unroll
-                for (int t = 0; t < R; ++t) col[lane + 32 * t] = fmaf(-li[t], l, col[lane + 32 * t]);
-            }
+            for (int t = 0; t < R; ++t) col[lane + 32 * t] = fmaf(-li[t], l, col[lane + 32 * t]);
+        };
+        if (p_next >= 0 && (p_next & 7) == crank && ((p_next >> 3) % WPC) == lwarp) {
+            update_column((p_next >> 3) / WPC);
+            __syncwarp();                                         // the send reads whole float4s of what the lanes updated
+            if (!send_pivot(p_next, k + 1)) { chol_failed = true; break; }
         }
+#pragma unroll
+        for (int u = 0; u < CW; ++u)
+            if ((colmask >> u) & 1u) update_column(u);
         if (tid == 0) { ord[p] = k; perm[k] = p; scl[k] = inv; }   // every CTA keeps its own copy of the tables
-        __syncwarp();                                             // the sender reads whole float4s of what the lanes updated
         if (lane == 0) mbar_arrive_local(&cdone[set]);            // this warp has finished step k
         if (lwarp == 0) {                                         // warp 0 reports the whole CTA to all 8 CTAs
-            bool fin = mbar_wait_cluster(&cdone[set], (uint32_t)(k >> 1) & 1u, &gflag[3]);
+            bool fin = mbar_wait_cluster(&cdone[set], (uint32_t)(k / 3) & 1u, &gflag[3]);
             fin = __all_sync(0xffffffffu, fin);
             if (!fin) {
                 if (lane == 0) atomicOr(&gflag[3], 1);
@@ -1173,6 +1191,7 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
             }
             if (lane < 8) mbar_arrive_remote(mapa_u32(smem_addr_u32(&alldone[set]), (uint32_t)lane));
         }
+        p = p_next;
     }
     __syncthreads();
     // ---- scale the pivot columns into the factor L (zero above the pivot order, zero unpivoted columns), into L2 ----
@@ -1681,11 +1700,11 @@ cudaError_t launch_eig_shrink(const float* K, int ldk, int n, int do_shrink, int
     if (variant == 0 && n > 64) {   // cluster of 8 CTAs, Jacobi columns in distributed shared memory (n <= 64: one CTA is as fast)
         const int T = n <= 128 ? 2 : n <= 192 ? 3 : n <= 256 ? 4 : 8;
         const int LD = 64 * T;
-        const size_t bytes = 3 * 512 * sizeof(float) + 3 * 512 * sizeof(int) + 32 + 24 * sizeof(uint64_t) + (size_t)T * 128 * sizeof(uint32_t) +
-                             2 * (size_t)LD * sizeof(float) + (size_t)(T <= 3 ? 2 : 1) * T * 8 * LD * sizeof(float);
+        const size_t bytes = 3 * 512 * sizeof(float) + 3 * 512 * sizeof(int) + 32 + 32 * sizeof(uint64_t) + (size_t)T * 128 * sizeof(uint32_t) +
+                             3 * (size_t)LD * sizeof(float) + (size_t)(T <= 3 ? 2 : 1) * T * 8 * LD * sizeof(float);
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(8);
-        cfg.blockDim = dim3(T <= 3 ? 512 : 256);
+        cfg.blockDim = dim3(256);
         cfg.dynamicSmemBytes = bytes;
         cfg.stream = st;
         cudaLaunchAttribute at[1];
@@ -1701,7 +1720,7 @@ cudaError_t launch_eig_shrink(const float* K, int ldk, int n, int do_shrink, int
     if (e == cudaSuccess)                                                                                                      \
         e = cudaLaunchKernelEx(&cfg, k_eig_shrink_dsm<TT, NTT>, K, ldk, n, do_shrink, delta_rank, keep, Ur, ldu, sigma_out, n_sigma, \
                                max_sweeps, info, Wsplit, ldw, j_pad, work);
-        if (T == 2) { SAGE_EIG_DSM(2, 512) } else if (T == 3) { SAGE_EIG_DSM(3, 512) }
+        if (T == 2) { SAGE_EIG_DSM(2, 256) } else if (T == 3) { SAGE_EIG_DSM(3, 256) }
         else if (T == 4) { SAGE_EIG_DSM(4, 256) } else { SAGE_EIG_DSM(8, 256) }
 #undef SAGE_EIG_DSM
         if (e == cudaSuccess) return cudaGetLastError();
