@@ -1275,41 +1275,15 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
                 bool loaded = false;
                 if (work) {
                     float* cur = kP2P ? sbuf + (size_t)((g & 1) * T + myslot) * 8 * LD : mybuf;
-                    bool ok = true;
-                    if (kP2P && g > 0) {                          // both blocks of this round have landed in this set
-                        if (lane == 0) mbar_arrive_expect_tx(&mbar[(g & 1) * 8 + myslot], 8u * LD * sizeof(float));
-                        ok = mbar_wait_cluster(&mbar[(g & 1) * 8 + myslot], (uint32_t)((g - 1) >> 1) & 1u, &gflag[3]);
-                        ok = __all_sync(0xffffffffu, ok);
-                        if (!ok) {
-                            failed = true;
-                            if (lane == 0) atomicOr(&gflag[3], 1);
-                        }
-                    }
-                    if (ok) {
-                        loaded = true;
-                        const uint32_t sc = mysched[br];
-                        const int ba = (int)(sc & 255u), bb = (int)((sc >> 8) & 255u);
-                        if (br == 0) {                            // pairs inside each block: quarters 0,1 -> ba, 2,3 -> bb
-                            const int half = (qd < 2) ? 0 : 1, base = 4 * (half ? bb : ba), h = qd & 1;
-                            float* blk = cur + half * 4 * LD;
-                            const int c0 = h ? 2 : 0, c1 = h ? 3 : 1, c2 = h ? 1 : 0, c3 = h ? 3 : 2, c4 = h ? 1 : 0, c5 = h ? 2 : 3;
-                            jacobi_pair_in_smem<Q>(blk + c0 * LD, blk + c1 * LD, base + c0 < rank && base + c1 < rank, l8, worst2);
-                            jacobi_pair_in_smem<Q>(blk + c2 * LD, blk + c3 * LD, base + c2 < rank && base + c3 < rank, l8, worst2);
-                            jacobi_pair_in_smem<Q>(blk + c4 * LD, blk + c5 * LD, base + c4 < rank && base + c5 < rank, l8, worst2);
-                        }
-                        const int lo = min(ba, bb);
-                        hi = max(ba, bb);
-                        const int half_lo = (ba < bb) ? 0 : 1;
-                        // quarter qd keeps column qd of block lo; the columns of block hi travel between quarters
-                        const float4* xa = reinterpret_cast<const float4*>(cur + (half_lo * 4 + qd) * LD) + l8;
-                        const float4* xb = reinterpret_cast<const float4*>(cur + ((1 - half_lo) * 4 + qd) * LD) + l8;
-                        va = 4 * lo + qd < rank;
-#pragma unroll
-                        for (int t = 0; t < Q; ++t) {
-                            x[t] = xa[8 * t];
-                            y[t] = xb[8 * t];
-                        }
-                        // where the next block round reads the two columns this quarter ends up with
+                    // Everything that does not depend on the incoming columns first (it runs while they are in flight):
+                    // the block pair of this round and where the next block round reads the columns this quarter ends with
+                    const uint32_t sc = mysched[br];
+                    const int ba = (int)(sc & 255u), bb = (int)((sc >> 8) & 255u);
+                    const int lo = min(ba, bb);
+                    hi = max(ba, bb);
+                    const int half_lo = (ba < bb) ? 0 : 1;
+                    va = 4 * lo + qd < rank;
+                    {
                         const int c_lo = (int)((sc >> 16) & 7u), l_lo = (int)((sc >> 19) & 7u), h_lo = (int)((sc >> 22) & 1u);
                         const int c_hi = (int)((sc >> 23) & 7u), l_hi = (int)((sc >> 26) & 7u), h_hi = (int)((sc >> 29) & 1u);
                         const int nset = kP2P ? ((g + 1) & 1) : 0;
@@ -1323,6 +1297,35 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
                         } else {
                             o_lo = reinterpret_cast<float4*>(cluster.map_shared_rank(d_lo, c_lo));
                             o_hi = reinterpret_cast<float4*>(cluster.map_shared_rank(d_hi, c_hi));
+                        }
+                    }
+                    bool ok = true;
+                    if (kP2P && g > 0) {                          // both blocks of this round have landed in this set
+                        if (lane == 0) mbar_arrive_expect_tx(&mbar[(g & 1) * 8 + myslot], 8u * LD * sizeof(float));
+                        ok = mbar_wait_cluster(&mbar[(g & 1) * 8 + myslot], (uint32_t)((g - 1) >> 1) & 1u, &gflag[3]);
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (!ok) {
+                            failed = true;
+                            if (lane == 0) atomicOr(&gflag[3], 1);
+                        }
+                    }
+                    if (ok) {
+                        loaded = true;
+                        if (br == 0) {                            // pairs inside each block: quarters 0,1 -> ba, 2,3 -> bb
+                            const int half = (qd < 2) ? 0 : 1, base = 4 * (half ? bb : ba), h = qd & 1;
+                            float* blk = cur + half * 4 * LD;
+                            const int c0 = h ? 2 : 0, c1 = h ? 3 : 1, c2 = h ? 1 : 0, c3 = h ? 3 : 2, c4 = h ? 1 : 0, c5 = h ? 2 : 3;
+                            jacobi_pair_in_smem<Q>(blk + c0 * LD, blk + c1 * LD, base + c0 < rank && base + c1 < rank, l8, worst2);
+                            jacobi_pair_in_smem<Q>(blk + c2 * LD, blk + c3 * LD, base + c2 < rank && base + c3 < rank, l8, worst2);
+                            jacobi_pair_in_smem<Q>(blk + c4 * LD, blk + c5 * LD, base + c4 < rank && base + c5 < rank, l8, worst2);
+                        }
+                        // quarter qd keeps column qd of block lo; the columns of block hi travel between quarters
+                        const float4* xa = reinterpret_cast<const float4*>(cur + (half_lo * 4 + qd) * LD) + l8;
+                        const float4* xb = reinterpret_cast<const float4*>(cur + ((1 - half_lo) * 4 + qd) * LD) + l8;
+#pragma unroll
+                        for (int t = 0; t < Q; ++t) {
+                            x[t] = xa[8 * t];
+                            y[t] = xb[8 * t];
                         }
                     }
                 }
