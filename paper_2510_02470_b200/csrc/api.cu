@@ -121,7 +121,8 @@ struct sage_fd {
     State state = SKETCHING;
     int delta_rank = 0, max_sweeps = 30;
     // Gram / eigen workspaces
-    float* gram_parts = nullptr;   // split-K partials of the Gram matrix (kGramPartFloats floats)
+    float* gram_parts = nullptr;   // split-K partials of the Gram matrix (gram_part_floats floats)
+    size_t gram_part_floats = 0;   // at least kGramPartFloats; 16 slices of m x m for buffers of more than 256 rows
     float* Wsplit = nullptr;       // rebuild factors split for the tensor cores: wsplit_ld rows x wsplit_ld floats
     int wsplit_ld = 256;           // 256 (buffers of up to 256 rows) or 512
     float* Kmat = nullptr;         // m x m
@@ -234,22 +235,17 @@ sage_status_t enqueue_gram(sage_fd* h, int r, cudaStream_t st) {
         const int ldc = ((r + 3) / 4) * 4;
         const int64_t stride = (int64_t)r * ldc;
         const int sym = r <= 128 ? 1 : 0;    // one diagonal tile: two MMAs per K step, transpose added in the reduction
-        int cap = (int)(kGramPartFloats / (size_t)stride);
+        int cap = (int)(h->gram_part_floats / (size_t)stride);
         if (cap > 148) cap = 148;
-        const int splits = pick_splits_waves(t * t, h->D, 256, cap);
-        cudaError_t e;
-        if (splits == 1 && !sym) {
-            e = timed(h, K_GRAM, 1, st, [&] { return launch_tc_gemm_nt_x3(Bc, h->pitch, Bc, h->pitch, r, r, h->D, 1, h->Kmat, h->m, 0, 0, h->tc_err, st); });
-        } else {
-            e = timed(h, K_GRAM, 1, st, [&] {
-                return launch_tc_gemm_nt_x3(Bc, h->pitch, Bc, h->pitch, r, r, h->D, splits, h->gram_parts, ldc, stride, sym, h->tc_err, st);
-            });
-        }
+        const int splits = pick_splits_waves(t * (t + 1) / 2, h->D, 256, cap);   // only the tiles on and above the diagonal run
+        cudaError_t e = timed(h, K_GRAM, 1, st, [&] {
+            return launch_tc_gemm_nt_x3(Bc, h->pitch, Bc, h->pitch, r, r, h->D, splits, h->gram_parts, ldc, stride, sym, h->tc_err, st);
+        });
         if (e == cudaSuccess) {
             if (sym)
                 CU_TRY(timed(h, K_GRAM_REDUCE, 1, st, [&] { return launch_gram_sym_reduce(h->gram_parts, splits, stride, r, ldc, h->Kmat, h->m, st); }));
-            else if (splits > 1)
-                CU_TRY(timed(h, K_GRAM_REDUCE, 1, st, [&] { return launch_split_reduce(h->gram_parts, splits, stride, r, r, ldc, h->Kmat, h->m, st); }));
+            else   // sums the K slices and fills the tiles below the diagonal from their mirror images
+                CU_TRY(timed(h, K_GRAM_REDUCE, 1, st, [&] { return launch_split_reduce(h->gram_parts, splits, stride, r, r, ldc, h->Kmat, h->m, st, 1); }));
             return SAGE_OK;
         }
         if (e != cudaErrorNotSupported) CU_TRY(e);
@@ -393,7 +389,9 @@ sage_status_t sage_fd_create(sage_fd_t** out, int64_t D, int32_t ell, sage_dtype
     cudaError_t e;
     for (int i = 0; i < 2; ++i)
         if ((e = cudaMalloc((void**)&h->B[i], bbytes)) != cudaSuccess) return fail(e, "cudaMalloc(buffer)");
-    if ((e = cudaMalloc((void**)&h->gram_parts, kGramPartFloats * sizeof(float))) != cudaSuccess) return fail(e, "cudaMalloc(gram)");
+    h->gram_part_floats = kGramPartFloats;
+    if ((size_t)16 * h->m * h->m > h->gram_part_floats) h->gram_part_floats = (size_t)16 * h->m * h->m;
+    if ((e = cudaMalloc((void**)&h->gram_parts, h->gram_part_floats * sizeof(float))) != cudaSuccess) return fail(e, "cudaMalloc(gram)");
     h->wsplit_ld = h->m <= 256 ? 256 : 512;
     if ((e = cudaMalloc((void**)&h->Wsplit, (size_t)h->wsplit_ld * h->wsplit_ld * sizeof(float))) != cudaSuccess)
         return fail(e, "cudaMalloc(W)");

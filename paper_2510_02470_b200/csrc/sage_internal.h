@@ -48,7 +48,8 @@ cudaError_t launch_tc_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const
 
 // fp32-faithful tensor-core C[z] = A_z * Bm_z^T for fp32 operands (three tf32 MMAs on hi/lo halves split in shared
 // memory, accumulator drained into registers every few K tiles). Same alignment rules and return convention as
-// launch_tc_gemm_nt; any N. When A == Bm (a Gram matrix) the diagonal tiles load one operand only.
+// launch_tc_gemm_nt; any N. When A == Bm (a Gram matrix) the diagonal tiles load one operand only and the 128 x 128
+// tiles below the diagonal are NOT computed (their part of C is left untouched): reduce with mirror = 1.
 // sym != 0 (only for a Gram matrix of at most 128 rows): two MMAs per K step instead of three; slice z then stores
 // T_z = hi*hi^T + 2*hi*lo^T and the Gram matrix is sum_z (T_z + T_z^T)/2: see launch_gram_sym_reduce.
 // sym == 2 (projection onto at most 64 sketch rows): Bm is the sketch already split by launch_split_tf32 (128 rows);
@@ -76,7 +77,7 @@ cudaError_t launch_to_bf16(const float* src, int64_t lds, int rows, int64_t cols
 cudaError_t launch_split_tf32(const float* src, int64_t lds, int rows, int64_t cols, float* out, int64_t ldo, cudaStream_t st);
 
 cudaError_t launch_split_reduce(const float* parts, int splits, int64_t split_stride, int M, int N, int64_t ldp,
-                                float* out, int64_t ldo, cudaStream_t st);
+                                float* out, int64_t ldo, cudaStream_t st, int mirror = 0);
 
 // out[j][d] = sum_{i<r} Ur[i*ldu + j] * Bsrc[i*pitch + d] for j < keep; rows keep..m_total-1 of out are zeroed.
 cudaError_t launch_rebuild(const float* Ur, int ldu, const float* Bsrc, float* Bdst, int64_t pitch, int64_t D, int r,

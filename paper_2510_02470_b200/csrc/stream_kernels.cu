@@ -163,13 +163,17 @@ __global__ void __launch_bounds__(256) k_split_tf32(const float* __restrict__ sr
     }
 }
 
+// mirror != 0 (a symmetric matrix of which only the 128 x 128 tiles on and above the diagonal were computed): elements of
+// the tiles below the diagonal are read from their mirror image.
 __global__ void __launch_bounds__(256) k_split_reduce(const float* __restrict__ parts, int splits, int64_t split_stride,
-                                                      int M, int N, int64_t ldp, float* __restrict__ out, int64_t ldo) {
+                                                      int M, int N, int64_t ldp, float* __restrict__ out, int64_t ldo, int mirror) {
     const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= (int64_t)M * N) return;
     const int i = (int)(e / N), j = (int)(e % N);
+    const bool below = mirror && (i >> 7) > (j >> 7);
+    const float* src = parts + (below ? (int64_t)j * ldp + i : (int64_t)i * ldp + j);
     double s = 0.0;
-    for (int z = 0; z < splits; ++z) s += (double)parts[(int64_t)z * split_stride + (int64_t)i * ldp + j];
+    for (int z = 0; z < splits; ++z) s += (double)src[(int64_t)z * split_stride];
     out[(int64_t)i * ldo + j] = (float)s;
 }
 
@@ -313,10 +317,10 @@ cudaError_t launch_split_tf32(const float* src, int64_t lds, int rows, int64_t c
 }
 
 cudaError_t launch_split_reduce(const float* parts, int splits, int64_t split_stride, int M, int N, int64_t ldp, float* out,
-                                int64_t ldo, cudaStream_t st) {
+                                int64_t ldo, cudaStream_t st, int mirror) {
     const int64_t total = (int64_t)M * N;
     if (total <= 0) return cudaSuccess;
-    k_split_reduce<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(parts, splits, split_stride, M, N, ldp, out, ldo);
+    k_split_reduce<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(parts, splits, split_stride, M, N, ldp, out, ldo, mirror);
     return cudaGetLastError();
 }
 

@@ -66,6 +66,7 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     const int m0 = blockIdx.x * kTileM, n0 = blockIdx.y * kTileN;
+    if (gram && m0 > n0) return;                          // a Gram matrix is symmetric: the reduction mirrors the upper tiles
     const bool proj = sym == 2;
     const bool wide = sym != 0;                           // one 256-wide MMA per K step
     const bool diag = gram && m0 == n0;                   // A tile == B tile: load once
