@@ -280,7 +280,7 @@ sage_status_t enqueue_factor(sage_fd* h, int r, int do_shrink, int keep, int zer
     const int m_total = zero_to > keep ? zero_to : keep;
     bool done = false;
     if (tc_rebuild) {
-        const int parts = (j_pad > 128 ? 2 : 1) * (r > 256 ? 2 : 1);     // launches: 128 output rows x 256 buffer rows each
+        const int parts = j_pad > 128 ? 2 : 1;                            // launches: 128 output rows each
         cudaError_t e = timed(h, K_REBUILD, parts, st, [&] {
             return launch_tc_rebuild(h->Wsplit, h->wsplit_ld, j_pad, h->B[h->cur], h->B[1 - h->cur], h->pitch, h->D, r, keep, h->tc_err, st);
         });

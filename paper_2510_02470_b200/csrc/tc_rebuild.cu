@@ -8,7 +8,9 @@
 // fp32 fidelity as in the Gram kernel: the tensor cores read a buffer value as hi (its low 13 bits ignored),
 // the split warps write lo = x - hi into a second buffer; W arrives already split from global memory as two stacked operands [W_hi; W_lo],
 // so one MMA of width 2*j_pad gives hi*W_hi and hi*W_lo side by side and a second one adds lo*W_hi; the
-// epilogue adds the two halves. A tile accumulates at most 8 chunks (256 buffer rows) in TMEM.
+// epilogue adds the two halves. One TMEM accumulator takes at most 8 chunks (256 buffer rows); with more buffer rows
+// (up to 512) a tile uses both accumulators, one per half of the rows, and the epilogue adds them in registers (the
+// tiles then no longer alternate between the accumulators, so a tile's MMAs start after the previous tile's epilogue).
 //
 //   warp 0    TMA producer: per chunk 4 boxes of [32 rows][32 columns] of the buffer (128-byte swizzle with
 //             32-byte atoms, the only layout the tensor cores take for 32-bit MN-major operands) and one box of W,
@@ -32,7 +34,7 @@ constexpr int kSpanBytes = kChunkRows * 128;         // 4 KB
 
 __global__ void __launch_bounds__(kThreads, 1)
 k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ CUtensorMap tmW, int r, int keep, int j_pad,
-             long long pitch, long long num_tiles, float* __restrict__ out, int stages, int accumulate, int* __restrict__ err) {
+             long long pitch, long long num_tiles, float* __restrict__ out, int stages, int* __restrict__ err) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     // stage layout: [buffer hi 16 KB][buffer lo 16 KB][W_hi ; W_lo: 2*j_pad rows of 128 bytes]
@@ -49,6 +51,7 @@ k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nchunk = (r + kChunkRows - 1) / kChunkRows;
     const int n_mma = 2 * j_pad;                           // <= 256
+    const bool two = nchunk > 8;                           // both accumulators serve one tile
     uint32_t tmem_cols = 32;
     while (tmem_cols < (uint32_t)(2 * n_mma)) tmem_cols <<= 1;
     // tiles of this CTA: blockIdx.x, blockIdx.x + gridDim.x, ...
@@ -105,11 +108,13 @@ k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ 
             long long q = 0;
             bool alive = true;
             for (long long lt = 0; lt < my_tiles && alive; ++lt) {
-                const int b = (int)(lt & 1);
-                alive = mbar_wait(&acc_empty[b], (((uint32_t)(lt >> 1)) & 1u) ^ 1u, abort);
+                const int b = two ? 0 : (int)(lt & 1);
+                const uint32_t par = two ? (uint32_t)lt : (uint32_t)(lt >> 1);
+                alive = mbar_wait(&acc_empty[b], (par & 1u) ^ 1u, abort);
                 if (!alive) break;
-                const uint32_t acc = tmem_base + (uint32_t)(b * n_mma);
                 for (int c = 0; c < nchunk; ++c, ++q) {
+                    const uint32_t acc = tmem_base + (uint32_t)((two ? (c >> 3) : b) * n_mma);
+                    const int c_in = two ? (c & 7) : c;       // position within this accumulator's run
                     const int s = (int)(q % stages);
                     const uint32_t use = (uint32_t)(q / stages);
                     if (!mbar_wait(&split_done[s], use & 1u, abort)) { alive = false; break; }
@@ -121,7 +126,7 @@ k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ 
                     for (int k = 0; k < 4; ++k) {          // 8 buffer rows per MMA: one 1024-byte row group
                         const uint64_t d_hi = smem_desc_mn_sw128_atom32(st + k * 1024, kSpanBytes);
                         const uint64_t d_lo = smem_desc_mn_sw128_atom32(st + kBufBytes + k * 1024, kSpanBytes);
-                        mma_tf32(acc, d_hi, d_w + 2 * k, idesc_fold, (c | k) != 0);   // hi*W_hi | hi*W_lo
+                        mma_tf32(acc, d_hi, d_w + 2 * k, idesc_fold, (c_in | k) != 0);   // hi*W_hi | hi*W_lo
                         mma_tf32(acc, d_lo, d_w + 2 * k, idesc_half, 1);              // + lo*W_hi
                     }
                     mma_commit(&empty[s]);
@@ -158,8 +163,9 @@ k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ 
         const int quarter = warp & 3;
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
         for (long long lt = 0; lt < my_tiles; ++lt) {
-            const int b = (int)(lt & 1);
-            bool ok = mbar_wait(&acc_full[b], ((uint32_t)(lt >> 1)) & 1u, abort);
+            const int b = two ? 0 : (int)(lt & 1);
+            const uint32_t par = two ? (uint32_t)lt : (uint32_t)(lt >> 1);
+            bool ok = mbar_wait(&acc_full[b], par & 1u, abort);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
@@ -169,13 +175,19 @@ k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ 
                 float v[16], w[16];
                 tmem_ld16(acc + (uint32_t)j0, v);
                 tmem_ld16(acc + (uint32_t)(j_pad + j0), w);
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[j] += w[j];
+                if (two) {                                  // the second half of the buffer rows, from the other accumulator
+                    float v2[16];
+                    tmem_ld16(acc + (uint32_t)(n_mma + j0), v2);
+                    tmem_ld16(acc + (uint32_t)(n_mma + j_pad + j0), w);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) v[j] += v2[j] + w[j];
+                }
                 if (d < pitch) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
-                        if (j0 + j < keep) {
-                            float* o = out + (long long)(j0 + j) * pitch + d;
-                            *o = accumulate ? *o + (v[j] + w[j]) : v[j] + w[j];   // second half of the buffer rows adds to the first
-                        }
+                        if (j0 + j < keep) out[(long long)(j0 + j) * pitch + d] = v[j];
                 }
             }
             tc_fence_before();
@@ -185,7 +197,8 @@ k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ 
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
-        if (my_tiles > 0 && !*abort) mbar_wait_quiet(&acc_full[(my_tiles - 1) & 1], ((uint32_t)((my_tiles - 1) >> 1)) & 1u, kWaitLimitCycles);
+        if (my_tiles > 0 && !*abort)
+            mbar_wait_quiet(&acc_full[two ? 0 : (my_tiles - 1) & 1], (uint32_t)(two ? my_tiles - 1 : (my_tiles - 1) >> 1) & 1u, kWaitLimitCycles);
         tc_fence_after();
         tmem_dealloc(tmem_base, tmem_cols);
     }
@@ -197,9 +210,9 @@ k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ 
 
 // See sage_internal.h.
 static cudaError_t launch_tc_rebuild_part(const float* Wsplit, int ldw, int j_pad, const float* Bsrc, float* Bdst, int64_t pitch, int r,
-                                          int keep, int accumulate, int* err, cudaStream_t st) {
+                                          int keep, int* err, cudaStream_t st) {
     if (keep <= 0 || r <= 0) return cudaSuccess;
-    if (j_pad < 16 || j_pad > 128 || (j_pad & 15) || keep > j_pad || r > 256) return cudaErrorNotSupported;
+    if (j_pad < 16 || j_pad > 128 || (j_pad & 15) || keep > j_pad || r > 512) return cudaErrorNotSupported;
     CUtensorMap tmBuf, tmW;
     // buffer: columns beyond D up to the pitch are zero and are rebuilt as zero, so the map spans the pitch
     if (!tc::make_tmap_2d(&tmBuf, Bsrc, 4, (uint64_t)r, (uint64_t)pitch, (uint64_t)pitch, tc::kChunkRows, 1)) return cudaErrorNotSupported;
@@ -215,32 +228,25 @@ static cudaError_t launch_tc_rebuild_part(const float* Wsplit, int ldw, int j_pa
     const int grid = (int)(num_tiles < 148 ? num_tiles : 148);
     cudaError_t e = cudaFuncSetAttribute(tc::k_tc_rebuild, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    tc::k_tc_rebuild<<<grid, tc::kThreads, smem, st>>>(tmBuf, tmW, r, keep, j_pad, pitch, num_tiles, Bdst, stages, accumulate, err);
+    tc::k_tc_rebuild<<<grid, tc::kThreads, smem, st>>>(tmBuf, tmW, r, keep, j_pad, pitch, num_tiles, Bdst, stages, err);
     return cudaGetLastError();
 }
 
-// See sage_internal.h. One launch takes at most 128 output rows and 256 buffer rows (accumulator width and the number
-// of accumulations one TMEM accumulator should take); larger problems (ell = 256: 255 rows out of 512) run as up to
-// 2 x 2 launches, the second half of the buffer rows adding to what the first half stored.
+// See sage_internal.h. One launch takes at most 128 output rows (accumulator width) of up to 512 buffer rows; 129 to 256
+// output rows (ell = 256: 255 rows out of 512) run as two launches over the same buffer rows.
 cudaError_t launch_tc_rebuild(const float* Wsplit, int ldw, int j_pad, const float* Bsrc, float* Bdst, int64_t pitch, int64_t D, int r,
                               int keep, int* err, cudaStream_t st) {
     (void)D;
     if (keep <= 0 || r <= 0) return cudaSuccess;
     if (j_pad < 16 || j_pad > 256 || (j_pad & 15) || keep > j_pad || r > 512) return cudaErrorNotSupported;
-    if (((reinterpret_cast<uintptr_t>(Bsrc) | reinterpret_cast<uintptr_t>(Wsplit)) & 15u) || (pitch & 3) || (ldw & 3)) return cudaErrorNotSupported;
-    const int jparts = j_pad > 128 ? 2 : 1, rparts = r > 256 ? 2 : 1;
-    if (rparts == 2 && ldw < 512) return cudaErrorNotSupported;
+    const int jparts = j_pad > 128 ? 2 : 1;
     for (int jh = 0; jh < jparts; ++jh) {
         const int jp = jparts == 2 ? 128 : j_pad;
         const int keep_h = keep - jh * 128 < jp ? keep - jh * 128 : jp;
         if (keep_h <= 0) continue;
         const float* Wb = Wsplit + (size_t)(jparts == 2 ? jh * 256 : 0) * ldw;
-        for (int rh = 0; rh < rparts; ++rh) {
-            const int r_h = r - rh * 256 < 256 ? r - rh * 256 : 256;
-            cudaError_t e = launch_tc_rebuild_part(Wb + rh * 256, ldw, jp, Bsrc + (size_t)rh * 256 * pitch, Bdst + (size_t)jh * 128 * pitch, pitch,
-                                                   r_h, keep_h, rh > 0 ? 1 : 0, err, st);
-            if (e != cudaSuccess) return e;
-        }
+        cudaError_t e = launch_tc_rebuild_part(Wb, ldw, jp, Bsrc, Bdst + (size_t)jh * 128 * pitch, pitch, r, keep_h, err, st);
+        if (e != cudaSuccess) return e;
     }
     return cudaSuccess;
 }
