@@ -176,6 +176,7 @@ def main():
     args.warmup = max(args.warmup, 3)
 
     import paper_2510_02470_b200 as sage
+    from paper_2510_02470_b200 import replicas
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -292,12 +293,8 @@ def main():
     gen_per_step = gen_total_ms / args.steps
     stats = fd.stats()
 
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([step_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        step_ms = float(t.item())
-    value = world * N / (step_ms * 1e-3)
+    step_ms = replicas.max_over_ranks(step_ms, dev)            # replicas only: the job is as slow as its slowest rank
+    value = replicas.whole_job_rows_per_s(N, world, step_ms)
 
     # ---- roofline of the dominant kernel -------------------------------------------------------------------
     peaks = measured_peaks()
@@ -378,12 +375,8 @@ def main():
             sc, ix = sage.sage_select_from_host(host_rows, D, ell, w.keep_rates[0], 0, local)
         torch.cuda.synchronize()
         dt = (time.perf_counter() - t_e) / reps
-        if world > 1:
-            import torch.distributed as dist
-            t = torch.tensor([dt], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
-        e2e = {"value": world * N / dt, "unit": UNIT, "h2d_bytes_per_step": 2 * N * w.ld * e,
+        dt = replicas.max_over_ranks(dt, dev)
+        e2e = {"value": replicas.whole_job_rows_per_s(N, world, dt * 1e3), "unit": UNIT, "h2d_bytes_per_step": 2 * N * w.ld * e,
                "d2h_bytes_per_step": N * 4 + int(ix.numel()) * 8, "ms_per_step": dt * 1e3,
                "call": "sage_select_from_host (pinned host rows, both passes streamed over PCIe, one keep_rate)"}
     elif not args.no_e2e:
