@@ -1234,11 +1234,21 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
         if (active) {                                             // columns of block round 0 from the factor in L2
             int ba, bb;
             rr_blocks(slot, 0, nbm1, ba, bb);
-            for (int hc = 0; hc < 8; ++hc) {
-                const int p = 4 * (hc < 4 ? ba : bb) + (hc & 3);
-                const float* src = X + (size_t)perm[p < rank ? p : 0] * LD;
+            for (int hc = 0; hc < 8; hc += 2) {                  // two columns' loads in flight (each is an L2 round trip)
+                const int p0 = 4 * (hc < 4 ? ba : bb) + (hc & 3), p1 = p0 + 1;
+                const float* s0 = X + (size_t)perm[p0 < rank ? p0 : 0] * LD;
+                const float* s1 = X + (size_t)perm[p1 < rank ? p1 : 0] * LD;
+                float v0[R], v1[R];
 #pragma unroll
-                for (int t = 0; t < R; ++t) mybuf[hc * LD + lane + 32 * t] = (p < rank) ? __ldcg(src + lane + 32 * t) : 0.f;
+                for (int t = 0; t < R; ++t) {
+                    v0[t] = (p0 < rank) ? __ldcg(s0 + lane + 32 * t) : 0.f;
+                    v1[t] = (p1 < rank) ? __ldcg(s1 + lane + 32 * t) : 0.f;
+                }
+#pragma unroll
+                for (int t = 0; t < R; ++t) {
+                    mybuf[hc * LD + lane + 32 * t] = v0[t];
+                    mybuf[(hc + 1) * LD + lane + 32 * t] = v1[t];
+                }
             }
         }
         // The tournament repeats every sweep: block pair and destinations of every block round, packed into one word
@@ -1391,16 +1401,25 @@ k_eig_shrink_dsm(const float* __restrict__ K, int ldk, int n, int do_shrink, int
     if (more == 2 && gtid == 0) atomicOr(&info->flags, kFlagExchangeTimeout);
     const int not_converged = rank >= 2 && more != 0;          // stopped at the sweep limit while still rotating visibly
     // ---- eigenvalues = squared column norms (pivot-step order), scaled back; sort descending, stable ----
-    for (int k = lwarp; k < n; k += WPC) {                          // every CTA forms all eigenvalues for its own tables
-        float a = 0.f;
-        if (k < rank) {
-            const float* x = X + perm[k] * LD;
+    for (int k0 = lwarp; k0 < n; k0 += 4 * WPC) {                  // every CTA forms all eigenvalues for its own tables;
+        float a[4] = {0.f, 0.f, 0.f, 0.f};                          // four columns' loads in flight (each is an L2 round trip)
+        float xv[4][R];
 #pragma unroll
-            for (int t = 0; t < R; ++t) { const float xv = __ldcg(x + lane + 32 * t); a = fmaf(xv, xv, a); }
+        for (int u = 0; u < 4; ++u) {
+            const int k = k0 + u * WPC;
+            const float* x = X + perm[k < rank ? k : 0] * LD;
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+            for (int t = 0; t < R; ++t) xv[u][t] = (k < rank) ? __ldcg(x + lane + 32 * t) : 0.f;
         }
-        if (lane == 0) lam[k] = a * dmax;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+#pragma unroll
+            for (int t = 0; t < R; ++t) a[u] = fmaf(xv[u][t], xv[u][t], a[u]);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) a[u] += __shfl_xor_sync(0xffffffffu, a[u], o);
+            const int k = k0 + u * WPC;
+            if (lane == 0 && k < n) lam[k] = a[u] * dmax;
+        }
     }
     __syncthreads();
     for (int t = tid; t < n; t += NT) {
