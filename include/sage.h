@@ -56,7 +56,7 @@ typedef enum { SAGE_F32 = 0, SAGE_BF16 = 1 } sage_dtype_t;
  */
 
 /* Frequent-Directions sketch state for rows of dimension D with sketch size ell (Method, first
- * paragraph; Algorithm 1 line "Initialize S"). The library keeps a buffer of 2*ell rows in fp32: rows
+ * paragraph; Algorithm 1, the initialisation step). The library keeps a buffer of 2*ell rows in fp32: rows
  * are appended into free rows and the buffer is shrunk when all 2*ell rows are in use.
  *   out        receives the handle (host pointer).
  *   D          row dimension, 1 <= D.
@@ -81,6 +81,13 @@ sage_status_t sage_fd_reset(sage_fd_t* h);
  * Asynchronous on the stream: the shrink schedule depends only on counts, so no device->host
  * synchronisation happens here. Device-side problems are reported by sage_fd_finalize. */
 sage_status_t sage_fd_update(sage_fd_t* h, const void* rows, int64_t n, int64_t ld, void* cuda_stream);
+
+/* Makes cuda_stream wait (on the device, without blocking the host) for everything this handle has enqueued on streams
+ * of its own: the merged form of pass 1 (option 6) runs its sketches on internal streams, and sage_fd_update only makes
+ * the caller's stream wait until the rows have been copied out of `rows`. sage_fd_finalize joins by itself; this call
+ * is for callers that want the handle's work ordered before other work of theirs (a benchmark that times what it
+ * enqueues next). The paper has no counterpart. */
+sage_status_t sage_fd_join(sage_fd_t* h, void* cuda_stream);
 
 /* Algorithm 1, the freeze step: orthogonalise what the buffer holds, apply the shrink only if
  * more than ell rows are in use (so N <= ell is exact), keep the first ell rows as S.
@@ -107,7 +114,11 @@ sage_status_t sage_score(sage_fd_t* h, const void* rows, int64_t n, int64_t ld, 
  * chunks (each read once), then finish. row_offset is the index of the chunk's first row in
  * [0, N_total); chunks must tile [0, N_total) without overlap and be given in ascending order.
  * The library keeps the N_total x ell normalised projections between chunk and end, because the
- * consensus direction is only known once every row has been seen. */
+ * consensus direction is only known once every row has been seen.
+ * sage_score / sage_score_end return as soon as the work is enqueued, so they cannot report what the device meets
+ * while it runs: after synchronising the stream, sage_fd_stats().device_flags tells whether a row was non-finite
+ * (bit 1; such rows score 0) or a kernel gave up a bounded wait (bits 2, 3; scores invalid). The synchronous
+ * sage_select_from_host checks those words itself and returns SAGE_ERR_NONFINITE / SAGE_ERR_CUDA. */
 sage_status_t sage_score_begin(sage_fd_t* h, int64_t N_total, void* cuda_stream);
 sage_status_t sage_score_chunk(sage_fd_t* h, const void* rows, int64_t n, int64_t ld, int64_t row_offset,
                                void* cuda_stream);
@@ -129,7 +140,7 @@ int64_t sage_select_count(int64_t N, double keep_rate);
 sage_status_t sage_select(const float* scores, int64_t N, double keep_rate, int64_t* idx, int64_t* k_out,
                           void* cuda_stream);
 
-/* Class-balanced variant (Algorithm 1, branch "class balance required"; "Agreement Scoring and Selection"): after a
+/* Class-balanced variant (Algorithm 1, the class-balanced branch; section on agreement scoring and selection): after a
  * finished scoring pass on this handle (sage_score or sage_score_end over N rows), replace the consensus u by the
  * per-class unit centroids u_c = zbar_c / ||zbar_c||, zbar_c the mean of zhat_i over the examples of class c (u_c = 0
  * when that mean is zero), and score every example against the centroid of its own class.
@@ -190,6 +201,7 @@ typedef struct {
                                bit 2: a tensor-core kernel gave up a bounded wait (results invalid),
                                bit 3: the cluster eigen-solve gave up a bounded wait (results invalid) */
     int64_t kernel_launches;/* kernels this handle has launched since create/reset */
+    int64_t tensor_core_launches; /* how many of them were tensor-core (tcgen05) kernels: Gram, rebuild, projection */
 } sage_stats_t;
 
 /* Synchronises the device and reads the counters back. */
@@ -202,7 +214,15 @@ sage_status_t sage_fd_stats(sage_fd_t* h, sage_stats_t* out);
  * aligned base, row pitch a multiple of 16 bytes), 0 to use the CUDA-core kernels everywhere; key 5 = which
  * kernels run the eigen-solve: 0 (default) a cluster of 8 thread blocks with the Jacobi columns in distributed
  * shared memory, 1 the single-block kernel (buffers of up to 192 rows) or the cluster kernel that keeps the
- * matrix in L2. Same algorithm either way; results agree up to rounding order. */
+ * matrix in L2. Same algorithm either way; results agree up to rounding order.
+ * Before the first update: key 6 = P, the number of sketches of the merged form of pass 1 (1 .. 64, default 1 = the
+ * paper's single sequential sketch); key 7 = rows per dealt block (default ell + 1). With P > 1 the row stream is cut into
+ * blocks of that many consecutive rows, block b (counted from the first row ever given, across calls) goes to sketch
+ * b mod P, and each sketch is a sequential Frequent-Directions sketch of its rows in stream order; sage_fd_finalize
+ * freezes every sketch and merges them pairwise (sketch a absorbs sketch a + s for s = 1, 2, 4, ...: the rows a + s
+ * kept are appended to a, which is frozen again). Frequent-Directions sketches are mergeable, so the result obeys
+ * the same error bound as the sequential sketch, but it is a different sketch. The P chains of Gram / eigen-solve /
+ * rebuild run on P streams of the library's own and overlap on the device; device memory grows P-fold. */
 sage_status_t sage_fd_set_option(sage_fd_t* h, int key, double value);
 
 /* Per-kernel device time of this handle's launches since the previous call, for the classes selected

@@ -146,9 +146,79 @@ def jacobi_eig(K: np.ndarray) -> Tuple[np.ndarray, np.ndarray, int]:
     return U, lam, sweeps
 
 
-def run(rows, D: int, ell: int, keep_rate: float, route: int = 0) -> dict:
-    """Whole path on resident rows: sketch -> finalize -> score -> select."""
-    fd = OracleFD(D, ell, route=route)
+class OracleMergedFD:
+    """P Frequent-Directions sketches over interleaved row blocks, merged pairwise at the freeze.
+
+    The paper's sketch is one sequential stream (Method section, first paragraph). Frequent-Directions sketches are
+    mergeable (a property of the works the paper cites for it): the sketch of the stacked rows of two sketches obeys
+    the same guarantee as a sketch of all the rows behind them. This class states the merged form the CUDA library
+    offers as an option, in terms of the sequential sketch above and nothing else:
+
+    * rows are dealt in blocks of ``block`` consecutive rows (default ell + 1, the number of rows between two
+      shrinks of one buffer): block b of the stream, counted from 0 over everything given to ``update``, goes to
+      sketch b mod P, and every sketch sees its rows in stream order;
+    * at the freeze every sketch is frozen on its own (orthogonalise, shrink only if more than ell rows are in use),
+      which leaves c_p <= ell non-trivial rows; then, for stride s = 1, 2, 4, ...: sketch a (a = 0, 2s, 4s, ...)
+      absorbs sketch a + s, if there is one: a fresh sequential sketch is fed the c_a rows of a, then the c_{a+s} rows
+      of a + s, and is frozen. Sketch 0 is the result.
+
+    With P = 1 nothing is dealt or merged: the result is the sequential sketch, bit for bit."""
+
+    def __init__(self, D: int, ell: int, sketches: int, block: Optional[int] = None, route: int = 0):
+        assert sketches >= 1
+        self.D, self.ell, self.P, self.route = int(D), int(ell), int(sketches), route
+        self.block = int(block) if block else self.ell + 1
+        self.subs = [OracleFD(D, ell, route=route) for _ in range(self.P)]
+        self.seen = 0
+        self.merge_stats = {"shrinks": 0, "sum_delta": 0.0}
+        self.frozen = None          # per sketch: (S, kept rows) as frozen before any merge
+
+    def update(self, rows) -> None:
+        kind, arr, n, ld = _rows_view(rows)
+        i = 0
+        while i < n:
+            b = self.seen // self.block
+            take = min(n - i, (b + 1) * self.block - self.seen)
+            self.subs[b % self.P].update(arr[i:i + take])
+            i += take
+            self.seen += take
+
+    @staticmethod
+    def _freeze(fd: OracleFD):
+        S, sigma = fd.finalize()
+        _, kept = fd.buffer()
+        return S, sigma, min(kept, fd.ell)
+
+    def finalize(self) -> Tuple[np.ndarray, np.ndarray]:
+        frozen = [self._freeze(fd) for fd in self.subs]
+        self.frozen = [(S.copy(), c) for S, _, c in frozen]
+        s = 1
+        while s < self.P:
+            for a in range(0, self.P, 2 * s):
+                b = a + s
+                if b >= self.P:
+                    continue
+                (Sa, _, ca), (Sb, _, cb) = frozen[a], frozen[b]
+                m = OracleFD(self.D, self.ell, route=self.route)
+                m.update(Sa[:ca])
+                m.update(Sb[:cb])
+                frozen[a] = self._freeze(m)
+                st = m.stats()
+                self.merge_stats["shrinks"] += st["shrinks"]
+                self.merge_stats["sum_delta"] += st["sum_delta"]
+            s *= 2
+        return frozen[0][0], frozen[0][1]
+
+    def stats(self) -> dict:
+        per = [fd.stats() for fd in self.subs]
+        return {"rows_seen": self.seen, "shrinks": sum(p["shrinks"] for p in per) + self.merge_stats["shrinks"],
+                "sum_delta": sum(p["sum_delta"] for p in per) + self.merge_stats["sum_delta"],
+                "last_sweeps": per[0]["last_sweeps"], "rows_per_sketch": [p["rows_seen"] for p in per]}
+
+
+def run(rows, D: int, ell: int, keep_rate: float, route: int = 0, sketches: int = 1, block: Optional[int] = None) -> dict:
+    """Whole path on resident rows: sketch -> finalize -> score -> select. sketches > 1: the merged form of pass 1."""
+    fd = OracleFD(D, ell, route=route) if sketches == 1 else OracleMergedFD(D, ell, sketches, block, route)
     fd.update(rows)
     S, sigma = fd.finalize()
     out = score(S, rows)

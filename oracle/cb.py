@@ -2,8 +2,8 @@
 
 TEST INFRASTRUCTURE ONLY, like the rest of this package: nothing on the product path imports it.
 
-What it follows: Algorithm 1, branch "class balance required", and the paragraph "Agreement Scoring and
-Selection": for each class c the mean of the normalised projections zhat_i over the class, its unit vector u_c (zero
+What it follows: Algorithm 1, the class-balanced branch, and the section on agreement scoring and
+selection: for each class c the mean of the normalised projections zhat_i over the class, its unit vector u_c (zero
 if the mean is zero), the score <zhat_i, u_c> of every example of the class, and the top-k_c examples per class
 with sum_c k_c = k.
 

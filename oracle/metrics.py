@@ -10,7 +10,7 @@ from __future__ import annotations
 import numpy as np
 
 
-def _signed_gram_eigs(P: np.ndarray, Q: np.ndarray) -> np.ndarray:
+def _signed_gram_eigs(P: np.ndarray, Q: np.ndarray, method: str = "auto") -> np.ndarray:
     """Eigenvalues of P^T P - Q^T Q on its range, from a (p+q) x (p+q) symmetric problem.
 
     With C = [P; Q] and J = diag(I_p, -I_q), P^T P - Q^T Q = C^T J C. If C^T = Y R (thin QR, Y with
@@ -21,7 +21,8 @@ def _signed_gram_eigs(P: np.ndarray, Q: np.ndarray) -> np.ndarray:
     Q = np.asarray(Q, dtype=np.float64)
     Cm = np.concatenate([P, Q], axis=0)
     J = np.concatenate([np.ones(P.shape[0]), -np.ones(Q.shape[0])])
-    if Cm.shape[0] <= Cm.shape[1] and Cm.size <= 2e8:
+    assert method in ("auto", "qr", "sqrt")
+    if method == "qr" or (method == "auto" and Cm.shape[0] <= Cm.shape[1] and Cm.size <= 2e8):
         R = np.linalg.qr(Cm.T, mode="r")
         M = (R * J[None, :]) @ R.T
     else:
@@ -32,9 +33,10 @@ def _signed_gram_eigs(P: np.ndarray, Q: np.ndarray) -> np.ndarray:
     return np.linalg.eigvalsh(0.5 * (M + M.T))
 
 
-def signed_gram_norm(P: np.ndarray, Q: np.ndarray) -> float:
-    """|| P^T P - Q^T Q ||_2 for P (p x D), Q (q x D) without forming a D x D matrix."""
-    ev = _signed_gram_eigs(P, Q)
+def signed_gram_norm(P: np.ndarray, Q: np.ndarray, method: str = "auto") -> float:
+    """|| P^T P - Q^T Q ||_2 for P (p x D), Q (q x D) without forming a D x D matrix. method: "qr", "sqrt" (the
+    W^(1/2) J W^(1/2) form) or "auto" (QR unless the stacked operand is very large)."""
+    ev = _signed_gram_eigs(P, Q, method)
     return float(np.max(np.abs(ev))) if ev.size else 0.0
 
 

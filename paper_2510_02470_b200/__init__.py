@@ -30,6 +30,7 @@ SIGNATURES = {
     "sage_fd_reset": (_i32, [_vp]),
     "sage_fd_update": (_i32, [_vp, _vp, _i64, _i64, _vp]),
     "sage_fd_finalize": (_i32, [_vp, _vp]),
+    "sage_fd_join": (_i32, [_vp, _vp]),
     "sage_fd_sketch": (_i32, [_vp, _vp, _vp, _vp]),
     "sage_fd_load_sketch": (_i32, [_vp, _vp, _i64, _vp]),
     "sage_score": (_i32, [_vp, _vp, _i64, _i64, _vp, _vp]),
@@ -56,7 +57,8 @@ SIGNATURES = {
 
 class SageStats(C.Structure):
     _fields_ = [("rows_seen", _i64), ("shrinks", _i64), ("sum_delta", _f64), ("last_sweeps", _i32),
-                ("max_sweeps", _i32), ("last_rank", _i32), ("device_flags", _u32), ("kernel_launches", _i64)]
+                ("max_sweeps", _i32), ("last_rank", _i32), ("device_flags", _u32), ("kernel_launches", _i64),
+                ("tensor_core_launches", _i64)]
 
 
 class SageError(RuntimeError):
@@ -132,6 +134,10 @@ def sage_fd_update(h: int, rows: torch.Tensor, D: int) -> None:
 
 def sage_fd_finalize(h: int, device=None, allow=()) -> int:
     return _check(lib().sage_fd_finalize(h, _stream(device)), allow)
+
+
+def sage_fd_join(h: int, device=None) -> None:
+    _check(lib().sage_fd_join(h, _stream(device)))
 
 
 def sage_fd_sketch(h: int, ell: int, D: int, device) -> Tuple[torch.Tensor, torch.Tensor]:
@@ -236,7 +242,7 @@ def sage_select_static(scores: torch.Tensor, keep_rate: float, idx: torch.Tensor
 
 
 def sage_select_from_host(rows: torch.Tensor, D: int, ell: int, keep_rate: float, chunk_rows: int = 0,
-                          device: int = 0, want_scores: bool = True):
+                          device: int = 0, want_scores: bool = True, allow=(6, 7)):
     """Whole path on HOST rows (pinned memory recommended). Returns (scores or None, idx) on the host."""
     assert rows.device.type == "cpu"
     ptr, N, ld = _rows_args(rows, D)
@@ -246,7 +252,7 @@ def sage_select_from_host(rows: torch.Tensor, D: int, ell: int, keep_rate: float
     k_out = _i64(0)
     st = lib().sage_select_from_host(ptr, N, D, ld, ell, _dtype_code(rows), keep_rate, chunk_rows, device,
                                      scores.data_ptr() if want_scores else None, idx.data_ptr(), C.byref(k_out))
-    _check(st, allow=(6, 7))
+    _check(st, allow=allow)
     return scores, idx[: k_out.value]
 
 
@@ -301,6 +307,9 @@ class SageFD:
 
     def finalize(self, allow=()) -> int:
         return sage_fd_finalize(self._h, self.device, allow)
+
+    def join(self) -> None:
+        sage_fd_join(self._h, self.device)
 
     def sketch(self):
         return sage_fd_sketch(self._h, self.ell, self.D, torch.device("cuda", self.device))

@@ -66,6 +66,23 @@ struct Prof {
     std::vector<Pending> pending;
     double ms[K_NCLASS] = {};
     int64_t n[K_NCLASS] = {};
+    // Adds the pairs whose second event has completed to the sums and recycles their events.
+    void fold_finished() {
+        size_t keep = 0;
+        for (size_t i = 0; i < pending.size(); ++i) {
+            Pending& p = pending[i];
+            float t = 0.f;
+            if (cudaEventQuery(p.b) == cudaSuccess && cudaEventElapsedTime(&t, p.a, p.b) == cudaSuccess) {
+                ms[p.cls] += t;
+                n[p.cls] += 1;
+                pool.push_back(p.a);
+                pool.push_back(p.b);
+            } else {
+                pending[keep++] = p;
+            }
+        }
+        pending.resize(keep);
+    }
     cudaEvent_t get() {
         if (!pool.empty()) { cudaEvent_t e = pool.back(); pool.pop_back(); return e; }
         cudaEvent_t e = nullptr;
@@ -154,7 +171,23 @@ struct sage_fd {
     bool use_tc = true;            // option 4: tensor-core kernels where their alignment rules hold
     int eig_variant = 0;           // option 5: 0 cluster eigen-solve in distributed shared memory, 1 the one-CTA / L2 kernels
     int64_t launches = 0;
+    int64_t tc_launches = 0;       // how many of them were tensor-core (tcgen05) kernels
     Prof prof;
+    // Merged form of pass 1 (option 6): P sketches over interleaved row blocks. This handle is sketch 0; sketches
+    // 1..P-1 are handles of their own that only sketch (no scoring state). With P > 1 every sketch runs its
+    // Gram / eigen-solve / rebuild chain on a stream of its own, so the chains of different sketches overlap.
+    int P = 1;
+    int64_t block = 0;             // rows per dealt block
+    int64_t dealt = 0;             // rows dealt so far (all sketches)
+    std::vector<sage_fd*> kids;
+    bool sketch_only = false;      // a sub-sketch: no scoring buffers
+    cudaStream_t chain = nullptr;  // P > 1: the stream of this sketch's chain (P == 1: the caller's stream)
+    bool app_pending = false;      // appends on `side` that the chain stream has not been made to wait for yet
+    int64_t in_epoch = -1;         // the update call whose entry event `side` already waits for
+    cudaEvent_t ev_in = nullptr;   // the caller's stream at the entry of an update call (sketch 0 only)
+    cudaEvent_t ev_rows = nullptr; // after the last append of the current update call
+    cudaEvent_t ev_done = nullptr; // end of the chain stream (joins)
+    bool used = false;             // fed during the current update call
 };
 
 namespace {
@@ -178,6 +211,7 @@ cudaError_t timed(sage_fd* h, int cls, int nlaunch, cudaStream_t st, F&& f) {
     if (on) {
         cudaEventRecord(b, st);
         h->prof.pending.push_back({cls, a, b});
+        if (h->prof.pending.size() >= 65536) h->prof.fold_finished();   // never grows without bound if nobody asks for the profile
     }
     count(h, nlaunch);
     return e;
@@ -234,7 +268,7 @@ sage_status_t enqueue_gram(sage_fd* h, int r, cudaStream_t st) {
         const int t = (r + 127) / 128;
         const int ldc = ((r + 3) / 4) * 4;
         const int64_t stride = (int64_t)r * ldc;
-        const int sym = r <= 128 ? 1 : 0;    // one diagonal tile: two MMAs per K step, transpose added in the reduction
+        const int sym = r <= 128 ? 1 : 0;    // one diagonal tile: one wide MMA per K step, transpose added in the reduction
         int cap = (int)(h->gram_part_floats / (size_t)stride);
         if (cap > 148) cap = 148;
         const int splits = pick_splits_waves(t * (t + 1) / 2, h->D, 256, cap);   // only the tiles on and above the diagonal run
@@ -242,6 +276,7 @@ sage_status_t enqueue_gram(sage_fd* h, int r, cudaStream_t st) {
             return launch_tc_gemm_nt_x3(Bc, h->pitch, Bc, h->pitch, r, r, h->D, splits, h->gram_parts, ldc, stride, sym, h->tc_err, st);
         });
         if (e == cudaSuccess) {
+            h->tc_launches += 1;
             if (sym)
                 CU_TRY(timed(h, K_GRAM_REDUCE, 1, st, [&] { return launch_gram_sym_reduce(h->gram_parts, splits, stride, r, ldc, h->Kmat, h->m, st); }));
             else   // sums the K slices and fills the tiles below the diagonal from their mirror images
@@ -286,12 +321,13 @@ sage_status_t enqueue_factor(sage_fd* h, int r, int do_shrink, int keep, int zer
         });
         if (e == cudaSuccess) {
             done = true;
+            h->tc_launches += parts;
             if (m_total > keep)
                 CU_TRY(cudaMemsetAsync(h->B[1 - h->cur] + (size_t)keep * h->pitch, 0, (size_t)(m_total - keep) * h->pitch * sizeof(float), st));
         } else if (e != cudaErrorNotSupported) {
             CU_TRY(e);
         } else {
-            count(h, -1);
+            count(h, -parts);
         }
     }
     if (!done)
@@ -356,7 +392,7 @@ int64_t sage_select_count(int64_t N, double keep_rate) {
     return (int64_t)k;
 }
 
-sage_status_t sage_fd_create(sage_fd_t** out, int64_t D, int32_t ell, sage_dtype_t row_dtype, int device) {
+static sage_status_t create_handle(sage_fd_t** out, int64_t D, int32_t ell, sage_dtype_t row_dtype, int device, bool sketch_only) {
     if (!out || D < 1 || (row_dtype != SAGE_F32 && row_dtype != SAGE_BF16) || device < 0) {
         set_err("sage_fd_create: bad argument (out=%p D=%lld dtype=%d device=%d)", (void*)out, (long long)D, (int)row_dtype, device);
         return SAGE_ERR_INVALID_ARG;
@@ -378,6 +414,8 @@ sage_status_t sage_fd_create(sage_fd_t** out, int64_t D, int32_t ell, sage_dtype
     h->dtype = row_dtype;
     h->device = device;
     h->delta_rank = ell;
+    h->sketch_only = sketch_only;
+    h->block = ell + 1;
     h->pitch = ((D + 31) / 32) * 32;
     const size_t bbytes = (size_t)h->m * h->pitch * sizeof(float);
     const size_t mm = (size_t)h->m * h->m * sizeof(float);
@@ -395,6 +433,9 @@ sage_status_t sage_fd_create(sage_fd_t** out, int64_t D, int32_t ell, sage_dtype
     h->wsplit_ld = h->m <= 256 ? 256 : 512;
     if ((e = cudaMalloc((void**)&h->Wsplit, (size_t)h->wsplit_ld * h->wsplit_ld * sizeof(float))) != cudaSuccess)
         return fail(e, "cudaMalloc(W)");
+    // rows of the split factors beyond the ones an eigen-solve writes are read by the rebuild's MMA (and ignored by its
+    // epilogue): they must hold finite values
+    if ((e = cudaMemset(h->Wsplit, 0, (size_t)h->wsplit_ld * h->wsplit_ld * sizeof(float))) != cudaSuccess) return fail(e, "cudaMemset");
     if ((e = cudaMalloc((void**)&h->Kmat, mm)) != cudaSuccess) return fail(e, "cudaMalloc(K)");
     if ((e = cudaMalloc((void**)&h->Ur, mm)) != cudaSuccess) return fail(e, "cudaMalloc(U)");
     // eigen workspace: the matrix padded to 256 or 512 rows/columns plus a few flag words
@@ -403,14 +444,16 @@ sage_status_t sage_fd_create(sage_fd_t** out, int64_t D, int32_t ell, sage_dtype
         return fail(e, "cudaMalloc(eig)");
     if ((e = cudaMalloc((void**)&h->sigma, ell * sizeof(float))) != cudaSuccess) return fail(e, "cudaMalloc(sigma)");
     if ((e = cudaMalloc((void**)&h->info, sizeof(EigInfo))) != cudaSuccess) return fail(e, "cudaMalloc(info)");
-    if ((e = cudaMalloc((void**)&h->zsum, 256 * sizeof(double))) != cudaSuccess) return fail(e, "cudaMalloc(zsum)");
-    if ((e = cudaMalloc((void**)&h->u, 256 * sizeof(float))) != cudaSuccess) return fail(e, "cudaMalloc(u)");
+    if (!sketch_only) {
+        if ((e = cudaMalloc((void**)&h->zsum, 256 * sizeof(double))) != cudaSuccess) return fail(e, "cudaMalloc(zsum)");
+        if ((e = cudaMalloc((void**)&h->u, 256 * sizeof(float))) != cudaSuccess) return fail(e, "cudaMalloc(u)");
+    }
     if ((e = cudaMalloc((void**)&h->tc_err, sizeof(int))) != cudaSuccess) return fail(e, "cudaMalloc(err)");
     if ((e = cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking)) != cudaSuccess) return fail(e, "cudaStreamCreate");
-    if ((e = cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
-    if ((e = cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
+    for (cudaEvent_t* ev : {&h->ev_fork, &h->ev_join, &h->ev_in, &h->ev_rows, &h->ev_done})
+        if ((e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
     if ((e = cudaMemset(h->tc_err, 0, sizeof(int))) != cudaSuccess) return fail(e, "cudaMemset");
-    if (row_dtype == SAGE_BF16) {
+    if (row_dtype == SAGE_BF16 && !sketch_only) {
         // Two-term bf16 sketch (16 significant bits) for short rows, where the rounding errors of a one-term
         // sketch would average over too few terms; long rows take the one-term sketch (half the operand traffic).
         h->p16_npad = ((ell + 15) / 16) * 16;
@@ -419,7 +462,7 @@ sage_status_t sage_fd_create(sage_fd_t** out, int64_t D, int32_t ell, sage_dtype
         if ((e = cudaMalloc((void**)&h->P16, prow * h->pitch * sizeof(__nv_bfloat16))) != cudaSuccess) return fail(e, "cudaMalloc(P16)");
         if ((e = cudaMemset(h->P16, 0, prow * h->pitch * sizeof(__nv_bfloat16))) != cudaSuccess) return fail(e, "cudaMemset");
     }
-    if (row_dtype == SAGE_F32 && ell <= 64) {
+    if (row_dtype == SAGE_F32 && ell <= 64 && !sketch_only) {
         // fp32 rows, small sketch: the projection multiplies the rows against the sketch pre-split into tf32 hi / lo rows
         if ((e = cudaMalloc((void**)&h->S32split, (size_t)128 * h->pitch * sizeof(float))) != cudaSuccess) return fail(e, "cudaMalloc(S split)");
         if ((e = cudaMemset(h->S32split, 0, (size_t)128 * h->pitch * sizeof(float))) != cudaSuccess) return fail(e, "cudaMemset");
@@ -431,10 +474,19 @@ sage_status_t sage_fd_create(sage_fd_t** out, int64_t D, int32_t ell, sage_dtype
     return SAGE_OK;
 }
 
+sage_status_t sage_fd_create(sage_fd_t** out, int64_t D, int32_t ell, sage_dtype_t row_dtype, int device) {
+    return create_handle(out, D, ell, row_dtype, device, false);
+}
+
 void sage_fd_destroy(sage_fd_t* h) {
     if (!h) return;
     DeviceGuard g(h->device);
     cudaDeviceSynchronize();
+    for (sage_fd* k : h->kids) sage_fd_destroy(k);
+    h->kids.clear();
+    if (h->chain) cudaStreamDestroy(h->chain);
+    for (cudaEvent_t ev : {h->ev_in, h->ev_rows, h->ev_done})
+        if (ev) cudaEventDestroy(ev);
     cudaFree(h->B[0]);
     cudaFree(h->B[1]);
     cudaFree(h->gram_parts);
@@ -475,10 +527,15 @@ sage_status_t sage_fd_reset(sage_fd_t* h) {
     CU_TRY(cudaMemset(h->tc_err, 0, sizeof(int)));
     h->fill = 0;
     h->rows_seen = 0;
+    h->dealt = 0;
     h->cur = 0;
     h->scored = false;
     h->state = SKETCHING;
     h->launches = 0;
+    h->tc_launches = 0;
+    h->app_pending = false;
+    h->in_epoch = -1;
+    for (sage_fd* k : h->kids) ST_TRY(sage_fd_reset(k));
     return SAGE_OK;
 }
 
@@ -486,31 +543,155 @@ sage_status_t sage_fd_set_option(sage_fd_t* h, int key, double value) {
     ST_TRY(check_handle(h));
     if (key == 3) {                          // per-kernel event timing mask: allowed at any time
         h->prof.mask = (unsigned)value & ((1u << K_NCLASS) - 1u);
+        for (sage_fd* k : h->kids) k->prof.mask = h->prof.mask;
         return SAGE_OK;
     }
     if (key == 4) {                          // 0: CUDA-core kernels only, 1: tensor-core kernels where possible
         h->use_tc = value != 0.0;
+        for (sage_fd* k : h->kids) k->use_tc = h->use_tc;
         return SAGE_OK;
     }
     if (key == 5) {                          // eigen-solve kernel family (same algorithm, same results up to rounding order)
         h->eig_variant = value != 0.0 ? 1 : 0;
+        for (sage_fd* k : h->kids) k->eig_variant = h->eig_variant;
         return SAGE_OK;
     }
-    if (h->rows_seen != 0 || h->state != SKETCHING) {
+    if (h->dealt != 0 || h->state != SKETCHING) {
         set_err("sage_fd_set_option: options must be set before the first update");
         return SAGE_ERR_BAD_STATE;
     }
     const int v = (int)value;
     if (key == 1 && v >= 2 && v <= h->m - 1) {
         h->delta_rank = v;
+        for (sage_fd* k : h->kids) k->delta_rank = v;
         return SAGE_OK;
     }
     if (key == 2 && v >= 1 && v <= 1000) {
         h->max_sweeps = v;
+        for (sage_fd* k : h->kids) k->max_sweeps = v;
+        return SAGE_OK;
+    }
+    if (key == 6 && v >= 1 && v <= 64 && (double)v == value) {      // number of sketches of the merged form of pass 1
+        if (v != h->P) {
+            DeviceGuard g(h->device);
+            cudaDeviceSynchronize();
+            for (sage_fd* k : h->kids) sage_fd_destroy(k);
+            h->kids.clear();
+            if (v == 1 && h->chain) {
+                cudaStreamDestroy(h->chain);
+                h->chain = nullptr;
+            }
+        }
+        h->P = v;
+        return SAGE_OK;
+    }
+    if (key == 7 && v >= 1 && v <= (1 << 20) && (double)v == value) { // rows per dealt block of the merged form
+        h->block = v;
         return SAGE_OK;
     }
     set_err("sage_fd_set_option: unknown key %d or value %g out of range", key, value);
     return SAGE_ERR_INVALID_ARG;
+}
+
+// ---- one sketch: feed rows, factor, freeze ------------------------------------------------------------------
+//
+// Streams of a sketch: every append runs on its `side` stream, the Gram / eigen-solve / rebuild chain on `chain` (the
+// caller's stream for a single sketch, the sketch's own stream in the merged form). An append writes rows
+// [fill, fill + take) of the current buffer copy and touches nothing the eigen-solve or the rebuild of the previous
+// shrink reads or writes (the rebuild fills rows [0, keep) of the same copy), so appends run beside the eigen-solve,
+// which leaves HBM idle. The side stream starts after the Gram kernel of the previous shrink (running beside it only
+// takes bandwidth from it; that also puts it after the rebuild before, which read the copy now being filled) and
+// the chain waits for the appends before the next Gram kernel.
+
+static sage_status_t sketch_join_appends(sage_fd* s, cudaStream_t chain) {
+    if (s->app_pending) {
+        CU_TRY(cudaEventRecord(s->ev_join, s->side));
+        CU_TRY(cudaStreamWaitEvent(chain, s->ev_join, 0));
+        s->app_pending = false;
+    }
+    return SAGE_OK;
+}
+
+static sage_status_t sketch_factor(sage_fd* s, int r, int do_shrink, int keep, int zero_to, cudaStream_t chain) {
+    ST_TRY(sketch_join_appends(s, chain));
+    ST_TRY(enqueue_factor(s, r, do_shrink, keep, zero_to, chain));
+    CU_TRY(cudaStreamWaitEvent(s->side, s->ev_fork, 0));
+    return SAGE_OK;
+}
+
+// Appends n rows of type dt and shrinks whenever the buffer fills. e_in (may be null): the event after which `rows`
+// are valid; epoch identifies the update call it belongs to. on_chain: appends run on the chain stream itself (used
+// where the rows to append are produced by that stream). Leaves s->ev_rows recorded after the last append.
+static sage_status_t sketch_feed(sage_fd* s, const void* rows, sage_dtype_t dt, int64_t n, int64_t ld, cudaStream_t chain,
+                                 cudaEvent_t e_in, int64_t epoch, bool on_chain) {
+    cudaStream_t as = on_chain ? chain : s->side;
+    if (!on_chain && e_in && s->in_epoch != epoch) {
+        CU_TRY(cudaStreamWaitEvent(as, e_in, 0));
+        s->in_epoch = epoch;
+    }
+    const char* p = static_cast<const char*>(rows);
+    const size_t row_bytes = (size_t)ld * elem_size(dt);
+    bool appended = false;
+    auto body = [&]() -> sage_status_t {
+        while (n > 0) {
+            const int64_t room = s->m - s->fill;
+            const int64_t take = n < room ? n : room;
+            CU_TRY(timed(s, K_APPEND, 1, as, [&] { return launch_append(p, dt, take, ld, s->D, s->B[s->cur], s->pitch, s->fill, as); }));
+            appended = true;
+            if (!on_chain) s->app_pending = true;
+            s->fill += (int)take;
+            s->rows_seen += take;
+            p += take * row_bytes;
+            n -= take;
+            if (s->fill == s->m) ST_TRY(sketch_factor(s, s->m, 1, s->delta_rank - 1, 0, chain));
+        }
+        return SAGE_OK;
+    };
+    const sage_status_t rc = body();
+    if (appended && !on_chain) {     // also on the error path: the caller's stream must not run ahead of appends that read `rows`
+        const cudaError_t e = cudaEventRecord(s->ev_rows, as);
+        if (rc == SAGE_OK) CU_TRY(e);
+        s->used = true;
+    }
+    return rc;
+}
+
+// The freeze of one sketch: orthogonalise what the buffer holds, shrink only if more than ell rows are in use.
+// Afterwards s->fill is the number of rows kept (at most ell) and rows up to ell are zero.
+static sage_status_t sketch_freeze(sage_fd* s, cudaStream_t chain) {
+    ST_TRY(sketch_join_appends(s, chain));
+    const int r = s->fill;
+    if (r == 0) {
+        CU_TRY(cudaMemsetAsync(s->B[s->cur], 0, (size_t)s->ell * s->pitch * sizeof(float), chain));
+        CU_TRY(cudaMemsetAsync(s->sigma, 0, s->ell * sizeof(float), chain));
+    } else {
+        const int do_shrink = r > s->ell ? 1 : 0;
+        const int keep = do_shrink ? s->delta_rank - 1 : (r < s->ell ? r : s->ell);
+        ST_TRY(sketch_factor(s, r, do_shrink, keep < s->ell ? keep : s->ell, s->ell, chain));
+    }
+    return SAGE_OK;
+}
+
+static sage_fd* sketch_at(sage_fd* h, int p) { return p == 0 ? h : h->kids[(size_t)p - 1]; }
+
+// Creates the sketches 1..P-1 and the chain streams of the merged form (first update after option 6).
+static sage_status_t ensure_sketches(sage_fd* h) {
+    if (h->P <= 1 || (int)h->kids.size() == h->P - 1) return SAGE_OK;
+    for (int p = (int)h->kids.size() + 1; p < h->P; ++p) {
+        sage_fd* k = nullptr;
+        ST_TRY(create_handle(&k, h->D, h->ell, h->dtype, h->device, true));
+        k->delta_rank = h->delta_rank;
+        k->max_sweeps = h->max_sweeps;
+        k->use_tc = h->use_tc;
+        k->eig_variant = h->eig_variant;
+        k->prof.mask = h->prof.mask;
+        h->kids.push_back(k);
+    }
+    for (int p = 0; p < h->P; ++p) {
+        sage_fd* s = sketch_at(h, p);
+        if (!s->chain) CU_TRY(cudaStreamCreateWithFlags(&s->chain, cudaStreamNonBlocking));
+    }
+    return SAGE_OK;
 }
 
 sage_status_t sage_fd_update(sage_fd_t* h, const void* rows, int64_t n, int64_t ld, void* cuda_stream) {
@@ -526,38 +707,54 @@ sage_status_t sage_fd_update(sage_fd_t* h, const void* rows, int64_t n, int64_t 
     if (n == 0) return SAGE_OK;
     DeviceGuard g(h->device);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    const char* p = static_cast<const char*>(rows);
-    const size_t row_bytes = (size_t)ld * elem_size(h->dtype);
-    // Appends that follow a shrink go to a side stream: they write rows [keep, m) of the buffer the rebuild is
-    // filling (rows [0, keep)) and touch nothing the eigen-solve / rebuild of that shrink read or write, so they run
-    // beside the eigen-solve, which leaves HBM idle. The side stream starts when the Gram kernel of the shrink has
-    // finished (running beside it only takes bandwidth from it) and is joined before the next Gram and before this
-    // call returns.
-    bool on_side = false, side_pending = false;
-    while (n > 0) {
-        const int64_t room = h->m - h->fill;
-        const int64_t take = n < room ? n : room;
-        cudaStream_t as = on_side ? h->side : st;
-        CU_TRY(timed(h, K_APPEND, 1, as, [&] { return launch_append(p, h->dtype, take, ld, h->D, h->B[h->cur], h->pitch, h->fill, as); }));
-        if (on_side) side_pending = true;
-        h->fill += (int)take;
-        h->rows_seen += take;
-        p += take * row_bytes;
-        n -= take;
-        if (h->fill == h->m) {
-            if (side_pending) {
-                CU_TRY(cudaEventRecord(h->ev_join, h->side));
-                CU_TRY(cudaStreamWaitEvent(st, h->ev_join, 0));
-                side_pending = false;
-            }
-            ST_TRY(enqueue_factor(h, h->m, 1, h->delta_rank - 1, 0, st));
-            CU_TRY(cudaStreamWaitEvent(h->side, h->ev_fork, 0));
-            on_side = true;
+    ST_TRY(ensure_sketches(h));
+    static std::atomic<long long> epochs{0};
+    const int64_t epoch = epochs.fetch_add(1) + 1;
+    CU_TRY(cudaEventRecord(h->ev_in, st));
+    sage_status_t rc = SAGE_OK;
+    if (h->P == 1) {
+        rc = sketch_feed(h, rows, h->dtype, n, ld, st, h->ev_in, epoch, false);
+        h->dealt += n;
+    } else {
+        // block b of the row stream (counted over all calls) goes to sketch b mod P
+        const char* p = static_cast<const char*>(rows);
+        const size_t row_bytes = (size_t)ld * elem_size(h->dtype);
+        while (n > 0 && rc == SAGE_OK) {
+            const int64_t b = h->dealt / h->block;
+            const int64_t left_in_block = (b + 1) * h->block - h->dealt;
+            const int64_t take = n < left_in_block ? n : left_in_block;
+            sage_fd* s = sketch_at(h, (int)(b % h->P));
+            rc = sketch_feed(s, p, h->dtype, take, ld, s->chain, h->ev_in, epoch, false);
+            h->dealt += take;
+            p += take * row_bytes;
+            n -= take;
         }
     }
-    if (side_pending) {
-        CU_TRY(cudaEventRecord(h->ev_join, h->side));
-        CU_TRY(cudaStreamWaitEvent(st, h->ev_join, 0));
+    // the caller's stream continues once every row of this call has been copied into a buffer
+    for (int p = 0; p < h->P && p <= (int)h->kids.size(); ++p) {
+        sage_fd* s = sketch_at(h, p);
+        if (s->used) {
+            const cudaError_t e = cudaStreamWaitEvent(st, s->ev_rows, 0);
+            if (rc == SAGE_OK) CU_TRY(e);
+            s->used = false;
+        }
+    }
+    return rc;
+}
+
+// Makes `cuda_stream` wait for everything the handle has enqueued on streams of its own.
+sage_status_t sage_fd_join(sage_fd_t* h, void* cuda_stream) {
+    ST_TRY(check_handle(h));
+    DeviceGuard g(h->device);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    for (int p = 0; p <= (int)h->kids.size(); ++p) {
+        sage_fd* s = sketch_at(h, p);
+        CU_TRY(cudaEventRecord(s->ev_join, s->side));
+        CU_TRY(cudaStreamWaitEvent(st, s->ev_join, 0));
+        if (s->chain) {
+            CU_TRY(cudaEventRecord(s->ev_done, s->chain));
+            CU_TRY(cudaStreamWaitEvent(st, s->ev_done, 0));
+        }
     }
     return SAGE_OK;
 }
@@ -570,14 +767,27 @@ sage_status_t sage_fd_finalize(sage_fd_t* h, void* cuda_stream) {
     }
     DeviceGuard g(h->device);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    const int r = h->fill;
-    if (r == 0) {
-        CU_TRY(cudaMemsetAsync(h->B[h->cur], 0, (size_t)h->ell * h->pitch * sizeof(float), st));
-        CU_TRY(cudaMemsetAsync(h->sigma, 0, h->ell * sizeof(float), st));
+    const int nsk = (int)h->kids.size() + 1;            // sketches that exist (1 unless the merged form has been fed)
+    if (nsk == 1) {
+        ST_TRY(sketch_freeze(h, (h->P > 1 && h->chain) ? h->chain : st));
     } else {
-        const int do_shrink = r > h->ell ? 1 : 0;
-        const int keep = do_shrink ? h->delta_rank - 1 : (r < h->ell ? r : h->ell);
-        ST_TRY(enqueue_factor(h, r, do_shrink, keep < h->ell ? keep : h->ell, h->ell, st));
+        // every sketch is frozen on its own, then sketch a absorbs sketch a + s for s = 1, 2, 4, ...: the rows the
+        // other one kept are appended to it and it is frozen again (a shrink happens if that fills its buffer)
+        for (int p = 0; p < nsk; ++p) ST_TRY(sketch_freeze(sketch_at(h, p), sketch_at(h, p)->chain));
+        for (int stride = 1; stride < nsk; stride *= 2)
+            for (int a = 0; a + stride < nsk; a += 2 * stride) {
+                sage_fd* A = sketch_at(h, a);
+                sage_fd* Bs = sketch_at(h, a + stride);
+                CU_TRY(cudaEventRecord(Bs->ev_done, Bs->chain));
+                CU_TRY(cudaStreamWaitEvent(A->chain, Bs->ev_done, 0));
+                if (Bs->fill > 0)
+                    ST_TRY(sketch_feed(A, Bs->B[Bs->cur], SAGE_F32, Bs->fill, Bs->pitch, A->chain, nullptr, 0, true));
+                ST_TRY(sketch_freeze(A, A->chain));
+            }
+    }
+    if (h->P > 1 && h->chain) {                          // merged form: sketch 0 holds the result; back to the caller's stream
+        CU_TRY(cudaEventRecord(h->ev_done, h->chain));
+        CU_TRY(cudaStreamWaitEvent(st, h->ev_done, 0));
     }
     ST_TRY(enqueue_freeze_aux(h, st));
     h->state = FROZEN;
@@ -586,6 +796,14 @@ sage_status_t sage_fd_finalize(sage_fd_t* h, void* cuda_stream) {
     CU_TRY(cudaMemcpyAsync(&info, h->info, sizeof info, cudaMemcpyDeviceToHost, st));
     CU_TRY(cudaMemcpyAsync(&tc_err, h->tc_err, sizeof tc_err, cudaMemcpyDeviceToHost, st));
     CU_TRY(cudaStreamSynchronize(st));
+    for (sage_fd* k : h->kids) {                         // their chains ended before sketch 0's did
+        EigInfo ki;
+        int kt = 0;
+        CU_TRY(cudaMemcpy(&ki, k->info, sizeof ki, cudaMemcpyDeviceToHost));
+        CU_TRY(cudaMemcpy(&kt, k->tc_err, sizeof kt, cudaMemcpyDeviceToHost));
+        info.flags |= ki.flags;
+        tc_err |= kt;
+    }
     if (tc_err) {
         set_err("sage_fd_finalize: a tensor-core kernel gave up waiting on its pipeline (results are not valid)");
         return SAGE_ERR_CUDA;
@@ -718,6 +936,7 @@ sage_status_t sage_score_chunk(sage_fd_t* h, const void* rows, int64_t n, int64_
             });
             if (e == cudaSuccess) {
                 done = true;
+                h->tc_launches += 1;
                 if (planes > 1)
                     CU_TRY(timed(h, K_PROJECT_REDUCE, 1, st,
                                  [&] { return launch_split_reduce(out, planes, (int64_t)sub * ell, (int)sub, ell, ell, Z, ell, st); }));
@@ -744,6 +963,7 @@ sage_status_t sage_score_chunk(sage_fd_t* h, const void* rows, int64_t n, int64_
             });
             if (e == cudaSuccess) {
                 done = true;
+                h->tc_launches += 1;
                 if (splits > 1)
                     CU_TRY(timed(h, K_PROJECT_REDUCE, 1, st,
                                  [&] { return launch_split_reduce(out, splits, (int64_t)sub * ell, (int)sub, ell, ell, Z, ell, st); }));
@@ -980,16 +1200,31 @@ sage_status_t sage_fd_stats(sage_fd_t* h, sage_stats_t* out) {
     CU_TRY(cudaDeviceSynchronize());
     EigInfo info;
     CU_TRY(cudaMemcpy(&info, h->info, sizeof info, cudaMemcpyDeviceToHost));
-    out->rows_seen = h->rows_seen;
+    int tc_err = 0;
+    CU_TRY(cudaMemcpy(&tc_err, h->tc_err, sizeof tc_err, cudaMemcpyDeviceToHost));
+    int64_t launches = h->launches, tc_launches = h->tc_launches;
+    for (sage_fd* k : h->kids) {             // merged form: counters of all sketches together
+        EigInfo ki;
+        int kt = 0;
+        CU_TRY(cudaMemcpy(&ki, k->info, sizeof ki, cudaMemcpyDeviceToHost));
+        CU_TRY(cudaMemcpy(&kt, k->tc_err, sizeof kt, cudaMemcpyDeviceToHost));
+        info.shrinks += ki.shrinks;
+        info.sum_delta += ki.sum_delta;
+        info.flags |= ki.flags;
+        if (ki.max_sweeps > info.max_sweeps) info.max_sweeps = ki.max_sweeps;
+        tc_err |= kt;
+        launches += k->launches;
+        tc_launches += k->tc_launches;
+    }
+    out->rows_seen = h->dealt;
     out->shrinks = info.shrinks;
     out->sum_delta = info.sum_delta;
     out->last_sweeps = info.sweeps;
     out->max_sweeps = info.max_sweeps;
     out->last_rank = info.rank;
-    int tc_err = 0;
-    CU_TRY(cudaMemcpy(&tc_err, h->tc_err, sizeof tc_err, cudaMemcpyDeviceToHost));
     out->device_flags = info.flags | (tc_err ? 4u : 0u);
-    out->kernel_launches = h->launches;
+    out->kernel_launches = launches;
+    out->tensor_core_launches = tc_launches;
     return SAGE_OK;
 }
 
@@ -1001,21 +1236,28 @@ sage_status_t sage_fd_profile(sage_fd_t* h, double* ms, int64_t* launches, int32
     }
     DeviceGuard g(h->device);
     CU_TRY(cudaDeviceSynchronize());
-    for (auto& p : h->prof.pending) {
-        float t = 0.f;
-        if (cudaEventElapsedTime(&t, p.a, p.b) == cudaSuccess) {
-            h->prof.ms[p.cls] += t;
-            h->prof.n[p.cls] += 1;
-        }
-        h->prof.pool.push_back(p.a);
-        h->prof.pool.push_back(p.b);
-    }
-    h->prof.pending.clear();
     for (int c = 0; c < K_NCLASS; ++c) {
-        ms[c] = h->prof.ms[c];
-        launches[c] = h->prof.n[c];
-        h->prof.ms[c] = 0.0;
-        h->prof.n[c] = 0;
+        ms[c] = 0.0;
+        launches[c] = 0;
+    }
+    for (int q = 0; q <= (int)h->kids.size(); ++q) {     // merged form: all sketches together (their kernels overlap in time)
+        Prof& pr = sketch_at(h, q)->prof;
+        for (auto& p : pr.pending) {
+            float t = 0.f;
+            if (cudaEventElapsedTime(&t, p.a, p.b) == cudaSuccess) {
+                pr.ms[p.cls] += t;
+                pr.n[p.cls] += 1;
+            }
+            pr.pool.push_back(p.a);
+            pr.pool.push_back(p.b);
+        }
+        pr.pending.clear();
+        for (int c = 0; c < K_NCLASS; ++c) {
+            ms[c] += pr.ms[c];
+            launches[c] += pr.n[c];
+            pr.ms[c] = 0.0;
+            pr.n[c] = 0;
+        }
     }
     return SAGE_OK;
 }
@@ -1088,6 +1330,19 @@ sage_status_t sage_select_from_host(const void* rows_host, int64_t N, int64_t D,
         if (k > 0) CU_TRY(cudaMemcpyAsync(idx_host, d_idx, (size_t)k * sizeof(int64_t), cudaMemcpyDeviceToHost, s_comp));
         CU_TRY(cudaStreamSynchronize(s_comp));
         CU_TRY(cudaStreamSynchronize(s_copy));
+        // what the device recorded during pass 2 (pass 1 was reported by the freeze)
+        int tc_err = 0;
+        EigInfo info;
+        CU_TRY(cudaMemcpy(&tc_err, h->tc_err, sizeof tc_err, cudaMemcpyDeviceToHost));
+        CU_TRY(cudaMemcpy(&info, h->info, sizeof info, cudaMemcpyDeviceToHost));
+        if (tc_err || (info.flags & kFlagExchangeTimeout)) {
+            set_err("sage_select_from_host: a kernel gave up a bounded wait during the scoring pass (results are not valid)");
+            return SAGE_ERR_CUDA;
+        }
+        if ((info.flags & kFlagNonFinite) && rc == SAGE_OK) {
+            set_err("sage_select_from_host: non-finite values were met in the rows (such rows score 0)");
+            rc = SAGE_ERR_NONFINITE;
+        }
         return SAGE_OK;
     };
     sage_status_t s = body();

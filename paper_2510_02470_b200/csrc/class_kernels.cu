@@ -1,4 +1,4 @@
-// Class-balanced variant (Algorithm 1, branch "class balance required"; "Agreement Scoring and Selection"):
+// Class-balanced variant (Algorithm 1, the class-balanced branch; section on agreement scoring and selection):
 // per-class unit centroids u_c of the stored normalised projections, scores <zhat_i, u_c(i)>, and the top-k_c
 // examples of every class. All reductions run in a fixed order (ascending example index), so results are
 // reproducible bit for bit.

@@ -61,8 +61,10 @@ cudaError_t launch_gram_sym_reduce(const float* parts, int splits, int64_t strid
 
 // Tensor-core rebuild: Bdst[j][d] = sum_{i<r} W[j][i] * Bsrc[i][d] for j < keep, d < pitch (fp32-faithful, see
 // tc_rebuild.cu). Wsplit holds W already split for tf32: rows [0, j_pad) = W rounded to 11 significant bits, rows
-// [j_pad, 2 j_pad) = the remainder; row pitch ldw floats, columns i >= r and rows j >= keep zero. Needs j_pad a
-// multiple of 16 with keep <= j_pad <= 128 and r <= 256; returns cudaErrorNotSupported otherwise.
+// [j_pad, 2 j_pad) = the remainder; row pitch ldw floats, columns i >= r and rows j >= keep zero (rows the eigen-solve
+// does not write, up to the next multiple of 128, are read by the MMA and must be finite: the caller zeroes the array
+// once). Needs j_pad a multiple of 16 with keep <= j_pad <= 256 (one launch per 128 output rows) and r <= 512;
+// returns cudaErrorNotSupported otherwise.
 cudaError_t launch_tc_rebuild(const float* Wsplit, int ldw, int j_pad, const float* Bsrc, float* Bdst, int64_t pitch, int64_t D, int r,
                               int keep, int* err, cudaStream_t st);
 

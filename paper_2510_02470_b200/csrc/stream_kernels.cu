@@ -178,8 +178,9 @@ __global__ void __launch_bounds__(256) k_split_reduce(const float* __restrict__ 
 }
 
 // Split reduction of a Gram matrix computed in the symmetric form: slice z left T_z = hi*hi^T + 2*hi*lo^T at
-// parts + z*stride; K = sum_z (T_z + T_z^T) / 2, ascending z, fp64. One block per 32 x 32 tile (I, J): thread
-// (ty, tx) sums T[I+ty][J+tx] and T[J+ty][I+tx] (both read along rows), the second is transposed through shared memory.
+// parts + z*stride; K = sum_z (T_z + T_z^T) / 2 in fp64. One block of 16 x 16 x 4 threads per 16 x 16 tile (I, J): thread
+// (ty, tx) of layer tz sums T[I+ty][J+tx] and T[J+ty][I+tx] (both read along rows) over the slices z = tz, tz+4, ...;
+// the four layers are added in a fixed order and the second sum is transposed through shared memory.
 __global__ void __launch_bounds__(1024) k_gram_sym_reduce(const float* __restrict__ parts, int splits, int64_t stride, int r,
                                                           int64_t ldp, float* __restrict__ out, int64_t ldo) {
     // 16 x 16 outputs per block; the four z-layers of the block each sum a quarter of the partial matrices

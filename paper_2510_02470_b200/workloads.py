@@ -238,21 +238,23 @@ class DeviceStream:
         if out is None:
             out = torch.zeros((n, w.ld), dtype=w.dtype, device=self.device)
         g = _dev_gen(self.device, self.seed, 42 if w.name == "c4" else 52, j)
+        # Three passes over a sub-block: the noise is drawn, the low-rank signal is added to it in place
+        # (x = sigma * noise + coef Q), and the row scale is applied while the result is rounded into the output.
         for r0 in range(0, n, self.sub_rows):
             r = min(self.sub_rows, n - r0)
             scale = torch.exp(0.5 * torch.randn((r, 1), generator=g, device=self.device))
             if w.name == "c4":
                 coef = torch.randn((r, 64), generator=g, device=self.device)
-                x = coef @ self.Q
-                x += 0.1 * torch.randn((r, w.D), generator=g, device=self.device)
-                out[r0:r0 + r, : w.D] = (scale * x).to(w.dtype)
+                x = torch.randn((r, w.D), generator=g, device=self.device)
+                x.addmm_(coef, self.Q, beta=0.1)
+                torch.mul(x, scale, out=out[r0:r0 + r, : w.D])
             else:
                 c0 = 0
                 for d, Q in zip(self.blocks, self.Qb):
                     coef = torch.randn((r, 8), generator=g, device=self.device)
-                    x = coef @ Q
-                    x += math.sqrt(2.0 / d) * torch.randn((r, d), generator=g, device=self.device)
-                    out[r0:r0 + r, c0:c0 + d] = (scale * x).to(w.dtype)
+                    x = torch.randn((r, d), generator=g, device=self.device)
+                    x.addmm_(coef, Q, beta=math.sqrt(2.0 / d))
+                    torch.mul(x, scale, out=out[r0:r0 + r, c0:c0 + d])
                     c0 += d
         return out[:n]
 

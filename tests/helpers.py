@@ -11,13 +11,17 @@ TOL_SKETCH = 1e-4          # ||S^T S - S_o^T S_o||_2 / ||A||_F^2
 TOL_SCORE = {torch.float32: 1e-4, torch.bfloat16: 2e-3}
 
 
-def gpu_run(rows_cpu: torch.Tensor, D: int, ell: int, keep_rate: float, chunks=None, score_chunks=None):
+def gpu_run(rows_cpu: torch.Tensor, D: int, ell: int, keep_rate: float, chunks=None, score_chunks=None, sketches=1, block=None):
     """rows_cpu: (N, ld) CPU tensor. Returns dict with S (ell x D fp64 numpy), sigma, alpha, idx, stats."""
     dev = torch.device("cuda", 0)
     rows = rows_cpu.to(dev)
     N = rows.shape[0]
     fd = sage.SageFD(D, ell, rows.dtype, 0)
     try:
+        if sketches > 1:
+            fd.set_option(6, sketches)
+        if block:
+            fd.set_option(7, block)
         if chunks is None:
             fd.update(rows)
         else:

@@ -336,3 +336,24 @@ def test_select_against_lexsort(kind):
         idx = oracle.select(a, rate)
         ref = np.lexsort((np.arange(N), -a))[: oracle.select_k(N, rate)]
         assert np.array_equal(idx, ref)
+
+
+# ------------------------------------------------------------------ the comparison helpers themselves
+
+@pytest.mark.parametrize("p,q,D", [(3, 2, 4), (8, 8, 300), (64, 64, 20000)])
+def test_signed_gram_norm_both_forms_against_the_dense_matrix(p, q, D):
+    """|| P^T P - Q^T Q ||_2 through the QR form and through the W^(1/2) J W^(1/2) form (the one taken for operands too
+    large for a QR) against numpy's eigvalsh of the D x D matrix itself where that is small, and against each other
+    on a mid-size case. The square-root form is accurate to about sqrt(eps) of the operands' scale."""
+    r = rng(p + q + D)
+    P = r.standard_normal((p, D)) * np.linspace(2.0, 0.1, p)[:, None]
+    Q = P[:q] + 1e-3 * r.standard_normal((q, D))
+    a = metrics.signed_gram_norm(P, Q, method="qr")
+    b = metrics.signed_gram_norm(P, Q, method="sqrt")
+    scale = np.linalg.norm(P) ** 2
+    assert abs(a - b) <= 1e-7 * scale
+    if D <= 300:
+        dense = np.abs(np.linalg.eigvalsh(P.T @ P - Q.T @ Q)).max()
+        assert abs(a - dense) <= 1e-12 * scale and abs(b - dense) <= 1e-7 * scale
+    lo, hi = metrics.signed_gram_extremes(P, Q)
+    assert np.isclose(max(abs(lo), abs(hi)), a)
