@@ -28,6 +28,7 @@
 #ifndef SAGE_B200_H_
 #define SAGE_B200_H_
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -124,6 +125,18 @@ sage_status_t sage_score_chunk(sage_fd_t* h, const void* rows, int64_t n, int64_
                                void* cuda_stream);
 sage_status_t sage_score_end(sage_fd_t* h, float* scores, void* cuda_stream);
 
+/* Strict-memory form of Phase II (Method, the complexity paragraph and the abstract: memory O(ell D), independent of N).
+ * The default keeps the N x ell normalised projections between the scoring pass and its end, because alpha_i needs the
+ * consensus u, which needs every row. With option 8 set to 1 nothing of size N is kept: sage_score_begin / _chunk / _end
+ * then only form u (sage_score_end accepts scores == NULL), holding the normalised projections of one sub-chunk at a
+ * time, and a third pass over the rows produces the scores:
+ *   sage_score_apply  alpha_i = <zhat_i, u> for the n given rows (any subset, any order, any chunking) against the u of
+ *                     the finished pass; scores: device, n floats. The rows are projected again, so this pass costs as much
+ *                     as the scoring pass; results equal the default's up to the rounding order of the consensus sum.
+ * Requires a pass finished in this mode; sage_score_intermediates and sage_score_classes need the default mode.
+ * Asynchronous on the stream. */
+sage_status_t sage_score_apply(sage_fd_t* h, const void* rows, int64_t n, int64_t ld, float* scores, void* cuda_stream);
+
 /* Borrowed device pointers to the last scoring pass's intermediates (for checks of the lemma in
  * "Energy preservation"): zhat N x ell fp32, znorm N fp32 (||z_i||), u ell fp32. Any may be NULL. */
 sage_status_t sage_score_intermediates(const sage_fd_t* h, const float** zhat, const float** znorm, const float** u);
@@ -190,6 +203,22 @@ sage_status_t sage_select_from_host(const void* rows_host, int64_t N, int64_t D,
                                     sage_dtype_t row_dtype, double keep_rate, int64_t chunk_rows, int device,
                                     float* scores_host, int64_t* idx_host, int64_t* k_out);
 
+/* Checkpoint of the sketch (Method, first paragraph and the complexity paragraph: the whole state of pass 1 is the buffer
+ * and a few counters, O(ell D) whatever N is). sage_fd_export writes it to HOST memory, sage_fd_import restores it into
+ * a handle created with the same D, ell and row type; a stream of rows can so be sketched in several sessions, or a frozen
+ * sketch kept for later scoring. Allowed while sketching (between updates) and when frozen, not during a scoring pass.
+ * A restored handle continues exactly where the exported one stood: feeding the remaining rows gives the same sketch,
+ * bit for bit, as the uninterrupted run. The merged form (option 6) is exported with all its sketches.
+ *   sage_fd_export_size  bytes the checkpoint needs now (it grows and shrinks with the rows in the buffer).
+ *   sage_fd_export       dst_host: host memory of `capacity` bytes; *written (may be NULL) receives the size. Synchronises
+ *                        the device.
+ *   sage_fd_import       src_host / bytes: a checkpoint; the handle is reset first and takes the checkpoint's options 1, 6
+ *                        and 7. SAGE_ERR_INVALID_ARG (handle untouched) if the data is not a checkpoint of this shape.
+ *                        Synchronises the device. */
+sage_status_t sage_fd_export_size(const sage_fd_t* h, size_t* bytes);
+sage_status_t sage_fd_export(sage_fd_t* h, void* dst_host, size_t capacity, size_t* written);
+sage_status_t sage_fd_import(sage_fd_t* h, const void* src_host, size_t bytes, void* cuda_stream);
+
 typedef struct {
     int64_t rows_seen;      /* rows given to sage_fd_update since create/reset */
     int64_t shrinks;        /* shrinks applied (including the one in finalize, if any) */
@@ -222,7 +251,9 @@ sage_status_t sage_fd_stats(sage_fd_t* h, sage_stats_t* out);
  * freezes every sketch and merges them pairwise (sketch a absorbs sketch a + s for s = 1, 2, 4, ...: the rows a + s
  * kept are appended to a, which is frozen again). Frequent-Directions sketches are mergeable, so the result obeys
  * the same error bound as the sequential sketch, but it is a different sketch. The P chains of Gram / eigen-solve /
- * rebuild run on P streams of the library's own and overlap on the device; device memory grows P-fold. */
+ * rebuild run on P streams of the library's own and overlap on the device; device memory grows P-fold.
+ * Outside a scoring pass: key 8 = 1 for the strict-memory form of Phase II (see sage_score_apply), 0 (default) to keep the
+ * N x ell normalised projections. */
 sage_status_t sage_fd_set_option(sage_fd_t* h, int key, double value);
 
 /* Per-kernel device time of this handle's launches since the previous call, for the classes selected

@@ -37,7 +37,11 @@ SIGNATURES = {
     "sage_score_begin": (_i32, [_vp, _i64, _vp]),
     "sage_score_chunk": (_i32, [_vp, _vp, _i64, _i64, _i64, _vp]),
     "sage_score_end": (_i32, [_vp, _vp, _vp]),
+    "sage_score_apply": (_i32, [_vp, _vp, _i64, _i64, _vp, _vp]),
     "sage_score_intermediates": (_i32, [_vp, _vp, _vp, _vp]),
+    "sage_fd_export_size": (_i32, [_vp, _vp]),
+    "sage_fd_export": (_i32, [_vp, _vp, C.c_size_t, _vp]),
+    "sage_fd_import": (_i32, [_vp, _vp, C.c_size_t, _vp]),
     "sage_select_count": (_i64, [_i64, _f64]),
     "sage_select": (_i32, [_vp, _i64, _f64, _vp, _vp, _vp]),
     "sage_score_classes": (_i32, [_vp, _vp, _i32, _vp, _vp]),
@@ -169,9 +173,34 @@ def sage_score_chunk(h: int, rows: torch.Tensor, D: int, row_offset: int) -> Non
     _check(lib().sage_score_chunk(h, ptr, n, ld, row_offset, _stream(rows.device)))
 
 
-def sage_score_end(h: int, scores: torch.Tensor) -> None:
+def sage_score_end(h: int, scores: Optional[torch.Tensor], device=None) -> None:
+    """scores may be None in the strict-memory mode (option 8), where this call only forms the consensus direction."""
+    if scores is None:
+        _check(lib().sage_score_end(h, None, _stream(device)))
+        return
     assert scores.dtype == torch.float32 and scores.is_contiguous()
     _check(lib().sage_score_end(h, scores.data_ptr(), _stream(scores.device)))
+
+
+def sage_score_apply(h: int, rows: torch.Tensor, D: int, scores: torch.Tensor) -> None:
+    ptr, n, ld = _rows_args(rows, D)
+    assert scores.dtype == torch.float32 and scores.is_contiguous() and scores.numel() >= n
+    _check(lib().sage_score_apply(h, ptr, n, ld, scores.data_ptr(), _stream(rows.device)))
+
+
+def sage_fd_export(h: int) -> torch.Tensor:
+    """The checkpoint of the sketch as a CPU uint8 tensor."""
+    need = C.c_size_t(0)
+    _check(lib().sage_fd_export_size(h, C.byref(need)))
+    buf = torch.empty((need.value,), dtype=torch.uint8)
+    written = C.c_size_t(0)
+    _check(lib().sage_fd_export(h, buf.data_ptr(), need.value, C.byref(written)))
+    return buf[: written.value]
+
+
+def sage_fd_import(h: int, blob: torch.Tensor, device=None) -> None:
+    assert blob.device.type == "cpu" and blob.dtype == torch.uint8 and blob.is_contiguous()
+    _check(lib().sage_fd_import(h, blob.data_ptr(), blob.numel(), _stream(device)))
 
 
 def sage_score_intermediates(h: int, N: int, ell: int, device) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor]:
@@ -329,8 +358,17 @@ class SageFD:
     def score_chunk(self, rows: torch.Tensor, row_offset: int) -> None:
         sage_score_chunk(self._h, rows, self.D, row_offset)
 
-    def score_end(self, scores: torch.Tensor) -> None:
+    def score_end(self, scores: Optional[torch.Tensor] = None) -> None:
         sage_score_end(self._h, scores)
+
+    def score_apply(self, rows: torch.Tensor, scores: torch.Tensor) -> None:
+        sage_score_apply(self._h, rows, self.D, scores)
+
+    def export_state(self) -> torch.Tensor:
+        return sage_fd_export(self._h)
+
+    def import_state(self, blob: torch.Tensor) -> None:
+        sage_fd_import(self._h, blob, self.device)
 
     def score_classes(self, labels: torch.Tensor, num_classes: int, scores: Optional[torch.Tensor] = None) -> torch.Tensor:
         if scores is None:

@@ -158,6 +158,8 @@ struct sage_fd {
     double* zsum = nullptr;
     float* u = nullptr;
     bool scored = false;           // a scoring pass over N_total rows has finished: zhat holds their normalised projections
+    bool strict = false;           // option 8: no N x ell store; scores come from a third pass (sage_score_apply)
+    bool scored_strict = false;    // the finished pass ran in strict-memory mode: u is known, zhat is not kept
     float* class_U = nullptr;      // class-balanced variant: unit centroids (class_cap x ell) and class sizes
     int* class_counts = nullptr;
     int class_cap = 0, class_num = 0;
@@ -530,6 +532,7 @@ sage_status_t sage_fd_reset(sage_fd_t* h) {
     h->dealt = 0;
     h->cur = 0;
     h->scored = false;
+    h->scored_strict = false;
     h->state = SKETCHING;
     h->launches = 0;
     h->tc_launches = 0;
@@ -549,6 +552,14 @@ sage_status_t sage_fd_set_option(sage_fd_t* h, int key, double value) {
     if (key == 4) {                          // 0: CUDA-core kernels only, 1: tensor-core kernels where possible
         h->use_tc = value != 0.0;
         for (sage_fd* k : h->kids) k->use_tc = h->use_tc;
+        return SAGE_OK;
+    }
+    if (key == 8) {                          // strict-memory scoring: no N x ell store, scores from a third pass
+        if (h->state == SCORING) {
+            set_err("sage_fd_set_option: a scoring pass is open");
+            return SAGE_ERR_BAD_STATE;
+        }
+        h->strict = value != 0.0;
         return SAGE_OK;
     }
     if (key == 5) {                          // eigen-solve kernel family (same algorithm, same results up to rounding order)
@@ -852,6 +863,7 @@ sage_status_t sage_fd_load_sketch(sage_fd_t* h, const float* S, int64_t ld, void
     ST_TRY(enqueue_freeze_aux(h, st));
     h->fill = h->ell;
     h->scored = false;
+    h->scored_strict = false;
     h->state = FROZEN;
     return SAGE_OK;
 }
@@ -868,7 +880,7 @@ sage_status_t sage_score_begin(sage_fd_t* h, int64_t N_total, void* cuda_stream)
     }
     DeviceGuard g(h->device);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    if (N_total > h->zcap) {
+    if (!h->strict && N_total > h->zcap) {
         CU_TRY(cudaStreamSynchronize(st));
         if (h->zhat) CU_TRY(cudaFree(h->zhat));
         if (h->znorm) CU_TRY(cudaFree(h->znorm));
@@ -882,24 +894,17 @@ sage_status_t sage_score_begin(sage_fd_t* h, int64_t N_total, void* cuda_stream)
     h->N_total = N_total;
     h->next_row = 0;
     h->scored = false;
+    h->scored_strict = false;
     h->state = SCORING;
     return SAGE_OK;
 }
 
-sage_status_t sage_score_chunk(sage_fd_t* h, const void* rows, int64_t n, int64_t ld, int64_t row_offset, void* cuda_stream) {
-    ST_TRY(check_handle(h));
-    if (h->state != SCORING) {
-        set_err("sage_score_chunk: no open scoring pass");
-        return SAGE_ERR_BAD_STATE;
-    }
-    if (n < 0 || (n > 0 && (!rows || ld < h->D)) || row_offset != h->next_row || row_offset + n > h->N_total) {
-        set_err("sage_score_chunk: bad argument (n=%lld ld=%lld offset=%lld expected offset=%lld N_total=%lld)", (long long)n,
-                (long long)ld, (long long)row_offset, (long long)h->next_row, (long long)h->N_total);
-        return SAGE_ERR_INVALID_ARG;
-    }
-    if (n == 0) return SAGE_OK;
-    DeviceGuard g(h->device);
-    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+// Projection, normalisation and consensus partials of n rows (sub-chunk by sub-chunk). store_at >= 0: the normalised
+// projections go to rows [store_at, store_at + n) of the handle's N x ell store; store_at < 0: to a scratch of one sub-chunk
+// (strict-memory mode). accumulate: the rows' sum is added to the consensus sum. scores_out != null (third pass of the
+// strict-memory mode): the scores of these rows against the finished consensus are written there.
+static sage_status_t score_rows(sage_fd* h, const void* rows, int64_t n, int64_t ld, cudaStream_t st, int64_t store_at, bool accumulate,
+                                float* scores_out) {
     const int ell = h->ell;
     int64_t sub_max = 148 * 128;             // one full wave of 128-row tiles
     const char* p = static_cast<const char*>(rows);
@@ -919,17 +924,27 @@ sage_status_t sage_score_chunk(sage_fd_t* h, const void* rows, int64_t n, int64_
         const int64_t sub = (n - r0 < sub_max) ? n - r0 : sub_max;
         const size_t nb = (size_t)((sub + 63) / 64);
         ST_TRY(ensure(&h->partials, &h->partials_bytes, nb * ell * sizeof(float)));
+        if (store_at < 0 && sub > h->zcap) {         // strict-memory mode: normalised projections of one sub-chunk only
+            CU_TRY(cudaStreamSynchronize(st));
+            if (h->zhat) CU_TRY(cudaFree(h->zhat));
+            if (h->znorm) CU_TRY(cudaFree(h->znorm));
+            h->zhat = h->znorm = nullptr;
+            h->zcap = 0;
+            CU_TRY(cudaMalloc((void**)&h->zhat, (size_t)sub * ell * sizeof(float)));
+            CU_TRY(cudaMalloc((void**)&h->znorm, (size_t)sub * sizeof(float)));
+            h->zcap = sub;
+        }
         const size_t zred = (size_t)sub * ell * sizeof(float);
         bool done = false;
-        float* Z = nullptr;
+        const float* Zparts = nullptr;       // the projections of this sub-chunk as nplanes partial planes of sub x ell floats
+        int nplanes = 1;
         if (tc32_ok) {
             const int splits = pick_splits_waves((int)((sub + 127) / 128), h->D, 2048, 64);
             // sketches of at most 64 rows: one wide MMA per K step against the pre-split sketch, two partial planes per K slice
             const bool wide = h->S32split != nullptr;
             const int planes = wide ? 2 * splits : splits;
-            ST_TRY(ensure(&h->zwork, &h->zwork_bytes, zred * (planes > 1 ? planes + 1 : 1)));
-            Z = h->zwork;
-            float* out = planes > 1 ? h->zwork + (size_t)sub * ell : Z;
+            ST_TRY(ensure(&h->zwork, &h->zwork_bytes, zred * planes));
+            float* out = h->zwork;
             cudaError_t e = timed(h, K_PROJECT, 1, st, [&] {
                 return launch_tc_gemm_nt_x3(reinterpret_cast<const float*>(p + r0 * row_bytes), ld, wide ? h->S32split : S, h->pitch, (int)sub,
                                             ell, h->D, splits, out, ell, (int64_t)sub * ell, wide ? 2 : 0, h->tc_err, st);
@@ -937,9 +952,8 @@ sage_status_t sage_score_chunk(sage_fd_t* h, const void* rows, int64_t n, int64_
             if (e == cudaSuccess) {
                 done = true;
                 h->tc_launches += 1;
-                if (planes > 1)
-                    CU_TRY(timed(h, K_PROJECT_REDUCE, 1, st,
-                                 [&] { return launch_split_reduce(out, planes, (int64_t)sub * ell, (int)sub, ell, ell, Z, ell, st); }));
+                Zparts = out;
+                nplanes = planes;
             } else if (e != cudaErrorNotSupported) {
                 CU_TRY(e);
             } else {
@@ -954,9 +968,8 @@ sage_status_t sage_score_chunk(sage_fd_t* h, const void* rows, int64_t n, int64_
             if (tiles >= 148 && mt > 2) mt = 2;   // measured: pairs of row tiles with two K slices beat single tiles by 25 %
             while (mt > 1 && (int64_t)((tiles + mt - 1) / mt) * (h->D / 4096 > 0 ? h->D / 4096 : 1) < 148) mt >>= 1;
             const int splits = pick_splits_waves((tiles + mt - 1) / mt, h->D, 4096, 148);
-            ST_TRY(ensure(&h->zwork, &h->zwork_bytes, zred * (splits > 1 ? splits + 1 : 1)));
-            Z = h->zwork;
-            float* out = splits > 1 ? h->zwork + (size_t)sub * ell : Z;
+            ST_TRY(ensure(&h->zwork, &h->zwork_bytes, zred * splits));
+            float* out = h->zwork;
             cudaError_t e = timed(h, K_PROJECT, 1, st, [&] {
                 return launch_tc_gemm_nt(p + r0 * row_bytes, SAGE_BF16, ld, h->P16, h->pitch, (int)sub, ell, h->p16_fold, mt, h->D, splits,
                                          out, ell, (int64_t)sub * ell, h->tc_err, st);
@@ -964,9 +977,8 @@ sage_status_t sage_score_chunk(sage_fd_t* h, const void* rows, int64_t n, int64_
             if (e == cudaSuccess) {
                 done = true;
                 h->tc_launches += 1;
-                if (splits > 1)
-                    CU_TRY(timed(h, K_PROJECT_REDUCE, 1, st,
-                                 [&] { return launch_split_reduce(out, splits, (int64_t)sub * ell, (int)sub, ell, ell, Z, ell, st); }));
+                Zparts = out;
+                nplanes = splits;
             } else if (e != cudaErrorNotSupported) {
                 CU_TRY(e);
             } else {
@@ -976,27 +988,43 @@ sage_status_t sage_score_chunk(sage_fd_t* h, const void* rows, int64_t n, int64_
         if (!done) {
             const int tiles = (int)((sub + 63) / 64) * ((ell + 63) / 64);
             const int splits = pick_splits(tiles, h->D, 1024);
-            ST_TRY(ensure(&h->zwork, &h->zwork_bytes, zred * (splits > 1 ? splits + 1 : 1)));
-            Z = h->zwork;
-            if (splits == 1) {
-                CU_TRY(timed(h, K_PROJECT, 1, st, [&] {
-                    return launch_gemm_nt(p + r0 * row_bytes, h->dtype, ld, S, h->pitch, (int)sub, ell, h->D, 1, Z, ell, 0, st);
-                }));
-            } else {
-                float* parts = h->zwork + (size_t)sub * ell;
-                CU_TRY(timed(h, K_PROJECT, 1, st, [&] {
-                    return launch_gemm_nt(p + r0 * row_bytes, h->dtype, ld, S, h->pitch, (int)sub, ell, h->D, splits, parts, ell,
-                                          (int64_t)sub * ell, st);
-                }));
-                CU_TRY(timed(h, K_PROJECT_REDUCE, 1, st,
-                             [&] { return launch_split_reduce(parts, splits, (int64_t)sub * ell, (int)sub, ell, ell, Z, ell, st); }));
-            }
+            ST_TRY(ensure(&h->zwork, &h->zwork_bytes, zred * splits));
+            CU_TRY(timed(h, K_PROJECT, 1, st, [&] {
+                return launch_gemm_nt(p + r0 * row_bytes, h->dtype, ld, S, h->pitch, (int)sub, ell, h->D, splits, h->zwork, ell,
+                                      (int64_t)sub * ell, st);
+            }));
+            Zparts = h->zwork;
+            nplanes = splits;
         }
-        const int64_t row = row_offset + r0;
-        CU_TRY(timed(h, K_NORMALISE, 2, st, [&] {
-            return launch_normalise(Z, ell, sub, ell, h->zhat + row * ell, h->znorm + row, h->partials, h->zsum, &h->info->flags, st);
+        // normalise (summing the K slices of the projection on the way), consensus partials, and in the third pass the scores
+        float* zh = store_at >= 0 ? h->zhat + (store_at + r0) * ell : h->zhat;
+        float* zn = store_at >= 0 ? h->znorm + (store_at + r0) : h->znorm;
+        CU_TRY(timed(h, K_NORMALISE, accumulate ? 2 : 1, st, [&] {
+            return launch_normalise(Zparts, nplanes, (int64_t)sub * ell, ell, sub, ell, zh, zn, h->partials, accumulate ? h->zsum : nullptr,
+                                    &h->info->flags, st);
         }));
+        if (scores_out)
+            CU_TRY(timed(h, K_SCORE, 1, st, [&] { return launch_consensus_score(h->zsum, zh, sub, ell, h->u, scores_out + r0, st); }));
     }
+    return SAGE_OK;
+}
+
+
+sage_status_t sage_score_chunk(sage_fd_t* h, const void* rows, int64_t n, int64_t ld, int64_t row_offset, void* cuda_stream) {
+    ST_TRY(check_handle(h));
+    if (h->state != SCORING) {
+        set_err("sage_score_chunk: no open scoring pass");
+        return SAGE_ERR_BAD_STATE;
+    }
+    if (n < 0 || (n > 0 && (!rows || ld < h->D)) || row_offset != h->next_row || row_offset + n > h->N_total) {
+        set_err("sage_score_chunk: bad argument (n=%lld ld=%lld offset=%lld expected offset=%lld N_total=%lld)", (long long)n,
+                (long long)ld, (long long)row_offset, (long long)h->next_row, (long long)h->N_total);
+        return SAGE_ERR_INVALID_ARG;
+    }
+    if (n == 0) return SAGE_OK;
+    DeviceGuard g(h->device);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    ST_TRY(score_rows(h, rows, n, ld, st, h->strict ? -1 : row_offset, true, nullptr));
     h->next_row += n;
     return SAGE_OK;
 }
@@ -1011,16 +1039,40 @@ sage_status_t sage_score_end(sage_fd_t* h, float* scores, void* cuda_stream) {
         set_err("sage_score_end: %lld of %lld rows were given", (long long)h->next_row, (long long)h->N_total);
         return SAGE_ERR_BAD_STATE;
     }
-    if (!scores && h->N_total > 0) {
+    if (!scores && h->N_total > 0 && !h->strict) {
         set_err("sage_score_end: null scores");
         return SAGE_ERR_INVALID_ARG;
     }
     DeviceGuard g(h->device);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    CU_TRY(timed(h, K_SCORE, 1, st, [&] { return launch_consensus_score(h->zsum, h->zhat, h->N_total, h->ell, h->u, scores, st); }));
-    h->scored = true;
+    if (h->strict) {     // only the consensus direction is formed here; the scores come from sage_score_apply
+        CU_TRY(timed(h, K_SCORE, 1, st, [&] { return launch_consensus_score(h->zsum, h->zhat, 0, h->ell, h->u, nullptr, st); }));
+        h->scored_strict = true;
+    } else {
+        CU_TRY(timed(h, K_SCORE, 1, st, [&] { return launch_consensus_score(h->zsum, h->zhat, h->N_total, h->ell, h->u, scores, st); }));
+        h->scored = true;
+    }
     h->state = FROZEN;
     return SAGE_OK;
+}
+
+sage_status_t sage_score_apply(sage_fd_t* h, const void* rows, int64_t n, int64_t ld, float* scores, void* cuda_stream) {
+    ST_TRY(check_handle(h));
+    if (h->state != FROZEN || !(h->scored || h->scored_strict)) {
+        set_err("sage_score_apply: needs a finished scoring pass (the consensus direction) on this handle");
+        return SAGE_ERR_BAD_STATE;
+    }
+    if (n < 0 || (n > 0 && (!rows || !scores || ld < h->D))) {
+        set_err("sage_score_apply: bad argument (n=%lld ld=%lld)", (long long)n, (long long)ld);
+        return SAGE_ERR_INVALID_ARG;
+    }
+    if (n == 0) return SAGE_OK;
+    if (h->scored) {     // the N x ell store of the finished pass must survive: this call works in a scratch of its own size class
+        set_err("sage_score_apply: the handle keeps the normalised projections of its last pass (option 8 is off); use sage_score");
+        return SAGE_ERR_BAD_STATE;
+    }
+    DeviceGuard g(h->device);
+    return score_rows(h, rows, n, ld, static_cast<cudaStream_t>(cuda_stream), -1, false, scores);
 }
 
 sage_status_t sage_score(sage_fd_t* h, const void* rows, int64_t n, int64_t ld, float* scores, void* cuda_stream) {
@@ -1037,8 +1089,8 @@ sage_status_t sage_score(sage_fd_t* h, const void* rows, int64_t n, int64_t ld, 
 
 sage_status_t sage_score_intermediates(const sage_fd_t* h, const float** zhat, const float** znorm, const float** u) {
     ST_TRY(check_handle(h));
-    if (h->state != FROZEN || !h->zhat) {
-        set_err("sage_score_intermediates: no finished scoring pass");
+    if (h->state != FROZEN || !h->zhat || !h->scored) {
+        set_err("sage_score_intermediates: no finished scoring pass that kept its projections");
         return SAGE_ERR_BAD_STATE;
     }
     if (zhat) *zhat = h->zhat;
@@ -1187,6 +1239,168 @@ sage_status_t sage_select_classes(const float* scores, const int32_t* labels, in
     if (k_per_class)
         for (int c = 0; c < C; ++c) k_per_class[c] = kc[c];
     if (k_out) *k_out = k;
+    return SAGE_OK;
+}
+
+// ---- checkpoint of the sketch state ---------------------------------------------------------------------------
+namespace {
+struct ExportHeader {
+    char magic[8];
+    int64_t D;
+    int32_t ell, dtype, P, frozen;
+    int64_t block, dealt;
+    int32_t nsk, delta_rank;
+};
+struct ExportSketch {
+    int32_t rows, pad;
+    EigInfo info;
+};
+const char kExportMagic[8] = {'S', 'A', 'G', 'E', 'F', 'D', '1', 0};
+
+int export_rows(const sage_fd* s, bool frozen) { return frozen ? s->ell : s->fill; }
+}  // namespace
+
+sage_status_t sage_fd_export_size(const sage_fd_t* h, size_t* bytes) {
+    ST_TRY(check_handle(h));
+    if (!bytes) {
+        set_err("sage_fd_export_size: null bytes");
+        return SAGE_ERR_INVALID_ARG;
+    }
+    if (h->state == SCORING) {
+        set_err("sage_fd_export_size: a scoring pass is open");
+        return SAGE_ERR_BAD_STATE;
+    }
+    const bool frozen = h->state == FROZEN;
+    size_t total = sizeof(ExportHeader);
+    const int nsk = frozen ? 1 : (int)h->kids.size() + 1;
+    for (int p = 0; p < nsk; ++p) {
+        const sage_fd* s = p == 0 ? h : h->kids[(size_t)p - 1];
+        total += sizeof(ExportSketch) + (size_t)export_rows(s, frozen) * h->D * sizeof(float);
+    }
+    if (frozen) total += (size_t)h->ell * sizeof(float);
+    *bytes = total;
+    return SAGE_OK;
+}
+
+sage_status_t sage_fd_export(sage_fd_t* h, void* dst_host, size_t capacity, size_t* written) {
+    size_t need = 0;
+    ST_TRY(sage_fd_export_size(h, &need));
+    if (!dst_host || capacity < need) {
+        set_err("sage_fd_export: destination of %zu bytes is too small (%zu needed)", capacity, need);
+        return SAGE_ERR_INVALID_ARG;
+    }
+    DeviceGuard g(h->device);
+    CU_TRY(cudaDeviceSynchronize());           // everything enqueued so far, on the caller's streams and the handle's own
+    const bool frozen = h->state == FROZEN;
+    char* out = static_cast<char*>(dst_host);
+    ExportHeader hd = {};
+    std::memcpy(hd.magic, kExportMagic, 8);
+    hd.D = h->D;
+    hd.ell = h->ell;
+    hd.dtype = (int32_t)h->dtype;
+    hd.P = h->P;
+    hd.frozen = frozen ? 1 : 0;
+    hd.block = h->block;
+    hd.dealt = h->dealt;
+    hd.nsk = frozen ? 1 : (int)h->kids.size() + 1;
+    hd.delta_rank = h->delta_rank;
+    std::memcpy(out, &hd, sizeof hd);
+    out += sizeof hd;
+    for (int p = 0; p < hd.nsk; ++p) {
+        sage_fd* s = sketch_at(h, p);
+        ExportSketch es = {};
+        es.rows = export_rows(s, frozen);
+        CU_TRY(cudaMemcpy(&es.info, s->info, sizeof(EigInfo), cudaMemcpyDeviceToHost));
+        if (frozen)                             // the counters of all sketches, as sage_fd_stats reports them
+            for (sage_fd* k : h->kids) {
+                EigInfo ki;
+                CU_TRY(cudaMemcpy(&ki, k->info, sizeof ki, cudaMemcpyDeviceToHost));
+                es.info.shrinks += ki.shrinks;
+                es.info.sum_delta += ki.sum_delta;
+                es.info.flags |= ki.flags;
+                if (ki.max_sweeps > es.info.max_sweeps) es.info.max_sweeps = ki.max_sweeps;
+            }
+        std::memcpy(out, &es, sizeof es);
+        out += sizeof es;
+        if (es.rows > 0)
+            CU_TRY(cudaMemcpy2D(out, (size_t)h->D * sizeof(float), s->B[s->cur], (size_t)s->pitch * sizeof(float),
+                                (size_t)h->D * sizeof(float), (size_t)es.rows, cudaMemcpyDeviceToHost));
+        out += (size_t)es.rows * h->D * sizeof(float);
+    }
+    if (frozen) {
+        CU_TRY(cudaMemcpy(out, h->sigma, (size_t)h->ell * sizeof(float), cudaMemcpyDeviceToHost));
+        out += (size_t)h->ell * sizeof(float);
+    }
+    if (written) *written = (size_t)(out - static_cast<char*>(dst_host));
+    return SAGE_OK;
+}
+
+sage_status_t sage_fd_import(sage_fd_t* h, const void* src_host, size_t bytes, void* cuda_stream) {
+    ST_TRY(check_handle(h));
+    ExportHeader hd;
+    if (!src_host || bytes < sizeof hd) {
+        set_err("sage_fd_import: no data");
+        return SAGE_ERR_INVALID_ARG;
+    }
+    std::memcpy(&hd, src_host, sizeof hd);
+    if (std::memcmp(hd.magic, kExportMagic, 8) != 0 || hd.D != h->D || hd.ell != h->ell || hd.dtype != (int32_t)h->dtype || hd.P < 1 ||
+        hd.P > 64 || hd.nsk < 1 || hd.nsk > hd.P || hd.block < 1 || hd.dealt < 0 || hd.delta_rank < 2 || hd.delta_rank > h->m - 1) {
+        set_err("sage_fd_import: not a checkpoint of a sketch with D=%lld ell=%d and this row type", (long long)h->D, h->ell);
+        return SAGE_ERR_INVALID_ARG;
+    }
+    // sizes first: nothing of the handle changes unless the whole checkpoint is consistent
+    {
+        const char* q = static_cast<const char*>(src_host) + sizeof hd;
+        size_t left = bytes - sizeof hd;
+        for (int p = 0; p < hd.nsk; ++p) {
+            ExportSketch es;
+            if (left < sizeof es) { set_err("sage_fd_import: truncated checkpoint"); return SAGE_ERR_INVALID_ARG; }
+            std::memcpy(&es, q, sizeof es);
+            const size_t rb = (size_t)(es.rows < 0 ? 0 : es.rows) * h->D * sizeof(float);
+            if (es.rows < 0 || es.rows >= h->m + (hd.frozen ? 1 : 0) || left < sizeof es + rb) {
+                set_err("sage_fd_import: truncated or inconsistent checkpoint");
+                return SAGE_ERR_INVALID_ARG;
+            }
+            q += sizeof es + rb;
+            left -= sizeof es + rb;
+        }
+        if (hd.frozen && left < (size_t)h->ell * sizeof(float)) { set_err("sage_fd_import: truncated checkpoint"); return SAGE_ERR_INVALID_ARG; }
+    }
+    DeviceGuard g(h->device);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    ST_TRY(sage_fd_reset(h));
+    ST_TRY(sage_fd_set_option(h, 6, (double)hd.P));
+    h->block = hd.block;
+    h->delta_rank = hd.delta_rank;
+    for (sage_fd* k : h->kids) k->delta_rank = hd.delta_rank;
+    if (hd.nsk > 1) ST_TRY(ensure_sketches(h));
+    const char* q = static_cast<const char*>(src_host) + sizeof hd;
+    for (int p = 0; p < hd.nsk; ++p) {
+        sage_fd* s = sketch_at(h, p);
+        s->delta_rank = hd.delta_rank;
+        ExportSketch es;
+        std::memcpy(&es, q, sizeof es);
+        q += sizeof es;
+        CU_TRY(cudaMemcpy(s->info, &es.info, sizeof(EigInfo), cudaMemcpyHostToDevice));
+        if (es.rows > 0)
+            CU_TRY(cudaMemcpy2D(s->B[0], (size_t)s->pitch * sizeof(float), q, (size_t)h->D * sizeof(float), (size_t)h->D * sizeof(float),
+                                (size_t)es.rows, cudaMemcpyHostToDevice));
+        if (s->pitch > h->D && es.rows > 0)     // columns between D and the pitch are zero in every buffer row
+            CU_TRY(cudaMemset2D(s->B[0] + h->D, (size_t)s->pitch * sizeof(float), 0, (size_t)(s->pitch - h->D) * sizeof(float), (size_t)es.rows));
+        q += (size_t)es.rows * h->D * sizeof(float);
+        s->cur = 0;
+        s->fill = hd.frozen ? h->ell : es.rows;
+    }
+    h->dealt = hd.dealt;
+    h->rows_seen = hd.dealt;
+    if (hd.frozen) {
+        CU_TRY(cudaMemcpy(h->sigma, q, (size_t)h->ell * sizeof(float), cudaMemcpyHostToDevice));
+        CU_TRY(cudaDeviceSynchronize());
+        ST_TRY(enqueue_freeze_aux(h, st));
+        h->state = FROZEN;
+    } else {
+        CU_TRY(cudaDeviceSynchronize());
+    }
     return SAGE_OK;
 }
 

@@ -99,10 +99,11 @@ cudaError_t launch_eig_shrink(const float* K, int ldk, int n, int do_shrink, int
                               int ldu, float* sigma_out, int n_sigma, float* work, int max_sweeps, EigInfo* info,
                               float* Wsplit, int ldw, int j_pad, int variant, cudaStream_t st);
 
-// Z (n x ell, pitch ldz, already reduced over splits) -> zhat rows, ||z|| and per-block partial sums of zhat.
-// zsum (ell doubles) += the partial sums in ascending block order (done by a second, single-block kernel).
-cudaError_t launch_normalise(const float* Z, int64_t ldz, int64_t n, int ell, float* zhat, float* znorm,
-                             float* partials, double* zsum, unsigned* flags, cudaStream_t st);
+// Z (n x ell, pitch ldz; planes > 1: that many partial planes plane_stride floats apart, summed in plane order with fp64
+// accumulation) -> zhat rows, ||z|| and per-block partial sums of zhat. zsum (ell doubles, may be null) += the partial sums in
+// a fixed order (done by a second, single-block kernel).
+cudaError_t launch_normalise(const float* Z, int planes, int64_t plane_stride, int64_t ldz, int64_t n, int ell, float* zhat,
+                             float* znorm, float* partials, double* zsum, unsigned* flags, cudaStream_t st);
 
 // u = zsum/||zsum|| (0 if zsum = 0); scores[i] = <zhat_i, u>.
 cudaError_t launch_consensus_score(const double* zsum, const float* zhat, int64_t N, int ell, float* u, float* scores,

@@ -11,8 +11,10 @@ constexpr int kRowsPerBlock = 64;   // rows whose zhat are summed into one parti
 constexpr int kMaxPerLane = 8;      // ell <= 256
 
 // One warp per row, 8 warps per block, each warp walks rows w, w+8, ... of the block's 64 rows.
-__global__ void __launch_bounds__(256) k_normalise(const float* __restrict__ Z, int64_t ldz, int64_t n, int ell,
-                                                   float* __restrict__ zhat, float* __restrict__ znorm,
+// planes > 1: the projections arrive as that many partial planes (K slices of the projection, `plane_stride` floats apart),
+// which are summed here in ascending plane order with fp64 accumulation before the row is normalised.
+__global__ void __launch_bounds__(256) k_normalise(const float* __restrict__ Z, int planes, int64_t plane_stride, int64_t ldz, int64_t n,
+                                                   int ell, float* __restrict__ zhat, float* __restrict__ znorm,
                                                    float* __restrict__ partials, unsigned* __restrict__ flags) {
     __shared__ float part[8][256];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -30,7 +32,25 @@ __global__ void __launch_bounds__(256) k_normalise(const float* __restrict__ Z, 
 #pragma unroll
         for (int t = 0; t < kMaxPerLane; ++t) {
             const int j = lane + 32 * t;
-            z[t] = (j < ell) ? Z[row * ldz + j] : 0.f;
+            if (j >= ell) {
+                z[t] = 0.f;
+            } else if (planes == 1) {
+                z[t] = Z[row * ldz + j];
+            } else {
+                const float* src = Z + row * ldz + j;
+                double acc = 0.0;
+                int pz = 0;
+                for (; pz + 4 <= planes; pz += 4) {      // four loads in flight, added in plane order
+                    const float a0 = src[(int64_t)pz * plane_stride], a1 = src[(int64_t)(pz + 1) * plane_stride];
+                    const float a2 = src[(int64_t)(pz + 2) * plane_stride], a3 = src[(int64_t)(pz + 3) * plane_stride];
+                    acc += (double)a0;
+                    acc += (double)a1;
+                    acc += (double)a2;
+                    acc += (double)a3;
+                }
+                for (; pz < planes; ++pz) acc += (double)src[(int64_t)pz * plane_stride];
+                z[t] = (float)acc;
+            }
             finite = finite && (fabsf(z[t]) <= 3.0e38f);   // false for NaN and Inf
             amax = fmaxf(amax, fabsf(z[t]));
         }
@@ -74,13 +94,24 @@ __global__ void __launch_bounds__(256) k_normalise(const float* __restrict__ Z, 
     if (bad && lane == 0) atomicOr(flags, kFlagNonFinite);
 }
 
-__global__ void __launch_bounds__(256) k_accumulate(const float* __restrict__ partials, int nblocks, int ell,
-                                                    double* __restrict__ zsum) {
-    const int j = threadIdx.x;
-    if (j >= ell) return;
-    double s = zsum[j];
-    for (int b = 0; b < nblocks; ++b) s += (double)partials[(int64_t)b * ell + j];
-    zsum[j] = s;
+// zsum[j] += sum over blocks b of partials[b][j], in a fixed order: the 1024 threads form 1024 / jw groups (jw = ell rounded up to
+// a power of two, at least 32); group g adds the partials of blocks g, g + G, g + 2G, ... in ascending order in fp64, and the
+// groups' sums are then added in ascending g.
+__global__ void __launch_bounds__(1024) k_accumulate(const float* __restrict__ partials, int nblocks, int ell, int jw,
+                                                     double* __restrict__ zsum) {
+    __shared__ double sh[1024];
+    const int G = 1024 / jw;
+    const int j = threadIdx.x % jw, g = threadIdx.x / jw;
+    double s = 0.0;
+    if (j < ell)
+        for (int b = g; b < nblocks; b += G) s += (double)partials[(int64_t)b * ell + j];
+    sh[threadIdx.x] = s;
+    __syncthreads();
+    if (g == 0 && j < ell) {
+        double t = zsum[j];
+        for (int q = 0; q < G; ++q) t += sh[q * jw + j];
+        zsum[j] = t;
+    }
 }
 
 // u = zsum/||zsum|| (the 1/N of the mean cancels); alpha_i = <zhat_i, u>. One warp per row.
@@ -114,14 +145,16 @@ __global__ void __launch_bounds__(256) k_consensus_score(const double* __restric
 
 }  // namespace
 
-cudaError_t launch_normalise(const float* Z, int64_t ldz, int64_t n, int ell, float* zhat, float* znorm, float* partials,
-                             double* zsum, unsigned* flags, cudaStream_t st) {
+cudaError_t launch_normalise(const float* Z, int planes, int64_t plane_stride, int64_t ldz, int64_t n, int ell, float* zhat,
+                             float* znorm, float* partials, double* zsum, unsigned* flags, cudaStream_t st) {
     if (n <= 0) return cudaSuccess;
     const int nblocks = (int)((n + kRowsPerBlock - 1) / kRowsPerBlock);
-    k_normalise<<<nblocks, 256, 0, st>>>(Z, ldz, n, ell, zhat, znorm, partials, flags);
+    k_normalise<<<nblocks, 256, 0, st>>>(Z, planes, plane_stride, ldz, n, ell, zhat, znorm, partials, flags);
     cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    k_accumulate<<<1, 256, 0, st>>>(partials, nblocks, ell, zsum);
+    if (e != cudaSuccess || !zsum) return e;
+    int jw = 32;
+    while (jw < ell) jw <<= 1;
+    k_accumulate<<<1, 1024, 0, st>>>(partials, nblocks, ell, jw, zsum);
     return cudaGetLastError();
 }
 

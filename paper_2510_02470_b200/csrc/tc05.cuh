@@ -73,12 +73,6 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* t
                  "l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(bar)), "r"(x), "r"(y)
                  : "memory");
 }
-// The same tile brought into L2 only (no shared memory, no completion to wait for): issued some tiles ahead of the
-// loads, it keeps more bytes in flight from HBM than the shared-memory stages alone can hold.
-__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* tmap, int x, int y) {
-    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];" ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y)
-                 : "memory");
-}
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* tmap) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tmap)) : "memory");
 }
@@ -194,8 +188,6 @@ __host__ __device__ inline uint32_t instr_desc(int fmt, int M, int N, int a_mn, 
 // with the 128-byte swizzle (atom32 != 0: its 32-byte-atom variant, for MN-major fp32 operands). elem_bytes 2
 // (bf16) or 4 (fp32). Returns false when TMA's alignment rules do not hold (base 16-byte aligned, pitch a
 // multiple of 16 bytes) or the driver refuses.
-// Tiles the producers prefetch into L2 ahead of their loads (0 = none).
-int prefetch_distance();
 bool make_tmap_2d(CUtensorMap* out, const void* base, int elem_bytes, uint64_t rows, uint64_t cols, uint64_t ld,
                   uint32_t box_rows, int atom32 = 0);
 

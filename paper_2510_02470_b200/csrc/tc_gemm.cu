@@ -9,21 +9,11 @@
 //   warps 2-5 read the fp32 accumulators out of TMEM (one row per thread) and store the partial result.
 // Rows and K elements outside the matrices are zero-filled by TMA, so no tail code exists. Split-K
 // partials are summed by a separate kernel in a fixed order.
-#include <cstdlib>
-
 #include "sage_internal.h"
 #include "tc05.cuh"
 
 namespace sage {
 namespace tc {
-
-int prefetch_distance() {
-    static int d = [] {
-        const char* e = getenv("SAGE_PF");
-        return e ? atoi(e) : 0;
-    }();
-    return d;
-}
 
 bool make_tmap_2d(CUtensorMap* out, const void* base, int elem_bytes, uint64_t rows, uint64_t cols, uint64_t ld,
                   uint32_t box_rows, int atom32) {
@@ -62,7 +52,7 @@ template <int kFmt>
 __global__ void __launch_bounds__(kThreads, 1)
 k_tc_gemm_nt(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, int M, int N, int n_pad, int fold,
              int mt, long long K, long long k_per_split, float* __restrict__ C, long long ldc, long long split_stride, int stages,
-             uint32_t tmem_cols, int pf, int* __restrict__ err) {
+             uint32_t tmem_cols, int* __restrict__ err) {
     constexpr int BK = kFmt == 1 ? 64 : 32;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -105,11 +95,6 @@ k_tc_gemm_nt(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             for (int kt = 0; kt < nkt; ++kt) {
                 const int s = kt % stages;
                 const uint32_t use = (uint32_t)(kt / stages);
-                if (pf > 0 && kt + pf < nkt) {
-                    const int xp = (int)(k_begin + (long long)(kt + pf) * BK);
-                    for (int t = 0; t < mt; ++t)
-                        if (m0 + t * kTileM < M) tma_prefetch_2d(&tmA, xp, m0 + t * kTileM);
-                }
                 if (!mbar_wait(&empty[s], (use & 1u) ^ 1u, abort)) break;
                 mbar_expect_tx(&full[s], tx_bytes);
                 const int x = (int)(k_begin + (long long)kt * BK);
@@ -227,12 +212,12 @@ cudaError_t launch_tc_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const
         e = cudaFuncSetAttribute(tc::k_tc_gemm_nt<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         tc::k_tc_gemm_nt<1><<<grid, tc::kThreads, smem, st>>>(tmA, tmB, M, N, n_pad, fold, mt, K, kps, C, ldc, split_stride, stages,
-                                                              tmem_cols, tc::prefetch_distance(), err);
+                                                              tmem_cols, err);
     } else {
         e = cudaFuncSetAttribute(tc::k_tc_gemm_nt<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         tc::k_tc_gemm_nt<2><<<grid, tc::kThreads, smem, st>>>(tmA, tmB, M, N, n_pad, fold, mt, K, kps, C, ldc, split_stride, stages,
-                                                              tmem_cols, tc::prefetch_distance(), err);
+                                                              tmem_cols, err);
     }
     return cudaGetLastError();
 }

@@ -62,7 +62,7 @@ __device__ __forceinline__ uint4 lo4(const uint4 v, float scale) {
 __global__ void __launch_bounds__(kThreads, 1)
 k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, int M, int N, int gram,
                 int b_box_rows, int sym, long long K, long long k_per_split, float* __restrict__ C, long long ldc, long long split_stride,
-                int stages, int stage_bytes, int pf, int* __restrict__ err) {
+                int stages, int stage_bytes, int* __restrict__ err) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     const int m0 = blockIdx.x * kTileM, n0 = blockIdx.y * kTileN;
@@ -119,11 +119,6 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             for (int kt = 0; kt < nkt; ++kt) {
                 const int s = kt % stages;
                 const uint32_t use = (uint32_t)(kt / stages);
-                if (pf > 0 && kt + pf < nkt) {
-                    const int xp = (int)(k_begin + (long long)(kt + pf) * BK);
-                    tma_prefetch_2d(&tmA, xp, m0);
-                    if (!proj && !diag) tma_prefetch_2d(&tmB, xp, n0);
-                }
                 if (!mbar_wait(&empty[s], (use & 1u) ^ 1u, abort)) break;
                 mbar_expect_tx(&full[s], (uint32_t)(proj ? 2 * kTileBytes : half_bytes));
                 const int x = (int)(k_begin + (long long)kt * BK);
@@ -326,7 +321,7 @@ cudaError_t launch_tc_gemm_nt_x3(const float* A, int64_t lda, const float* Bm, i
     cudaError_t e = cudaFuncSetAttribute(tc::k_tc_gemm_nt_x3, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     tc::k_tc_gemm_nt_x3<<<grid, tc::kThreads, smem, st>>>(tmA, tmB, M, N, gram, b_box_rows, sym, K, kps, C, ldc, split_stride, stages,
-                                                                 stage_bytes, tc::prefetch_distance(), err);
+                                                                 stage_bytes, err);
     return cudaGetLastError();
 }
 

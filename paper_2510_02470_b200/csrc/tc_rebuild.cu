@@ -34,7 +34,7 @@ constexpr int kSpanBytes = kChunkRows * 128;         // 4 KB
 
 __global__ void __launch_bounds__(kThreads, 1)
 k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ CUtensorMap tmW, int r, int keep, int j_pad,
-             long long pitch, long long num_tiles, float* __restrict__ out, int stages, int pf, int* __restrict__ err) {
+             long long pitch, long long num_tiles, float* __restrict__ out, int stages, int* __restrict__ err) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     // stage layout: [buffer hi 16 KB][buffer lo 16 KB][W_hi ; W_lo: 2*j_pad rows of 128 bytes]
@@ -87,16 +87,6 @@ k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ 
                 for (int c = 0; c < nchunk; ++c, ++q) {
                     const int s = (int)(q % stages);
                     const uint32_t use = (uint32_t)(q / stages);
-                    if (pf > 0) {                      // the chunk pf steps ahead, possibly in a later tile of this CTA
-                        long long lt2 = lt;
-                        int c2 = c + pf;
-                        while (c2 >= nchunk) { c2 -= nchunk; ++lt2; }
-                        if (lt2 < my_tiles) {
-                            const long long dp = (blockIdx.x + lt2 * gridDim.x) * kTileD;
-#pragma unroll
-                            for (int sp = 0; sp < 4; ++sp) tma_prefetch_2d(&tmBuf, (int)(dp + 32 * sp), c2 * kChunkRows);
-                        }
-                    }
                     if (!mbar_wait(&empty[s], (use & 1u) ^ 1u, abort)) { alive = false; break; }
                     mbar_expect_tx(&full[s], (uint32_t)(kBufBytes + w_bytes));
                     uint8_t* st = smem + (size_t)s * stage_bytes;
@@ -238,7 +228,7 @@ static cudaError_t launch_tc_rebuild_part(const float* Wsplit, int ldw, int j_pa
     const int grid = (int)(num_tiles < 148 ? num_tiles : 148);
     cudaError_t e = cudaFuncSetAttribute(tc::k_tc_rebuild, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    tc::k_tc_rebuild<<<grid, tc::kThreads, smem, st>>>(tmBuf, tmW, r, keep, j_pad, pitch, num_tiles, Bdst, stages, tc::prefetch_distance(), err);
+    tc::k_tc_rebuild<<<grid, tc::kThreads, smem, st>>>(tmBuf, tmW, r, keep, j_pad, pitch, num_tiles, Bdst, stages, err);
     return cudaGetLastError();
 }
 
