@@ -30,6 +30,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# The merged form of pass 1 runs one stream per sketch; CUDA gives every stream a hardware queue of its own only up to this
+# number (default 8). It is read when CUDA is initialised, so it has to be set before torch touches the device.
+os.environ.setdefault("CUDA_DEVICE_MAX_CONNECTIONS", "32")
+
 import torch  # noqa: E402
 
 METRIC = "gradient rows/s (FD sketch + agreement scoring + top-k, whole path)"

@@ -125,6 +125,24 @@ sage_status_t sage_score_chunk(sage_fd_t* h, const void* rows, int64_t n, int64_
                                void* cuda_stream);
 sage_status_t sage_score_end(sage_fd_t* h, float* scores, void* cuda_stream);
 
+/* Structured last-layer rows (Method, the definition of the per-example gradient; Limitations, on last-layer gradients).
+ * For a softmax head with C classes on F features the per-example gradient with respect to (weights, bias) is the outer
+ * product q_i (x) [h_i ; 1], q_i = softmax - onehot(label): row i is [vec_rowmajor(q_i h_i^T) (C x F) ; q_i (C)], D = C F + C.
+ * These entry points take the two factors instead of the row, so the N x D matrix is never formed in the caller's memory
+ * nor read from HBM: pass 1 writes each row straight into the sketch buffer, pass 2 expands a sub-chunk of rows at a time
+ * into a scratch that stays in L2 and projects it from there. Results are those of sage_fd_update / sage_score_chunk /
+ * sage_score on the materialised rows (products taken in fp32, exact for bfloat16 factors); both kinds of call may be
+ * mixed on one handle.
+ *   q     device, n x ldq elements of the handle's row dtype, C values used per row (ldq >= C).
+ *   feat  device, n x ldf elements of the handle's row dtype, F values used per row (ldf >= F).
+ * C F + C must equal the handle's D. Stream semantics, state machine and errors are those of the dense calls. */
+sage_status_t sage_fd_update_outer(sage_fd_t* h, const void* q, int64_t ldq, const void* feat, int64_t ldf, int64_t n, int32_t C, int32_t F,
+                                   void* cuda_stream);
+sage_status_t sage_score_chunk_outer(sage_fd_t* h, const void* q, int64_t ldq, const void* feat, int64_t ldf, int64_t n, int32_t C,
+                                     int32_t F, int64_t row_offset, void* cuda_stream);
+sage_status_t sage_score_outer(sage_fd_t* h, const void* q, int64_t ldq, const void* feat, int64_t ldf, int64_t n, int32_t C, int32_t F,
+                               float* scores, void* cuda_stream);
+
 /* Strict-memory form of Phase II (Method, the complexity paragraph and the abstract: memory O(ell D), independent of N).
  * The default keeps the N x ell normalised projections between the scoring pass and its end, because alpha_i needs the
  * consensus u, which needs every row. With option 8 set to 1 nothing of size N is kept: sage_score_begin / _chunk / _end
@@ -251,7 +269,9 @@ sage_status_t sage_fd_stats(sage_fd_t* h, sage_stats_t* out);
  * freezes every sketch and merges them pairwise (sketch a absorbs sketch a + s for s = 1, 2, 4, ...: the rows a + s
  * kept are appended to a, which is frozen again). Frequent-Directions sketches are mergeable, so the result obeys
  * the same error bound as the sequential sketch, but it is a different sketch. The P chains of Gram / eigen-solve /
- * rebuild run on P streams of the library's own and overlap on the device; device memory grows P-fold.
+ * rebuild run on P streams of the library's own and overlap on the device; device memory grows P-fold. (CUDA maps streams onto
+ * a limited number of hardware queues, 8 unless the environment variable CUDA_DEVICE_MAX_CONNECTIONS says otherwise when CUDA
+ * is initialised; streams that share a queue do not overlap, so with P > 8 set it to 32 before the process touches CUDA.)
  * Outside a scoring pass: key 8 = 1 for the strict-memory form of Phase II (see sage_score_apply), 0 (default) to keep the
  * N x ell normalised projections. */
 sage_status_t sage_fd_set_option(sage_fd_t* h, int key, double value);

@@ -38,6 +38,9 @@ SIGNATURES = {
     "sage_score_chunk": (_i32, [_vp, _vp, _i64, _i64, _i64, _vp]),
     "sage_score_end": (_i32, [_vp, _vp, _vp]),
     "sage_score_apply": (_i32, [_vp, _vp, _i64, _i64, _vp, _vp]),
+    "sage_fd_update_outer": (_i32, [_vp, _vp, _i64, _vp, _i64, _i64, _i32, _i32, _vp]),
+    "sage_score_chunk_outer": (_i32, [_vp, _vp, _i64, _vp, _i64, _i64, _i32, _i32, _i64, _vp]),
+    "sage_score_outer": (_i32, [_vp, _vp, _i64, _vp, _i64, _i64, _i32, _i32, _vp, _vp]),
     "sage_score_intermediates": (_i32, [_vp, _vp, _vp, _vp]),
     "sage_fd_export_size": (_i32, [_vp, _vp]),
     "sage_fd_export": (_i32, [_vp, _vp, C.c_size_t, _vp]),
@@ -180,6 +183,29 @@ def sage_score_end(h: int, scores: Optional[torch.Tensor], device=None) -> None:
         return
     assert scores.dtype == torch.float32 and scores.is_contiguous()
     _check(lib().sage_score_end(h, scores.data_ptr(), _stream(scores.device)))
+
+
+def _outer_args(q: torch.Tensor, feat: torch.Tensor, C: int, F: int):
+    assert q.dim() == 2 and feat.dim() == 2 and q.shape[0] == feat.shape[0] and q.dtype == feat.dtype
+    assert q.shape[1] >= C and feat.shape[1] >= F and q.stride(1) == 1 and feat.stride(1) == 1
+    n = q.shape[0]
+    return q.data_ptr(), (q.stride(0) if n > 1 else q.shape[1]), feat.data_ptr(), (feat.stride(0) if n > 1 else feat.shape[1]), n
+
+
+def sage_fd_update_outer(h: int, q: torch.Tensor, feat: torch.Tensor, C: int, F: int) -> None:
+    qp, ldq, fp, ldf, n = _outer_args(q, feat, C, F)
+    _check(lib().sage_fd_update_outer(h, qp, ldq, fp, ldf, n, C, F, _stream(q.device)))
+
+
+def sage_score_chunk_outer(h: int, q: torch.Tensor, feat: torch.Tensor, C: int, F: int, row_offset: int) -> None:
+    qp, ldq, fp, ldf, n = _outer_args(q, feat, C, F)
+    _check(lib().sage_score_chunk_outer(h, qp, ldq, fp, ldf, n, C, F, row_offset, _stream(q.device)))
+
+
+def sage_score_outer(h: int, q: torch.Tensor, feat: torch.Tensor, C: int, F: int, scores: torch.Tensor) -> None:
+    qp, ldq, fp, ldf, n = _outer_args(q, feat, C, F)
+    assert scores.dtype == torch.float32 and scores.is_contiguous() and scores.numel() >= n
+    _check(lib().sage_score_outer(h, qp, ldq, fp, ldf, n, C, F, scores.data_ptr(), _stream(q.device)))
 
 
 def sage_score_apply(h: int, rows: torch.Tensor, D: int, scores: torch.Tensor) -> None:
@@ -351,6 +377,18 @@ class SageFD:
             scores = torch.empty((rows.shape[0],), dtype=torch.float32, device=rows.device)
         sage_score(self._h, rows, self.D, scores)
         return scores
+
+    def update_outer(self, q: torch.Tensor, feat: torch.Tensor, C: int, F: int) -> None:
+        sage_fd_update_outer(self._h, q, feat, C, F)
+
+    def score_outer(self, q: torch.Tensor, feat: torch.Tensor, C: int, F: int, scores: Optional[torch.Tensor] = None) -> torch.Tensor:
+        if scores is None:
+            scores = torch.empty((q.shape[0],), dtype=torch.float32, device=q.device)
+        sage_score_outer(self._h, q, feat, C, F, scores)
+        return scores
+
+    def score_chunk_outer(self, q: torch.Tensor, feat: torch.Tensor, C: int, F: int, row_offset: int) -> None:
+        sage_score_chunk_outer(self._h, q, feat, C, F, row_offset)
 
     def score_begin(self, N_total: int) -> None:
         sage_score_begin(self._h, N_total, self.device)

@@ -158,6 +158,8 @@ struct sage_fd {
     double* zsum = nullptr;
     float* u = nullptr;
     bool scored = false;           // a scoring pass over N_total rows has finished: zhat holds their normalised projections
+    float* xwork = nullptr;        // structured rows expanded a sub-chunk at a time for the scoring pass (fp32, pitch D rounded up to 4)
+    size_t xwork_bytes = 0;
     bool strict = false;           // option 8: no N x ell store; scores come from a third pass (sage_score_apply)
     bool scored_strict = false;    // the finished pass ran in strict-memory mode: u is known, zhat is not kept
     float* class_U = nullptr;      // class-balanced variant: unit centroids (class_cap x ell) and class sizes
@@ -502,6 +504,7 @@ void sage_fd_destroy(sage_fd_t* h) {
     cudaFree(h->znorm);
     cudaFree(h->zwork);
     cudaFree(h->partials);
+    cudaFree(h->xwork);
     cudaFree(h->zsum);
     cudaFree(h->u);
     cudaFree(h->class_U);
@@ -630,36 +633,62 @@ static sage_status_t sketch_factor(sage_fd* s, int r, int do_shrink, int keep, i
     return SAGE_OK;
 }
 
+// Where the rows of an update come from: a dense matrix (rows, pitch ld), or the two factors of structured last-layer
+// rows (q: pitch ldq, C values per row; feat: pitch ldf, F values per row), expanded on the fly.
+struct RowSrc {
+    const void* rows = nullptr;
+    int64_t ld = 0;
+    const void* q = nullptr;
+    const void* feat = nullptr;
+    int64_t ldq = 0, ldf = 0;
+    int C = 0, F = 0;
+    sage_dtype_t dt = SAGE_F32;
+    bool outer() const { return q != nullptr; }
+    RowSrc advanced(int64_t k) const {       // the same source, k rows further on
+        RowSrc r = *this;
+        const size_t es = elem_size(dt);
+        if (rows) r.rows = static_cast<const char*>(rows) + (size_t)k * ld * es;
+        if (q) r.q = static_cast<const char*>(q) + (size_t)k * ldq * es;
+        if (feat) r.feat = static_cast<const char*>(feat) + (size_t)k * ldf * es;
+        return r;
+    }
+    cudaError_t append(int64_t take, int64_t D, float* B, int64_t pitch, int dst_row0, cudaStream_t st) const {
+        if (outer()) return launch_append_outer(q, ldq, feat, ldf, dt, take, C, F, B, pitch, dst_row0, st);
+        return launch_append(rows, dt, take, ld, D, B, pitch, dst_row0, st);
+    }
+};
+
 // Appends n rows of type dt and shrinks whenever the buffer fills. e_in (may be null): the event after which `rows`
 // are valid; epoch identifies the update call it belongs to. on_chain: appends run on the chain stream itself (used
 // where the rows to append are produced by that stream). Leaves s->ev_rows recorded after the last append.
-static sage_status_t sketch_feed(sage_fd* s, const void* rows, sage_dtype_t dt, int64_t n, int64_t ld, cudaStream_t chain,
-                                 cudaEvent_t e_in, int64_t epoch, bool on_chain) {
+static sage_status_t sketch_feed(sage_fd* s, RowSrc src, int64_t n, cudaStream_t chain, cudaEvent_t e_in, int64_t epoch, bool on_chain) {
+    // merged form: the appends run on the chain stream too (the chains of the other sketches fill the device while this
+    // one waits, and half as many streams keep every chain on a hardware queue of its own)
+    const bool from_caller = !on_chain;
+    if (s->chain && chain == s->chain) on_chain = true;
     cudaStream_t as = on_chain ? chain : s->side;
-    if (!on_chain && e_in && s->in_epoch != epoch) {
+    if (from_caller && e_in && s->in_epoch != epoch) {
         CU_TRY(cudaStreamWaitEvent(as, e_in, 0));
         s->in_epoch = epoch;
     }
-    const char* p = static_cast<const char*>(rows);
-    const size_t row_bytes = (size_t)ld * elem_size(dt);
     bool appended = false;
     auto body = [&]() -> sage_status_t {
         while (n > 0) {
             const int64_t room = s->m - s->fill;
             const int64_t take = n < room ? n : room;
-            CU_TRY(timed(s, K_APPEND, 1, as, [&] { return launch_append(p, dt, take, ld, s->D, s->B[s->cur], s->pitch, s->fill, as); }));
+            CU_TRY(timed(s, K_APPEND, 1, as, [&] { return src.append(take, s->D, s->B[s->cur], s->pitch, s->fill, as); }));
             appended = true;
             if (!on_chain) s->app_pending = true;
             s->fill += (int)take;
             s->rows_seen += take;
-            p += take * row_bytes;
+            src = src.advanced(take);
             n -= take;
             if (s->fill == s->m) ST_TRY(sketch_factor(s, s->m, 1, s->delta_rank - 1, 0, chain));
         }
         return SAGE_OK;
     };
     const sage_status_t rc = body();
-    if (appended && !on_chain) {     // also on the error path: the caller's stream must not run ahead of appends that read `rows`
+    if (appended && from_caller) {   // also on the error path: the caller's stream must not run ahead of appends that read `rows`
         const cudaError_t e = cudaEventRecord(s->ev_rows, as);
         if (rc == SAGE_OK) CU_TRY(e);
         s->used = true;
@@ -705,39 +734,28 @@ static sage_status_t ensure_sketches(sage_fd* h) {
     return SAGE_OK;
 }
 
-sage_status_t sage_fd_update(sage_fd_t* h, const void* rows, int64_t n, int64_t ld, void* cuda_stream) {
-    ST_TRY(check_handle(h));
-    if (n < 0 || (n > 0 && (!rows || ld < h->D))) {
-        set_err("sage_fd_update: bad argument (rows=%p n=%lld ld=%lld D=%lld)", rows, (long long)n, (long long)ld, (long long)h->D);
-        return SAGE_ERR_INVALID_ARG;
-    }
-    if (h->state != SKETCHING) {
-        set_err("sage_fd_update: the sketch is frozen (call sage_fd_reset to start over)");
-        return SAGE_ERR_BAD_STATE;
-    }
-    if (n == 0) return SAGE_OK;
+// Algorithm 1, Phase I for n rows from `src` (dense rows or the factors of structured rows): shared by sage_fd_update and
+// sage_fd_update_outer.
+static sage_status_t update_from(sage_fd* h, RowSrc src, int64_t n, cudaStream_t st) {
     DeviceGuard g(h->device);
-    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     ST_TRY(ensure_sketches(h));
     static std::atomic<long long> epochs{0};
     const int64_t epoch = epochs.fetch_add(1) + 1;
     CU_TRY(cudaEventRecord(h->ev_in, st));
     sage_status_t rc = SAGE_OK;
     if (h->P == 1) {
-        rc = sketch_feed(h, rows, h->dtype, n, ld, st, h->ev_in, epoch, false);
+        rc = sketch_feed(h, src, n, st, h->ev_in, epoch, false);
         h->dealt += n;
     } else {
         // block b of the row stream (counted over all calls) goes to sketch b mod P
-        const char* p = static_cast<const char*>(rows);
-        const size_t row_bytes = (size_t)ld * elem_size(h->dtype);
         while (n > 0 && rc == SAGE_OK) {
             const int64_t b = h->dealt / h->block;
             const int64_t left_in_block = (b + 1) * h->block - h->dealt;
             const int64_t take = n < left_in_block ? n : left_in_block;
             sage_fd* s = sketch_at(h, (int)(b % h->P));
-            rc = sketch_feed(s, p, h->dtype, take, ld, s->chain, h->ev_in, epoch, false);
+            rc = sketch_feed(s, src, take, s->chain, h->ev_in, epoch, false);
             h->dealt += take;
-            p += take * row_bytes;
+            src = src.advanced(take);
             n -= take;
         }
     }
@@ -751,6 +769,58 @@ sage_status_t sage_fd_update(sage_fd_t* h, const void* rows, int64_t n, int64_t 
         }
     }
     return rc;
+}
+
+sage_status_t sage_fd_update(sage_fd_t* h, const void* rows, int64_t n, int64_t ld, void* cuda_stream) {
+    ST_TRY(check_handle(h));
+    if (n < 0 || (n > 0 && (!rows || ld < h->D))) {
+        set_err("sage_fd_update: bad argument (rows=%p n=%lld ld=%lld D=%lld)", rows, (long long)n, (long long)ld, (long long)h->D);
+        return SAGE_ERR_INVALID_ARG;
+    }
+    if (h->state != SKETCHING) {
+        set_err("sage_fd_update: the sketch is frozen (call sage_fd_reset to start over)");
+        return SAGE_ERR_BAD_STATE;
+    }
+    if (n == 0) return SAGE_OK;
+    RowSrc src;
+    src.rows = rows;
+    src.ld = ld;
+    src.dt = h->dtype;
+    return update_from(h, src, n, static_cast<cudaStream_t>(cuda_stream));
+}
+
+// Checks the arguments of the entry points that take structured last-layer rows.
+static sage_status_t check_outer(const sage_fd* h, const char* who, const void* q, int64_t ldq, const void* feat, int64_t ldf, int64_t n,
+                                 int32_t C, int32_t F) {
+    if (C < 1 || F < 1 || (int64_t)C * F + C != h->D) {
+        set_err("%s: C=%d classes x F=%d features + C biases is not the handle's row dimension D=%lld", who, (int)C, (int)F, (long long)h->D);
+        return SAGE_ERR_INVALID_ARG;
+    }
+    if (n < 0 || (n > 0 && (!q || !feat || ldq < C || ldf < F))) {
+        set_err("%s: bad argument (q=%p ldq=%lld feat=%p ldf=%lld n=%lld)", who, q, (long long)ldq, feat, (long long)ldf, (long long)n);
+        return SAGE_ERR_INVALID_ARG;
+    }
+    return SAGE_OK;
+}
+
+sage_status_t sage_fd_update_outer(sage_fd_t* h, const void* q, int64_t ldq, const void* feat, int64_t ldf, int64_t n, int32_t C, int32_t F,
+                                   void* cuda_stream) {
+    ST_TRY(check_handle(h));
+    ST_TRY(check_outer(h, "sage_fd_update_outer", q, ldq, feat, ldf, n, C, F));
+    if (h->state != SKETCHING) {
+        set_err("sage_fd_update_outer: the sketch is frozen (call sage_fd_reset to start over)");
+        return SAGE_ERR_BAD_STATE;
+    }
+    if (n == 0) return SAGE_OK;
+    RowSrc src;
+    src.q = q;
+    src.ldq = ldq;
+    src.feat = feat;
+    src.ldf = ldf;
+    src.C = C;
+    src.F = F;
+    src.dt = h->dtype;
+    return update_from(h, src, n, static_cast<cudaStream_t>(cuda_stream));
 }
 
 // Makes `cuda_stream` wait for everything the handle has enqueued on streams of its own.
@@ -792,7 +862,13 @@ sage_status_t sage_fd_finalize(sage_fd_t* h, void* cuda_stream) {
                 CU_TRY(cudaEventRecord(Bs->ev_done, Bs->chain));
                 CU_TRY(cudaStreamWaitEvent(A->chain, Bs->ev_done, 0));
                 if (Bs->fill > 0)
-                    ST_TRY(sketch_feed(A, Bs->B[Bs->cur], SAGE_F32, Bs->fill, Bs->pitch, A->chain, nullptr, 0, true));
+                {
+                    RowSrc kept;
+                    kept.rows = Bs->B[Bs->cur];
+                    kept.ld = Bs->pitch;
+                    kept.dt = SAGE_F32;
+                    ST_TRY(sketch_feed(A, kept, Bs->fill, A->chain, nullptr, 0, true));
+                }
                 ST_TRY(sketch_freeze(A, A->chain));
             }
     }
@@ -903,19 +979,19 @@ sage_status_t sage_score_begin(sage_fd_t* h, int64_t N_total, void* cuda_stream)
 // projections go to rows [store_at, store_at + n) of the handle's N x ell store; store_at < 0: to a scratch of one sub-chunk
 // (strict-memory mode). accumulate: the rows' sum is added to the consensus sum. scores_out != null (third pass of the
 // strict-memory mode): the scores of these rows against the finished consensus are written there.
-static sage_status_t score_rows(sage_fd* h, const void* rows, int64_t n, int64_t ld, cudaStream_t st, int64_t store_at, bool accumulate,
-                                float* scores_out) {
+static sage_status_t score_rows(sage_fd* h, const void* rows, sage_dtype_t dt, int64_t n, int64_t ld, cudaStream_t st, int64_t store_at,
+                                bool accumulate, float* scores_out) {
     const int ell = h->ell;
     int64_t sub_max = 148 * 128;             // one full wave of 128-row tiles
     const char* p = static_cast<const char*>(rows);
-    const size_t row_bytes = (size_t)ld * elem_size(h->dtype);
+    const size_t row_bytes = (size_t)ld * elem_size(dt);
     const float* S = h->B[h->cur];
     // Tensor-core path: bf16 rows against the bf16 copy of the sketch (a one-term bf16 sketch is only used for
     // long rows, where its rounding errors average out). 
-    const bool tc_ok = h->use_tc && h->dtype == SAGE_BF16 && h->P16 && (h->p16_fold || h->D >= 16384) &&
+    const bool tc_ok = h->use_tc && dt == SAGE_BF16 && h->P16 && (h->p16_fold || h->D >= 16384) &&
                        (reinterpret_cast<uintptr_t>(rows) & 15u) == 0 && (row_bytes & 15u) == 0;
     // fp32 rows: the fp32-faithful three-MMA kernel against the fp32 sketch itself (one 128-wide tile of S)
-    const bool tc32_ok = h->use_tc && h->dtype == SAGE_F32 && ell <= 128 && (reinterpret_cast<uintptr_t>(rows) & 15u) == 0 &&
+    const bool tc32_ok = h->use_tc && dt == SAGE_F32 && ell <= 128 && (reinterpret_cast<uintptr_t>(rows) & 15u) == 0 &&
                          (row_bytes & 15u) == 0;
     // fp32 rows against a small sketch: the projections of a sub-chunk are small (ell <= 64 floats per row and plane), so
     // up to 8 waves go into one launch (fewer launch-scale overheads per pass)
@@ -990,7 +1066,7 @@ static sage_status_t score_rows(sage_fd* h, const void* rows, int64_t n, int64_t
             const int splits = pick_splits(tiles, h->D, 1024);
             ST_TRY(ensure(&h->zwork, &h->zwork_bytes, zred * splits));
             CU_TRY(timed(h, K_PROJECT, 1, st, [&] {
-                return launch_gemm_nt(p + r0 * row_bytes, h->dtype, ld, S, h->pitch, (int)sub, ell, h->D, splits, h->zwork, ell,
+                return launch_gemm_nt(p + r0 * row_bytes, dt, ld, S, h->pitch, (int)sub, ell, h->D, splits, h->zwork, ell,
                                       (int64_t)sub * ell, st);
             }));
             Zparts = h->zwork;
@@ -1024,7 +1100,56 @@ sage_status_t sage_score_chunk(sage_fd_t* h, const void* rows, int64_t n, int64_
     if (n == 0) return SAGE_OK;
     DeviceGuard g(h->device);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    ST_TRY(score_rows(h, rows, n, ld, st, h->strict ? -1 : row_offset, true, nullptr));
+    ST_TRY(score_rows(h, rows, h->dtype, n, ld, st, h->strict ? -1 : row_offset, true, nullptr));
+    h->next_row += n;
+    return SAGE_OK;
+}
+
+// Scoring pass over structured last-layer rows: a sub-chunk of rows is expanded from its factors into a scratch small enough
+// to stay in L2 (products in fp32, exact for bf16 factors) and projected from there; the C F + C values of a row never
+// exist in the caller's memory and are not streamed from HBM.
+static sage_status_t score_rows_outer(sage_fd* h, RowSrc src, int64_t n, cudaStream_t st, int64_t store_at, bool accumulate,
+                                      float* scores_out) {
+    const int64_t pitch_x = ((h->D + 3) / 4) * 4;
+    int64_t sub = (int64_t)((48ull << 20) / ((size_t)pitch_x * sizeof(float)));     // about 48 MB of expanded rows at a time
+    sub = (sub / 128) * 128;
+    if (sub < 128) sub = 128;
+    if (sub > 148 * 128) sub = 148 * 128;
+    ST_TRY(ensure(&h->xwork, &h->xwork_bytes, (size_t)(sub < n ? sub : n) * pitch_x * sizeof(float)));
+    for (int64_t r0 = 0; r0 < n; r0 += sub) {
+        const int64_t take = n - r0 < sub ? n - r0 : sub;
+        const RowSrc part = src.advanced(r0);
+        CU_TRY(timed(h, K_APPEND, 1, st, [&] { return part.append(take, h->D, h->xwork, pitch_x, 0, st); }));
+        ST_TRY(score_rows(h, h->xwork, SAGE_F32, take, pitch_x, st, store_at >= 0 ? store_at + r0 : -1, accumulate,
+                          scores_out ? scores_out + r0 : nullptr));
+    }
+    return SAGE_OK;
+}
+
+sage_status_t sage_score_chunk_outer(sage_fd_t* h, const void* q, int64_t ldq, const void* feat, int64_t ldf, int64_t n, int32_t C,
+                                     int32_t F, int64_t row_offset, void* cuda_stream) {
+    ST_TRY(check_handle(h));
+    if (h->state != SCORING) {
+        set_err("sage_score_chunk_outer: no open scoring pass");
+        return SAGE_ERR_BAD_STATE;
+    }
+    ST_TRY(check_outer(h, "sage_score_chunk_outer", q, ldq, feat, ldf, n, C, F));
+    if (row_offset != h->next_row || row_offset + n > h->N_total) {
+        set_err("sage_score_chunk_outer: bad argument (n=%lld offset=%lld expected offset=%lld N_total=%lld)", (long long)n,
+                (long long)row_offset, (long long)h->next_row, (long long)h->N_total);
+        return SAGE_ERR_INVALID_ARG;
+    }
+    if (n == 0) return SAGE_OK;
+    DeviceGuard g(h->device);
+    RowSrc src;
+    src.q = q;
+    src.ldq = ldq;
+    src.feat = feat;
+    src.ldf = ldf;
+    src.C = C;
+    src.F = F;
+    src.dt = h->dtype;
+    ST_TRY(score_rows_outer(h, src, n, static_cast<cudaStream_t>(cuda_stream), h->strict ? -1 : row_offset, true, nullptr));
     h->next_row += n;
     return SAGE_OK;
 }
@@ -1072,12 +1197,27 @@ sage_status_t sage_score_apply(sage_fd_t* h, const void* rows, int64_t n, int64_
         return SAGE_ERR_BAD_STATE;
     }
     DeviceGuard g(h->device);
-    return score_rows(h, rows, n, ld, static_cast<cudaStream_t>(cuda_stream), -1, false, scores);
+    return score_rows(h, rows, h->dtype, n, ld, static_cast<cudaStream_t>(cuda_stream), -1, false, scores);
 }
 
 sage_status_t sage_score(sage_fd_t* h, const void* rows, int64_t n, int64_t ld, float* scores, void* cuda_stream) {
     ST_TRY(sage_score_begin(h, n, cuda_stream));
     sage_status_t s = sage_score_chunk(h, rows, n, ld, 0, cuda_stream);
+    if (s != SAGE_OK) {
+        h->state = FROZEN;
+        return s;
+    }
+    s = sage_score_end(h, scores, cuda_stream);
+    if (s != SAGE_OK) h->state = FROZEN;
+    return s;
+}
+
+sage_status_t sage_score_outer(sage_fd_t* h, const void* q, int64_t ldq, const void* feat, int64_t ldf, int64_t n, int32_t C, int32_t F,
+                               float* scores, void* cuda_stream) {
+    ST_TRY(check_handle(h));
+    ST_TRY(check_outer(h, "sage_score_outer", q, ldq, feat, ldf, n, C, F));
+    ST_TRY(sage_score_begin(h, n, cuda_stream));
+    sage_status_t s = sage_score_chunk_outer(h, q, ldq, feat, ldf, n, C, F, 0, cuda_stream);
     if (s != SAGE_OK) {
         h->state = FROZEN;
         return s;

@@ -45,6 +45,36 @@ __global__ void __launch_bounds__(256) k_append(const T* __restrict__ rows, int6
     }
 }
 
+// Append of structured last-layer rows (the per-example gradient of a softmax head, Method section): row i is
+// [vec_rowmajor(q_i h_i^T) ; q_i] with q_i (C values) = softmax - onehot and h_i (F values) the features; it is formed here
+// from the two factors and written straight into the destination rows, so the C F + C values never exist in the caller's
+// memory. Products are taken in fp32 (exact for bf16 factors). Columns from C F + C up to the pitch are zeroed.
+template <typename T>
+__global__ void __launch_bounds__(256) k_append_outer(const T* __restrict__ q, int64_t ldq, const T* __restrict__ feat, int64_t ldf, int C,
+                                                      int F, float* __restrict__ B, int64_t pitch, int dst_row0) {
+    const int64_t row = blockIdx.y;
+    const T* qr = q + row * ldq;
+    const T* hr = feat + row * ldf;
+    float* dst = B + (int64_t)(dst_row0 + row) * pitch;
+    const int64_t CF = (int64_t)C * F, D = CF + C;
+    const int64_t c0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x * 4;
+    for (int64_t d = c0; d < pitch; d += stride) {          // the pitch is a multiple of 4 floats, rows are 16-byte aligned
+        float v[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int64_t e = d + i;
+            if (e < CF) {
+                const int c = (int)(e / F), f = (int)(e - (int64_t)c * F);
+                v[i] = to_f32(qr[c]) * to_f32(hr[f]);
+            } else {
+                v[i] = e < D ? to_f32(qr[e - CF]) : 0.f;
+            }
+        }
+        *reinterpret_cast<float4*>(dst + d) = make_float4(v[0], v[1], v[2], v[3]);
+    }
+}
+
 // ------------------------------------------------------------------------------------------------
 // C[z] = A_z * Bm_z^T over the z-th slice of the contraction index (both operands k-contiguous).
 // 64 x 64 output tile, 32-deep k tiles, 256 threads with 4 x 4 register tiles. The register
@@ -282,6 +312,22 @@ cudaError_t launch_append(const void* rows, sage_dtype_t dt, int64_t n, int64_t 
         k_append<float><<<grid, 256, 0, st>>>(static_cast<const float*>(rows), n, ld, D, B, pitch, dst_row0);
     else
         k_append<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(rows), n, ld, D, B, pitch, dst_row0);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_append_outer(const void* q, int64_t ldq, const void* feat, int64_t ldf, sage_dtype_t dt, int64_t n, int C, int F,
+                                float* B, int64_t pitch, int dst_row0, cudaStream_t st) {
+    if (n <= 0) return cudaSuccess;
+    int64_t bx = (pitch / 4 + 255) / 256;
+    if (bx > 592) bx = 592;
+    if (bx < 1) bx = 1;
+    dim3 grid((unsigned)bx, (unsigned)n);
+    if (dt == SAGE_F32)
+        k_append_outer<float><<<grid, 256, 0, st>>>(static_cast<const float*>(q), ldq, static_cast<const float*>(feat), ldf, C, F, B, pitch,
+                                                    dst_row0);
+    else
+        k_append_outer<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(q), ldq, static_cast<const __nv_bfloat16*>(feat),
+                                                            ldf, C, F, B, pitch, dst_row0);
     return cudaGetLastError();
 }
 

@@ -120,8 +120,9 @@ def _lowrank_chunk(w: Workload, seed: int, chunk: int, rank: int, noise_frac: fl
     return (scale[:, None] * (signal + noise)).astype(np.float32)
 
 
-def _lastlayer_chunk(w: Workload, seed: int, chunk: int, classes: int, flip_frac: float) -> np.ndarray:
-    """Rows [vec((p - e_y) h^T) ; (p - e_y)] for a nearest-mean softmax head over a Gaussian mixture."""
+def _lastlayer_chunk(w: Workload, seed: int, chunk: int, classes: int, flip_frac: float, factors: bool = False):
+    """Rows [vec((p - e_y) h^T) ; (p - e_y)] for a nearest-mean softmax head over a Gaussian mixture; with
+    ``factors`` the pair (p - e_y, h) the rows are outer products of, instead of the rows."""
     feat = (w.D - classes) // classes
     assert classes * feat + classes == w.D, "D must equal classes*features + classes"
     n0 = chunk * w.chunk_rows
@@ -143,6 +144,8 @@ def _lastlayer_chunk(w: Workload, seed: int, chunk: int, classes: int, flip_frac
     p = np.exp(logits)
     p /= p.sum(axis=1, keepdims=True)
     p[np.arange(n), y] -= 1.0                                       # p - onehot(y)
+    if factors:
+        return p.astype(np.float32), h.astype(np.float32)
     rows = np.empty((n, w.D), dtype=np.float32)
     rows[:, : classes * feat] = (p[:, :, None] * h[:, None, :]).reshape(n, classes * feat)
     rows[:, classes * feat:] = p
@@ -161,6 +164,29 @@ def host_chunk(w: Workload, seed: int, chunk: int) -> torch.Tensor:
         raise ValueError(f"{w.name} is generated on the device; use device_chunk")
     t = torch.from_numpy(_pad_to(rows, padded_pitch(w.D, 4 if w.dtype == torch.float32 else 2)))
     return t if w.dtype == torch.float32 else t.to(torch.bfloat16)
+
+
+def host_factors(w: Workload, seed: int = 0, n_rows: Optional[int] = None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """The last-layer workloads (c2, c3) in factored form: q = softmax - onehot (n x C) and the features h (n x F), in the
+    workload's dtype and with padded pitches, such that row i of the workload's structured variant is
+    [vec_rowmajor(q_i h_i^T) ; q_i] with the products taken exactly from the stored values. (For fp32 this is the
+    workload's own row up to the rounding of the product; for bf16 the factors are rounded, not the products.)"""
+    classes = {"c2": 10, "c3": 100}[w.name]
+    flip = {"c2": 0.2, "c3": 0.1}[w.name]
+    n_rows = w.N if n_rows is None else min(n_rows, w.N)
+    feat = (w.D - classes) // classes
+    eb = w.elem_bytes
+    q = torch.zeros((n_rows, padded_pitch(classes, eb)), dtype=w.dtype)
+    h = torch.zeros((n_rows, padded_pitch(feat, eb)), dtype=w.dtype)
+    done = chunk = 0
+    while done < n_rows:
+        qc, hc = _lastlayer_chunk(w, seed, chunk, classes, flip, factors=True)
+        take = min(qc.shape[0], n_rows - done)
+        q[done:done + take, :classes] = torch.from_numpy(qc[:take]).to(w.dtype)
+        h[done:done + take, :feat] = torch.from_numpy(hc[:take]).to(w.dtype)
+        done += take
+        chunk += 1
+    return q, h
 
 
 def host_rows(w: Workload, seed: int = 0, n_rows: Optional[int] = None) -> torch.Tensor:
