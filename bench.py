@@ -12,7 +12,9 @@ summed over ranks; with more than one GPU every rank runs an independent replica
 One invocation runs every listed workload and prints ONE JSON line (rank 0). The top-level fields are those of
 the headline workload (default: c5, the largest one that fits one GPU), timed over exactly K steps after W
 warm-up steps; the other workloads follow under "workloads" with the same fields, each timed over
-min(K, 5) steps so that the whole run stays within minutes. `--impl reference` times the fp64 CPU oracle on
+min(K, 5) steps so that the whole run stays within minutes: c1..c4 with the paper's sequential sketch, the same four
+with the merged form of pass 1 (16 sketches, "cN_merged16"), and c2 / c3 given as the factors of their rows
+("cN_factored"). `--impl reference` times the fp64 CPU oracle on
 the host cores instead, on a bounded sample of the headline workload.
 """
 from __future__ import annotations
@@ -118,7 +120,7 @@ class ClockSampler:
 
 
 # Rows of each workload the oracle is timed on: chosen so that one run costs roughly 10 to 40 s of host time.
-CPU_SAMPLE_ROWS = {"c1": 4096, "c2": 20000, "c3": 2000, "c4": 768, "c5": 256}
+CPU_SAMPLE_ROWS = {"c1": 4096, "c2": 20000, "c3": 2000, "c4": 768, "c5": 100}
 
 
 def sample_rows_for(w, n):
@@ -148,7 +150,7 @@ def cpu_oracle_sample(w, sample_rows, rows=None):
 
 
 # Rough cost model of the oracle (host seconds) used only to size the reference arm's sample: flops of the Gram route per
-# shrink and per scored row at a nominal 12 GFLOP/s for its naive fp64 loops on the host cores.
+# shrink and per scored row at a nominal 8 GFLOP/s for its naive fp64 loops on the host cores.
 def oracle_seconds_estimate(w, n):
     full, r_final = shrink_schedule(n, w.ell)
     m = 2 * w.ell
@@ -157,7 +159,7 @@ def oracle_seconds_estimate(w, n):
     else:
         flop = full * (m * m + 2.0 * w.ell * m) * w.D + (r_final * r_final + 2.0 * w.ell * r_final) * w.D
     flop += 2.0 * n * w.ell * w.D
-    return flop / 12e9
+    return flop / 8e9
 
 
 def run_reference(args, w):
@@ -188,7 +190,7 @@ def run_reference(args, w):
     print(json.dumps(line))
 
 
-def run_workload(w, args, steps, warmup, ctx, want_e2e, want_cpu, sketches):
+def run_workload(w, args, steps, warmup, ctx, want_e2e, want_cpu, sketches, factored=False):
     """Times `steps` steps of one workload after `warmup` warm-up steps; returns the fields of its JSON entry."""
     import paper_2510_02470_b200 as sage
     from paper_2510_02470_b200 import replicas
@@ -202,7 +204,14 @@ def run_workload(w, args, steps, warmup, ctx, want_e2e, want_cpu, sketches):
     stream = None
     rows = None
     chunk_buf = None
-    if w.on_device:
+    qf = hf = None
+    C_out = F_out = 0
+    if factored:             # last-layer workloads given as the factors of their rows (no N x D matrix anywhere)
+        C_out = {"c2": 10, "c3": 100}[w.name]
+        F_out = (D - C_out) // C_out
+        q_host, h_host = wl.host_factors(w, args.seed, N)
+        qf, hf = q_host.to(dev), h_host.to(dev)
+    elif w.on_device:
         stream = wl.DeviceStream(w, args.seed, dev)
         chunk_buf = torch.zeros((w.chunk_rows, w.ld), dtype=w.dtype, device=dev)
     else:
@@ -226,7 +235,9 @@ def run_workload(w, args, steps, warmup, ctx, want_e2e, want_cpu, sketches):
         marks = [ev() for _ in range(4)] if phase_events is not None else None
         fd.reset()
         if marks: marks[0].record()
-        if stream is None:
+        if factored:
+            fd.update_outer(qf, hf, C_out, F_out)
+        elif stream is None:
             fd.update(rows)
         else:
             for j in range(w.num_chunks):
@@ -241,7 +252,9 @@ def run_workload(w, args, steps, warmup, ctx, want_e2e, want_cpu, sketches):
                     phase_events.setdefault("gen1", []).append((g0, g1))
         fd.finalize(allow=(6, 7))
         if marks: marks[1].record()
-        if stream is None:
+        if factored:
+            fd.score_outer(qf, hf, C_out, F_out, scores)
+        elif stream is None:
             fd.score(rows, scores)
         else:
             fd.score_begin(N)
@@ -324,7 +337,7 @@ def run_workload(w, args, steps, warmup, ctx, want_e2e, want_cpu, sketches):
     eig_flops = 9.0 * (full * m ** 3 + r_final ** 3)
     dom_ms_per_step = prof_dom["ms"] / steps
     dom_launches_per_step = prof_dom["launches"] / steps
-    if dominant == "eig_shrink" and sketches <= 1:
+    if dominant == "eig_shrink":
         achieved = eig_flops / (dom_ms_per_step * 1e-3) / 1e12
         roof = {"kernel": "k_eig_shrink_fast" if 2 * ell <= 64 else "k_eig_shrink_dsm", "bound": "alu", "achieved": achieved,
                 "peak": FP32_ALU_PEAK_TFLOPS, "unit": "TFLOP/s", "frac": achieved / FP32_ALU_PEAK_TFLOPS, "traffic": None,
@@ -340,6 +353,9 @@ def run_workload(w, args, steps, warmup, ctx, want_e2e, want_cpu, sketches):
                 "frac": gbs / peaks["hbm_gbs"], "traffic": traffic * D if traffic else None,
                 "peak_source": f"{peaks['source']} STREAM-style copy",
                 "algorithmic_bytes_per_launch": per_step_bytes.get(dominant, 0) / max(dom_launches_per_step, 1)}
+    if sketches > 1:
+        roof["note"] = (f"{sketches} sketches run their kernels side by side: the per-kernel times are sums over launches that overlap "
+                        "in time, so achieved / share_of_step describe one launch's pace, not the device's")
     roof["avg_launch_ms"] = dom_ms_per_step / max(dom_launches_per_step, 1)
     roof["launches_per_step"] = dom_launches_per_step
     roof["share_of_step"] = dom_ms_per_step / step_ms
@@ -380,12 +396,12 @@ def run_workload(w, args, steps, warmup, ctx, want_e2e, want_cpu, sketches):
         cb_info = {"error": str(exc)}
 
     fd.close()
-    del rows, chunk_buf, stream, scores, idx_buf
+    del rows, chunk_buf, stream, scores, idx_buf, qf, hf
     torch.cuda.empty_cache()
 
     # ---- end to end through the host-pointer entry point ------------------------------------------------
     e2e = None
-    if want_e2e:
+    if want_e2e and not factored:
         note = None
         if host_rows is None:
             # streamed workloads do not fit host memory as N x D: a prefix of the same rows, copied to pinned host memory
@@ -420,7 +436,8 @@ def run_workload(w, args, steps, warmup, ctx, want_e2e, want_cpu, sketches):
     return {
         "value": value, "unit": UNIT, "steps": steps, "warmup": warmup, "ms_per_step": step_ms,
         "config": {"workload": w.name, "N": N, "D": D, "ell": ell, "rows_dtype": str(w.dtype).replace("torch.", ""),
-                   "ld": w.ld, "keep_rates": list(w.keep_rates), "sketches": sketches, "multi_gpu": "replicas only",
+                   "ld": w.ld, "keep_rates": list(w.keep_rates), "sketches": sketches,
+                   "input": "factors of the rows (softmax - onehot, features)" if factored else "rows", "multi_gpu": "replicas only",
                    "l2": "inputs larger than L2" if N * D * e > 200e6 else "inputs fit in L2 (no flush: stated, c1 only)",
                    "generator_ms_per_step_excluded": gen_per_step, "input_generation_s": t_gen},
         "passes": {"pass1_ms": p1, "pass2_ms": p2, "select_ms": p3,
@@ -449,6 +466,7 @@ def main():
     ap.add_argument("--rows", type=int, default=0, help="use only the first ROWS rows of each workload (debugging)")
     ap.add_argument("--dim", type=int, default=0, help="override the row dimension D (small cases for profiler captures)")
     ap.add_argument("--sketches", type=int, default=1, help="number of sub-sketches of pass 1 (1 = the sequential sketch)")
+    ap.add_argument("--no-variants", action="store_true", help="skip the merged-sketch and factored-input runs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--seed", type=int, default=0)
@@ -488,14 +506,22 @@ def main():
     sage.lib()
     ctx = {"dev": dev, "local": local, "world": world, "rank": rank}
 
+    # Every workload with the paper's sequential sketch; beside it (unless --no-variants) the merged form of pass 1 with 16
+    # sketches on the workloads whose pass 1 is a chain of eigen-solves, and the last-layer workloads given as factors.
+    # The headline comes last and is the only one timed over exactly --steps steps.
+    runs = [(n, n, args.sketches, False) for n in names if n != headline]
+    if not args.no_variants and args.sketches == 1 and not args.rows and not args.dim:
+        runs += [(f"{n}_merged16", n, 16, False) for n in names if n in ("c1", "c2", "c3", "c4") and n != headline]
+        runs += [(f"{n}_factored", n, 1, True) for n in names if n in ("c2", "c3") and n != headline]
+    runs.append((headline, headline, args.sketches, False))
     results = {}
-    for n in [x for x in names if x != headline] + [headline]:
+    for key, n, P, fact in runs:
         w = shaped(n)
-        is_head = n == headline
+        is_head = key == headline
         steps = args.steps if is_head else min(args.steps, 5)
         warm = args.warmup if is_head else 3
-        results[n] = run_workload(w, args, steps, warm, ctx, want_e2e=not args.no_e2e and (is_head or not w.on_device),
-                                  want_cpu=not args.no_cpu_baseline and is_head, sketches=args.sketches)
+        results[key] = run_workload(w, args, steps, warm, ctx, want_e2e=not args.no_e2e and not fact and P == args.sketches and (is_head or not w.on_device),
+                                    want_cpu=not args.no_cpu_baseline and is_head, sketches=P, factored=fact)
 
     if rank == 0:
         head = results[headline]

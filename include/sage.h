@@ -129,10 +129,11 @@ sage_status_t sage_score_end(sage_fd_t* h, float* scores, void* cuda_stream);
  * For a softmax head with C classes on F features the per-example gradient with respect to (weights, bias) is the outer
  * product q_i (x) [h_i ; 1], q_i = softmax - onehot(label): row i is [vec_rowmajor(q_i h_i^T) (C x F) ; q_i (C)], D = C F + C.
  * These entry points take the two factors instead of the row, so the N x D matrix is never formed in the caller's memory
- * nor read from HBM: pass 1 writes each row straight into the sketch buffer, pass 2 expands a sub-chunk of rows at a time
- * into a scratch that stays in L2 and projects it from there. Results are those of sage_fd_update / sage_score_chunk /
- * sage_score on the materialised rows (products taken in fp32, exact for bfloat16 factors); both kinds of call may be
- * mixed on one handle.
+ * memory: pass 1 writes each row straight into the sketch buffer, pass 2 expands a sub-chunk of rows at a time
+ * (one wave of row tiles) into a scratch of the library's own and projects it from there. Results are those of sage_fd_update /
+ * sage_score_chunk / sage_score on the materialised rows: pass 1 takes the products in fp32 (exact for bfloat16 factors); the
+ * scoring pass of a bfloat16 handle rounds each product to bfloat16, as a caller storing bfloat16 rows would have. Both kinds
+ * of call may be mixed on one handle.
  *   q     device, n x ldq elements of the handle's row dtype, C values used per row (ldq >= C).
  *   feat  device, n x ldf elements of the handle's row dtype, F values used per row (ldf >= F).
  * C F + C must equal the handle's D. Stream semantics, state machine and errors are those of the dense calls. */

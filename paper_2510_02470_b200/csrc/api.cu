@@ -158,7 +158,9 @@ struct sage_fd {
     double* zsum = nullptr;
     float* u = nullptr;
     bool scored = false;           // a scoring pass over N_total rows has finished: zhat holds their normalised projections
-    float* xwork = nullptr;        // structured rows expanded a sub-chunk at a time for the scoring pass (fp32, pitch D rounded up to 4)
+    float* zred = nullptr;         // projections of a sub-chunk summed over their K slices (when there are many slices)
+    size_t zred_bytes = 0;
+    float* xwork = nullptr;        // structured rows expanded a sub-chunk at a time for the scoring pass (the handle's row type)
     size_t xwork_bytes = 0;
     bool strict = false;           // option 8: no N x ell store; scores come from a third pass (sage_score_apply)
     bool scored_strict = false;    // the finished pass ran in strict-memory mode: u is known, zhat is not kept
@@ -505,6 +507,7 @@ void sage_fd_destroy(sage_fd_t* h) {
     cudaFree(h->zwork);
     cudaFree(h->partials);
     cudaFree(h->xwork);
+    cudaFree(h->zred);
     cudaFree(h->zsum);
     cudaFree(h->u);
     cudaFree(h->class_U);
@@ -653,7 +656,7 @@ struct RowSrc {
         return r;
     }
     cudaError_t append(int64_t take, int64_t D, float* B, int64_t pitch, int dst_row0, cudaStream_t st) const {
-        if (outer()) return launch_append_outer(q, ldq, feat, ldf, dt, take, C, F, B, pitch, dst_row0, st);
+        if (outer()) return launch_append_outer(q, ldq, feat, ldf, dt, take, C, F, B, SAGE_F32, pitch, dst_row0, st);
         return launch_append(rows, dt, take, ld, D, B, pitch, dst_row0, st);
     }
 };
@@ -1072,6 +1075,17 @@ static sage_status_t score_rows(sage_fd* h, const void* rows, sage_dtype_t dt, i
             Zparts = h->zwork;
             nplanes = splits;
         }
+        // Many K slices (few rows per launch, as in the 512-row chunks of very long rows): summed first by a kernel with a
+        // thread per element; the normalise kernel has a warp per row and would walk the slices one after the other.
+        if (nplanes > 4) {
+            ST_TRY(ensure(&h->zred, &h->zred_bytes, zred));
+            const float* parts = Zparts;
+            const int np = nplanes;
+            CU_TRY(timed(h, K_PROJECT_REDUCE, 1, st,
+                         [&] { return launch_split_reduce(parts, np, (int64_t)sub * ell, (int)sub, ell, ell, h->zred, ell, st); }));
+            Zparts = h->zred;
+            nplanes = 1;
+        }
         // normalise (summing the K slices of the projection on the way), consensus partials, and in the third pass the scores
         float* zh = store_at >= 0 ? h->zhat + (store_at + r0) * ell : h->zhat;
         float* zn = store_at >= 0 ? h->znorm + (store_at + r0) : h->znorm;
@@ -1105,22 +1119,27 @@ sage_status_t sage_score_chunk(sage_fd_t* h, const void* rows, int64_t n, int64_
     return SAGE_OK;
 }
 
-// Scoring pass over structured last-layer rows: a sub-chunk of rows is expanded from its factors into a scratch small enough
-// to stay in L2 (products in fp32, exact for bf16 factors) and projected from there; the C F + C values of a row never
-// exist in the caller's memory and are not streamed from HBM.
+// Scoring pass over structured last-layer rows: up to one full wave of row tiles at a time is expanded from its factors
+// into a scratch of the handle's row type and projected from there by the kernels of the dense path. fp32 handles: the
+// products are exact. bfloat16 handles: each product is rounded to bfloat16, the row as a caller holding bfloat16 rows would
+// have stored it (pass 1 wrote the exact products into the fp32 buffer; the difference stays far inside the tolerance of
+// bfloat16 rows). The C F + C values of a row never exist in the caller's memory.
 static sage_status_t score_rows_outer(sage_fd* h, RowSrc src, int64_t n, cudaStream_t st, int64_t store_at, bool accumulate,
                                       float* scores_out) {
-    const int64_t pitch_x = ((h->D + 3) / 4) * 4;
-    int64_t sub = (int64_t)((48ull << 20) / ((size_t)pitch_x * sizeof(float)));     // about 48 MB of expanded rows at a time
-    sub = (sub / 128) * 128;
-    if (sub < 128) sub = 128;
-    if (sub > 148 * 128) sub = 148 * 128;
-    ST_TRY(ensure(&h->xwork, &h->xwork_bytes, (size_t)(sub < n ? sub : n) * pitch_x * sizeof(float)));
+    const size_t es = elem_size(h->dtype);
+    const int64_t per16 = (int64_t)(16 / es);
+    const int64_t pitch_x = ((h->D + per16 - 1) / per16) * per16;
+    int64_t sub = 148 * 128;                      // one full wave of 128-row tiles
+    if (h->dtype == SAGE_F32 && h->S32split) sub *= 8;
+    if (sub > n) sub = n;
+    ST_TRY(ensure(&h->xwork, &h->xwork_bytes, (size_t)sub * pitch_x * es));
     for (int64_t r0 = 0; r0 < n; r0 += sub) {
         const int64_t take = n - r0 < sub ? n - r0 : sub;
         const RowSrc part = src.advanced(r0);
-        CU_TRY(timed(h, K_APPEND, 1, st, [&] { return part.append(take, h->D, h->xwork, pitch_x, 0, st); }));
-        ST_TRY(score_rows(h, h->xwork, SAGE_F32, take, pitch_x, st, store_at >= 0 ? store_at + r0 : -1, accumulate,
+        CU_TRY(timed(h, K_APPEND, 1, st, [&] {
+            return launch_append_outer(part.q, part.ldq, part.feat, part.ldf, part.dt, take, part.C, part.F, h->xwork, h->dtype, pitch_x, 0, st);
+        }));
+        ST_TRY(score_rows(h, h->xwork, h->dtype, take, pitch_x, st, store_at >= 0 ? store_at + r0 : -1, accumulate,
                           scores_out ? scores_out + r0 : nullptr));
     }
     return SAGE_OK;

@@ -32,9 +32,11 @@ cudaError_t launch_append(const void* rows, sage_dtype_t dt, int64_t n, int64_t 
                           int64_t pitch, int dst_row0, cudaStream_t st);
 
 // Structured last-layer rows: B[dst_row0 + i, :] = [vec_rowmajor(q_i feat_i^T) ; q_i] for i < n, with q n x C (pitch ldq) and feat
-// n x F (pitch ldf) of element type dt; products in fp32; columns C F + C .. pitch-1 zeroed. pitch must be a multiple of 4.
+// n x F (pitch ldf) of element type dt; products in fp32; columns C F + C .. pitch-1 zeroed. B holds elements of type out_dt
+// (fp32, or bf16 for bf16 factors: the products are then rounded to nearest even); pitch in elements, a multiple of 4 (8 for
+// bf16 output so that rows stay 16-byte aligned).
 cudaError_t launch_append_outer(const void* q, int64_t ldq, const void* feat, int64_t ldf, sage_dtype_t dt, int64_t n, int C, int F,
-                                float* B, int64_t pitch, int dst_row0, cudaStream_t st);
+                                void* B, sage_dtype_t out_dt, int64_t pitch, int dst_row0, cudaStream_t st);
 
 // C[z][i][j] = sum over the z-th K-slice of A[i][k] * Bm[j][k]   (both operands contiguous along k).
 // A is M x K (element type dt, pitch lda), Bm is N x K fp32 (pitch ldb). splits >= 1 slices of k.

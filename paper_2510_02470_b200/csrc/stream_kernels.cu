@@ -49,17 +49,27 @@ __global__ void __launch_bounds__(256) k_append(const T* __restrict__ rows, int6
 // [vec_rowmajor(q_i h_i^T) ; q_i] with q_i (C values) = softmax - onehot and h_i (F values) the features; it is formed here
 // from the two factors and written straight into the destination rows, so the C F + C values never exist in the caller's
 // memory. Products are taken in fp32 (exact for bf16 factors). Columns from C F + C up to the pitch are zeroed.
-template <typename T>
+// Out = float: the buffer rows of pass 1 and the scoring scratch of fp32 handles. Out = bfloat16: the scoring scratch of
+// bfloat16 handles, each product rounded to nearest even (the row as a caller holding bfloat16 rows would have stored it).
+__device__ __forceinline__ void store4(float* p, const float v[4]) { *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]); }
+__device__ __forceinline__ void store4(__nv_bfloat16* p, const float v[4]) {
+    __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
+    uint2 raw;
+    raw.x = *reinterpret_cast<uint32_t*>(&a);
+    raw.y = *reinterpret_cast<uint32_t*>(&b);
+    *reinterpret_cast<uint2*>(p) = raw;
+}
+template <typename T, typename Out>
 __global__ void __launch_bounds__(256) k_append_outer(const T* __restrict__ q, int64_t ldq, const T* __restrict__ feat, int64_t ldf, int C,
-                                                      int F, float* __restrict__ B, int64_t pitch, int dst_row0) {
+                                                      int F, Out* __restrict__ B, int64_t pitch, int dst_row0) {
     const int64_t row = blockIdx.y;
     const T* qr = q + row * ldq;
     const T* hr = feat + row * ldf;
-    float* dst = B + (int64_t)(dst_row0 + row) * pitch;
+    Out* dst = B + (int64_t)(dst_row0 + row) * pitch;
     const int64_t CF = (int64_t)C * F, D = CF + C;
     const int64_t c0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x * 4;
-    for (int64_t d = c0; d < pitch; d += stride) {          // the pitch is a multiple of 4 floats, rows are 16-byte aligned
+    for (int64_t d = c0; d < pitch; d += stride) {          // the pitch is a multiple of 4 elements, rows are 16-byte aligned
         float v[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -71,7 +81,7 @@ __global__ void __launch_bounds__(256) k_append_outer(const T* __restrict__ q, i
                 v[i] = e < D ? to_f32(qr[e - CF]) : 0.f;
             }
         }
-        *reinterpret_cast<float4*>(dst + d) = make_float4(v[0], v[1], v[2], v[3]);
+        store4(dst + d, v);
     }
 }
 
@@ -316,18 +326,23 @@ cudaError_t launch_append(const void* rows, sage_dtype_t dt, int64_t n, int64_t 
 }
 
 cudaError_t launch_append_outer(const void* q, int64_t ldq, const void* feat, int64_t ldf, sage_dtype_t dt, int64_t n, int C, int F,
-                                float* B, int64_t pitch, int dst_row0, cudaStream_t st) {
+                                void* B, sage_dtype_t out_dt, int64_t pitch, int dst_row0, cudaStream_t st) {
     if (n <= 0) return cudaSuccess;
+    if ((pitch & 3) || (out_dt == SAGE_BF16 && dt != SAGE_BF16)) return cudaErrorInvalidValue;
     int64_t bx = (pitch / 4 + 255) / 256;
     if (bx > 592) bx = 592;
     if (bx < 1) bx = 1;
     dim3 grid((unsigned)bx, (unsigned)n);
     if (dt == SAGE_F32)
-        k_append_outer<float><<<grid, 256, 0, st>>>(static_cast<const float*>(q), ldq, static_cast<const float*>(feat), ldf, C, F, B, pitch,
-                                                    dst_row0);
+        k_append_outer<float, float><<<grid, 256, 0, st>>>(static_cast<const float*>(q), ldq, static_cast<const float*>(feat), ldf, C, F,
+                                                           static_cast<float*>(B), pitch, dst_row0);
+    else if (out_dt == SAGE_F32)
+        k_append_outer<__nv_bfloat16, float><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(q), ldq, static_cast<const __nv_bfloat16*>(feat),
+                                                                   ldf, C, F, static_cast<float*>(B), pitch, dst_row0);
     else
-        k_append_outer<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(q), ldq, static_cast<const __nv_bfloat16*>(feat),
-                                                            ldf, C, F, B, pitch, dst_row0);
+        k_append_outer<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(q), ldq,
+                                                                           static_cast<const __nv_bfloat16*>(feat), ldf, C, F,
+                                                                           static_cast<__nv_bfloat16*>(B), pitch, dst_row0);
     return cudaGetLastError();
 }
 
