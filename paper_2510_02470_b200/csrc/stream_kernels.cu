@@ -71,14 +71,22 @@ __global__ void __launch_bounds__(256) k_append_outer(const T* __restrict__ q, i
     const int64_t stride = (int64_t)gridDim.x * blockDim.x * 4;
     for (int64_t d = c0; d < pitch; d += stride) {          // the pitch is a multiple of 4 elements, rows are 16-byte aligned
         float v[4];
+        const int c0q = (int)(d / F);
+        const int f0 = (int)(d - (int64_t)c0q * F);
+        if (d + 3 < CF && f0 + 3 < F) {              // the four columns belong to one class: one factor, four features
+            const float qc = to_f32(qr[c0q]);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int64_t e = d + i;
-            if (e < CF) {
-                const int c = (int)(e / F), f = (int)(e - (int64_t)c * F);
-                v[i] = to_f32(qr[c]) * to_f32(hr[f]);
-            } else {
-                v[i] = e < D ? to_f32(qr[e - CF]) : 0.f;
+            for (int i = 0; i < 4; ++i) v[i] = qc * to_f32(hr[f0 + i]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int64_t e = d + i;
+                if (e < CF) {
+                    const int c = (int)(e / F), f = (int)(e - (int64_t)c * F);
+                    v[i] = to_f32(qr[c]) * to_f32(hr[f]);
+                } else {
+                    v[i] = e < D ? to_f32(qr[e - CF]) : 0.f;
+                }
             }
         }
         store4(dst + d, v);

@@ -54,3 +54,32 @@ def test_static_select_edges_and_limit():
     assert b"262144" in lib.sage_last_error()
     assert lib.sage_select_static(None, 5, 0.5, idx.data_ptr(), None, None) == 1
     assert lib.sage_select_static(None, 0, 0.5, None, C.byref(k_out), None) == 0 and k_out.value == 0
+
+
+def test_static_select_allocates_nothing_and_follows_the_stream():
+    """What the entry point is for: after its first call on the device, further calls leave the device's free memory and
+    torch's allocator untouched (the output buffer is the caller's, the scratch is inside the library), also when they
+    are enqueued on a stream other than the default one."""
+    s = _scores(100000, 5, False)
+    k = sage.sage_select_count(100000, 0.25)
+    idx = torch.empty((k,), dtype=torch.int64, device=DEV)
+    want = sage.sage_select(s, 0.25)
+    sage.sage_select_static(s, 0.25, idx)                        # first call on the device: looks up the array's address
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    held0 = torch.cuda.memory_allocated()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    for i in range(4):
+        idx.zero_()
+        torch.cuda.synchronize()
+        if i % 2:
+            with torch.cuda.stream(side):
+                got = sage.sage_select_static(s, 0.25, idx)
+            side.synchronize()
+        else:
+            got = sage.sage_select_static(s, 0.25, idx)
+            torch.cuda.synchronize()
+        assert torch.equal(got, want)
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0 and torch.cuda.memory_allocated() == held0
