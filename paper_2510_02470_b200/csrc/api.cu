@@ -6,7 +6,6 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
-#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -1047,7 +1046,6 @@ static sage_status_t score_rows(sage_fd* h, const void* rows, sage_dtype_t dt, i
             int mt = 512 / n_mma >= 4 ? 4 : (512 / n_mma >= 2 ? 2 : 1);
             if (tiles >= 148 && mt > 2) mt = 2;   // measured: pairs of row tiles with two K slices beat single tiles by 25 %
             while (mt > 1 && (int64_t)((tiles + mt - 1) / mt) * (h->D / 4096 > 0 ? h->D / 4096 : 1) < 148) mt >>= 1;
-            { static const int forced = getenv("SAGE_MT") ? atoi(getenv("SAGE_MT")) : 0; if (forced > 0 && forced <= mt) mt = forced; }
             const int splits = pick_splits_waves((tiles + mt - 1) / mt, h->D, 4096, 148);
             ST_TRY(ensure(&h->zwork, &h->zwork_bytes, zred * splits));
             float* out = h->zwork;

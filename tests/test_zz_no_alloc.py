@@ -65,11 +65,14 @@ def test_static_select_allocates_nothing_and_follows_the_stream():
     idx = torch.empty((k,), dtype=torch.int64, device=DEV)
     want = sage.sage_select(s, 0.25)
     sage.sage_select_static(s, 0.25, idx)                        # first call on the device: looks up the array's address
+    side = torch.cuda.Stream()                                   # the stream itself (torch's and the driver's doing) comes first
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        sage.sage_select_static(s, 0.25, idx)
+    idx.zero_()
     torch.cuda.synchronize()
     free0, _ = torch.cuda.mem_get_info()
     held0 = torch.cuda.memory_allocated()
-    side = torch.cuda.Stream()
-    side.wait_stream(torch.cuda.current_stream())
     for i in range(4):
         idx.zero_()
         torch.cuda.synchronize()
