@@ -128,12 +128,14 @@ sage_status_t sage_score_end(sage_fd_t* h, float* scores, void* cuda_stream);
 /* Structured last-layer rows (Method, the definition of the per-example gradient; Limitations, on last-layer gradients).
  * For a softmax head with C classes on F features the per-example gradient with respect to (weights, bias) is the outer
  * product q_i (x) [h_i ; 1], q_i = softmax - onehot(label): row i is [vec_rowmajor(q_i h_i^T) (C x F) ; q_i (C)], D = C F + C.
- * These entry points take the two factors instead of the row, so the N x D matrix is never formed in the caller's memory
- * memory: pass 1 writes each row straight into the sketch buffer, pass 2 expands a sub-chunk of rows at a time
- * (one wave of row tiles) into a scratch of the library's own and projects it from there. Results are those of sage_fd_update /
- * sage_score_chunk / sage_score on the materialised rows: pass 1 takes the products in fp32 (exact for bfloat16 factors); the
- * scoring pass of a bfloat16 handle rounds each product to bfloat16, as a caller storing bfloat16 rows would have. Both kinds
- * of call may be mixed on one handle.
+ * These entry points take the two factors instead of the row, so the N x D matrix is never formed, neither in the caller's
+ * memory nor in the library's: pass 1 writes each row straight into the sketch buffer (products in fp32, exact for bfloat16
+ * factors); pass 2 uses z_i = S g_i = sum_c q_ic (S_c h_i + b_c), with S_c the columns [c F, c F + F) of the sketch and b_c
+ * column c of its last C columns: one launch of the projection kernel of the dense path contracts the features with every
+ * class block (the classes take the place of its K slices), a second kernel folds the per-class planes with the factors
+ * q_ic. The planes of a sub-chunk of rows are scratch of the library's own (C x ell floats per row, at most 1 GiB at a time).
+ * Results are those of sage_fd_update / sage_score_chunk / sage_score on the materialised rows up to rounding. Both kinds of
+ * call may be mixed on one handle.
  *   q     device, n x ldq elements of the handle's row dtype, C values used per row (ldq >= C).
  *   feat  device, n x ldf elements of the handle's row dtype, F values used per row (ldf >= F).
  * C F + C must equal the handle's D. Stream semantics, state machine and errors are those of the dense calls. */

@@ -158,10 +158,10 @@ struct sage_fd {
     double* zsum = nullptr;
     float* u = nullptr;
     bool scored = false;           // a scoring pass over N_total rows has finished: zhat holds their normalised projections
+    float* bias_t = nullptr;       // structured rows: the bias block of the sketch transposed (C x ell)
+    size_t bias_t_bytes = 0;
     float* zred = nullptr;         // projections of a sub-chunk summed over their K slices (when there are many slices)
     size_t zred_bytes = 0;
-    float* xwork = nullptr;        // structured rows expanded a sub-chunk at a time for the scoring pass (the handle's row type)
-    size_t xwork_bytes = 0;
     bool strict = false;           // option 8: no N x ell store; scores come from a third pass (sage_score_apply)
     bool scored_strict = false;    // the finished pass ran in strict-memory mode: u is known, zhat is not kept
     float* class_U = nullptr;      // class-balanced variant: unit centroids (class_cap x ell) and class sizes
@@ -506,8 +506,8 @@ void sage_fd_destroy(sage_fd_t* h) {
     cudaFree(h->znorm);
     cudaFree(h->zwork);
     cudaFree(h->partials);
-    cudaFree(h->xwork);
     cudaFree(h->zred);
+    cudaFree(h->bias_t);
     cudaFree(h->zsum);
     cudaFree(h->u);
     cudaFree(h->class_U);
@@ -656,7 +656,7 @@ struct RowSrc {
         return r;
     }
     cudaError_t append(int64_t take, int64_t D, float* B, int64_t pitch, int dst_row0, cudaStream_t st) const {
-        if (outer()) return launch_append_outer(q, ldq, feat, ldf, dt, take, C, F, B, SAGE_F32, pitch, dst_row0, st);
+        if (outer()) return launch_append_outer(q, ldq, feat, ldf, dt, take, C, F, B, pitch, dst_row0, st);
         return launch_append(rows, dt, take, ld, D, B, pitch, dst_row0, st);
     }
 };
@@ -982,15 +982,32 @@ sage_status_t sage_score_begin(sage_fd_t* h, int64_t N_total, void* cuda_stream)
 // projections go to rows [store_at, store_at + n) of the handle's N x ell store; store_at < 0: to a scratch of one sub-chunk
 // (strict-memory mode). accumulate: the rows' sum is added to the consensus sum. scores_out != null (third pass of the
 // strict-memory mode): the scores of these rows against the finished consensus are written there.
+// Projection, normalisation, consensus partials (and, with scores_out, the scores) of n rows, a sub-chunk at a time.
+// Dense rows: `rows` with pitch ld. Structured last-layer rows (outer != nullptr; rows and ld unused): the projection
+// factorises over the classes,
+//     z_i = S g_i = sum_c q_ic (S_c h_i) + S_b q_i      (S_c: columns [c F, c F + F) of the sketch, S_b: its last C columns),
+// so the row g_i is never formed: ONE launch of the projection kernel takes the classes as its K slices (every slice reads
+// the same F feature columns, slice c the class block c of the sketch) and leaves the planes T_c = H S_c^T, which a second
+// kernel folds with the factors q_ic and the bias block.
 static sage_status_t score_rows(sage_fd* h, const void* rows, sage_dtype_t dt, int64_t n, int64_t ld, cudaStream_t st, int64_t store_at,
-                                bool accumulate, float* scores_out) {
+                                bool accumulate, float* scores_out, const RowSrc* outer = nullptr) {
     const int ell = h->ell;
+    const bool structured = outer != nullptr;
+    const void* oq = structured ? outer->q : nullptr;
+    const int64_t oldq = structured ? outer->ldq : 0;
+    const int oC = structured ? outer->C : 0, oF = structured ? outer->F : 0;
+    if (structured) {
+        rows = outer->feat;
+        ld = outer->ldf;
+    }
+    const int64_t K = structured ? (int64_t)oC * oF : h->D;      // contraction length against the sketch
+    const int64_t class_F = structured ? oF : 0;
     int64_t sub_max = 148 * 128;             // one full wave of 128-row tiles
     const char* p = static_cast<const char*>(rows);
     const size_t row_bytes = (size_t)ld * elem_size(dt);
     const float* S = h->B[h->cur];
     // Tensor-core path: bf16 rows against the bf16 copy of the sketch (a one-term bf16 sketch is only used for
-    // long rows, where its rounding errors average out). 
+    // long rows, where its rounding errors average out).
     const bool tc_ok = h->use_tc && dt == SAGE_BF16 && h->P16 && (h->p16_fold || h->D >= 16384) &&
                        (reinterpret_cast<uintptr_t>(rows) & 15u) == 0 && (row_bytes & 15u) == 0;
     // fp32 rows: the fp32-faithful three-MMA kernel against the fp32 sketch itself (one 128-wide tile of S)
@@ -999,6 +1016,13 @@ static sage_status_t score_rows(sage_fd* h, const void* rows, sage_dtype_t dt, i
     // fp32 rows against a small sketch: the projections of a sub-chunk are small (ell <= 64 floats per row and plane), so
     // up to 8 waves go into one launch (fewer launch-scale overheads per pass)
     if (tc32_ok && h->S32split) sub_max *= 8;
+    if (structured) {
+        // one plane per class (two with the pre-split sketch): keep the planes of a sub-chunk within 1 GiB
+        const int64_t per_row = (int64_t)oC * ((tc32_ok && h->S32split) ? 2 : 1) * ell * (int64_t)sizeof(float);
+        int64_t fit = ((int64_t)1 << 30) / per_row / 128 * 128;
+        if (fit < 128) fit = 128;
+        if (sub_max > fit) sub_max = fit;
+    }
     for (int64_t r0 = 0; r0 < n; r0 += sub_max) {
         const int64_t sub = (n - r0 < sub_max) ? n - r0 : sub_max;
         const size_t nb = (size_t)((sub + 63) / 64);
@@ -1018,7 +1042,7 @@ static sage_status_t score_rows(sage_fd* h, const void* rows, sage_dtype_t dt, i
         const float* Zparts = nullptr;       // the projections of this sub-chunk as nplanes partial planes of sub x ell floats
         int nplanes = 1;
         if (tc32_ok) {
-            const int splits = pick_splits_waves((int)((sub + 127) / 128), h->D, 2048, 64);
+            const int splits = structured ? oC : pick_splits_waves((int)((sub + 127) / 128), K, 2048, 64);
             // sketches of at most 64 rows: one wide MMA per K step against the pre-split sketch, two partial planes per K slice
             const bool wide = h->S32split != nullptr;
             const int planes = wide ? 2 * splits : splits;
@@ -1026,7 +1050,7 @@ static sage_status_t score_rows(sage_fd* h, const void* rows, sage_dtype_t dt, i
             float* out = h->zwork;
             cudaError_t e = timed(h, K_PROJECT, 1, st, [&] {
                 return launch_tc_gemm_nt_x3(reinterpret_cast<const float*>(p + r0 * row_bytes), ld, wide ? h->S32split : S, h->pitch, (int)sub,
-                                            ell, h->D, splits, out, ell, (int64_t)sub * ell, wide ? 2 : 0, h->tc_err, st);
+                                            ell, K, splits, out, ell, (int64_t)sub * ell, wide ? 2 : 0, h->tc_err, st, class_F);
             });
             if (e == cudaSuccess) {
                 done = true;
@@ -1045,13 +1069,14 @@ static sage_status_t score_rows(sage_fd* h, const void* rows, sage_dtype_t dt, i
             const int tiles = (int)((sub + 127) / 128);
             int mt = 512 / n_mma >= 4 ? 4 : (512 / n_mma >= 2 ? 2 : 1);
             if (tiles >= 148 && mt > 2) mt = 2;   // measured: pairs of row tiles with two K slices beat single tiles by 25 %
-            while (mt > 1 && (int64_t)((tiles + mt - 1) / mt) * (h->D / 4096 > 0 ? h->D / 4096 : 1) < 148) mt >>= 1;
-            const int splits = pick_splits_waves((tiles + mt - 1) / mt, h->D, 4096, 148);
+            const int64_t slices_at_least = structured ? oC : (K / 4096 > 0 ? K / 4096 : 1);
+            while (mt > 1 && (int64_t)((tiles + mt - 1) / mt) * slices_at_least < 148) mt >>= 1;
+            const int splits = structured ? oC : pick_splits_waves((tiles + mt - 1) / mt, K, 4096, 148);
             ST_TRY(ensure(&h->zwork, &h->zwork_bytes, zred * splits));
             float* out = h->zwork;
             cudaError_t e = timed(h, K_PROJECT, 1, st, [&] {
-                return launch_tc_gemm_nt(p + r0 * row_bytes, SAGE_BF16, ld, h->P16, h->pitch, (int)sub, ell, h->p16_fold, mt, h->D, splits,
-                                         out, ell, (int64_t)sub * ell, h->tc_err, st);
+                return launch_tc_gemm_nt(p + r0 * row_bytes, SAGE_BF16, ld, h->P16, h->pitch, (int)sub, ell, h->p16_fold, mt, K, splits,
+                                         out, ell, (int64_t)sub * ell, h->tc_err, st, class_F);
             });
             if (e == cudaSuccess) {
                 done = true;
@@ -1066,14 +1091,27 @@ static sage_status_t score_rows(sage_fd* h, const void* rows, sage_dtype_t dt, i
         }
         if (!done) {
             const int tiles = (int)((sub + 63) / 64) * ((ell + 63) / 64);
-            const int splits = pick_splits(tiles, h->D, 1024);
+            const int splits = structured ? oC : pick_splits(tiles, K, 1024);
             ST_TRY(ensure(&h->zwork, &h->zwork_bytes, zred * splits));
             CU_TRY(timed(h, K_PROJECT, 1, st, [&] {
-                return launch_gemm_nt(p + r0 * row_bytes, dt, ld, S, h->pitch, (int)sub, ell, h->D, splits, h->zwork, ell,
-                                      (int64_t)sub * ell, st);
+                return launch_gemm_nt(p + r0 * row_bytes, dt, ld, S, h->pitch, (int)sub, ell, K, splits, h->zwork, ell,
+                                      (int64_t)sub * ell, st, class_F);
             }));
             Zparts = h->zwork;
             nplanes = splits;
+        }
+        if (structured) {
+            // z = sum_c q_c (T_c + bias column c), classes in ascending order
+            ST_TRY(ensure(&h->zred, &h->zred_bytes, zred));
+            const float* parts = Zparts;
+            const int pp = nplanes / oC;
+            const char* qsub = static_cast<const char*>(oq) + (size_t)r0 * oldq * elem_size(dt);
+            ST_TRY(ensure(&h->bias_t, &h->bias_t_bytes, (size_t)oC * ell * sizeof(float)));
+            CU_TRY(timed(h, K_PROJECT_REDUCE, 2, st, [&] {
+                return launch_outer_combine(qsub, oldq, dt, oC, parts, pp, (int64_t)sub * ell, S + K, h->pitch, h->bias_t, sub, ell, h->zred, st);
+            }));
+            Zparts = h->zred;
+            nplanes = 1;
         }
         // Many K slices (few rows per launch, as in the 512-row chunks of very long rows): summed first by a kernel with a
         // thread per element; the normalise kernel has a warp per row and would walk the slices one after the other.
@@ -1119,32 +1157,6 @@ sage_status_t sage_score_chunk(sage_fd_t* h, const void* rows, int64_t n, int64_
     return SAGE_OK;
 }
 
-// Scoring pass over structured last-layer rows: up to one full wave of row tiles at a time is expanded from its factors
-// into a scratch of the handle's row type and projected from there by the kernels of the dense path. fp32 handles: the
-// products are exact. bfloat16 handles: each product is rounded to bfloat16, the row as a caller holding bfloat16 rows would
-// have stored it (pass 1 wrote the exact products into the fp32 buffer; the difference stays far inside the tolerance of
-// bfloat16 rows). The C F + C values of a row never exist in the caller's memory.
-static sage_status_t score_rows_outer(sage_fd* h, RowSrc src, int64_t n, cudaStream_t st, int64_t store_at, bool accumulate,
-                                      float* scores_out) {
-    const size_t es = elem_size(h->dtype);
-    const int64_t per16 = (int64_t)(16 / es);
-    const int64_t pitch_x = ((h->D + per16 - 1) / per16) * per16;
-    int64_t sub = 148 * 128;                      // one full wave of 128-row tiles
-    if (h->dtype == SAGE_F32 && h->S32split) sub *= 8;
-    if (sub > n) sub = n;
-    ST_TRY(ensure(&h->xwork, &h->xwork_bytes, (size_t)sub * pitch_x * es));
-    for (int64_t r0 = 0; r0 < n; r0 += sub) {
-        const int64_t take = n - r0 < sub ? n - r0 : sub;
-        const RowSrc part = src.advanced(r0);
-        CU_TRY(timed(h, K_APPEND, 1, st, [&] {
-            return launch_append_outer(part.q, part.ldq, part.feat, part.ldf, part.dt, take, part.C, part.F, h->xwork, h->dtype, pitch_x, 0, st);
-        }));
-        ST_TRY(score_rows(h, h->xwork, h->dtype, take, pitch_x, st, store_at >= 0 ? store_at + r0 : -1, accumulate,
-                          scores_out ? scores_out + r0 : nullptr));
-    }
-    return SAGE_OK;
-}
-
 sage_status_t sage_score_chunk_outer(sage_fd_t* h, const void* q, int64_t ldq, const void* feat, int64_t ldf, int64_t n, int32_t C,
                                      int32_t F, int64_t row_offset, void* cuda_stream) {
     ST_TRY(check_handle(h));
@@ -1168,7 +1180,7 @@ sage_status_t sage_score_chunk_outer(sage_fd_t* h, const void* q, int64_t ldq, c
     src.C = C;
     src.F = F;
     src.dt = h->dtype;
-    ST_TRY(score_rows_outer(h, src, n, static_cast<cudaStream_t>(cuda_stream), h->strict ? -1 : row_offset, true, nullptr));
+    ST_TRY(score_rows(h, nullptr, h->dtype, n, 0, static_cast<cudaStream_t>(cuda_stream), h->strict ? -1 : row_offset, true, nullptr, &src));
     h->next_row += n;
     return SAGE_OK;
 }

@@ -32,16 +32,25 @@ cudaError_t launch_append(const void* rows, sage_dtype_t dt, int64_t n, int64_t 
                           int64_t pitch, int dst_row0, cudaStream_t st);
 
 // Structured last-layer rows: B[dst_row0 + i, :] = [vec_rowmajor(q_i feat_i^T) ; q_i] for i < n, with q n x C (pitch ldq) and feat
-// n x F (pitch ldf) of element type dt; products in fp32; columns C F + C .. pitch-1 zeroed. B holds elements of type out_dt
-// (fp32, or bf16 for bf16 factors: the products are then rounded to nearest even); pitch in elements, a multiple of 4 (8 for
-// bf16 output so that rows stay 16-byte aligned).
+// n x F (pitch ldf) of element type dt; products in fp32 (exact for bf16 factors); columns C F + C .. pitch-1 zeroed. pitch
+// must be a multiple of 4.
 cudaError_t launch_append_outer(const void* q, int64_t ldq, const void* feat, int64_t ldf, sage_dtype_t dt, int64_t n, int C, int F,
-                                void* B, sage_dtype_t out_dt, int64_t pitch, int dst_row0, cudaStream_t st);
+                                float* B, int64_t pitch, int dst_row0, cudaStream_t st);
+
+// Projection of structured rows from per-class planes: with T[c] = feat * S_c^T (n x ell, the sum of pp consecutive planes of
+// `planes`, plane_stride floats apart, n x ell each with pitch ell) and S_c the columns [c F, c F + F) of the sketch,
+//     Z[i][j] = sum_c q[i][c] * (T[c][i][j] + Sb[j][c]),      Sb = S + C F (the bias columns of the sketch, pitch lds).
+// Classes are added in ascending order in fp32. q is n x C of element type dt (pitch ldq); Z is n x ell, pitch ell. biasT:
+// scratch of C x ell floats (receives Sb transposed). Two launches.
+cudaError_t launch_outer_combine(const void* q, int64_t ldq, sage_dtype_t dt, int C, const float* planes, int pp, int64_t plane_stride,
+                                 const float* Sb, int64_t lds, float* biasT, int64_t n, int ell, float* Z, cudaStream_t st);
 
 // C[z][i][j] = sum over the z-th K-slice of A[i][k] * Bm[j][k]   (both operands contiguous along k).
 // A is M x K (element type dt, pitch lda), Bm is N x K fp32 (pitch ldb). splits >= 1 slices of k.
+// class_F > 0 ("class slices", needs splits * class_F == K): A is M x class_F and slice z contracts ALL of it with the columns
+// [z class_F, (z + 1) class_F) of Bm, so C[z] = A * Bm_z^T: the per-class projections of structured rows in one launch.
 cudaError_t launch_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const float* Bm, int64_t ldb, int M, int N,
-                           int64_t K, int splits, float* C, int64_t ldc, int64_t split_stride, cudaStream_t st);
+                           int64_t K, int splits, float* C, int64_t ldc, int64_t split_stride, cudaStream_t st, int64_t class_F = 0);
 
 // Tensor-core version of launch_gemm_nt (tcgen05 + TMA). Both operands have element type dt (fp32 operands are
 // read as tf32) and must satisfy TMA's rules: 16-byte aligned base, pitch a multiple of 16 bytes.
@@ -51,7 +60,8 @@ cudaError_t launch_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const fl
 // Without fold N <= 256. *err (device) is set to 1 if a bounded wait inside the kernel ran out.
 // mt (1, 2 or 4) row tiles of 128 share each B tile inside one CTA; needs mt * (fold ? 2 n_pad : n_pad) <= 512.
 cudaError_t launch_tc_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const void* Bm, int64_t ldb, int M, int N, int fold,
-                              int mt, int64_t K, int splits, float* C, int64_t ldc, int64_t split_stride, int* err, cudaStream_t st);
+                              int mt, int64_t K, int splits, float* C, int64_t ldc, int64_t split_stride, int* err, cudaStream_t st,
+                              int64_t class_F = 0);   // class slices as in launch_gemm_nt; needs class_F * element size a multiple of 16
 
 // fp32-faithful tensor-core C[z] = A_z * Bm_z^T for fp32 operands (three tf32 MMAs on hi/lo halves split in shared
 // memory, accumulator drained into registers every few K tiles). Same alignment rules and return convention as
@@ -62,7 +72,8 @@ cudaError_t launch_tc_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const
 // sym == 2 (projection onto at most 64 sketch rows): Bm is the sketch already split by launch_split_tf32 (128 rows);
 // one MMA per K step; C receives 2 * splits partial planes (split_stride apart) whose sum is A * S^T (M x N).
 cudaError_t launch_tc_gemm_nt_x3(const float* A, int64_t lda, const float* Bm, int64_t ldb, int M, int N, int64_t K, int splits,
-                                 float* C, int64_t ldc, int64_t split_stride, int sym, int* err, cudaStream_t st);
+                                 float* C, int64_t ldc, int64_t split_stride, int sym, int* err, cudaStream_t st,
+                                 int64_t class_F = 0);   // class slices as in launch_gemm_nt; needs class_F a multiple of 4
 cudaError_t launch_gram_sym_reduce(const float* parts, int splits, int64_t stride, int r, int64_t ldp, float* out, int64_t ldo,
                                    cudaStream_t st);
 

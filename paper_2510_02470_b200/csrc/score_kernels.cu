@@ -143,6 +143,80 @@ __global__ void __launch_bounds__(256) k_consensus_score(const double* __restric
     if (lane == 0) scores[row] = fminf(1.f, fmaxf(-1.f, acc));
 }
 
+
+// Structured rows: the projection z_i = sum_c q_ic (S_c h_i + b_c), b_c = column c of the bias block of the sketch, from the
+// per-class planes T_c = H S_c^T. A thread owns four consecutive columns of one row of Z and walks the classes in ascending
+// order (fp32), four classes' loads in flight at a time. biasT is the bias block transposed (C x ell, by k_bias_transpose), so
+// that its reads are contiguous and shared by all rows. Needs ell a multiple of 4 and 16-byte aligned planes.
+template <typename T>
+__global__ void __launch_bounds__(256) k_outer_combine(const T* __restrict__ q, int64_t ldq, int C, const float* __restrict__ planes, int pp,
+                                                       int64_t plane_stride, const float* __restrict__ biasT, int64_t total4, int ell,
+                                                       float* __restrict__ Z) {
+    const int64_t e4 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e4 >= total4) return;
+    const int ell4 = ell >> 2;
+    const int64_t i = e4 / ell4;
+    const int j = (int)(e4 - i * ell4) * 4;
+    const T* qr = q + i * ldq;
+    const float* t = planes + i * ell + j;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int cb = 0; cb < C; cb += 4) {
+        float4 v[4];
+        float qc[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int c = cb + u;
+            qc[u] = c < C ? (float)qr[c] : 0.f;
+            v[u] = c < C ? __ldg(reinterpret_cast<const float4*>(biasT + (int64_t)c * ell + j)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        for (int p = 0; p < pp; ++p) {
+            float4 w[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                w[u] = cb + u < C ? __ldcs(reinterpret_cast<const float4*>(t + ((int64_t)(cb + u) * pp + p) * plane_stride))
+                                  : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) { v[u].x += w[u].x; v[u].y += w[u].y; v[u].z += w[u].z; v[u].w += w[u].w; }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            acc.x = fmaf(qc[u], v[u].x, acc.x);
+            acc.y = fmaf(qc[u], v[u].y, acc.y);
+            acc.z = fmaf(qc[u], v[u].z, acc.z);
+            acc.w = fmaf(qc[u], v[u].w, acc.w);
+        }
+    }
+    *reinterpret_cast<float4*>(Z + i * ell + j) = acc;
+}
+
+// biasT[c][j] = Sb[j][c] (Sb: ell rows of pitch lds)
+__global__ void __launch_bounds__(256) k_bias_transpose(const float* __restrict__ Sb, int64_t lds, int C, int ell, float* __restrict__ biasT) {
+    const int x = blockIdx.x * blockDim.x + threadIdx.x;
+    if (x >= C * ell) return;
+    const int j = x / C, c = x - j * C;
+    biasT[(int64_t)c * ell + j] = Sb[(int64_t)j * lds + c];
+}
+
+// any ell: one thread per element
+template <typename T>
+__global__ void __launch_bounds__(256) k_outer_combine_scalar(const T* __restrict__ q, int64_t ldq, int C, const float* __restrict__ planes,
+                                                              int pp, int64_t plane_stride, const float* __restrict__ biasT,
+                                                              int64_t total, int ell, float* __restrict__ Z) {
+    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= total) return;
+    const int64_t i = e / ell;
+    const int j = (int)(e - i * ell);
+    const T* qr = q + i * ldq;
+    const float* t = planes + e;
+    float acc = 0.f;
+    for (int c = 0; c < C; ++c) {
+        float v = __ldg(biasT + (int64_t)c * ell + j);
+        for (int p = 0; p < pp; ++p) v += t[((int64_t)c * pp + p) * plane_stride];
+        acc = fmaf((float)qr[c], v, acc);
+    }
+    Z[e] = acc;
+}
+
 }  // namespace
 
 cudaError_t launch_normalise(const float* Z, int planes, int64_t plane_stride, int64_t ldz, int64_t n, int ell, float* zhat,
@@ -155,6 +229,34 @@ cudaError_t launch_normalise(const float* Z, int planes, int64_t plane_stride, i
     int jw = 32;
     while (jw < ell) jw <<= 1;
     k_accumulate<<<1, 1024, 0, st>>>(partials, nblocks, ell, jw, zsum);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_outer_combine(const void* q, int64_t ldq, sage_dtype_t dt, int C, const float* planes, int pp, int64_t plane_stride,
+                                 const float* Sb, int64_t lds, float* biasT, int64_t n, int ell, float* Z, cudaStream_t st) {
+    const int64_t total = n * ell;
+    if (total <= 0 || C <= 0) return cudaSuccess;
+    k_bias_transpose<<<(unsigned)(((int64_t)C * ell + 255) / 256), 256, 0, st>>>(Sb, lds, C, ell, biasT);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const bool vec = ell % 4 == 0 && plane_stride % 4 == 0 && (reinterpret_cast<uintptr_t>(planes) & 15u) == 0 &&
+                     (reinterpret_cast<uintptr_t>(Z) & 15u) == 0 && (reinterpret_cast<uintptr_t>(biasT) & 15u) == 0;
+    if (vec) {
+        const int64_t total4 = total / 4;
+        const unsigned blocks = (unsigned)((total4 + 255) / 256);
+        if (dt == SAGE_F32)
+            k_outer_combine<float><<<blocks, 256, 0, st>>>(static_cast<const float*>(q), ldq, C, planes, pp, plane_stride, biasT, total4, ell, Z);
+        else
+            k_outer_combine<__nv_bfloat16><<<blocks, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(q), ldq, C, planes, pp, plane_stride,
+                                                                   biasT, total4, ell, Z);
+        return cudaGetLastError();
+    }
+    const unsigned blocks = (unsigned)((total + 255) / 256);
+    if (dt == SAGE_F32)
+        k_outer_combine_scalar<float><<<blocks, 256, 0, st>>>(static_cast<const float*>(q), ldq, C, planes, pp, plane_stride, biasT, total, ell, Z);
+    else
+        k_outer_combine_scalar<__nv_bfloat16><<<blocks, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(q), ldq, C, planes, pp, plane_stride,
+                                                                      biasT, total, ell, Z);
     return cudaGetLastError();
 }
 

@@ -49,23 +49,13 @@ __global__ void __launch_bounds__(256) k_append(const T* __restrict__ rows, int6
 // [vec_rowmajor(q_i h_i^T) ; q_i] with q_i (C values) = softmax - onehot and h_i (F values) the features; it is formed here
 // from the two factors and written straight into the destination rows, so the C F + C values never exist in the caller's
 // memory. Products are taken in fp32 (exact for bf16 factors). Columns from C F + C up to the pitch are zeroed.
-// Out = float: the buffer rows of pass 1 and the scoring scratch of fp32 handles. Out = bfloat16: the scoring scratch of
-// bfloat16 handles, each product rounded to nearest even (the row as a caller holding bfloat16 rows would have stored it).
-__device__ __forceinline__ void store4(float* p, const float v[4]) { *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]); }
-__device__ __forceinline__ void store4(__nv_bfloat16* p, const float v[4]) {
-    __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
-    uint2 raw;
-    raw.x = *reinterpret_cast<uint32_t*>(&a);
-    raw.y = *reinterpret_cast<uint32_t*>(&b);
-    *reinterpret_cast<uint2*>(p) = raw;
-}
-template <typename T, typename Out>
+template <typename T>
 __global__ void __launch_bounds__(256) k_append_outer(const T* __restrict__ q, int64_t ldq, const T* __restrict__ feat, int64_t ldf, int C,
-                                                      int F, Out* __restrict__ B, int64_t pitch, int dst_row0) {
+                                                      int F, float* __restrict__ B, int64_t pitch, int dst_row0) {
     const int64_t row = blockIdx.y;
     const T* qr = q + row * ldq;
     const T* hr = feat + row * ldf;
-    Out* dst = B + (int64_t)(dst_row0 + row) * pitch;
+    float* dst = B + (int64_t)(dst_row0 + row) * pitch;
     const int64_t CF = (int64_t)C * F, D = CF + C;
     const int64_t c0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x * 4;
@@ -89,7 +79,7 @@ __global__ void __launch_bounds__(256) k_append_outer(const T* __restrict__ q, i
                 }
             }
         }
-        store4(dst + d, v);
+        *reinterpret_cast<float4*>(dst + d) = make_float4(v[0], v[1], v[2], v[3]);
     }
 }
 
@@ -121,7 +111,7 @@ __device__ __forceinline__ void load4(const T* p, bool vec, int64_t k, int64_t k
 
 template <typename T>
 __global__ void __launch_bounds__(256) k_gemm_nt(const T* __restrict__ A, int64_t lda, const float* __restrict__ Bm,
-                                                 int64_t ldb, int M, int N, int64_t K, int64_t k_per_split,
+                                                 int64_t ldb, int M, int N, int64_t K, int64_t k_per_split, int a_shared,
                                                  float* __restrict__ C, int64_t ldc, int64_t split_stride) {
     __shared__ float As[BK][BM + PAD];
     __shared__ float Bs[BK][BN + PAD];
@@ -132,8 +122,10 @@ __global__ void __launch_bounds__(256) k_gemm_nt(const T* __restrict__ A, int64_
     const int lrow = tid >> 3;          // 0..31
     const int lk = (tid & 7) * 4;       // 0,4,..,28
     const int ty = tid >> 4, tx = tid & 15;
+    // class slices (a_shared): slice z contracts columns [0, k_per_split) of A with columns [k_begin, k_end) of Bm
+    const int64_t a_back = a_shared ? k_begin : 0;
     const bool a_vec = (lda * sizeof(T)) % (4 * sizeof(T)) == 0 && (reinterpret_cast<uintptr_t>(A) % (4 * sizeof(T))) == 0 &&
-                       (lda % 4 == 0) && (k_begin % 4 == 0);
+                       (lda % 4 == 0) && ((k_begin - a_back) % 4 == 0);
     const bool b_vec = (ldb % 4 == 0) && (reinterpret_cast<uintptr_t>(Bm) % 16 == 0) && (k_begin % 4 == 0);
 
     float acc[4][4] = {}, tot[4][4] = {};
@@ -143,7 +135,7 @@ __global__ void __launch_bounds__(256) k_gemm_nt(const T* __restrict__ A, int64_
         for (int h = 0; h < 2; ++h) {
             const int r = lrow + h * 32;
             float v[4] = {0.f, 0.f, 0.f, 0.f};
-            if (m0 + r < M) load4(A + (int64_t)(m0 + r) * lda, a_vec, k0 + lk, k_end, v);
+            if (m0 + r < M) load4(A + (int64_t)(m0 + r) * lda, a_vec, k0 + lk - a_back, k_end - a_back, v);
 #pragma unroll
             for (int i = 0; i < 4; ++i) As[lk + i][r] = v[i];
             float w[4] = {0.f, 0.f, 0.f, 0.f};
@@ -334,37 +326,36 @@ cudaError_t launch_append(const void* rows, sage_dtype_t dt, int64_t n, int64_t 
 }
 
 cudaError_t launch_append_outer(const void* q, int64_t ldq, const void* feat, int64_t ldf, sage_dtype_t dt, int64_t n, int C, int F,
-                                void* B, sage_dtype_t out_dt, int64_t pitch, int dst_row0, cudaStream_t st) {
+                                float* B, int64_t pitch, int dst_row0, cudaStream_t st) {
     if (n <= 0) return cudaSuccess;
-    if ((pitch & 3) || (out_dt == SAGE_BF16 && dt != SAGE_BF16)) return cudaErrorInvalidValue;
+    if (pitch & 3) return cudaErrorInvalidValue;
     int64_t bx = (pitch / 4 + 255) / 256;
     if (bx > 592) bx = 592;
     if (bx < 1) bx = 1;
     dim3 grid((unsigned)bx, (unsigned)n);
     if (dt == SAGE_F32)
-        k_append_outer<float, float><<<grid, 256, 0, st>>>(static_cast<const float*>(q), ldq, static_cast<const float*>(feat), ldf, C, F,
-                                                           static_cast<float*>(B), pitch, dst_row0);
-    else if (out_dt == SAGE_F32)
-        k_append_outer<__nv_bfloat16, float><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(q), ldq, static_cast<const __nv_bfloat16*>(feat),
-                                                                   ldf, C, F, static_cast<float*>(B), pitch, dst_row0);
+        k_append_outer<float><<<grid, 256, 0, st>>>(static_cast<const float*>(q), ldq, static_cast<const float*>(feat), ldf, C, F, B, pitch,
+                                                    dst_row0);
     else
-        k_append_outer<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(q), ldq,
-                                                                           static_cast<const __nv_bfloat16*>(feat), ldf, C, F,
-                                                                           static_cast<__nv_bfloat16*>(B), pitch, dst_row0);
+        k_append_outer<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(q), ldq, static_cast<const __nv_bfloat16*>(feat),
+                                                            ldf, C, F, B, pitch, dst_row0);
     return cudaGetLastError();
 }
 
 cudaError_t launch_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const float* Bm, int64_t ldb, int M, int N,
-                           int64_t K, int splits, float* C, int64_t ldc, int64_t split_stride, cudaStream_t st) {
+                           int64_t K, int splits, float* C, int64_t ldc, int64_t split_stride, cudaStream_t st, int64_t class_F) {
     if (M <= 0 || N <= 0) return cudaSuccess;
+    if (class_F > 0 && (int64_t)splits * class_F != K) return cudaErrorInvalidValue;
     int64_t kps = (K + splits - 1) / splits;
     kps = ((kps + BK - 1) / BK) * BK;
+    if (class_F > 0) kps = class_F;
+    const int a_shared = class_F > 0 ? 1 : 0;
     dim3 grid((M + BM - 1) / BM, (N + BN - 1) / BN, splits);
     if (dt == SAGE_F32)
-        k_gemm_nt<float><<<grid, 256, 0, st>>>(static_cast<const float*>(A), lda, Bm, ldb, M, N, K, kps, C, ldc, split_stride);
+        k_gemm_nt<float><<<grid, 256, 0, st>>>(static_cast<const float*>(A), lda, Bm, ldb, M, N, K, kps, a_shared, C, ldc, split_stride);
     else
-        k_gemm_nt<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(A), lda, Bm, ldb, M, N, K, kps, C, ldc,
-                                                       split_stride);
+        k_gemm_nt<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(A), lda, Bm, ldb, M, N, K, kps, a_shared, C,
+                                                       ldc, split_stride);
     return cudaGetLastError();
 }
 

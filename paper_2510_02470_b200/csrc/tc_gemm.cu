@@ -51,8 +51,8 @@ constexpr int kATileBytes = kTileM * 128;
 template <int kFmt>
 __global__ void __launch_bounds__(kThreads, 1)
 k_tc_gemm_nt(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, int M, int N, int n_pad, int fold,
-             int mt, long long K, long long k_per_split, float* __restrict__ C, long long ldc, long long split_stride, int stages,
-             uint32_t tmem_cols, int* __restrict__ err) {
+             int mt, long long K, long long k_per_split, int a_shared, float* __restrict__ C, long long ldc, long long split_stride,
+             int stages, uint32_t tmem_cols, int* __restrict__ err) {
     constexpr int BK = kFmt == 1 ? 64 : 32;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -98,8 +98,9 @@ k_tc_gemm_nt(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 if (!mbar_wait(&empty[s], (use & 1u) ^ 1u, abort)) break;
                 mbar_expect_tx(&full[s], tx_bytes);
                 const int x = (int)(k_begin + (long long)kt * BK);
+                const int xa = a_shared ? kt * BK : x;   // class slices: every slice reads the same columns of A
                 for (int t = 0; t < mt; ++t)     // row tiles past the end of A are zero-filled by TMA
-                    tma_load_2d(smem + (size_t)s * stage_bytes + (size_t)t * kATileBytes, &tmA, &full[s], x, m0 + t * kTileM);
+                    tma_load_2d(smem + (size_t)s * stage_bytes + (size_t)t * kATileBytes, &tmA, &full[s], xa, m0 + t * kTileM);
                 tma_load_2d(smem + (size_t)s * stage_bytes + a_bytes, &tmB, &full[s], x, 0);
                 issued = kt + 1;
             }
@@ -183,7 +184,8 @@ k_tc_gemm_nt(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 }  // namespace tc
 
 cudaError_t launch_tc_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const void* Bm, int64_t ldb, int M, int N, int fold,
-                              int mt, int64_t K, int splits, float* C, int64_t ldc, int64_t split_stride, int* err, cudaStream_t st) {
+                              int mt, int64_t K, int splits, float* C, int64_t ldc, int64_t split_stride, int* err, cudaStream_t st,
+                              int64_t class_F) {
     if (M <= 0 || N <= 0 || K <= 0) return cudaSuccess;
     const int es = dt == SAGE_F32 ? 4 : 2;
     const int BK = 128 / es;
@@ -192,11 +194,17 @@ cudaError_t launch_tc_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const
     if (n_mma > 256 || splits < 1 || splits > 65535) return cudaErrorNotSupported;
     if ((mt != 1 && mt != 2 && mt != 4) || mt * n_mma > 512) return cudaErrorNotSupported;
     CUtensorMap tmA, tmB;
-    if (!tc::make_tmap_2d(&tmA, A, es, (uint64_t)M, (uint64_t)K, (uint64_t)lda, tc::kTileM)) return cudaErrorNotSupported;
+    // class slices: A has class_F columns, slice c contracts them with columns [c class_F, (c + 1) class_F) of Bm. A slice
+    // starts at a multiple of class_F, which TMA wants on a 16-byte boundary; its last K tile may reach into the next
+    // slice's columns of Bm, where A reads as zero (beyond its extent).
+    if (class_F > 0 && ((class_F * es) % 16 != 0 || (int64_t)splits * class_F != K)) return cudaErrorNotSupported;
+    if (!tc::make_tmap_2d(&tmA, A, es, (uint64_t)M, (uint64_t)(class_F > 0 ? class_F : K), (uint64_t)lda, tc::kTileM)) return cudaErrorNotSupported;
     if (!tc::make_tmap_2d(&tmB, Bm, es, (uint64_t)(fold ? n_pad + N : N), (uint64_t)K, (uint64_t)ldb, (uint32_t)n_mma))
         return cudaErrorNotSupported;
     int64_t kps = (K + splits - 1) / splits;
     kps = ((kps + BK - 1) / BK) * BK;
+    if (class_F > 0) kps = class_F;
+    const int a_shared = class_F > 0 ? 1 : 0;
     // a trailing slice may be empty after rounding to whole K tiles: its CTAs store zeros
     const int stage_bytes = mt * tc::kATileBytes + n_mma * 128;
     int stages = (200 * 1024) / stage_bytes;
@@ -211,12 +219,12 @@ cudaError_t launch_tc_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const
     if (dt == SAGE_BF16) {
         e = cudaFuncSetAttribute(tc::k_tc_gemm_nt<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        tc::k_tc_gemm_nt<1><<<grid, tc::kThreads, smem, st>>>(tmA, tmB, M, N, n_pad, fold, mt, K, kps, C, ldc, split_stride, stages,
+        tc::k_tc_gemm_nt<1><<<grid, tc::kThreads, smem, st>>>(tmA, tmB, M, N, n_pad, fold, mt, K, kps, a_shared, C, ldc, split_stride, stages,
                                                               tmem_cols, err);
     } else {
         e = cudaFuncSetAttribute(tc::k_tc_gemm_nt<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        tc::k_tc_gemm_nt<2><<<grid, tc::kThreads, smem, st>>>(tmA, tmB, M, N, n_pad, fold, mt, K, kps, C, ldc, split_stride, stages,
+        tc::k_tc_gemm_nt<2><<<grid, tc::kThreads, smem, st>>>(tmA, tmB, M, N, n_pad, fold, mt, K, kps, a_shared, C, ldc, split_stride, stages,
                                                               tmem_cols, err);
     }
     return cudaGetLastError();

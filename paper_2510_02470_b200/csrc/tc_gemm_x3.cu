@@ -61,8 +61,8 @@ __device__ __forceinline__ uint4 lo4(const uint4 v, float scale) {
 
 __global__ void __launch_bounds__(kThreads, 1)
 k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, int M, int N, int gram,
-                int b_box_rows, int sym, long long K, long long k_per_split, float* __restrict__ C, long long ldc, long long split_stride,
-                int stages, int stage_bytes, int* __restrict__ err) {
+                int b_box_rows, int sym, long long K, long long k_per_split, int a_shared, float* __restrict__ C, long long ldc,
+                long long split_stride, int stages, int stage_bytes, int* __restrict__ err) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     const int m0 = blockIdx.x * kTileM, n0 = blockIdx.y * kTileN;
@@ -123,7 +123,7 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 mbar_expect_tx(&full[s], (uint32_t)(proj ? 2 * kTileBytes : half_bytes));
                 const int x = (int)(k_begin + (long long)kt * BK);
                 uint8_t* st = smem + (size_t)s * stage_bytes;
-                tma_load_2d(st, &tmA, &full[s], x, m0);
+                tma_load_2d(st, &tmA, &full[s], a_shared ? kt * BK : x, m0);   // class slices: the same columns of A for every slice
                 if (proj) tma_load_2d(st + 2 * kTileBytes, &tmB, &full[s], x, 0);
                 else if (!diag) tma_load_2d(st + kTileBytes, &tmB, &full[s], x, n0);
                 issued = kt + 1;
@@ -298,19 +298,22 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 }  // namespace tc
 
 cudaError_t launch_tc_gemm_nt_x3(const float* A, int64_t lda, const float* Bm, int64_t ldb, int M, int N, int64_t K, int splits,
-                                 float* C, int64_t ldc, int64_t split_stride, int sym, int* err, cudaStream_t st) {
+                                 float* C, int64_t ldc, int64_t split_stride, int sym, int* err, cudaStream_t st, int64_t class_F) {
     if (M <= 0 || N <= 0 || K <= 0) return cudaSuccess;
     if (splits < 1 || splits > 65535) return cudaErrorNotSupported;
     const int gram = (A == Bm && lda == ldb && M == N) ? 1 : 0;
     const bool proj = sym == 2;       // Bm: the sketch split into [hi (64 rows) ; lo (64 rows)], 128 rows of pitch ldb; N <= 64
     if (sym == 1 && !(gram && M <= tc::kTileM)) return cudaErrorInvalidValue;
     if (proj && (N > 64 || gram)) return cudaErrorInvalidValue;
+    // class slices: see launch_tc_gemm_nt
+    if (class_F > 0 && (gram || class_F % 4 != 0 || (int64_t)splits * class_F != K)) return cudaErrorNotSupported;
     CUtensorMap tmA, tmB;
-    if (!tc::make_tmap_2d(&tmA, A, 4, (uint64_t)M, (uint64_t)K, (uint64_t)lda, tc::kTileM)) return cudaErrorNotSupported;
+    if (!tc::make_tmap_2d(&tmA, A, 4, (uint64_t)M, (uint64_t)(class_F > 0 ? class_F : K), (uint64_t)lda, tc::kTileM)) return cudaErrorNotSupported;
     const int b_box_rows = proj ? tc::kTileN : (N >= tc::kTileN ? tc::kTileN : ((N + 15) / 16) * 16);
     if (!tc::make_tmap_2d(&tmB, Bm, 4, (uint64_t)(proj ? 128 : N), (uint64_t)K, (uint64_t)ldb, (uint32_t)b_box_rows)) return cudaErrorNotSupported;
     int64_t kps = (K + splits - 1) / splits;
     kps = ((kps + tc::BK - 1) / tc::BK) * tc::BK;
+    if (class_F > 0) kps = class_F;
     // a trailing slice may be empty after rounding to whole K tiles: its CTAs store zeros
     // a Gram matrix of at most 128 rows has diagonal tiles only: one operand per stage
     const int stage_bytes = proj ? 3 * tc::kTileBytes : 2 * ((gram && M <= tc::kTileM) ? tc::kTileBytes : tc::kTileBytes + b_box_rows * 128);
@@ -320,7 +323,7 @@ cudaError_t launch_tc_gemm_nt_x3(const float* A, int64_t lda, const float* Bm, i
     dim3 grid((unsigned)((M + tc::kTileM - 1) / tc::kTileM), proj ? 1u : (unsigned)((N + tc::kTileN - 1) / tc::kTileN), (unsigned)splits);
     cudaError_t e = cudaFuncSetAttribute(tc::k_tc_gemm_nt_x3, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    tc::k_tc_gemm_nt_x3<<<grid, tc::kThreads, smem, st>>>(tmA, tmB, M, N, gram, b_box_rows, sym, K, kps, C, ldc, split_stride, stages,
+    tc::k_tc_gemm_nt_x3<<<grid, tc::kThreads, smem, st>>>(tmA, tmB, M, N, gram, b_box_rows, sym, K, kps, class_F > 0 ? 1 : 0, C, ldc, split_stride, stages,
                                                                  stage_bytes, err);
     return cudaGetLastError();
 }

@@ -1,6 +1,7 @@
 """GPU parity for structured last-layer rows: the library is given the factors (q = softmax - onehot, h = features) and
 must give what the oracle gives on the materialised rows [vec(q h^T) ; q]. Through the C ABI's binding; tolerances as
-in the dense tests (pass 1 forms the products exactly; the scoring pass of a bfloat16 handle rounds them to bfloat16)."""
+in the dense tests (pass 1 forms the products exactly; the scoring pass never forms the rows: it projects the features onto
+every class block of the sketch and folds the results with the other factor)."""
 import numpy as np
 import pytest
 import torch
@@ -78,7 +79,6 @@ def test_structured_rows_match_oracle(dtype, N, C, F, ell, ldq, ldf):
     q, h = factors(N, C, F, N + C, dtype, ldq, ldf)
     ref = structured.run(q[:, :C], h[:, :F], ell, 0.2, route=1)
     S, a, idx, st = gpu_outer(q, h, C, F, ell, 0.2, cuts=[N // 3, N - N // 3])
-    # pass 1 forms the products q_c h_f exactly; the scoring pass of a bfloat16 handle rounds them to bfloat16 rows
     print(check(q, h, C, F, ell, 0.2, S, a, idx, st, ref, TOL_SCORE[dtype]))
 
 
@@ -102,6 +102,41 @@ def test_structured_and_dense_calls_mix_and_agree():
     fd.close()
     assert metrics.signed_gram_norm(S.double().cpu().numpy(), ref["S"]) / float(np.linalg.norm(G.double().numpy()) ** 2) <= TOL_SKETCH
     assert np.max(np.abs(a - ref["alpha"])) <= 1e-4 and np.max(np.abs(a - b)) <= 1e-5
+
+
+@pytest.mark.parametrize("dtype,ell,tol", [(torch.float32, 64, 2e-5), (torch.bfloat16, 128, TOL_SCORE[torch.bfloat16])])
+def test_structured_scoring_over_several_sub_chunks_agrees_with_dense_rows(dtype, ell, tol):
+    """c3-shaped factors (100 classes x 512 features), 45,000 rows: the per-class planes of that many rows do not fit the
+    1 GiB the library allows itself, so the scoring pass takes several sub-chunks. The reference is the dense scoring
+    pass of the same handle on rows materialised on the device a chunk at a time (itself checked against the oracle
+    by the dense tests); fp32 products are exact, bfloat16 rows carry the rounding of each product."""
+    N, C, F = 45000, 100, 512
+    D = C * F + C
+    g = torch.Generator(device=DEV).manual_seed(11)
+    cls = torch.randint(0, C, (N,), device=DEV, generator=g)
+    mu = torch.randn((C, F), device=DEV, generator=g)
+    h = torch.relu(mu[cls] + torch.randn((N, F), device=DEV, generator=g))
+    q = torch.softmax(h @ torch.relu(mu).T / F ** 0.5, dim=1)
+    q[torch.arange(N, device=DEV), cls] -= 1.0
+    q, h = q.to(dtype).contiguous(), h.to(dtype).contiguous()
+    fd = sage.SageFD(D, ell, dtype, 0)
+    fd.update_outer(q[:3 * ell], h[:3 * ell], C, F)
+    fd.finalize()
+    a = fd.score_outer(q, h, C, F).double().cpu().numpy()
+    b = torch.empty((N,), dtype=torch.float32, device=DEV)
+    fd.score_begin(N)
+    for r0 in range(0, N, 9000):
+        qs, hs = q[r0:r0 + 9000].float(), h[r0:r0 + 9000].float()
+        rows = torch.cat([(qs[:, :, None] * hs[:, None, :]).reshape(qs.shape[0], C * F), qs], dim=1).to(dtype)
+        fd.score_chunk(rows, r0)
+        torch.cuda.synchronize()
+        del rows
+    fd.score_end(b)
+    torch.cuda.synchronize()
+    st = fd.stats()
+    fd.close()
+    assert st["device_flags"] == 0
+    assert np.max(np.abs(a - b.double().cpu().numpy())) <= tol
 
 
 def test_structured_rows_merged_sketches_and_errors():
