@@ -15,16 +15,22 @@
 // One CTA owns a 128 x (<=128) output tile and one K slice:
 //   warp 0    TMA producer (raw fp32 tiles, 128-byte swizzle),
 //   warp 1    TMEM allocation and MMA issue into a ring of four accumulators,
-//   warps 2-9 write the lo part of each landed stage into its second buffer, as two groups of four warps that take
-//             alternate stages; every kChunk stages each warp also drains its lanes and columns of the accumulator
+//   warps 2-9 write the lo part of each landed stage into its second buffer. The stage slots are dealt to G groups of
+//             8 / G warps (G = the number of stages where that is at most 8: one warp per slot), so as many
+//             wait -> load -> remainder -> store -> fence -> arrive chains are in flight as there are slots (measured on the
+//             128 x 11.2 M Gram matrix: two groups of four warps 1.64 ms, six groups of one 1.54 ms, seven stages with seven
+//             groups 1.46 ms). Every kChunk stages each warp also drains its lanes and columns of the accumulator
 //             that was finished ring / 2 chunks earlier (its MMAs are long done, so the drain hardly waits) into
 //             registers, and stores them at the end. Warp w drains TMEM lanes 32 * (w % 4), columns 64 * ((w - 2) / 4).
+// The producer and the MMA thread keep running stage / phase / chunk counters and advance the operand descriptors by a
+// constant per stage: with integer divisions and freshly built descriptors in its loop the single MMA-issuing thread took
+// 1,500 cycles per K tile and was what bounded the kernel (now about 600).
 // On the diagonal tiles of a Gram matrix only one operand tile is loaded and used on both sides. A Gram matrix
-// of at most 128 rows (sym mode) needs ONE 256-wide MMA per K step: the hi tile and the (doubled) lo tile lie
-// back to back in the stage and serve as one 256-row B operand, so the accumulator holds hi*hi^T | 2*hi*lo^T side
-// by side; their sum T satisfies (T + T^T)/2 = hi*hi^T + hi*lo^T + lo*hi^T, formed by the split reduction. (Issuing
-// a tf32 MMA costs the issuing thread about 110 cycles whatever its width, and a 128 x 128 x 8 one executes in
-// about 70: narrow MMAs leave the tensor pipe idle, wide ones do not.)
+// of at most 128 rows (sym mode) needs ONE 256-wide MMA per K step: the hi tile and the lo tile lie back to back
+// in the stage and serve as one 256-row B operand, so the accumulator holds hi*hi^T | hi*lo^T side by side; the drain
+// forms T = hi*hi^T + 2*hi*lo^T (the doubling is exact), which satisfies (T + T^T)/2 = hi*hi^T + hi*lo^T + lo*hi^T,
+// formed by the split reduction. (A 128 x 128 x 8 tf32 MMA executes in about 70 cycles, less than issuing it costs
+// the issuing thread: narrow MMAs leave the tensor pipe idle, wide ones do not.)
 // The projection of fp32 rows onto a sketch of at most 64 rows (proj mode, sym = 2) uses the same wide form with the
 // operands' roles exchanged: the sketch, split once into [hi (64 rows) ; lo (64 rows)] when it was frozen, is the
 // 128-row A operand and needs no work per stage; the tile of 128 data rows is split by the workers into hi | lo and
@@ -50,19 +56,17 @@ constexpr int kAccs = 4;                    // accumulators in TMEM (4 x 128 col
 // The tensor cores read an fp32 word as tf32 by ignoring its low 13 bits, so the raw tile already is the hi operand
 // (hi = x with those bits cleared) and only the remainder has to be written: lo = x - hi, exact, then rounded to 11
 // significant bits so that the hardware's truncation of lo finds nothing to cut (a truncated lo would bias sums of
-// like-signed products). `scale` is 1 or, for the doubled remainder of sym mode, 2.
-__device__ __forceinline__ uint32_t lo_of(uint32_t x, float scale) {
-    const float l = scale * (__uint_as_float(x) - __uint_as_float(x & 0xffffe000u));
+// like-signed products).
+__device__ __forceinline__ uint32_t lo_of(uint32_t x) {
+    const float l = __uint_as_float(x) - __uint_as_float(x & 0xffffe000u);
     return (__float_as_uint(l) + 0x1000u) & 0xffffe000u;
 }
-__device__ __forceinline__ uint4 lo4(const uint4 v, float scale) {
-    return make_uint4(lo_of(v.x, scale), lo_of(v.y, scale), lo_of(v.z, scale), lo_of(v.w, scale));
-}
+__device__ __forceinline__ uint4 lo4(const uint4 v) { return make_uint4(lo_of(v.x), lo_of(v.y), lo_of(v.z), lo_of(v.w)); }
 
 __global__ void __launch_bounds__(kThreads, 1)
 k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, int M, int N, int gram,
                 int b_box_rows, int sym, long long K, long long k_per_split, int a_shared, float* __restrict__ C, long long ldc,
-                long long split_stride, int stages, int stage_bytes, int* __restrict__ err) {
+                long long split_stride, int stages, int stage_bytes, int G, int* __restrict__ err) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     const int m0 = blockIdx.x * kTileM, n0 = blockIdx.y * kTileN;
@@ -95,7 +99,7 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
             mbar_init(&full[s], 1);
-            mbar_init(&split_done[s], (stages & 1) ? kWorkers / 32 : kWorkers / 64);   // one arrival per warp that handles the stage
+            mbar_init(&split_done[s], 8 / G);                           // one arrival per warp of the group that owns the slot
             mbar_init(&empty[s], 1);
         }
         for (int b = 0; b < kAccs; ++b) {
@@ -116,17 +120,21 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     if (warp == 0) {
         if (lane == 0) {
             int issued = 0;
+            int s = 0;
+            uint32_t ph = 1;                                    // parity of the empty-barrier phase to wait for
+            int x = (int)k_begin, xa = a_shared ? 0 : (int)k_begin;   // class slices: the same columns of A for every slice
+            uint8_t* st = smem;
+            const uint32_t tx_bytes = (uint32_t)(proj ? 2 * kTileBytes : half_bytes);
             for (int kt = 0; kt < nkt; ++kt) {
-                const int s = kt % stages;
-                const uint32_t use = (uint32_t)(kt / stages);
-                if (!mbar_wait(&empty[s], (use & 1u) ^ 1u, abort)) break;
-                mbar_expect_tx(&full[s], (uint32_t)(proj ? 2 * kTileBytes : half_bytes));
-                const int x = (int)(k_begin + (long long)kt * BK);
-                uint8_t* st = smem + (size_t)s * stage_bytes;
-                tma_load_2d(st, &tmA, &full[s], a_shared ? kt * BK : x, m0);   // class slices: the same columns of A for every slice
+                if (!mbar_wait(&empty[s], ph, abort)) break;
+                mbar_expect_tx(&full[s], tx_bytes);
+                tma_load_2d(st, &tmA, &full[s], xa, m0);
                 if (proj) tma_load_2d(st + 2 * kTileBytes, &tmB, &full[s], x, 0);
                 else if (!diag) tma_load_2d(st + kTileBytes, &tmB, &full[s], x, n0);
                 issued = kt + 1;
+                x += BK;
+                xa += BK;
+                if (++s == stages) { s = 0; ph ^= 1u; st = smem; } else { st += stage_bytes; }
             }
             if (*abort) {
                 for (int kt = issued > stages ? issued - stages : 0; kt < issued; ++kt)
@@ -136,38 +144,51 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     } else if (warp == 1) {
         if (lane == 0) {
             const uint32_t idesc = instr_desc(2, kTileM, wide ? 2 * kTileN : n_pad, 0, 0);
-            bool alive = true;
-            for (int kt = 0; kt < nkt && alive; ++kt) {
-                const int s = kt % stages;
-                const uint32_t use = (uint32_t)(kt / stages);
-                const int c = kt / kChunk, b = c % ring, in_chunk = kt - c * kChunk;
-                if (in_chunk == 0) alive = mbar_wait(&acc_empty[b], (((uint32_t)c / ring) & 1u) ^ 1u, abort);
-                if (alive) alive = mbar_wait(&split_done[s], use & 1u, abort);
-                if (!alive) break;
+            // everything but the start address of an operand descriptor (see smem_desc_k_sw128); the addresses advance by
+            // stage_bytes per stage
+            const uint64_t desc_hi = smem_desc_k_sw128(0);
+            const uint32_t st0 = smem_u32(smem);
+            const uint32_t a_hi_off = proj ? 2 * kTileBytes : 0, a_lo_off = half_bytes;   // proj: A = the split sketch
+            const uint32_t b_hi_off = (diag || proj) ? 0 : kTileBytes, b_lo_off = b_hi_off + half_bytes;
+            int s = 0, in_chunk = 0, b = 0;
+            uint32_t ph = 0, acc_par = 1;
+            uint32_t st = st0;
+            for (int kt = 0; kt < nkt; ++kt) {
+                if (in_chunk == 0 && !mbar_wait(&acc_empty[b], acc_par, abort)) break;
+                if (!mbar_wait(&split_done[s], ph, abort)) break;
                 tc_fence_after();
-                const uint32_t st = smem_u32(smem + (size_t)s * stage_bytes);
-                const uint32_t a_hi = proj ? st + 2 * kTileBytes : st, a_lo = st + half_bytes;   // proj: A = the split sketch
-                const uint32_t b_hi = (diag || proj) ? st : st + kTileBytes, b_lo = b_hi + half_bytes;
-                const uint64_t d_ahi = smem_desc_k_sw128(a_hi), d_alo = smem_desc_k_sw128(a_lo);
-                const uint64_t d_bhi = smem_desc_k_sw128(b_hi), d_blo = smem_desc_k_sw128(b_lo);
+                const uint64_t d_ahi = desc_hi | ((st + a_hi_off) >> 4), d_bhi = desc_hi | ((st + b_hi_off) >> 4);
                 const uint32_t acc = tmem_base + (uint32_t)(b * acc_cols);
+                if (wide) {                                 // sym: B = [hi ; lo] (the drain doubles the lo half), proj: [hi ; lo]
+                    mma_tf32(acc, d_ahi, d_bhi, idesc, in_chunk != 0);
+                    mma_tf32(acc, d_ahi + 2, d_bhi + 2, idesc, 1);       // 4 x 8 tf32 elements per 128-byte row
+                    mma_tf32(acc, d_ahi + 4, d_bhi + 4, idesc, 1);
+                    mma_tf32(acc, d_ahi + 6, d_bhi + 6, idesc, 1);
+                } else {
+                    const uint64_t d_alo = desc_hi | ((st + a_lo_off) >> 4), d_blo = desc_hi | ((st + b_lo_off) >> 4);
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {          // 4 x 8 tf32 elements per 128-byte row
-                    mma_tf32(acc, d_ahi + 2 * k, d_bhi + 2 * k, idesc, (in_chunk | k) != 0);   // sym: B = [hi ; 2 lo], proj: [hi ; lo]
-                    if (!wide) {
+                    for (int k = 0; k < 4; ++k) {
+                        mma_tf32(acc, d_ahi + 2 * k, d_bhi + 2 * k, idesc, (in_chunk | k) != 0);
                         mma_tf32(acc, d_ahi + 2 * k, d_blo + 2 * k, idesc, 1);
                         mma_tf32(acc, d_alo + 2 * k, d_bhi + 2 * k, idesc, 1);
                     }
                 }
                 mma_commit(&empty[s]);
-                if (in_chunk == kChunk - 1 || kt == nkt - 1) mma_commit(&acc_full[b]);
+                if (in_chunk == kChunk - 1 || kt == nkt - 1) {
+                    mma_commit(&acc_full[b]);
+                    in_chunk = 0;
+                    if (++b == ring) { b = 0; acc_par ^= 1u; }
+                } else {
+                    ++in_chunk;
+                }
+                if (++s == stages) { s = 0; ph ^= 1u; st = st0; } else { st += (uint32_t)stage_bytes; }
             }
         }
     } else {
         // ---- workers: write the lo part of landed stages; drain finished accumulators ----
         const int t = threadIdx.x - 64;                 // 0..255
         const int chunks16 = half_bytes / 16;
-        const float lo_scale = sym == 1 ? 2.f : 1.f;
+        const float lo_scale = sym == 1 ? 2.f : 1.f;          // sym: the lo half of the accumulator counts twice (folded into the drain)
         const int quarter = warp & 3, chalf = (warp - 2) >> 2;
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + (uint32_t)(chalf * 64);
         float acc[64];
@@ -192,7 +213,7 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         tmem_ld_use(v0);
                         tmem_ld_use(v1);
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) acc[16 * q + j] += __uint_as_float(v0[j]) + __uint_as_float(v1[j]);
+                        for (int j = 0; j < 16; ++j) acc[16 * q + j] += fmaf(lo_scale, __uint_as_float(v1[j]), __uint_as_float(v0[j]));
                     }
                 }
             } else {
@@ -219,35 +240,37 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[b]);
         };
-        // The eight warps work as two groups of four (warps 2-5 and 6-9) that take alternate stages: a stage's
-        // load -> remainder -> store -> fence -> arrive chain is latency, and two chains in flight hide half of it.
-        // Only with an even number of stages, though: a stage slot then always belongs to the same group, which sees
-        // every phase of its barrier in turn. With an odd number the slots would alternate between the groups, a
-        // group would skip every other phase, and a parity wait cannot tell "two phases back" from "done".
+        // The stage slots are dealt to G groups of 8 / G warps: group g takes the K tiles kt = g, g + G, ... A slot then
+        // always belongs to the same group (stages is a multiple of G), which sees every phase of its barrier in turn: a
+        // group that skipped a phase could not tell "two phases back" from "done" with a parity wait. Warps beyond
+        // G * (8 / G) only drain.
         int drained = 0;                                // chunks drained so far
-        const bool alt = (stages & 1) == 0;
-        const int grp = alt ? chalf : 0, tg = alt ? t - 128 * grp : t;      // group and thread index within it
-        const int kGroup = alt ? kWorkers / 2 : kWorkers, kstep = alt ? 2 : 1;
-        for (int kt = grp; kt < nkt && ok; kt += kstep) {
-            const int s = kt % stages;
-            const uint32_t use = (uint32_t)(kt / stages);
-            bool landed = mbar_wait(&full[s], use & 1u, abort);
+        const int wpg = 8 / G, ww = warp - 2;
+        const int grp = ww / wpg, tg = (ww - grp * wpg) * 32 + lane;      // group, thread index within it
+        const int kGroup = 32 * wpg, kstep = G;
+        int s = grp % stages;
+        uint32_t ph = (uint32_t)(grp / stages) & 1u;
+        for (int kt = ww < wpg * G ? grp : nkt; kt < nkt && ok; kt += kstep) {
+            bool landed = mbar_wait(&full[s], ph, abort);
             landed = __all_sync(0xffffffffu, landed);
             if (!landed) { ok = false; break; }
             uint4* hi = reinterpret_cast<uint4*>(smem + (size_t)s * stage_bytes);
             uint4* lo = reinterpret_cast<uint4*>(smem + (size_t)s * stage_bytes + half_bytes);
-            for (int c = tg; c < chunks16; c += 4 * kGroup) {      // four independent 16-byte pieces in flight
+            const int s_now = s;
+            s += kstep;                                 // the slot and phase of this group's next K tile
+            while (s >= stages) { s -= stages; ph ^= 1u; }
+            for (int c = tg; c < chunks16; c += 4 * kGroup) {      // four independent 16-byte pieces in flight (eight: slower)
                 uint4 v[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u)
                     if (c + u * kGroup < chunks16) v[u] = hi[c + u * kGroup];
 #pragma unroll
                 for (int u = 0; u < 4; ++u)
-                    if (c + u * kGroup < chunks16) lo[c + u * kGroup] = lo4(v[u], lo_scale);   // sym: doubled remainder
+                    if (c + u * kGroup < chunks16) lo[c + u * kGroup] = lo4(v[u]);
             }
             fence_proxy_async_smem();                   // the tensor cores read these writes
             __syncwarp();                               // one arrival per warp
-            if (lane == 0) mbar_arrive(&split_done[s]);
+            if (lane == 0) mbar_arrive(&split_done[s_now]);
             // a chunk is folded into the registers once the stages of the following ring / 2 chunks have been handled
             // (its MMAs are long done by then); every warp drains its own lanes and columns of every chunk
             while (ok && drained < nchunks && (drained + 1 + ring / 2) * kChunk - kstep <= kt) drain(drained++);
@@ -317,14 +340,22 @@ cudaError_t launch_tc_gemm_nt_x3(const float* A, int64_t lda, const float* Bm, i
     // a trailing slice may be empty after rounding to whole K tiles: its CTAs store zeros
     // a Gram matrix of at most 128 rows has diagonal tiles only: one operand per stage
     const int stage_bytes = proj ? 3 * tc::kTileBytes : 2 * ((gram && M <= tc::kTileM) ? tc::kTileBytes : tc::kTileBytes + b_box_rows * 128);
-    int stages = (200 * 1024) / stage_bytes;
+    // Long K slices of the one-MMA-per-step forms (16 KB of remainders per stage): as many stages as fit the 227 KB a block
+    // may have (7 of 32 KB, 4 of 48 KB), each slot with a worker group of its own (8 / stages warps), so that many
+    // remainder chains overlap. Short slices, and the three-MMA form (32 KB of remainders per stage, 3 stages): the
+    // eight warps work on a stage together (odd number of stages) or as two groups of four on alternate stages, which
+    // finishes a single stage sooner.
+    const bool deep = sym != 0 && kps / tc::BK >= 64;
+    int stages = ((deep ? 227 * 1024 - 1536 : 200 * 1024)) / stage_bytes;
     if (stages > 8) stages = 8;
+    if (stages < 2) return cudaErrorNotSupported;
+    const int G = deep ? stages : ((stages & 1) ? 1 : 2);
     const size_t smem = (size_t)stages * stage_bytes + 1024 + (3 * stages + 2 * tc::kAccs) * 8 + 16;
     dim3 grid((unsigned)((M + tc::kTileM - 1) / tc::kTileM), proj ? 1u : (unsigned)((N + tc::kTileN - 1) / tc::kTileN), (unsigned)splits);
     cudaError_t e = cudaFuncSetAttribute(tc::k_tc_gemm_nt_x3, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     tc::k_tc_gemm_nt_x3<<<grid, tc::kThreads, smem, st>>>(tmA, tmB, M, N, gram, b_box_rows, sym, K, kps, class_F > 0 ? 1 : 0, C, ldc, split_stride, stages,
-                                                                 stage_bytes, err);
+                                                                 stage_bytes, G, err);
     return cudaGetLastError();
 }
 
