@@ -13,7 +13,8 @@
 // tiles then no longer alternate between the accumulators, so a tile's MMAs start after the previous tile's epilogue).
 //
 //   warp 0    TMA producer: per chunk 4 boxes of [32 rows][32 columns] of the buffer (128-byte swizzle with
-//             32-byte atoms, the only layout the tensor cores take for 32-bit MN-major operands) and one box of W,
+//             32-byte atoms, the only layout the tensor cores take for 32-bit MN-major operands) and one box of W; where
+//             all chunk boxes of W fit 64 KB (up to 128 buffer rows onto 64 output rows) they are loaded once and stay,
 //   warp 1    TMEM allocation, MMA issue into two ping-pong accumulators (one per column tile),
 //   warps 2-5 write the lo part of the buffer tile of each landed stage,
 //   warps 6-9 epilogue: TMEM -> registers -> out.
@@ -34,22 +35,25 @@ constexpr int kSpanBytes = kChunkRows * 128;         // 4 KB
 
 __global__ void __launch_bounds__(kThreads, 1)
 k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ CUtensorMap tmW, int r, int keep, int j_pad,
-             long long pitch, long long num_tiles, float* __restrict__ out, int stages, int* __restrict__ err) {
+             long long pitch, long long num_tiles, float* __restrict__ out, int stages, int w_res, int* __restrict__ err) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-    // stage layout: [buffer hi 16 KB][buffer lo 16 KB][W_hi ; W_lo: 2*j_pad rows of 128 bytes]
+    // stage layout: [buffer hi 16 KB][buffer lo 16 KB][W_hi ; W_lo: 2*j_pad rows of 128 bytes]; w_res: the W boxes of all
+    // chunks are loaded once and stay behind the ring (W does not depend on the column tile), the stages hold buffer data only
     const int w_bytes = 2 * j_pad * 128;
-    const int stage_bytes = 2 * kBufBytes + w_bytes;
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)stages * stage_bytes);
+    const int stage_bytes = w_res ? 2 * kBufBytes : 2 * kBufBytes + w_bytes;
+    const int nchunk = (r + kChunkRows - 1) / kChunkRows;
+    uint8_t* wres = smem + (size_t)stages * stage_bytes;
+    uint64_t* full = reinterpret_cast<uint64_t*>(wres + (w_res ? (size_t)nchunk * w_bytes : 0));
     uint64_t* split_done = full + stages;
     uint64_t* empty = split_done + stages;
     uint64_t* acc_full = empty + stages;                   // [2]
     uint64_t* acc_empty = acc_full + 2;                    // [2]
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    uint64_t* w_full = acc_empty + 2;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(w_full + 1);
     volatile int* abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int nchunk = (r + kChunkRows - 1) / kChunkRows;
     const int n_mma = 2 * j_pad;                           // <= 256
     const bool two = nchunk > 8;                           // both accumulators serve one tile
     uint32_t tmem_cols = 32;
@@ -63,6 +67,7 @@ k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ 
             mbar_init(&split_done[s], kSplitThreads);
             mbar_init(&empty[s], 1);
         }
+        mbar_init(w_full, 1);
         for (int b = 0; b < 2; ++b) {
             mbar_init(&acc_full[b], 1);
             mbar_init(&acc_empty[b], kEpiThreads);
@@ -80,23 +85,30 @@ k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ 
 
     if (warp == 0) {
         if (lane == 0) {
-            long long q = 0, issued = 0;
+            long long issued = 0;
             bool alive = true;
+            int s = 0;
+            uint32_t ph = 1;                                // parity of the empty-barrier phase to wait for
+            uint8_t* st = smem;
+            const uint32_t tx_bytes = (uint32_t)(w_res ? kBufBytes : kBufBytes + w_bytes);
+            if (w_res) {
+                mbar_expect_tx(w_full, (uint32_t)(nchunk * w_bytes));
+                for (int c = 0; c < nchunk; ++c) tma_load_2d(wres + (size_t)c * w_bytes, &tmW, w_full, c * kChunkRows, 0);
+            }
             for (long long lt = 0; lt < my_tiles && alive; ++lt) {
-                const long long d0 = (blockIdx.x + lt * gridDim.x) * kTileD;
-                for (int c = 0; c < nchunk; ++c, ++q) {
-                    const int s = (int)(q % stages);
-                    const uint32_t use = (uint32_t)(q / stages);
-                    if (!mbar_wait(&empty[s], (use & 1u) ^ 1u, abort)) { alive = false; break; }
-                    mbar_expect_tx(&full[s], (uint32_t)(kBufBytes + w_bytes));
-                    uint8_t* st = smem + (size_t)s * stage_bytes;
+                const int d0 = (int)((blockIdx.x + lt * gridDim.x) * kTileD);
+                for (int c = 0; c < nchunk; ++c) {
+                    if (!mbar_wait(&empty[s], ph, abort)) { alive = false; break; }
+                    mbar_expect_tx(&full[s], tx_bytes);
 #pragma unroll
-                    for (int sp = 0; sp < 4; ++sp) tma_load_2d(st + sp * kSpanBytes, &tmBuf, &full[s], (int)(d0 + 32 * sp), c * kChunkRows);
-                    tma_load_2d(st + 2 * kBufBytes, &tmW, &full[s], c * kChunkRows, 0);
-                    issued = q + 1;
+                    for (int sp = 0; sp < 4; ++sp) tma_load_2d(st + sp * kSpanBytes, &tmBuf, &full[s], d0 + 32 * sp, c * kChunkRows);
+                    if (!w_res) tma_load_2d(st + 2 * kBufBytes, &tmW, &full[s], c * kChunkRows, 0);
+                    ++issued;
+                    if (++s == stages) { s = 0; ph ^= 1u; st = smem; } else { st += stage_bytes; }
                 }
             }
             if (*abort) {
+                if (w_res) mbar_wait_quiet(w_full, 0, 20000000ll);
                 for (long long k = issued > stages ? issued - stages : 0; k < issued; ++k)
                     mbar_wait_quiet(&full[k % stages], (uint32_t)(k / stages) & 1u, 20000000ll);
             }
@@ -105,31 +117,34 @@ k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ 
         if (lane == 0) {
             const uint32_t idesc_fold = instr_desc(2, kTileD, n_mma, 1, 0);   // A (buffer) MN-major, B (W) K-major
             const uint32_t idesc_half = instr_desc(2, kTileD, j_pad, 1, 0);
-            long long q = 0;
+            // running stage / phase counters and descriptors advanced by a constant per stage: the loop of the single issuing
+            // thread bounds the kernel, so it holds no division and builds no descriptor from scratch
+            const uint64_t desc_w = smem_desc_k_sw128(0), desc_buf = smem_desc_mn_sw128_atom32(0, kSpanBytes);
+            const uint32_t st0 = smem_u32(smem);
             bool alive = true;
+            int s = 0;
+            uint32_t ph = 0, st = st0;
+            const uint32_t wres0 = smem_u32(wres);
+            if (w_res) alive = mbar_wait(w_full, 0, abort);
             for (long long lt = 0; lt < my_tiles && alive; ++lt) {
                 const int b = two ? 0 : (int)(lt & 1);
                 const uint32_t par = two ? (uint32_t)lt : (uint32_t)(lt >> 1);
                 alive = mbar_wait(&acc_empty[b], (par & 1u) ^ 1u, abort);
                 if (!alive) break;
-                for (int c = 0; c < nchunk; ++c, ++q) {
+                for (int c = 0; c < nchunk; ++c) {
                     const uint32_t acc = tmem_base + (uint32_t)((two ? (c >> 3) : b) * n_mma);
                     const int c_in = two ? (c & 7) : c;       // position within this accumulator's run
-                    const int s = (int)(q % stages);
-                    const uint32_t use = (uint32_t)(q / stages);
-                    if (!mbar_wait(&split_done[s], use & 1u, abort)) { alive = false; break; }
+                    if (!mbar_wait(&split_done[s], ph, abort)) { alive = false; break; }
                     tc_fence_after();
-                    const uint32_t st = smem_u32(smem + (size_t)s * stage_bytes);
-                    const uint32_t w_addr = st + 2 * kBufBytes;
-                    const uint64_t d_w = smem_desc_k_sw128(w_addr);
+                    const uint64_t d_w = desc_w | ((w_res ? wres0 + (uint32_t)(c * w_bytes) : st + 2 * kBufBytes) >> 4);
+                    const uint64_t d_hi = desc_buf | (st >> 4), d_lo = desc_buf | ((st + kBufBytes) >> 4);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {          // 8 buffer rows per MMA: one 1024-byte row group
-                        const uint64_t d_hi = smem_desc_mn_sw128_atom32(st + k * 1024, kSpanBytes);
-                        const uint64_t d_lo = smem_desc_mn_sw128_atom32(st + kBufBytes + k * 1024, kSpanBytes);
-                        mma_tf32(acc, d_hi, d_w + 2 * k, idesc_fold, (c_in | k) != 0);   // hi*W_hi | hi*W_lo
-                        mma_tf32(acc, d_lo, d_w + 2 * k, idesc_half, 1);              // + lo*W_hi
+                    for (int k = 0; k < 4; ++k) {          // 8 buffer rows per MMA: one 1024-byte row group (64 descriptor units)
+                        mma_tf32(acc, d_hi + 64 * k, d_w + 2 * k, idesc_fold, (c_in | k) != 0);   // hi*W_hi | hi*W_lo
+                        mma_tf32(acc, d_lo + 64 * k, d_w + 2 * k, idesc_half, 1);              // + lo*W_hi
                     }
                     mma_commit(&empty[s]);
+                    if (++s == stages) { s = 0; ph ^= 1u; st = st0; } else { st += (uint32_t)stage_bytes; }
                 }
                 if (alive) mma_commit(&acc_full[b]);
             }
@@ -137,10 +152,10 @@ k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ 
     } else if (warp < 6) {
         const int t = threadIdx.x - 64;
         const long long total = my_tiles * nchunk;
+        int s = 0;
+        uint32_t ph = 0;
         for (long long q = 0; q < total; ++q) {
-            const int s = (int)(q % stages);
-            const uint32_t use = (uint32_t)(q / stages);
-            if (!mbar_wait(&full[s], use & 1u, abort)) break;
+            if (!mbar_wait(&full[s], ph, abort)) break;
             uint4* hi = reinterpret_cast<uint4*>(smem + (size_t)s * stage_bytes);
             uint4* lo = reinterpret_cast<uint4*>(smem + (size_t)s * stage_bytes + kBufBytes);
 #pragma unroll
@@ -158,6 +173,7 @@ k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ 
             }
             fence_proxy_async_smem();
             mbar_arrive(&split_done[s]);
+            if (++s == stages) { s = 0; ph ^= 1u; }
         }
     } else {
         const int quarter = warp & 3;
@@ -171,23 +187,56 @@ k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ 
             tc_fence_after();
             const long long d = (blockIdx.x + lt * gridDim.x) * kTileD + quarter * 32 + lane;
             const uint32_t acc = lane_base + (uint32_t)(b * n_mma);
-            for (int j0 = 0; j0 < j_pad; j0 += 16) {
-                float v[16], w[16];
-                tmem_ld16(acc + (uint32_t)j0, v);
-                tmem_ld16(acc + (uint32_t)(j_pad + j0), w);
+            for (int j0 = 0; j0 < j_pad; j0 += 32) {
+                // four TMEM loads in flight per wait (hi*W_hi | hi*W_lo halves of two groups of 16 output rows)
+                const bool second = j0 + 16 < j_pad;
+                uint32_t v0[16], w0[16], v1[16], w1[16];
+                tmem_ld16_issue(acc + (uint32_t)j0, v0);
+                tmem_ld16_issue(acc + (uint32_t)(j_pad + j0), w0);
+                if (second) {
+                    tmem_ld16_issue(acc + (uint32_t)(j0 + 16), v1);
+                    tmem_ld16_issue(acc + (uint32_t)(j_pad + j0 + 16), w1);
+                }
+                tmem_ld_wait();
+                tmem_ld_use(v0);
+                tmem_ld_use(w0);
+                float a0[16], a1[16];
 #pragma unroll
-                for (int j = 0; j < 16; ++j) v[j] += w[j];
+                for (int j = 0; j < 16; ++j) a0[j] = __uint_as_float(v0[j]) + __uint_as_float(w0[j]);
+                if (second) {
+                    tmem_ld_use(v1);
+                    tmem_ld_use(w1);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) a1[j] = __uint_as_float(v1[j]) + __uint_as_float(w1[j]);
+                }
                 if (two) {                                  // the second half of the buffer rows, from the other accumulator
-                    float v2[16];
-                    tmem_ld16(acc + (uint32_t)(n_mma + j0), v2);
-                    tmem_ld16(acc + (uint32_t)(n_mma + j_pad + j0), w);
+                    tmem_ld16_issue(acc + (uint32_t)(n_mma + j0), v0);
+                    tmem_ld16_issue(acc + (uint32_t)(n_mma + j_pad + j0), w0);
+                    if (second) {
+                        tmem_ld16_issue(acc + (uint32_t)(n_mma + j0 + 16), v1);
+                        tmem_ld16_issue(acc + (uint32_t)(n_mma + j_pad + j0 + 16), w1);
+                    }
+                    tmem_ld_wait();
+                    tmem_ld_use(v0);
+                    tmem_ld_use(w0);
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) v[j] += v2[j] + w[j];
+                    for (int j = 0; j < 16; ++j) a0[j] += __uint_as_float(v0[j]) + __uint_as_float(w0[j]);
+                    if (second) {
+                        tmem_ld_use(v1);
+                        tmem_ld_use(w1);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) a1[j] += __uint_as_float(v1[j]) + __uint_as_float(w1[j]);
+                    }
                 }
                 if (d < pitch) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
-                        if (j0 + j < keep) out[(long long)(j0 + j) * pitch + d] = v[j];
+                        if (j0 + j < keep) out[(long long)(j0 + j) * pitch + d] = a0[j];
+                    if (second) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (j0 + 16 + j < keep) out[(long long)(j0 + 16 + j) * pitch + d] = a1[j];
+                    }
                 }
             }
             tc_fence_before();
@@ -220,15 +269,20 @@ static cudaError_t launch_tc_rebuild_part(const float* Wsplit, int ldw, int j_pa
     if (kcols > ldw) return cudaErrorNotSupported;
     if (!tc::make_tmap_2d(&tmW, Wsplit, 4, (uint64_t)(2 * j_pad), (uint64_t)kcols, (uint64_t)ldw, (uint32_t)(2 * j_pad)))
         return cudaErrorNotSupported;
-    const int stage_bytes = 2 * tc::kBufBytes + 2 * j_pad * 128;
-    int stages = (200 * 1024) / stage_bytes;
+    // W resident in shared memory when all its chunk boxes take at most 64 KB (up to 128 buffer rows onto 64 output rows)
+    const int nchunk = (r + tc::kChunkRows - 1) / tc::kChunkRows;
+    const size_t w_all = (size_t)nchunk * 2 * j_pad * 128;
+    const int w_res = w_all <= 64 * 1024 ? 1 : 0;
+    const int stage_bytes = w_res ? 2 * tc::kBufBytes : 2 * tc::kBufBytes + 2 * j_pad * 128;
+    int stages = (int)((227 * 1024 - 1536 - (w_res ? w_all : 0)) / stage_bytes);
     if (stages > 8) stages = 8;
-    const size_t smem = (size_t)stages * stage_bytes + 1024 + (3 * stages + 4) * 8 + 16;
+    if (stages < 2) return cudaErrorNotSupported;
+    const size_t smem = (size_t)stages * stage_bytes + (w_res ? w_all : 0) + 1024 + (3 * stages + 5) * 8 + 16;
     const long long num_tiles = (pitch + tc::kTileD - 1) / tc::kTileD;
     const int grid = (int)(num_tiles < 148 ? num_tiles : 148);
     cudaError_t e = cudaFuncSetAttribute(tc::k_tc_rebuild, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    tc::k_tc_rebuild<<<grid, tc::kThreads, smem, st>>>(tmBuf, tmW, r, keep, j_pad, pitch, num_tiles, Bdst, stages, err);
+    tc::k_tc_rebuild<<<grid, tc::kThreads, smem, st>>>(tmBuf, tmW, r, keep, j_pad, pitch, num_tiles, Bdst, stages, w_res, err);
     return cudaGetLastError();
 }
 
