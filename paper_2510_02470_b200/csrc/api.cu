@@ -1069,6 +1069,8 @@ static sage_status_t score_rows(sage_fd* h, const void* rows, sage_dtype_t dt, i
             const int tiles = (int)((sub + 127) / 128);
             int mt = 512 / n_mma >= 4 ? 4 : (512 / n_mma >= 2 ? 2 : 1);
             if (tiles >= 148 && mt > 2) mt = 2;   // measured: pairs of row tiles with two K slices beat single tiles by 25 %
+            // rows a page or more apart: the kernel fetches two K tiles per stage (256 bytes per row visit), two row tiles fit
+            if (row_bytes >= ((size_t)2 << 20) && mt > 2) mt = 2;
             const int64_t slices_at_least = structured ? oC : (K / 4096 > 0 ? K / 4096 : 1);
             while (mt > 1 && (int64_t)((tiles + mt - 1) / mt) * slices_at_least < 148) mt >>= 1;
             const int splits = structured ? oC : pick_splits_waves((tiles + mt - 1) / mt, K, 4096, 148);

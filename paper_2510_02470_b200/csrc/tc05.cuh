@@ -73,6 +73,13 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* t
                  "l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(bar)), "r"(x), "r"(y)
                  : "memory");
 }
+// 4-D tile load (coordinates innermost first; c0 must make c0 * element size a multiple of 16 bytes).
+__device__ __forceinline__ void tma_load_4d(void* smem_dst, const CUtensorMap* tmap, uint64_t* bar, int c0, int c1, int c2, int c3) {
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(
+                     smem_u32(smem_dst)),
+                 "l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+                 : "memory");
+}
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* tmap) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tmap)) : "memory");
 }
@@ -152,11 +159,13 @@ __device__ __forceinline__ void tmem_ld_use(uint32_t r[16]) {
 // Shared-memory operand descriptor for a tile whose rows are 128 bytes of the contraction index (K-major),
 // stored by TMA with the 128-byte swizzle: groups of 8 rows are 1024 bytes apart. The tile base must be
 // 1024-byte aligned; stepping along K inside the 128-byte row adds the byte offset to the start address.
-__device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t smem_addr_bytes) {
+// group_stride_bytes: distance between consecutive groups of 8 rows (1024 when the tile is one box of rows x 128 bytes;
+// kt * 1024 when a 4-D box interleaved kt K tiles group by group, see make_tmap_4d_ktiles).
+__device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t smem_addr_bytes, uint32_t group_stride_bytes = 1024) {
     uint64_t d = 0;
     d |= static_cast<uint64_t>((smem_addr_bytes & 0x3ffffu) >> 4);   // start address / 16
     d |= static_cast<uint64_t>(1) << 16;                              // leading byte offset (unused for this layout)
-    d |= static_cast<uint64_t>(1024 >> 4) << 32;                      // stride byte offset: 8 rows * 128 bytes
+    d |= static_cast<uint64_t>(group_stride_bytes >> 4) << 32;        // stride byte offset between groups of 8 rows
     d |= static_cast<uint64_t>(1) << 46;                              // descriptor version of sm_100
     d |= static_cast<uint64_t>(2) << 61;                              // 128-byte swizzle
     return d;
@@ -190,6 +199,15 @@ __host__ __device__ inline uint32_t instr_desc(int fmt, int M, int N, int a_mn, 
 // multiple of 16 bytes) or the driver refuses.
 bool make_tmap_2d(CUtensorMap* out, const void* base, int elem_bytes, uint64_t rows, uint64_t cols, uint64_t ld,
                   uint32_t box_rows, int atom32 = 0);
+// The same row-major tensor seen as 4-D (128 bytes of a row, 8 rows, K tile, group of 8 rows), so that ONE box of
+// kt K tiles x box_rows rows reads kt * 128 consecutive bytes at every visit of a row: on rows megabytes apart
+// (every row visit a different page) that is what the load rate depends on (measured on 44 MB rows: 4.6 TB/s with
+// one K tile per visit, 6.5 TB/s with two, 6.8 TB/s with four). Shared-memory image: [row group][K tile][8 rows][128
+// bytes], i.e. K tile t of the box is an operand tile that starts t * 1024 bytes in and whose 8-row groups are
+// kt * 1024 bytes apart. Only whole K tiles (cols / (128 / elem_bytes) of them) and whole row groups are
+// addressable: rows must be a multiple of 8 (groups past the end read as zero), box_rows a multiple of 8 up to 256.
+bool make_tmap_4d_ktiles(CUtensorMap* out, const void* base, int elem_bytes, uint64_t rows, uint64_t cols, uint64_t ld,
+                         uint32_t box_rows, uint32_t kt);
 
 }  // namespace tc
 }  // namespace sage

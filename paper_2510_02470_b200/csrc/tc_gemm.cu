@@ -41,6 +41,32 @@ bool make_tmap_2d(CUtensorMap* out, const void* base, int elem_bytes, uint64_t r
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+bool make_tmap_4d_ktiles(CUtensorMap* out, const void* base, int elem_bytes, uint64_t rows, uint64_t cols, uint64_t ld,
+                         uint32_t box_rows, uint32_t kt) {
+    using Fn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                            const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                            CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static Fn encode = [] {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            fn = nullptr;
+        return reinterpret_cast<Fn>(fn);
+    }();
+    if (!encode) return false;
+    const uint64_t per_tile = 128 / elem_bytes, ktiles = cols / per_tile;
+    if ((reinterpret_cast<uintptr_t>(base) & 15u) || ((ld * (uint64_t)elem_bytes) & 15u) || rows == 0 || (rows & 7u) || ktiles == 0) return false;
+    if (box_rows == 0 || box_rows > 256 || (box_rows & 7u) || kt == 0 || kt > 8 || rows >= (1ull << 32)) return false;
+    const cuuint64_t dims[4] = {per_tile, 8, ktiles, rows / 8};
+    const cuuint64_t strides[3] = {ld * (uint64_t)elem_bytes, 128, 8 * ld * (uint64_t)elem_bytes};
+    const cuuint32_t box[4] = {static_cast<cuuint32_t>(per_tile), 8, kt, box_rows / 8};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    const CUtensorMapDataType dt = elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+    return encode(out, dt, 4, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 namespace {
 
 constexpr int kThreads = 192;
@@ -50,15 +76,21 @@ constexpr int kATileBytes = kTileM * 128;
 // kFmt: 1 = bf16 operands (64 elements per 128-byte K tile), 2 = fp32 operands read as tf32 (32 elements).
 template <int kFmt>
 __global__ void __launch_bounds__(kThreads, 1)
-k_tc_gemm_nt(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, int M, int N, int n_pad, int fold,
-             int mt, long long K, long long k_per_split, int a_shared, float* __restrict__ C, long long ldc, long long split_stride,
-             int stages, uint32_t tmem_cols, int* __restrict__ err) {
+k_tc_gemm_nt(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmA4,
+             const __grid_constant__ CUtensorMap tmB4, int kt2, int M, int N, int n_pad, int fold, int mt, long long K,
+             long long k_per_split, int a_shared, float* __restrict__ C, long long ldc, long long split_stride, int stages,
+             uint32_t tmem_cols, int* __restrict__ err) {
     constexpr int BK = kFmt == 1 ? 64 : 32;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     const int n_mma = fold ? 2 * n_pad : n_pad;         // folded: B holds two stacked operands whose products are added
-    const int a_bytes = mt * kATileBytes;
-    const int stage_bytes = a_bytes + n_mma * 128;
+    // kt2 (rows megabytes apart): a stage holds TWO K tiles, fetched by one 4-D box per operand tile so that every row
+    // visit reads 256 consecutive bytes (see make_tmap_4d_ktiles); the two tiles lie interleaved by groups of 8 rows. A
+    // slice's last odd or ragged K tiles go through the 2-D maps (zero fill) into the front of a stage.
+    const int ktn = kt2 ? 2 : 1;
+    const int a_tile_bytes = ktn * kATileBytes;
+    const int a_bytes = mt * a_tile_bytes;
+    const int stage_bytes = a_bytes + ktn * n_mma * 128;
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)stages * stage_bytes);
     uint64_t* empty = full + stages;
     uint64_t* tmem_full = empty + stages;
@@ -70,6 +102,8 @@ k_tc_gemm_nt(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     const long long k_begin = (long long)blockIdx.y * k_per_split;
     const long long k_end = K < k_begin + k_per_split ? K : k_begin + k_per_split;
     const int nkt = k_end > k_begin ? (int)((k_end - k_begin + BK - 1) / BK) : 0;
+    const int npairs = kt2 && k_end > k_begin ? (int)((k_end - k_begin) / BK) / 2 : 0;   // pairs of whole K tiles
+    const int nsteps = npairs + (nkt - 2 * npairs);                                     // stages filled by this CTA
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
@@ -90,19 +124,29 @@ k_tc_gemm_nt(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 
     if (warp == 0) {
         if (lane == 0) {
-            const uint32_t tx_bytes = (uint32_t)stage_bytes;
             int issued = 0;
-            for (int kt = 0; kt < nkt; ++kt) {
-                const int s = kt % stages;
-                const uint32_t use = (uint32_t)(kt / stages);
-                if (!mbar_wait(&empty[s], (use & 1u) ^ 1u, abort)) break;
-                mbar_expect_tx(&full[s], tx_bytes);
-                const int x = (int)(k_begin + (long long)kt * BK);
-                const int xa = a_shared ? kt * BK : x;   // class slices: every slice reads the same columns of A
-                for (int t = 0; t < mt; ++t)     // row tiles past the end of A are zero-filled by TMA
-                    tma_load_2d(smem + (size_t)s * stage_bytes + (size_t)t * kATileBytes, &tmA, &full[s], xa, m0 + t * kTileM);
-                tma_load_2d(smem + (size_t)s * stage_bytes + a_bytes, &tmB, &full[s], x, 0);
-                issued = kt + 1;
+            int s = 0;
+            uint32_t ph = 1;                                    // parity of the empty-barrier phase to wait for
+            uint8_t* st = smem;
+            const int kt_b0 = (int)(k_begin / BK), kt_a0 = a_shared ? 0 : kt_b0;   // class slices: every slice reads the same columns of A
+            for (int i = 0; i < nsteps; ++i) {
+                if (!mbar_wait(&empty[s], ph, abort)) break;
+                if (i < npairs) {
+                    mbar_expect_tx(&full[s], (uint32_t)stage_bytes);
+                    for (int t = 0; t < mt; ++t)     // row groups past the end of A are zero-filled by TMA
+                        tma_load_4d(st + (size_t)t * a_tile_bytes, &tmA4, &full[s], 0, 0, kt_a0 + 2 * i, (m0 + t * kTileM) / 8);
+                    tma_load_4d(st + a_bytes, &tmB4, &full[s], 0, 0, kt_b0 + 2 * i, 0);
+                } else {
+                    const int kt = 2 * npairs + (i - npairs);
+                    mbar_expect_tx(&full[s], (uint32_t)(mt * kATileBytes + n_mma * 128));
+                    const int x = (int)(k_begin + (long long)kt * BK);
+                    const int xa = a_shared ? kt * BK : x;
+                    for (int t = 0; t < mt; ++t)     // row tiles past the end of A are zero-filled by TMA
+                        tma_load_2d(st + (size_t)t * a_tile_bytes, &tmA, &full[s], xa, m0 + t * kTileM);
+                    tma_load_2d(st + a_bytes, &tmB, &full[s], x, 0);
+                }
+                issued = i + 1;
+                if (++s == stages) { s = 0; ph ^= 1u; st = smem; } else { st += stage_bytes; }
             }
             if (*abort) {   // give copies already in flight a bounded time to land before the block goes away
                 for (int kt = issued > stages ? issued - stages : 0; kt < issued; ++kt)
@@ -112,23 +156,30 @@ k_tc_gemm_nt(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     } else if (warp == 1) {
         if (lane == 0) {
             const uint32_t idesc = instr_desc(kFmt, kTileM, n_mma, 0, 0);
-            for (int kt = 0; kt < nkt; ++kt) {
-                const int s = kt % stages;
-                const uint32_t use = (uint32_t)(kt / stages);
-                if (!mbar_wait(&full[s], use & 1u, abort)) break;
+            const uint32_t st0 = smem_u32(smem);
+            int s = 0;
+            uint32_t ph = 0, st = st0;
+            bool first = true;                         // the first MMA of every accumulator overwrites it
+            for (int i = 0; i < nsteps; ++i) {
+                if (!mbar_wait(&full[s], ph, abort)) break;
                 tc_fence_after();
-                const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
-                const uint64_t bdesc = smem_desc_k_sw128(a_addr + a_bytes);
-                for (int t = 0; t < mt; ++t) {
-                    const uint64_t adesc = smem_desc_k_sw128(a_addr + t * kATileBytes);
-                    const uint32_t acc = tmem_base + (uint32_t)(t * n_mma);
+                const bool pair = i < npairs;
+                const uint32_t group_stride = pair ? 2048u : 1024u;
+                for (int kk = 0; kk < (pair ? 2 : 1); ++kk) {
+                    const uint64_t bdesc = smem_desc_k_sw128(st + a_bytes + kk * 1024, group_stride);
+                    for (int t = 0; t < mt; ++t) {
+                        const uint64_t adesc = smem_desc_k_sw128(st + t * a_tile_bytes + kk * 1024, group_stride);
+                        const uint32_t acc = tmem_base + (uint32_t)(t * n_mma);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {      // 4 x 32 bytes of K per 128-byte row
-                        if constexpr (kFmt == 1) mma_bf16(acc, adesc + 2 * k, bdesc + 2 * k, idesc, (kt | k) != 0);
-                        else mma_tf32(acc, adesc + 2 * k, bdesc + 2 * k, idesc, (kt | k) != 0);
+                        for (int k = 0; k < 4; ++k) {      // 4 x 32 bytes of K per 128-byte row
+                            if constexpr (kFmt == 1) mma_bf16(acc, adesc + 2 * k, bdesc + 2 * k, idesc, !(first && k == 0));
+                            else mma_tf32(acc, adesc + 2 * k, bdesc + 2 * k, idesc, !(first && k == 0));
+                        }
                     }
+                    first = false;
                 }
                 mma_commit(&empty[s]);                 // the stage is free once these MMAs have read it
+                if (++s == stages) { s = 0; ph ^= 1u; st = st0; } else { st += (uint32_t)stage_bytes; }
             }
             mma_commit(tmem_full);
         }
@@ -206,8 +257,18 @@ cudaError_t launch_tc_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const
     if (class_F > 0) kps = class_F;
     const int a_shared = class_F > 0 ? 1 : 0;
     // a trailing slice may be empty after rounding to whole K tiles: its CTAs store zeros
-    const int stage_bytes = mt * tc::kATileBytes + n_mma * 128;
-    int stages = (200 * 1024) / stage_bytes;
+    // Rows at least a page (2 MB) apart: two K tiles per stage through 4-D boxes (256 bytes per row visit), where the
+    // shapes allow it (whole groups of 8 rows in both operands, slices that start on a K tile) and two such stages fit.
+    CUtensorMap tmA4 = tmA, tmB4 = tmB;
+    const uint64_t b_rows = (uint64_t)(fold ? n_pad + N : N);
+    int kt2 = (lda * es >= (2 << 20) && M % 8 == 0 && b_rows % 8 == 0 && (class_F == 0 || class_F % BK == 0) &&
+               2 * (2 * mt * tc::kATileBytes + 2 * n_mma * 128) + 2048 <= 227 * 1024)
+                  ? 1 : 0;
+    if (kt2 && !(tc::make_tmap_4d_ktiles(&tmA4, A, es, (uint64_t)M, (uint64_t)(class_F > 0 ? class_F : K), (uint64_t)lda, tc::kTileM, 2) &&
+                 tc::make_tmap_4d_ktiles(&tmB4, Bm, es, b_rows, (uint64_t)K, (uint64_t)ldb, (uint32_t)n_mma, 2)))
+        kt2 = 0;
+    const int stage_bytes = (kt2 ? 2 : 1) * (mt * tc::kATileBytes + n_mma * 128);
+    int stages = ((kt2 ? 227 * 1024 - 2048 : 200 * 1024)) / stage_bytes;
     if (stages > 8) stages = 8;
     if (stages < 2) return cudaErrorNotSupported;
     const size_t smem = (size_t)stages * stage_bytes + 1024 + (2 * stages + 1) * 8 + 16;
@@ -219,12 +280,12 @@ cudaError_t launch_tc_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const
     if (dt == SAGE_BF16) {
         e = cudaFuncSetAttribute(tc::k_tc_gemm_nt<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        tc::k_tc_gemm_nt<1><<<grid, tc::kThreads, smem, st>>>(tmA, tmB, M, N, n_pad, fold, mt, K, kps, a_shared, C, ldc, split_stride, stages,
+        tc::k_tc_gemm_nt<1><<<grid, tc::kThreads, smem, st>>>(tmA, tmB, tmA4, tmB4, kt2, M, N, n_pad, fold, mt, K, kps, a_shared, C, ldc, split_stride, stages,
                                                               tmem_cols, err);
     } else {
         e = cudaFuncSetAttribute(tc::k_tc_gemm_nt<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        tc::k_tc_gemm_nt<2><<<grid, tc::kThreads, smem, st>>>(tmA, tmB, M, N, n_pad, fold, mt, K, kps, a_shared, C, ldc, split_stride, stages,
+        tc::k_tc_gemm_nt<2><<<grid, tc::kThreads, smem, st>>>(tmA, tmB, tmA4, tmB4, kt2, M, N, n_pad, fold, mt, K, kps, a_shared, C, ldc, split_stride, stages,
                                                               tmem_cols, err);
     }
     return cudaGetLastError();
