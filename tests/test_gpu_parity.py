@@ -272,6 +272,37 @@ def test_tensor_core_path_agrees_with_cuda_core_path(dtype, N, D, ell):
         assert np.max(np.abs(a - ref["alpha"])) <= TOL_SCORE[dtype]
 
 
+@pytest.mark.parametrize("N,D,ell,ld", [(520, 1000, 16, 1100008), (515, 1000, 16, 1100008), (264, 20008, 24, 1200000),
+                                        (392, 16456, 64, 1048576)])
+def test_bf16_rows_a_page_or_more_apart_score_like_packed_rows(N, D, ell, ld):
+    """bfloat16 rows held in a much wider matrix (row pitch of 2 MB and more): the projection then fetches two K tiles
+    per row visit through 4-D TMA boxes where the shapes allow it (row counts that are multiples of 8; 515 rows take the
+    2-D boxes), with the two-term sketch (D = 1000), the one-term sketch, odd numbers of K tiles and ragged last tiles.
+    The scores must be those of the same rows packed tightly, far inside the tolerance, and match the oracle."""
+    rows = lowrank_rows(N, D, 5, 0.4, N + D, torch.bfloat16)
+    dev = torch.device("cuda", 0)
+    wide = torch.zeros((N, ld), dtype=torch.bfloat16, device=dev)
+    wide[:, :D] = rows.to(dev)
+    wide[:, D:D + 64] = float("nan")                       # what follows a row must never be read as data
+    packed = rows.to(dev)
+    out = []
+    for g in (wide[:, :D], packed):
+        fd = sage.SageFD(D, ell, torch.bfloat16, 0)
+        fd.update(g)
+        fd.finalize()
+        a = fd.score(g)
+        torch.cuda.synchronize()
+        st = fd.stats()
+        S, _ = fd.sketch()
+        fd.close()
+        assert st["device_flags"] == 0
+        out.append((S.double().cpu().numpy(), a.double().cpu().numpy()))
+    assert np.array_equal(out[0][0], out[1][0])                                    # pass 1 does not depend on the pitch
+    assert np.max(np.abs(out[0][1] - out[1][1])) <= 2e-5
+    ref = oracle.run(rows, D, ell, 0.1, route=1)
+    assert np.max(np.abs(out[0][1] - ref["alpha"])) <= TOL_SCORE[torch.bfloat16]
+
+
 # ------------------------------------------------------------------ the two eigen-solve kernel families
 
 def _run_with_eig_variant(rows, D, ell, variant):
