@@ -327,10 +327,13 @@ def run_workload(w, args, steps, warmup, ctx, want_e2e, want_cpu, sketches, fact
     full, r_final = shrink_schedule(N, ell)
     m, keep = 2 * ell, ell - 1
     keep_final = (ell - 1) if r_final > ell else min(r_final, ell)
+    # rows that whole shrink cycles read in place (never appended; bf16, 2 bytes instead of the buffer's 4): counted by the
+    # library since the reset at the start of the last step
+    in_place = stats.get("rows_in_place", 0)
     per_step_bytes = {
-        "append": N * D * (e + 4),
-        "gram": (full * m + r_final) * D * 4,
-        "rebuild": (full * (m + keep) + (r_final + max(keep_final, ell))) * D * 4,
+        "append": (N - in_place) * D * (e + 4),
+        "gram": (full * m + r_final) * D * 4 - in_place * D * (4 - e),
+        "rebuild": (full * (m + keep) + (r_final + max(keep_final, ell))) * D * 4 - in_place * D * (4 - e),
         "project": N * D * e,
         "normalise": N * ell * 8,
         "score": N * ell * 4 + N * 4,
@@ -370,7 +373,9 @@ def run_workload(w, args, steps, warmup, ctx, want_e2e, want_cpu, sketches, fact
             entry["frac_of_hbm"] = entry["GBps"] / peaks["hbm_gbs"]
         kernels[name] = entry
     roof_pass2_s = max(N * D * e / (peaks["hbm_gbs"] * 1e9), 2.0 * N * ell * D / (peaks["bf16_tflops_sustained"] * 1e12))
-    p1_bytes = per_step_bytes["append"] + per_step_bytes["gram"] + per_step_bytes["rebuild"]
+    # pass-1 roofline: the bytes of the method with every row appended to an fp32 buffer (append read + write, Gram read,
+    # rebuild read + write); cycles that read their rows in place move fewer, so the fraction compares TIME with that model
+    p1_bytes = N * D * (e + 4) + (full * m + r_final) * D * 4 + (full * (m + keep) + (r_final + max(keep_final, ell))) * D * 4
     roof_pass1_s = p1_bytes / (peaks["hbm_gbs"] * 1e9)
     stream_ms = sum(prof_all[k]["ms"] for k in ("append", "gram", "gram_reduce", "rebuild"))
 

@@ -252,6 +252,7 @@ typedef struct {
                                bit 3: the cluster eigen-solve gave up a bounded wait (results invalid) */
     int64_t kernel_launches;/* kernels this handle has launched since create/reset */
     int64_t tensor_core_launches; /* how many of them were tensor-core (tcgen05) kernels: Gram, rebuild, projection */
+    int64_t rows_in_place;  /* rows of sage_fd_update that whole shrink cycles read where the caller held them (option 9) */
 } sage_stats_t;
 
 /* Synchronises the device and reads the counters back. */
@@ -276,7 +277,13 @@ sage_status_t sage_fd_stats(sage_fd_t* h, sage_stats_t* out);
  * a limited number of hardware queues, 8 unless the environment variable CUDA_DEVICE_MAX_CONNECTIONS says otherwise when CUDA
  * is initialised; streams that share a queue do not overlap, so with P > 8 set it to 32 before the process touches CUDA.)
  * Outside a scoring pass: key 8 = 1 for the strict-memory form of Phase II (see sage_score_apply), 0 (default) to keep the
- * N x ell normalised projections. */
+ * N x ell normalised projections.
+ * At any time: key 9 = 1 (default) lets a shrink cycle whose ell + 1 new rows all lie in one sage_fd_update call read them
+ * where the caller holds them instead of appending them to the buffer first (bfloat16 rows, ell = 32 or 64, tensor-core
+ * kernels, the paper's single sketch: the Gram and rebuild kernels take rows 0 .. ell - 2 from the buffer and convert the
+ * caller's rows on the way into the operand tiles; same arithmetic and the same results as the appended form); rows that do
+ * not fill a cycle are appended as before. 0: always append. Either way `rows` must stay unchanged until the work enqueued by
+ * the call has run (stream order on cuda_stream takes care of that for work enqueued there afterwards). */
 sage_status_t sage_fd_set_option(sage_fd_t* h, int key, double value);
 
 /* Per-kernel device time of this handle's launches since the previous call, for the classes selected

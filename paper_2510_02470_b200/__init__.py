@@ -65,7 +65,7 @@ SIGNATURES = {
 class SageStats(C.Structure):
     _fields_ = [("rows_seen", _i64), ("shrinks", _i64), ("sum_delta", _f64), ("last_sweeps", _i32),
                 ("max_sweeps", _i32), ("last_rank", _i32), ("device_flags", _u32), ("kernel_launches", _i64),
-                ("tensor_core_launches", _i64)]
+                ("tensor_core_launches", _i64), ("rows_in_place", _i64)]
 
 
 class SageError(RuntimeError):

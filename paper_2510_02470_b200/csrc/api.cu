@@ -162,6 +162,7 @@ struct sage_fd {
     size_t bias_t_bytes = 0;
     float* zred = nullptr;         // projections of a sub-chunk summed over their K slices (when there are many slices)
     size_t zred_bytes = 0;
+    bool direct_rows = true;       // option 9: shrink cycles read bfloat16 rows from the caller's memory where the shapes allow it
     bool strict = false;           // option 8: no N x ell store; scores come from a third pass (sage_score_apply)
     bool scored_strict = false;    // the finished pass ran in strict-memory mode: u is known, zhat is not kept
     float* class_U = nullptr;      // class-balanced variant: unit centroids (class_cap x ell) and class sizes
@@ -178,6 +179,7 @@ struct sage_fd {
     int eig_variant = 0;           // option 5: 0 cluster eigen-solve in distributed shared memory, 1 the one-CTA / L2 kernels
     int64_t launches = 0;
     int64_t tc_launches = 0;       // how many of them were tensor-core (tcgen05) kernels
+    int64_t rows_in_place = 0;     // rows that shrink cycles read where the caller held them (never appended)
     Prof prof;
     // Merged form of pass 1 (option 6): P sketches over interleaved row blocks. This handle is sketch 0; sketches
     // 1..P-1 are handles of their own that only sketch (no scoring state). With P > 1 every sketch runs its
@@ -542,6 +544,7 @@ sage_status_t sage_fd_reset(sage_fd_t* h) {
     h->state = SKETCHING;
     h->launches = 0;
     h->tc_launches = 0;
+    h->rows_in_place = 0;
     h->app_pending = false;
     h->in_epoch = -1;
     for (sage_fd* k : h->kids) ST_TRY(sage_fd_reset(k));
@@ -558,6 +561,11 @@ sage_status_t sage_fd_set_option(sage_fd_t* h, int key, double value) {
     if (key == 4) {                          // 0: CUDA-core kernels only, 1: tensor-core kernels where possible
         h->use_tc = value != 0.0;
         for (sage_fd* k : h->kids) k->use_tc = h->use_tc;
+        return SAGE_OK;
+    }
+    if (key == 9) {                          // 1: whole shrink cycles read their new rows in place (no append), 0: always append
+        h->direct_rows = value != 0.0;
+        for (sage_fd* k : h->kids) k->direct_rows = h->direct_rows;
         return SAGE_OK;
     }
     if (key == 8) {                          // strict-memory scoring: no N x ell store, scores from a third pass
@@ -636,6 +644,61 @@ static sage_status_t sketch_factor(sage_fd* s, int r, int do_shrink, int keep, i
     return SAGE_OK;
 }
 
+// A whole shrink cycle whose new rows (m - fill of them, bfloat16, pitch ld) are read where the caller holds them instead of
+// being appended first: the Gram and rebuild kernels take rows 0 .. fill - 1 from the buffer and the rest from `rows`
+// (same arithmetic, same results as the appended form). *done = false (and nothing enqueued) when the kernels do not
+// support the shape: the caller then appends as usual.
+static sage_status_t sketch_factor_direct(sage_fd* s, const void* rows, int64_t ld, cudaStream_t chain, bool* done) {
+    *done = false;
+    const int r = s->m, old_rows = s->fill, n_new = s->m - s->fill, keep = s->delta_rank - 1;
+    const int j_pad = ((keep + 15) / 16) * 16;
+    if (!s->use_tc || !s->Wsplit || r > 128 || keep != old_rows || keep <= 0 || (old_rows + 1) % 32 != 0 || r % 32 != 0 ||
+        j_pad > s->wsplit_ld / 2 || r > s->wsplit_ld || j_pad > 64 || (reinterpret_cast<uintptr_t>(rows) & 15u) || ((ld * 2) & 15))
+        return SAGE_OK;
+    ST_TRY(sketch_join_appends(s, chain));
+    const int ldc = ((r + 3) / 4) * 4;
+    const int64_t stride = (int64_t)r * ldc;
+    int cap = (int)(s->gram_part_floats / (size_t)stride);
+    if (cap > 148) cap = 148;
+    const int splits = pick_splits_waves(1, s->D, 256, cap);
+    float* Bc = s->B[s->cur];
+    cudaError_t e = timed(s, K_GRAM, 1, chain, [&] {
+        return launch_tc_gram_direct(Bc, s->pitch, old_rows, rows, ld, n_new, s->D, splits, s->gram_parts, ldc, stride, s->tc_err, chain);
+    });
+    if (e == cudaErrorNotSupported) {
+        count(s, -1);
+        return SAGE_OK;
+    }
+    CU_TRY(e);
+    s->tc_launches += 1;
+    CU_TRY(timed(s, K_GRAM_REDUCE, 1, chain, [&] { return launch_gram_sym_reduce(s->gram_parts, splits, stride, r, ldc, s->Kmat, s->m, chain); }));
+    CU_TRY(cudaEventRecord(s->ev_fork, chain));
+    CU_TRY(timed(s, K_EIG, 1, chain, [&] {
+        return launch_eig_shrink(s->Kmat, s->m, r, 1, s->delta_rank, keep, s->Ur, s->m, s->sigma, s->ell, s->eig_work, s->max_sweeps, s->info,
+                                 s->Wsplit, s->wsplit_ld, j_pad, s->eig_variant, chain);
+    }));
+    e = timed(s, K_REBUILD, 1, chain, [&] {
+        return launch_tc_rebuild_direct(s->Wsplit, s->wsplit_ld, j_pad, Bc, s->B[1 - s->cur], s->pitch, s->D, r, keep, rows, ld, n_new, s->tc_err,
+                                        chain);
+    });
+    if (e == cudaErrorNotSupported) {
+        // the factors exist already: bring the rows into the buffer after all and rebuild from there
+        count(s, -1);
+        CU_TRY(timed(s, K_APPEND, 1, chain, [&] { return launch_append(rows, SAGE_BF16, n_new, ld, s->D, Bc, s->pitch, old_rows, chain); }));
+        CU_TRY(timed(s, K_REBUILD, 1, chain, [&] {
+            return launch_tc_rebuild(s->Wsplit, s->wsplit_ld, j_pad, Bc, s->B[1 - s->cur], s->pitch, s->D, r, keep, s->tc_err, chain);
+        }));
+    } else {
+        CU_TRY(e);
+    }
+    s->tc_launches += 1;
+    s->cur = 1 - s->cur;
+    s->fill = keep;
+    CU_TRY(cudaStreamWaitEvent(s->side, s->ev_fork, 0));
+    *done = true;
+    return SAGE_OK;
+}
+
 // Where the rows of an update come from: a dense matrix (rows, pitch ld), or the two factors of structured last-layer
 // rows (q: pitch ldq, C values per row; feat: pitch ldf, F values per row), expanded on the fly.
 struct RowSrc {
@@ -679,6 +742,19 @@ static sage_status_t sketch_feed(sage_fd* s, RowSrc src, int64_t n, cudaStream_t
         while (n > 0) {
             const int64_t room = s->m - s->fill;
             const int64_t take = n < room ? n : room;
+            // a whole cycle's rows at hand, bfloat16, on the caller's own stream: no append, the kernels read them in place
+            if (s->direct_rows && from_caller && !s->chain && !src.outer() && src.dt == SAGE_BF16 && take == room && s->fill > 0 &&
+                s->fill == s->delta_rank - 1) {
+                bool direct = false;
+                ST_TRY(sketch_factor_direct(s, src.rows, src.ld, chain, &direct));
+                if (direct) {
+                    s->rows_in_place += take;
+                    s->rows_seen += take;
+                    src = src.advanced(take);
+                    n -= take;
+                    continue;
+                }
+            }
             CU_TRY(timed(s, K_APPEND, 1, as, [&] { return src.append(take, s->D, s->B[s->cur], s->pitch, s->fill, as); }));
             appended = true;
             if (!on_chain) s->app_pending = true;
@@ -1589,7 +1665,7 @@ sage_status_t sage_fd_stats(sage_fd_t* h, sage_stats_t* out) {
     CU_TRY(cudaMemcpy(&info, h->info, sizeof info, cudaMemcpyDeviceToHost));
     int tc_err = 0;
     CU_TRY(cudaMemcpy(&tc_err, h->tc_err, sizeof tc_err, cudaMemcpyDeviceToHost));
-    int64_t launches = h->launches, tc_launches = h->tc_launches;
+    int64_t launches = h->launches, tc_launches = h->tc_launches, in_place = h->rows_in_place;
     for (sage_fd* k : h->kids) {             // merged form: counters of all sketches together
         EigInfo ki;
         int kt = 0;
@@ -1602,6 +1678,7 @@ sage_status_t sage_fd_stats(sage_fd_t* h, sage_stats_t* out) {
         tc_err |= kt;
         launches += k->launches;
         tc_launches += k->tc_launches;
+        in_place += k->rows_in_place;
     }
     out->rows_seen = h->dealt;
     out->shrinks = info.shrinks;
@@ -1612,6 +1689,7 @@ sage_status_t sage_fd_stats(sage_fd_t* h, sage_stats_t* out) {
     out->device_flags = info.flags | (tc_err ? 4u : 0u);
     out->kernel_launches = launches;
     out->tensor_core_launches = tc_launches;
+    out->rows_in_place = in_place;
     return SAGE_OK;
 }
 

@@ -74,6 +74,11 @@ cudaError_t launch_tc_gemm_nt(const void* A, sage_dtype_t dt, int64_t lda, const
 cudaError_t launch_tc_gemm_nt_x3(const float* A, int64_t lda, const float* Bm, int64_t ldb, int M, int N, int64_t K, int splits,
                                  float* C, int64_t ldc, int64_t split_stride, int sym, int* err, cudaStream_t st,
                                  int64_t class_F = 0);   // class slices as in launch_gemm_nt; needs class_F a multiple of 4
+// The symmetric form of launch_tc_gemm_nt_x3 (sym = 1) for a buffer whose last n_new rows have not been appended: rows
+// 0 .. old_rows - 1 come from Bold (fp32, pitch elements; one more row must be readable), the n_new rows after them are
+// bfloat16 rows at src (pitch ld_src). old_rows + n_new <= 128, old_rows + 1 a multiple of 8. Same output as the appended form.
+cudaError_t launch_tc_gram_direct(const float* Bold, int64_t pitch, int old_rows, const void* src, int64_t ld_src, int n_new, int64_t D,
+                                  int splits, float* C, int64_t ldc, int64_t split_stride, int* err, cudaStream_t st);
 cudaError_t launch_gram_sym_reduce(const float* parts, int splits, int64_t stride, int r, int64_t ldp, float* out, int64_t ldo,
                                    cudaStream_t st);
 
@@ -85,6 +90,11 @@ cudaError_t launch_gram_sym_reduce(const float* parts, int splits, int64_t strid
 // returns cudaErrorNotSupported otherwise.
 cudaError_t launch_tc_rebuild(const float* Wsplit, int ldw, int j_pad, const float* Bsrc, float* Bdst, int64_t pitch, int64_t D, int r,
                               int keep, int* err, cudaStream_t st);
+// The same rebuild for a buffer whose last n_new rows have not been appended: rows 0 .. r - n_new - 1 come from Bsrc (one
+// more row must be readable), the n_new rows after them are bfloat16 rows at src (pitch ld_src, D columns). Needs r <= 128,
+// r and r - n_new + 1 multiples of 32, and the factors resident (at most 64 output rows); cudaErrorNotSupported otherwise.
+cudaError_t launch_tc_rebuild_direct(const float* Wsplit, int ldw, int j_pad, const float* Bsrc, float* Bdst, int64_t pitch, int64_t D,
+                                     int r, int keep, const void* src, int64_t ld_src, int n_new, int* err, cudaStream_t st);
 
 // hi[i][0:cols] = bf16(src[i][0:cols]) (round to nearest even) for i < rows; when lo != nullptr also
 // lo[i][:] = bf16(src - float(hi)), so that hi + lo carries 16 significant bits of src.

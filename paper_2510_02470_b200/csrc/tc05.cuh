@@ -199,6 +199,10 @@ __host__ __device__ inline uint32_t instr_desc(int fmt, int M, int N, int a_mn, 
 // multiple of 16 bytes) or the driver refuses.
 bool make_tmap_2d(CUtensorMap* out, const void* base, int elem_bytes, uint64_t rows, uint64_t cols, uint64_t ld,
                   uint32_t box_rows, int atom32 = 0);
+// Row-major tensor -> boxes of box_rows x box_cols elements WITHOUT swizzle (the box image in shared memory is plain
+// row-major); box_cols * elem_bytes must be a multiple of 16.
+bool make_tmap_2d_plain(CUtensorMap* out, const void* base, int elem_bytes, uint64_t rows, uint64_t cols, uint64_t ld,
+                        uint32_t box_cols, uint32_t box_rows);
 // The same row-major tensor seen as 4-D (128 bytes of a row, 8 rows, K tile, group of 8 rows), so that ONE box of
 // kt K tiles x box_rows rows reads kt * 128 consecutive bytes at every visit of a row: on rows megabytes apart
 // (every row visit a different page) that is what the load rate depends on (measured on 44 MB rows: 4.6 TB/s with

@@ -66,7 +66,7 @@ __device__ __forceinline__ uint4 lo4(const uint4 v) { return make_uint4(lo_of(v.
 __global__ void __launch_bounds__(kThreads, 1)
 k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, int M, int N, int gram,
                 int b_box_rows, int sym, long long K, long long k_per_split, int a_shared, float* __restrict__ C, long long ldc,
-                long long split_stride, int stages, int stage_bytes, int G, int* __restrict__ err) {
+                long long split_stride, int stages, int stage_bytes, int G, int direct_new, int direct_box, int* __restrict__ err) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     const int m0 = blockIdx.x * kTileM, n0 = blockIdx.y * kTileN;
@@ -76,6 +76,13 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const bool diag = gram && m0 == n0;                   // A tile == B tile: load once
     // stage layout: [hi: A | B][lo: A | B]; on diagonal tiles there is no separate B; proj: [hi: rows][lo: rows][sketch]
     const int half_bytes = (diag || proj) ? kTileBytes : kTileBytes + b_box_rows * 128;
+    // direct_new > 0 (a symmetric Gram matrix of at most 128 rows whose last direct_new rows are still bfloat16 rows in the
+    // caller's memory): tmA covers the first M - direct_new + 1 buffer rows (the last of them is a placeholder), tmB the
+    // caller's rows (boxes of direct_box rows x 64 bytes, no swizzle) which land behind the two tiles of the stage; the
+    // workers convert them and put them where rows M - direct_new ... M - 1 of the operand tile belong (128-byte swizzle:
+    // 16-byte chunk j of row r sits in slot j ^ (r & 7)). Their remainders are zero (bfloat16 has 8 significant bits):
+    // the remainder tiles are cleared once and only rows below M - direct_new are ever written.
+    const int old_rows = direct_new ? M - direct_new : 0;
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)stages * stage_bytes);
     uint64_t* split_done = full + stages;
     uint64_t* empty = split_done + stages;
@@ -111,6 +118,13 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         tma_prefetch_desc(&tmA);
         tma_prefetch_desc(&tmB);
     }
+    if (direct_new) {
+        for (int s = 0; s < stages; ++s) {
+            uint4* lo = reinterpret_cast<uint4*>(smem + (size_t)s * stage_bytes + kTileBytes);
+            for (int c = threadIdx.x; c < kTileBytes / 16; c += kThreads) lo[c] = make_uint4(0u, 0u, 0u, 0u);
+        }
+        fence_proxy_async_smem();
+    }
     if (warp == 1) tmem_alloc(tmem_slot, kAccs * kTileN);
     tc_fence_before();
     __syncthreads();
@@ -124,12 +138,12 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             uint32_t ph = 1;                                    // parity of the empty-barrier phase to wait for
             int x = (int)k_begin, xa = a_shared ? 0 : (int)k_begin;   // class slices: the same columns of A for every slice
             uint8_t* st = smem;
-            const uint32_t tx_bytes = (uint32_t)(proj ? 2 * kTileBytes : half_bytes);
+            const uint32_t tx_bytes = direct_new ? (uint32_t)((old_rows + 1) * 128 + direct_box * 64) : (uint32_t)(proj ? 2 * kTileBytes : half_bytes);
             for (int kt = 0; kt < nkt; ++kt) {
                 if (!mbar_wait(&empty[s], ph, abort)) break;
                 mbar_expect_tx(&full[s], tx_bytes);
                 tma_load_2d(st, &tmA, &full[s], xa, m0);
-                if (proj) tma_load_2d(st + 2 * kTileBytes, &tmB, &full[s], x, 0);
+                if (proj || direct_new) tma_load_2d(st + 2 * kTileBytes, &tmB, &full[s], x, 0);
                 else if (!diag) tma_load_2d(st + kTileBytes, &tmB, &full[s], x, n0);
                 issued = kt + 1;
                 x += BK;
@@ -187,7 +201,7 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     } else {
         // ---- workers: write the lo part of landed stages; drain finished accumulators ----
         const int t = threadIdx.x - 64;                 // 0..255
-        const int chunks16 = half_bytes / 16;
+        const int chunks16 = direct_new ? old_rows * 8 : half_bytes / 16;     // direct: remainders of the buffer rows only
         const float lo_scale = sym == 1 ? 2.f : 1.f;          // sym: the lo half of the accumulator counts twice (folded into the drain)
         const int quarter = warp & 3, chalf = (warp - 2) >> 2;
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + (uint32_t)(chalf * 64);
@@ -267,6 +281,18 @@ k_tc_gemm_nt_x3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 #pragma unroll
                 for (int u = 0; u < 4; ++u)
                     if (c + u * kGroup < chunks16) lo[c + u * kGroup] = lo4(v[u]);
+            }
+            if (direct_new) {
+                // the caller's bfloat16 rows: 4 x 16 bytes (32 values) per row and K tile -> 8 chunks of 4 floats in the operand tile
+                const uint4* src = reinterpret_cast<const uint4*>(smem + (size_t)s_now * stage_bytes + 2 * kTileBytes);
+                for (int i = tg; i < direct_new * 4; i += kGroup) {
+                    const int row = i >> 2, q = i & 3, R = old_rows + row;
+                    const uint4 v = src[i];
+                    const uint4 a = make_uint4(v.x << 16, v.x & 0xffff0000u, v.y << 16, v.y & 0xffff0000u);
+                    const uint4 b = make_uint4(v.z << 16, v.z & 0xffff0000u, v.w << 16, v.w & 0xffff0000u);
+                    hi[R * 8 + ((2 * q) ^ (R & 7))] = a;
+                    hi[R * 8 + ((2 * q + 1) ^ (R & 7))] = b;
+                }
             }
             fence_proxy_async_smem();                   // the tensor cores read these writes
             __syncwarp();                               // one arrival per warp
@@ -355,7 +381,35 @@ cudaError_t launch_tc_gemm_nt_x3(const float* A, int64_t lda, const float* Bm, i
     cudaError_t e = cudaFuncSetAttribute(tc::k_tc_gemm_nt_x3, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     tc::k_tc_gemm_nt_x3<<<grid, tc::kThreads, smem, st>>>(tmA, tmB, M, N, gram, b_box_rows, sym, K, kps, class_F > 0 ? 1 : 0, C, ldc, split_stride, stages,
-                                                                 stage_bytes, G, err);
+                                                                 stage_bytes, G, 0, 0, err);
+    return cudaGetLastError();
+}
+
+// See sage_internal.h.
+cudaError_t launch_tc_gram_direct(const float* Bold, int64_t pitch, int old_rows, const void* src, int64_t ld_src, int n_new, int64_t D,
+                                  int splits, float* C, int64_t ldc, int64_t split_stride, int* err, cudaStream_t st) {
+    const int M = old_rows + n_new;
+    if (old_rows < 1 || n_new < 1 || M > tc::kTileM || D <= 0 || splits < 1 || splits > 65535) return cudaErrorNotSupported;
+    const int old_box = old_rows + 1;                         // one placeholder row, overwritten by the first new row
+    const int src_box = ((n_new + 7) / 8) * 8;
+    if ((old_box & 7) || src_box > 128) return cudaErrorNotSupported;
+    CUtensorMap tmA, tmB;
+    if (!tc::make_tmap_2d(&tmA, Bold, 4, (uint64_t)old_box, (uint64_t)D, (uint64_t)pitch, (uint32_t)old_box)) return cudaErrorNotSupported;
+    if (!tc::make_tmap_2d_plain(&tmB, src, 2, (uint64_t)n_new, (uint64_t)D, (uint64_t)ld_src, 32, (uint32_t)src_box)) return cudaErrorNotSupported;
+    int64_t kps = (D + splits - 1) / splits;
+    kps = ((kps + tc::BK - 1) / tc::BK) * tc::BK;
+    const int stage_bytes = 2 * tc::kTileBytes + ((src_box * 64 + 1023) / 1024) * 1024;
+    const bool deep = kps / tc::BK >= 64;
+    int stages = ((deep ? 227 * 1024 - 1536 : 200 * 1024)) / stage_bytes;
+    if (stages > 8) stages = 8;
+    if (stages < 2) return cudaErrorNotSupported;
+    const int G = deep ? stages : ((stages & 1) ? 1 : 2);
+    const size_t smem = (size_t)stages * stage_bytes + 1024 + (3 * stages + 2 * tc::kAccs) * 8 + 16;
+    dim3 grid(1u, 1u, (unsigned)splits);
+    cudaError_t e = cudaFuncSetAttribute(tc::k_tc_gemm_nt_x3, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    tc::k_tc_gemm_nt_x3<<<grid, tc::kThreads, smem, st>>>(tmA, tmB, M, M, 1, 0, 1, D, kps, 0, C, ldc, split_stride, stages, stage_bytes, G, n_new,
+                                                         src_box, err);
     return cudaGetLastError();
 }
 

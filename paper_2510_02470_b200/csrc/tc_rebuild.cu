@@ -34,14 +34,22 @@ constexpr int kBufBytes = kChunkRows * kTileD * 4;   // 16 KB: 4 spans of [32 ro
 constexpr int kSpanBytes = kChunkRows * 128;         // 4 KB
 
 __global__ void __launch_bounds__(kThreads, 1)
-k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ CUtensorMap tmW, int r, int keep, int j_pad,
+k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmSrc,
+             const __grid_constant__ CUtensorMap tmSrc1, int direct_new, int r, int keep, int j_pad,
              long long pitch, long long num_tiles, float* __restrict__ out, int stages, int w_res, int* __restrict__ err) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     // stage layout: [buffer hi 16 KB][buffer lo 16 KB][W_hi ; W_lo: 2*j_pad rows of 128 bytes]; w_res: the W boxes of all
     // chunks are loaded once and stay behind the ring (W does not depend on the column tile), the stages hold buffer data only
     const int w_bytes = 2 * j_pad * 128;
-    const int stage_bytes = w_res ? 2 * kBufBytes : 2 * kBufBytes + w_bytes;
+    // direct_new > 0 (needs w_res): the last direct_new of the r rows are bfloat16 rows in the caller's memory. Rows
+    // 0 .. r - direct_new - 1 come from the buffer as usual; r - direct_new is the last row of its chunk of 32 (cb), so that
+    // chunk gets one bfloat16 row (tmSrc1) and the chunks after it 32 each (tmSrc) into an 8 KB staging area behind the two
+    // buffer tiles; the split warps convert them into the operand layout (32-byte atoms: chunk j of k row rr sits in slot
+    // ((j >> 1) ^ (rr & 3)) * 2 + (j & 1) of its 128-byte span row). Their remainders are zero, so chunks after cb take one
+    // MMA per K step instead of two.
+    const int stage_bytes = (w_res ? 2 * kBufBytes : 2 * kBufBytes + w_bytes) + (direct_new ? 8192 : 0);
+    const int cb = direct_new ? (r - direct_new) / kChunkRows : 1 << 30;
     const int nchunk = (r + kChunkRows - 1) / kChunkRows;
     uint8_t* wres = smem + (size_t)stages * stage_bytes;
     uint64_t* full = reinterpret_cast<uint64_t*>(wres + (w_res ? (size_t)nchunk * w_bytes : 0));
@@ -99,10 +107,16 @@ k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ 
                 const int d0 = (int)((blockIdx.x + lt * gridDim.x) * kTileD);
                 for (int c = 0; c < nchunk; ++c) {
                     if (!mbar_wait(&empty[s], ph, abort)) { alive = false; break; }
-                    mbar_expect_tx(&full[s], tx_bytes);
+                    if (c > cb) {                               // caller's rows only
+                        mbar_expect_tx(&full[s], 8192u);
+                        tma_load_2d(st + 2 * kBufBytes, &tmSrc, &full[s], d0, 1 + (c - cb - 1) * kChunkRows);
+                    } else {
+                        mbar_expect_tx(&full[s], c == cb ? tx_bytes + 256u : tx_bytes);
 #pragma unroll
-                    for (int sp = 0; sp < 4; ++sp) tma_load_2d(st + sp * kSpanBytes, &tmBuf, &full[s], d0 + 32 * sp, c * kChunkRows);
-                    if (!w_res) tma_load_2d(st + 2 * kBufBytes, &tmW, &full[s], c * kChunkRows, 0);
+                        for (int sp = 0; sp < 4; ++sp) tma_load_2d(st + sp * kSpanBytes, &tmBuf, &full[s], d0 + 32 * sp, c * kChunkRows);
+                        if (c == cb) tma_load_2d(st + 2 * kBufBytes, &tmSrc1, &full[s], d0, 0);
+                        if (!w_res) tma_load_2d(st + 2 * kBufBytes, &tmW, &full[s], c * kChunkRows, 0);
+                    }
                     ++issued;
                     if (++s == stages) { s = 0; ph ^= 1u; st = smem; } else { st += stage_bytes; }
                 }
@@ -141,7 +155,7 @@ k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ 
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {          // 8 buffer rows per MMA: one 1024-byte row group (64 descriptor units)
                         mma_tf32(acc, d_hi + 64 * k, d_w + 2 * k, idesc_fold, (c_in | k) != 0);   // hi*W_hi | hi*W_lo
-                        mma_tf32(acc, d_lo + 64 * k, d_w + 2 * k, idesc_half, 1);              // + lo*W_hi
+                        if (c <= cb) mma_tf32(acc, d_lo + 64 * k, d_w + 2 * k, idesc_half, 1);     // + lo*W_hi (zero for bfloat16 rows)
                     }
                     mma_commit(&empty[s]);
                     if (++s == stages) { s = 0; ph ^= 1u; st = st0; } else { st += (uint32_t)stage_bytes; }
@@ -152,25 +166,45 @@ k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ 
     } else if (warp < 6) {
         const int t = threadIdx.x - 64;
         const long long total = my_tiles * nchunk;
-        int s = 0;
+        int s = 0, c = 0;                               // stage slot and chunk (32 buffer rows) of the current tile
         uint32_t ph = 0;
         for (long long q = 0; q < total; ++q) {
             if (!mbar_wait(&full[s], ph, abort)) break;
             uint4* hi = reinterpret_cast<uint4*>(smem + (size_t)s * stage_bytes);
             uint4* lo = reinterpret_cast<uint4*>(smem + (size_t)s * stage_bytes + kBufBytes);
+            if (c <= cb) {
 #pragma unroll
-            for (int c = 0; c < kBufBytes / 16 / kSplitThreads; ++c) {
-                const int idx = t + c * kSplitThreads;
-                // the tensor cores ignore the low 13 bits of an fp32 word, so the raw tile is the hi operand as it stands;
-                // lo = x - hi (exact), rounded to 11 significant bits so that the same truncation cuts nothing from it
-                const uint4 v = hi[idx];
-                uint4 l;
-                l.x = (__float_as_uint(__uint_as_float(v.x) - __uint_as_float(v.x & 0xffffe000u)) + 0x1000u) & 0xffffe000u;
-                l.y = (__float_as_uint(__uint_as_float(v.y) - __uint_as_float(v.y & 0xffffe000u)) + 0x1000u) & 0xffffe000u;
-                l.z = (__float_as_uint(__uint_as_float(v.z) - __uint_as_float(v.z & 0xffffe000u)) + 0x1000u) & 0xffffe000u;
-                l.w = (__float_as_uint(__uint_as_float(v.w) - __uint_as_float(v.w & 0xffffe000u)) + 0x1000u) & 0xffffe000u;
-                lo[idx] = l;
+                for (int cc = 0; cc < kBufBytes / 16 / kSplitThreads; ++cc) {
+                    const int idx = t + cc * kSplitThreads;
+                    // the tensor cores ignore the low 13 bits of an fp32 word, so the raw tile is the hi operand as it stands;
+                    // lo = x - hi (exact), rounded to 11 significant bits so that the same truncation cuts nothing from it
+                    const uint4 v = hi[idx];
+                    uint4 l;
+                    l.x = (__float_as_uint(__uint_as_float(v.x) - __uint_as_float(v.x & 0xffffe000u)) + 0x1000u) & 0xffffe000u;
+                    l.y = (__float_as_uint(__uint_as_float(v.y) - __uint_as_float(v.y & 0xffffe000u)) + 0x1000u) & 0xffffe000u;
+                    l.z = (__float_as_uint(__uint_as_float(v.z) - __uint_as_float(v.z & 0xffffe000u)) + 0x1000u) & 0xffffe000u;
+                    l.w = (__float_as_uint(__uint_as_float(v.w) - __uint_as_float(v.w & 0xffffe000u)) + 0x1000u) & 0xffffe000u;
+                    // the last row of chunk cb is a placeholder for the caller's first row (a bfloat16 row: remainder zero)
+                    if (c == cb && ((idx >> 3) & 31) == kChunkRows - 1) l = make_uint4(0u, 0u, 0u, 0u);
+                    lo[idx] = l;
+                }
             }
+            if (c >= cb) {
+                // bfloat16 rows from the staging area (256 bytes = 128 columns per row): 8 values -> two chunks of 4 floats
+                const uint4* src = reinterpret_cast<const uint4*>(smem + (size_t)s * stage_bytes + 2 * kBufBytes);
+                const int n_in = c == cb ? 16 : kChunkRows * 16;
+                for (int i = t; i < n_in; i += kSplitThreads) {
+                    const int rr = c == cb ? kChunkRows - 1 : i >> 4, q8 = i & 15;     // k row within the chunk, group of 8 columns
+                    const uint4 v = src[i];
+                    const uint4 a = make_uint4(v.x << 16, v.x & 0xffff0000u, v.y << 16, v.y & 0xffff0000u);
+                    const uint4 b = make_uint4(v.z << 16, v.z & 0xffff0000u, v.w << 16, v.w & 0xffff0000u);
+                    const int span = q8 >> 2, j = (q8 & 3) * 2;                          // 32-column span, 16-byte chunk within its row
+                    uint4* row = hi + span * (kSpanBytes / 16) + rr * 8;
+                    row[(((j >> 1) ^ (rr & 3)) << 1) | (j & 1)] = a;
+                    row[((((j + 1) >> 1) ^ (rr & 3)) << 1) | ((j + 1) & 1)] = b;
+                }
+            }
+            if (++c == nchunk) c = 0;
             fence_proxy_async_smem();
             mbar_arrive(&split_done[s]);
             if (++s == stages) { s = 0; ph ^= 1u; }
@@ -259,12 +293,15 @@ k_tc_rebuild(const __grid_constant__ CUtensorMap tmBuf, const __grid_constant__ 
 
 // See sage_internal.h.
 static cudaError_t launch_tc_rebuild_part(const float* Wsplit, int ldw, int j_pad, const float* Bsrc, float* Bdst, int64_t pitch, int r,
-                                          int keep, int* err, cudaStream_t st) {
+                                          int keep, int* err, cudaStream_t st, const void* src = nullptr, int64_t ld_src = 0, int n_new = 0,
+                                          int64_t D = 0) {
     if (keep <= 0 || r <= 0) return cudaSuccess;
     if (j_pad < 16 || j_pad > 128 || (j_pad & 15) || keep > j_pad || r > 512) return cudaErrorNotSupported;
     CUtensorMap tmBuf, tmW;
     // buffer: columns beyond D up to the pitch are zero and are rebuilt as zero, so the map spans the pitch
-    if (!tc::make_tmap_2d(&tmBuf, Bsrc, 4, (uint64_t)r, (uint64_t)pitch, (uint64_t)pitch, tc::kChunkRows, 1)) return cudaErrorNotSupported;
+    // direct form (src != nullptr): only the rows that are in the buffer, plus the placeholder row, are addressable
+    if (!tc::make_tmap_2d(&tmBuf, Bsrc, 4, (uint64_t)(src ? r - n_new + 1 : r), (uint64_t)pitch, (uint64_t)pitch, tc::kChunkRows, 1))
+        return cudaErrorNotSupported;
     const int kcols = ((r + tc::kChunkRows - 1) / tc::kChunkRows) * tc::kChunkRows;
     if (kcols > ldw) return cudaErrorNotSupported;
     if (!tc::make_tmap_2d(&tmW, Wsplit, 4, (uint64_t)(2 * j_pad), (uint64_t)kcols, (uint64_t)ldw, (uint32_t)(2 * j_pad)))
@@ -273,7 +310,14 @@ static cudaError_t launch_tc_rebuild_part(const float* Wsplit, int ldw, int j_pa
     const int nchunk = (r + tc::kChunkRows - 1) / tc::kChunkRows;
     const size_t w_all = (size_t)nchunk * 2 * j_pad * 128;
     const int w_res = w_all <= 64 * 1024 ? 1 : 0;
-    const int stage_bytes = w_res ? 2 * tc::kBufBytes : 2 * tc::kBufBytes + 2 * j_pad * 128;
+    CUtensorMap tmSrc = tmW, tmSrc1 = tmW;
+    if (src) {
+        if (!w_res || n_new < 2 || n_new >= r || (r - n_new + 1) % tc::kChunkRows != 0 || r % tc::kChunkRows != 0) return cudaErrorNotSupported;
+        if (!tc::make_tmap_2d_plain(&tmSrc, src, 2, (uint64_t)n_new, (uint64_t)D, (uint64_t)ld_src, 128, (uint32_t)tc::kChunkRows) ||
+            !tc::make_tmap_2d_plain(&tmSrc1, src, 2, (uint64_t)n_new, (uint64_t)D, (uint64_t)ld_src, 128, 1))
+            return cudaErrorNotSupported;
+    }
+    const int stage_bytes = (w_res ? 2 * tc::kBufBytes : 2 * tc::kBufBytes + 2 * j_pad * 128) + (src ? 8192 : 0);
     int stages = (int)((227 * 1024 - 1536 - (w_res ? w_all : 0)) / stage_bytes);
     if (stages > 8) stages = 8;
     if (stages < 2) return cudaErrorNotSupported;
@@ -282,7 +326,8 @@ static cudaError_t launch_tc_rebuild_part(const float* Wsplit, int ldw, int j_pa
     const int grid = (int)(num_tiles < 148 ? num_tiles : 148);
     cudaError_t e = cudaFuncSetAttribute(tc::k_tc_rebuild, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    tc::k_tc_rebuild<<<grid, tc::kThreads, smem, st>>>(tmBuf, tmW, r, keep, j_pad, pitch, num_tiles, Bdst, stages, w_res, err);
+    tc::k_tc_rebuild<<<grid, tc::kThreads, smem, st>>>(tmBuf, tmW, tmSrc, tmSrc1, src ? n_new : 0, r, keep, j_pad, pitch, num_tiles, Bdst, stages,
+                                                       w_res, err);
     return cudaGetLastError();
 }
 
@@ -303,6 +348,14 @@ cudaError_t launch_tc_rebuild(const float* Wsplit, int ldw, int j_pad, const flo
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;
+}
+
+// See sage_internal.h.
+cudaError_t launch_tc_rebuild_direct(const float* Wsplit, int ldw, int j_pad, const float* Bsrc, float* Bdst, int64_t pitch, int64_t D,
+                                     int r, int keep, const void* src, int64_t ld_src, int n_new, int* err, cudaStream_t st) {
+    if (keep <= 0 || r <= 0 || !src) return cudaErrorNotSupported;
+    if (j_pad < 16 || j_pad > 128 || (j_pad & 15) || keep > j_pad || r > 128) return cudaErrorNotSupported;
+    return launch_tc_rebuild_part(Wsplit, ldw, j_pad, Bsrc, Bdst, pitch, r, keep, err, st, src, ld_src, n_new, D);
 }
 
 }  // namespace sage

@@ -303,6 +303,41 @@ def test_bf16_rows_a_page_or_more_apart_score_like_packed_rows(N, D, ell, ld):
     assert np.max(np.abs(out[0][1] - ref["alpha"])) <= TOL_SCORE[torch.bfloat16]
 
 
+@pytest.mark.parametrize("N,D,ell,cuts", [(1000, 4104, 64, [300, 300, 400]), (777, 1000, 32, [97] * 8 + [1]), (900, 20008, 64, [66, 65, 64, 705]),
+                                          (500, 2056, 64, [500])])
+def test_rows_read_in_place_give_the_appended_result_bit_for_bit(N, D, ell, cuts):
+    """bfloat16 rows, ell = 32 / 64: shrink cycles whose ell + 1 new rows lie inside one update call read them where the
+    caller holds them (option 9, default) instead of appending them. The arithmetic is the same, so sketch and scores must
+    equal those of the always-append form (option 9 = 0) bit for bit, whatever the calls' sizes (leftover rows, cycles that
+    straddle two calls, calls shorter than a cycle); the counter of rows read in place must move, and both match the oracle."""
+    assert sum(cuts) == N
+    rows = lowrank_rows(N, D, 6, 0.4, N + D + ell, torch.bfloat16)
+    g = rows.to(torch.device("cuda", 0))
+    out = []
+    for direct in (1, 0):
+        fd = sage.SageFD(D, ell, torch.bfloat16, 0)
+        fd.set_option(9, direct)
+        r0 = 0
+        for c in cuts:
+            fd.update(g[r0:r0 + c])
+            r0 += c
+        fd.finalize()
+        S, sigma = fd.sketch()
+        a = fd.score(g)
+        torch.cuda.synchronize()
+        st = fd.stats()
+        fd.close()
+        assert st["device_flags"] == 0
+        out.append((S.cpu().numpy().copy(), sigma.cpu().numpy().copy(), a.cpu().numpy().copy(), st))
+    assert out[0][3]["rows_in_place"] > 0 and out[0][3]["rows_in_place"] % (ell + 1) == 0 and out[1][3]["rows_in_place"] == 0
+    assert out[0][3]["shrinks"] == out[1][3]["shrinks"]
+    assert np.array_equal(out[0][0], out[1][0]) and np.array_equal(out[0][1], out[1][1]) and np.array_equal(out[0][2], out[1][2])
+    ref = oracle.run(rows, D, ell, 0.1, route=1)
+    F2 = float(np.linalg.norm(metrics.rows_as_f64(rows, D)) ** 2)
+    assert metrics.signed_gram_norm(out[0][0].astype(np.float64), ref["S"]) / F2 <= 1e-4
+    assert np.max(np.abs(out[0][2].astype(np.float64) - ref["alpha"])) <= TOL_SCORE[torch.bfloat16]
+
+
 # ------------------------------------------------------------------ the two eigen-solve kernel families
 
 def _run_with_eig_variant(rows, D, ell, variant):
