@@ -44,7 +44,8 @@ FP32_ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12     # SMs x FMA lanes x 2 
 ALL = ("c1", "c2", "c3", "c4", "c5")
 # DRAM bytes per launch of the dominant streaming kernels from one ncu capture each (profiles/): the capture ran on a
 # scaled-down D and the traffic grows in proportion to D, so the figure is stored per buffer column.
-NCU_TRAFFIC_PER_COLUMN = {("c5", "rebuild"): (572.255e6 + 252.071e6) / 1117396, ("c5", "gram"): (573.417e6 + 3.676e6) / 1117396,
+# (Gram and rebuild: launches of cycles that read their 65 new rows in place, as 7 of 8 cycles of c5 do.)
+NCU_TRAFFIC_PER_COLUMN = {("c5", "rebuild"): (431.471e6 + 246.243e6) / 1117396, ("c5", "gram"): (433.734e6 + 3.507e6) / 1117396,
                           ("c5", "project"): (1294.674e6 + 3.727e6) / 1117396}
 
 
