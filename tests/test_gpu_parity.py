@@ -681,6 +681,19 @@ def test_select_from_host_matches_device_path():
     assert np.max(np.abs(scores.double().numpy() - ref["alpha"])) <= 1e-4
 
 
+def test_select_from_host_bf16_rows_read_in_place():
+    """The host pipeline with bfloat16 rows and ell = 64: inside it most shrink cycles read their rows straight from the
+    staging buffers the copies land in, so a copy that overwrote a buffer too early would show here. Same result as the
+    device path on the same rows, and both inside the tolerance of the oracle."""
+    N, D, ell = 1500, 2056, 64
+    rows = lowrank_rows(N, D, 6, 0.4, 21, torch.bfloat16)
+    ref = oracle.run(rows, D, ell, 0.1, route=1)
+    scores, idx = sage.sage_select_from_host(rows.pin_memory(), D, ell, 0.1, chunk_rows=400)
+    dev = gpu_run(rows, D, ell, 0.1, score_chunks=[400, 400, 400, 300])
+    assert np.max(np.abs(scores.double().numpy() - dev["alpha"])) <= 1e-6 and np.array_equal(idx.numpy(), dev["idx"])
+    assert np.max(np.abs(scores.double().numpy() - ref["alpha"])) <= TOL_SCORE[torch.bfloat16]
+
+
 def test_state_machine_and_errors():
     D, ell = 64, 4
     fd = sage.SageFD(D, ell, torch.float32, 0)
