@@ -78,7 +78,10 @@ sage_status_t sage_fd_reset(sage_fd_t* h);
  * delta = sigma_ell^2, Sigma'_jj = sqrt(max(sigma_j^2 - delta, 0)) and rebuild S <- Sigma' V^T
  * (Method, first paragraph). ell-1 rows survive a shrink, so after the first 2*ell rows a shrink
  * happens every ell+1 rows.
- *   rows  device, n x ld elements of the handle's dtype; n == 0 is a no-op.
+ *   rows  device, n x ld elements of the handle's dtype; n == 0 is a no-op. The library only reads them, by work
+ *         enqueued on cuda_stream (or ordered before what the caller enqueues there next): they may be changed by
+ *         later work on that stream, not before it. Rows that do not fill the buffer are copied into it; a shrink
+ *         whose new rows all come from this call may read them in place instead (option 9 of sage_fd_set_option).
  * Asynchronous on the stream: the shrink schedule depends only on counts, so no device->host
  * synchronisation happens here. Device-side problems are reported by sage_fd_finalize. */
 sage_status_t sage_fd_update(sage_fd_t* h, const void* rows, int64_t n, int64_t ld, void* cuda_stream);
