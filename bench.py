@@ -12,7 +12,7 @@ summed over ranks; with more than one GPU every rank runs an independent replica
 One invocation runs every listed workload and prints ONE JSON line (rank 0). The top-level fields are those of
 the headline workload (default: c5, the largest one that fits one GPU), timed over exactly K steps after W
 warm-up steps; the other workloads follow under "workloads" with the same fields, each timed over
-min(K, 5) steps so that the whole run stays within minutes: c1..c4 with the paper's sequential sketch, the same four
+10 steps (c1-c3) or min(K, 5) steps (c4) so that the whole run stays within minutes: c1..c4 with the paper's sequential sketch, the same four
 with the merged form of pass 1 (16 sketches, "cN_merged16"), and c2 / c3 given as the factors of their rows
 ("cN_factored"). `--impl reference` times the fp64 CPU oracle on
 the host cores instead, on a bounded sample of the headline workload.
@@ -525,7 +525,9 @@ def main():
     for key, n, P, fact in runs:
         w = shaped(n)
         is_head = key == headline
-        steps = args.steps if is_head else min(args.steps, 5)
+        # the headline is timed over exactly --steps steps; beside it the short workloads (c1-c3: a step is 6-460 ms) get
+        # ten timed steps, the long one (c4) at most five, unless fewer were asked for
+        steps = args.steps if is_head else (min(args.steps, 5) if (n in ("c4", "c5") or args.steps < 3) else 10)
         warm = args.warmup if is_head else 3
         results[key] = run_workload(w, args, steps, warm, ctx, want_e2e=not args.no_e2e and not fact and P == args.sketches and (is_head or not w.on_device),
                                     want_cpu=not args.no_cpu_baseline and is_head, sketches=P, factored=fact)
